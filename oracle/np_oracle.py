@@ -1,0 +1,336 @@
+"""CPU oracle for the delta-prefetch decode hot path.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, fp64 restatement of what one decode step computes, written from
+the paper (Sections 3.1, 3.4, 3.5) and from the workload definition, for the
+sole purpose of checking the CUDA library.  It shares no code with that library
+and imports nothing from it; only tests, the smoke check and the benchmark's
+CPU-baseline leg may import this file.  It is not tuned for speed.
+
+Conventions (same symbols as the C header):
+  L layers, D model width, M FFN width (multiple of 32), H predictor width,
+  k rows selected per layer per sequence, C resident capacity in rows,
+  W = M / 32 bitmap words per layer; bit j of word w is neuron 32*w + j.
+  bf16 tensors are passed as ``uint16`` bit patterns.
+
+Pins (see tests/test_oracle_*.py): exact rational brute force and structured
+closed forms for ``predict``; full-sort brute force, constructed ties and
+degenerate k for ``topk_bitmap``; the set identities of Eq. 2-3, slot-map
+bijection invariants and a set-based brute force for ``Residency.delta``;
+byte identity for ``install``; the dense SwiGLU library form when every row is
+active, linearity over disjoint sets and a scalar loop for ``sparse_mlp``; the
+paper's buffer-size arithmetic (Section 4.3) for ``record_bytes``.
+
+Parity unpinned against the paper (the paper is silent; these are this build's
+definitions, pinned only by invariants and determinism): the victim order of
+the LRU policy, and the truncation rule when a predicted set exceeds capacity.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+EVICT_EXACT = 0   # Eq. 3: every row that leaves the predicted set frees its slot
+EVICT_LRU = 1     # keep rows while capacity allows; evict least recently predicted
+
+
+# --------------------------------------------------------------------------
+# layout arithmetic (Section 3.5: neuron-centric records; Section 4.3: sizes)
+# --------------------------------------------------------------------------
+def record_bytes(D: int, elem_bytes: int = 2) -> int:
+    """One neuron record = its gate, up and transposed-down rows, back to back."""
+    return 3 * D * elem_bytes
+
+
+def resident_buffer_bytes(C: int, D: int, elem_bytes: int = 2) -> int:
+    """Bytes of one layer's resident row buffers (three projections, C rows each)."""
+    return C * record_bytes(D, elem_bytes)
+
+
+def record_offset_bytes(layer: int, neuron: int, M: int, D: int) -> int:
+    """Byte offset of a record in the layer-major store: consecutive neuron IDs
+    of a layer occupy consecutive byte ranges (Section 3.5)."""
+    return (layer * M + neuron) * record_bytes(D)
+
+
+def count_from_percent(pct: int, M: int) -> int:
+    """Rows for a density or capacity given in percent of M (rounded to nearest)."""
+    return (pct * M + 50) // 100
+
+
+# --------------------------------------------------------------------------
+# number formats
+# --------------------------------------------------------------------------
+def bf16_to_f64(u16: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to fp64."""
+    u16 = np.ascontiguousarray(u16, dtype=np.uint16)
+    return (u16.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def fp32_order_key(z32: np.ndarray) -> np.ndarray:
+    """Order-preserving map from fp32 bit patterns to uint32 (larger float ->
+    larger key; +0 above -0): flip all bits of negatives, set the sign bit of
+    the rest."""
+    b = np.ascontiguousarray(z32, dtype=np.float32).view(np.uint32)
+    neg = (b >> np.uint32(31)).astype(bool)
+    return np.where(neg, ~b, b | np.uint32(0x80000000)).astype(np.uint32)
+
+
+def bitmap_to_bool(words: np.ndarray, M: int) -> np.ndarray:
+    """uint32 words ``[..., W]`` -> bool ``[..., M]``."""
+    words = np.ascontiguousarray(words).view(np.uint32)
+    shifts = np.arange(32, dtype=np.uint32)
+    bits = (words[..., :, None] >> shifts) & np.uint32(1)
+    return bits.reshape(*words.shape[:-1], words.shape[-1] * 32)[..., :M].astype(bool)
+
+
+def bool_to_bitmap(bits: np.ndarray) -> np.ndarray:
+    """bool ``[..., M]`` (M multiple of 32) -> uint32 words ``[..., M/32]``."""
+    bits = np.asarray(bits, dtype=bool)
+    M = bits.shape[-1]
+    assert M % 32 == 0
+    b = bits.reshape(*bits.shape[:-1], M // 32, 32).astype(np.uint64)
+    weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
+    return (b * weights).sum(axis=-1).astype(np.uint32)
+
+
+# --------------------------------------------------------------------------
+# stage 1: predictor forward (one pass after layer 0 scores every FFN neuron of
+# every downstream layer; Section 3.1 step 2, in the workload's MLP form
+# D -> H (ReLU) -> L*M, no biases)
+# --------------------------------------------------------------------------
+def predict(w1_u16: np.ndarray, w2_u16: np.ndarray, x_u16: np.ndarray, L: int, M: int) -> np.ndarray:
+    """logits[b, l, n] = sum_m W2[l*M + n, m] * max(0, sum_j W1[m, j] * x[b, j]), fp64.
+
+    The hidden vector is kept in fp64 (never rounded)."""
+    W1 = bf16_to_f64(w1_u16)                       # [H, D]
+    x = bf16_to_f64(x_u16)                         # [B, D]
+    h = np.maximum(0.0, x @ W1.T)                  # [B, H]
+    B = x.shape[0]
+    z = np.empty((B, L, M), dtype=np.float64)
+    for l in range(L):                             # layer by layer only to bound memory
+        W2l = bf16_to_f64(w2_u16[l * M:(l + 1) * M])   # [M, H]
+        z[:, l, :] = h @ W2l.T
+    return z
+
+
+# --------------------------------------------------------------------------
+# stage 2: per-layer top-k -> active bitmaps (replaces the paper's centroid
+# lookup by a fixed budget of k rows per layer, Section 4.1's K_max budgets)
+# --------------------------------------------------------------------------
+def topk_bitmap(logits_f32: np.ndarray, k: int) -> np.ndarray:
+    """For every (sequence, layer): the k largest logits under the total order
+    (fp32 key descending, neuron index ascending); OR over sequences.
+
+    ``logits_f32`` is ``[B, L, M]`` float32; returns uint32 ``[L, M/32]``."""
+    z = np.ascontiguousarray(logits_f32, dtype=np.float32)
+    B, L, M = z.shape
+    bits = np.zeros((L, M), dtype=bool)
+    for b in range(B):
+        for l in range(L):
+            key = fp32_order_key(z[b, l]).astype(np.int64)
+            order = np.argsort(-key, kind="stable")     # ties keep ascending index
+            bits[l, order[:k]] = True
+    return bool_to_bitmap(bits)
+
+
+# --------------------------------------------------------------------------
+# stage 3a: delta / residency (Section 3.4, Eq. 2-3, slot map S in Z^M)
+# --------------------------------------------------------------------------
+class LayerDelta:
+    """What one layer's delta step emits (all ascending neuron index)."""
+
+    def __init__(self):
+        self.delta_ids = np.zeros(0, np.int32)     # incoming rows that got a slot
+        self.delta_slots = np.zeros(0, np.int32)   # their slots
+        self.evict_ids = np.zeros(0, np.int32)     # rows that released their slot
+        self.overflow_ids = np.zeros(0, np.int32)  # incoming rows left non-resident
+        self.active_ids = np.zeros(0, np.int32)    # predicted AND resident, after update
+        self.active_slots = np.zeros(0, np.int32)
+        self.n_pred = 0
+        self.n_kept = 0
+
+
+class Residency:
+    """Per-layer resident-row state: bitmap R, slot map S (-1 = not resident),
+    owner (slot -> neuron, -1 = free) and last-predicted step stamps."""
+
+    def __init__(self, L: int, M: int, C: int, policy: int = EVICT_EXACT):
+        assert M % 32 == 0 and 0 < C <= M
+        self.L, self.M, self.C, self.policy = L, M, C, policy
+        self.reset()
+
+    def reset(self):
+        L, M, C = self.L, self.M, self.C
+        self.R = np.zeros((L, M), dtype=bool)
+        self.S = np.full((L, M), -1, dtype=np.int32)
+        self.owner = np.full((L, C), -1, dtype=np.int32)
+        self.stamp = np.full((L, M), -1, dtype=np.int32)
+        self.t = 0
+
+    def delta(self, pred_words: np.ndarray) -> list:
+        """One decode step for all layers.  ``pred_words`` uint32 ``[L, W]``."""
+        P_all = bitmap_to_bool(pred_words, self.M)
+        out = [self._delta_layer(l, P_all[l]) for l in range(self.L)]
+        self.t += 1
+        return out
+
+    def _delta_layer(self, l: int, P: np.ndarray) -> LayerDelta:
+        R, S, owner, stamp = self.R[l], self.S[l], self.owner[l], self.stamp[l]
+        C = self.C
+        res = LayerDelta()
+        # 1. kept rows, incoming rows (Eq. 2) and eviction candidates (Eq. 3's set)
+        kept = np.flatnonzero(P & R)
+        D_in = np.flatnonzero(P & ~R)               # ascending neuron index
+        cand = np.flatnonzero(R & ~P)
+        res.n_pred = int(P.sum())
+        res.n_kept = int(kept.size)
+        # 2. every predicted row is stamped with the current step
+        stamp[P] = self.t
+        # 3. victims
+        if self.policy == EVICT_EXACT:
+            E = cand
+        else:
+            free = C - int(R.sum())
+            need = max(0, int(D_in.size) - free)
+            if need >= cand.size:
+                E = cand
+            else:
+                # least recently predicted first, ties by lower neuron index
+                order = np.lexsort((cand, stamp[cand]))
+                E = np.sort(cand[order[:need]])
+        # 4. outgoing rows release their slots
+        for n in E:
+            owner[S[n]] = -1
+            S[n] = -1
+            R[n] = False
+        res.evict_ids = E.astype(np.int32)
+        # 5. i-th incoming row (ascending neuron) takes the i-th free slot (ascending slot)
+        avail = np.flatnonzero(owner == -1)
+        n_fit = min(int(D_in.size), int(avail.size))
+        for i in range(n_fit):
+            n, s = int(D_in[i]), int(avail[i])
+            S[n] = s
+            owner[s] = n
+            R[n] = True
+        res.delta_ids = D_in[:n_fit].astype(np.int32)
+        res.delta_slots = avail[:n_fit].astype(np.int32)
+        res.overflow_ids = D_in[n_fit:].astype(np.int32)
+        # 6. the rows the sparse MLP will use: predicted and resident
+        act = np.flatnonzero(P & R)
+        res.active_ids = act.astype(np.int32)
+        res.active_slots = S[act].astype(np.int32)
+        return res
+
+    def resident_words(self) -> np.ndarray:
+        return bool_to_bitmap(self.R)
+
+
+# --------------------------------------------------------------------------
+# stage 3b/3c: install (Section 3.5: interleaved records -> three row buffers)
+# --------------------------------------------------------------------------
+def coalesce_runs(ids: np.ndarray) -> list:
+    """Ascending IDs -> list of (first_id, count) with adjacent IDs merged."""
+    runs = []
+    for n in np.asarray(ids, dtype=np.int64):
+        if runs and runs[-1][0] + runs[-1][1] == n:
+            runs[-1][1] += 1
+        else:
+            runs.append([int(n), 1])
+    return [(a, c) for a, c in runs]
+
+
+def install(backing_u16: np.ndarray, gate: np.ndarray, up: np.ndarray, downT: np.ndarray,
+            layer: int, delta_ids: np.ndarray, delta_slots: np.ndarray) -> int:
+    """Copy record (layer, n) to slot s of the three buffers for every (n, s).
+
+    ``backing_u16`` is ``[L, M, 3, D]``; the buffers are ``[L, C, D]``.  Returns
+    the bytes copied.  Reads go run by run, as the transfer path would issue
+    them; the result does not depend on that grouping."""
+    pos = 0
+    for first, count in coalesce_runs(delta_ids):
+        block = backing_u16[layer, first:first + count]      # [count, 3, D]
+        for r in range(count):
+            s = int(delta_slots[pos])
+            gate[layer, s] = block[r, 0]
+            up[layer, s] = block[r, 1]
+            downT[layer, s] = block[r, 2]
+            pos += 1
+    assert pos == len(delta_ids)
+    return pos * backing_u16.shape[-1] * 3 * 2
+
+
+# --------------------------------------------------------------------------
+# stage 4: sparse SwiGLU MLP through the slot map (Section 3.4)
+# --------------------------------------------------------------------------
+def sparse_mlp(gate: np.ndarray, up: np.ndarray, downT: np.ndarray, layer: int,
+               slots: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """y[b] = sum_i silu(g_i) * u_i * downT[s_i], g_i = gate[s_i] . x[b], u_i = up[s_i] . x[b].
+
+    ``slots`` are the buffer slots of the active rows; ``x`` is fp64 ``[B, D]``."""
+    slots = np.asarray(slots, dtype=np.int64)
+    x = np.asarray(x, dtype=np.float64)
+    G = bf16_to_f64(gate[layer, slots])          # [n, D]
+    U = bf16_to_f64(up[layer, slots])
+    Dn = bf16_to_f64(downT[layer, slots])
+    g = x @ G.T                                  # [B, n]
+    u = x @ U.T
+    a = g / (1.0 + np.exp(-g)) * u
+    return a @ Dn                                # [B, D]
+
+
+def sparse_mlp_from_store(backing_u16: np.ndarray, layer: int, ids: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """Same sum, rows taken straight from the record store by neuron ID."""
+    ids = np.asarray(ids, dtype=np.int64)
+    x = np.asarray(x, dtype=np.float64)
+    rec = backing_u16[layer, ids]                # [n, 3, D]
+    G, U, Dn = bf16_to_f64(rec[:, 0]), bf16_to_f64(rec[:, 1]), bf16_to_f64(rec[:, 2])
+    g = x @ G.T
+    u = x @ U.T
+    a = g / (1.0 + np.exp(-g)) * u
+    return a @ Dn
+
+
+# --------------------------------------------------------------------------
+# one whole decode step of the stack (residual chain x_{l+1} = x_l + MLP_l(x_l))
+# --------------------------------------------------------------------------
+class Engine:
+    """State carried across decode steps: residency tables and resident buffers."""
+
+    def __init__(self, L, D, M, H, k, C, policy, w1_u16, w2_u16, backing_u16):
+        self.L, self.D, self.M, self.H, self.k, self.C = L, D, M, H, k, C
+        self.w1, self.w2, self.backing = w1_u16, w2_u16, backing_u16
+        self.res = Residency(L, M, C, policy)
+        self.gate = np.zeros((L, C, D), dtype=np.uint16)
+        self.up = np.zeros((L, C, D), dtype=np.uint16)
+        self.downT = np.zeros((L, C, D), dtype=np.uint16)
+
+    def step(self, x_u16: np.ndarray, pred_words: np.ndarray = None, logits_f32: np.ndarray = None):
+        """Run predict -> top-k -> delta -> install -> MLP chain for one token.
+
+        ``pred_words`` (or ``logits_f32``) may be supplied to take the selection
+        (or the logits) from elsewhere; returns a dict of everything produced."""
+        out = {}
+        if pred_words is None:
+            if logits_f32 is None:
+                z = predict(self.w1, self.w2, x_u16, self.L, self.M)
+                out["logits"] = z
+                logits_f32 = z.astype(np.float32)
+            pred_words = topk_bitmap(logits_f32, self.k)
+        out["pred"] = pred_words
+        deltas = self.res.delta(pred_words)
+        out["deltas"] = deltas
+        nbytes = 0
+        for l, d in enumerate(deltas):
+            nbytes += install(self.backing, self.gate, self.up, self.downT, l, d.delta_ids, d.delta_slots)
+        out["installed_bytes"] = nbytes
+        x = bf16_to_f64(x_u16)
+        ys = []
+        xs = [x]
+        for l, d in enumerate(deltas):
+            y = sparse_mlp(self.gate, self.up, self.downT, l, d.active_slots, x)
+            ys.append(y)
+            x = x + y
+            xs.append(x)
+        out["y_layers"] = ys
+        out["x_layers"] = xs
+        out["x_final"] = x
+        return out

@@ -1,0 +1,192 @@
+"""Seeded synthetic workloads shaped like the paper's MLP stacks.
+
+This module only draws random numbers and lays bytes out; it contains none of
+the method's arithmetic (no predictor, selection, residency or MLP math), so
+the CPU oracle and the CUDA path can both be fed from it without sharing code.
+
+Everything is handed out as raw bf16 bit patterns (``torch.bfloat16`` tensors,
+or ``uint16`` views of them): those bytes are the ground truth both sides read.
+
+Recipe
+------
+* Weights: one ``torch.Generator`` per tensor, seeded with
+  ``seed * 1_000_003 + tensor_id``; ``randn * 0.02`` rounded to bf16.
+  ``tensor_id``: 0 = W1 ``[H, D]``, 1 = W2 ``[L*M, H]``, ``2 + l`` = the
+  neuron-centric record block of layer ``l``, ``[M, 3, D]`` with the three rows
+  of a record being gate, up and transposed-down (the layer-major repacked
+  layout of Section 3.5 of the paper, with a pinned-host array standing in for
+  the NVMe file).
+* Hidden states: ``x_0 ~ N(0, I)``, ``x_t = rho * x_{t-1} + sqrt(1 - rho^2) *
+  eps_t`` in fp32 (generator seeded ``seed * 1_000_003 + 999``), rounded to
+  bf16.  For batches, every sequence mixes one shared AR(1) driver with its own
+  AR(1) process: ``x^(b) = sqrt(gamma) * s + sqrt(1 - gamma) * u^(b)``.
+
+The paper's own activations (Mistral-7B / Llama-3-8B on WikiText-2 and
+HellaSwag) are not available; these inputs stand in for them and reproduce only
+the shapes and the token-to-token persistence statistic.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Optional
+
+import torch
+
+_SEED_MUL = 1_000_003
+
+
+@dataclasses.dataclass(frozen=True)
+class StackConfig:
+    """Shapes of one synthetic MLP stack (notation: L, D, M, H, k, C)."""
+
+    name: str
+    n_layers: int      # L
+    d_model: int       # D
+    d_ffn: int         # M
+    d_pred: int        # H
+    density_pct: int   # top-k density, percent of M
+    capacity_pct: int  # resident capacity, percent of M
+    n_tokens: int
+    seed: int
+    rho: float
+
+    @property
+    def top_k(self) -> int:
+        return (self.density_pct * self.d_ffn + 50) // 100
+
+    @property
+    def capacity(self) -> int:
+        return (self.capacity_pct * self.d_ffn + 50) // 100
+
+    @property
+    def record_elems(self) -> int:
+        return 3 * self.d_model
+
+    @property
+    def record_bytes(self) -> int:
+        return 3 * self.d_model * 2
+
+    def with_(self, **kw) -> "StackConfig":
+        return dataclasses.replace(self, **kw)
+
+
+# rho of the 7B-class shapes is the value at which this generator gives ~83 %
+# token-to-token overlap of the top-k sets (measured by the bench and printed).
+CONFIGS = {
+    "tiny": StackConfig("tiny", 2, 256, 1024, 64, 10, 20, 16, 0, 0.9),
+    "small": StackConfig("small", 3, 512, 2048 + 32, 96, 10, 25, 12, 7, 0.95),
+    "7b": StackConfig("7b", 32, 4096, 11008, 512, 10, 25, 128, 1, 0.97),
+    "13b": StackConfig("13b", 40, 5120, 13824, 640, 8, 25, 256, 2, 0.97),
+    "70b": StackConfig("70b", 80, 8192, 28672, 1024, 5, 20, 128, 3, 0.97),
+    "stress": StackConfig("stress", 32, 4096, 11008, 512, 10, 25, 512, 4, 0.97),
+}
+
+
+def _gen(seed: int, tensor_id: int, device: str) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(seed * _SEED_MUL + tensor_id)
+    return g
+
+
+def _randn_bf16(shape, seed: int, tensor_id: int, device: str, out: Optional[torch.Tensor] = None,
+                chunk_elems: int = 1 << 26) -> torch.Tensor:
+    """``randn * 0.02`` rounded to bf16, drawn in bounded chunks from one generator."""
+    n = math.prod(shape)
+    g = _gen(seed, tensor_id, device)
+    if out is None:
+        out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+    flat = out.view(-1)
+    assert flat.numel() == n
+    for lo in range(0, n, chunk_elems):
+        hi = min(n, lo + chunk_elems)
+        blk = torch.randn(hi - lo, generator=g, device=device, dtype=torch.float32)
+        flat[lo:hi].copy_(blk.mul_(0.02).to(torch.bfloat16))
+    return out
+
+
+def predictor_weights(cfg: StackConfig, device: str = "cpu"):
+    """W1 ``[H, D]`` and W2 ``[L*M, H]`` (row-major, layer-major), bf16."""
+    w1 = _randn_bf16((cfg.d_pred, cfg.d_model), cfg.seed, 0, device)
+    w2 = _randn_bf16((cfg.n_layers * cfg.d_ffn, cfg.d_pred), cfg.seed, 1, device)
+    return w1, w2
+
+
+def fill_backing_store(cfg: StackConfig, out: torch.Tensor, gen_device: str = "cpu") -> torch.Tensor:
+    """Fill ``out`` (bf16 ``[L, M, 3, D]``, usually pinned host memory) layer by layer.
+
+    ``gen_device`` may be ``"cuda"`` to draw the large stores quickly; the bytes
+    then come from the CUDA generator stream of the same seeds and are copied
+    into ``out``.
+    """
+    L, M, D = cfg.n_layers, cfg.d_ffn, cfg.d_model
+    assert tuple(out.shape) == (L, M, 3, D) and out.dtype == torch.bfloat16
+    for l in range(L):
+        if gen_device == "cpu" and out.device.type == "cpu":
+            _randn_bf16((M, 3, D), cfg.seed, 2 + l, "cpu", out=out[l])
+        else:
+            blk = _randn_bf16((M, 3, D), cfg.seed, 2 + l, gen_device)
+            out[l].copy_(blk)
+    return out
+
+
+def backing_store(cfg: StackConfig, pin: bool = False, gen_device: str = "cpu") -> torch.Tensor:
+    out = torch.empty((cfg.n_layers, cfg.d_ffn, 3, cfg.d_model), dtype=torch.bfloat16,
+                      pin_memory=pin)
+    return fill_backing_store(cfg, out, gen_device)
+
+
+def hidden_states(cfg: StackConfig, n_tokens: Optional[int] = None, batch: int = 1,
+                  rho: Optional[float] = None, gamma: float = 0.9) -> torch.Tensor:
+    """AR(1) layer-0 hidden states, bf16 ``[T, B, D]`` (CPU generator, fp32 recursion)."""
+    T = cfg.n_tokens if n_tokens is None else n_tokens
+    rho = cfg.rho if rho is None else rho
+    D = cfg.d_model
+    g = _gen(cfg.seed, 999, "cpu")
+    nproc = 1 if batch == 1 else batch + 1   # [shared driver] + one per sequence
+    innov = math.sqrt(max(0.0, 1.0 - rho * rho))
+    state = torch.randn(nproc, D, generator=g, dtype=torch.float32)
+    out = torch.empty(T, batch, D, dtype=torch.bfloat16)
+    for t in range(T):
+        if t > 0:
+            eps = torch.randn(nproc, D, generator=g, dtype=torch.float32)
+            state = rho * state + innov * eps
+        if batch == 1:
+            out[t, 0] = state[0].to(torch.bfloat16)
+        else:
+            mix = math.sqrt(gamma) * state[0:1] + math.sqrt(1.0 - gamma) * state[1:]
+            out[t] = mix.to(torch.bfloat16)
+    return out
+
+
+def random_bitmaps(n_layers: int, d_ffn: int, n_set: int, seed: int, n_steps: int,
+                   persistence: float = 0.8) -> torch.Tensor:
+    """Sequence of random predicted bitmaps, int32-typed uint32 words ``[T, L, M/32]``.
+
+    Each step keeps about ``persistence`` of the previous set and redraws the
+    rest uniformly; used to drive the residency manager without a predictor.
+    Bit ``j`` of word ``w`` stands for neuron ``32 * w + j``.
+    """
+    assert d_ffn % 32 == 0
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed * _SEED_MUL + 31337)
+    W = d_ffn // 32
+    out = torch.zeros(n_steps, n_layers, W, dtype=torch.int64)
+    weights = (1 << torch.arange(32, dtype=torch.int64))
+    for l in range(n_layers):
+        cur = torch.randperm(d_ffn, generator=g)[:n_set]
+        for t in range(n_steps):
+            if t > 0:
+                keep_n = int(round(persistence * n_set))
+                keep = cur[torch.randperm(cur.numel(), generator=g)[:keep_n]]
+                mask = torch.ones(d_ffn, dtype=torch.bool)
+                mask[cur] = False
+                pool = mask.nonzero().flatten()
+                new = pool[torch.randperm(pool.numel(), generator=g)[: n_set - keep_n]]
+                cur = torch.cat([keep, new])
+            bits = torch.zeros(d_ffn, dtype=torch.int64)
+            bits[cur] = 1
+            out[t, l] = (bits.view(W, 32) * weights).sum(dim=1)
+    # store as the uint32 bit pattern inside int32
+    out = torch.where(out >= (1 << 31), out - (1 << 32), out)
+    return out.to(torch.int32)
