@@ -1,0 +1,247 @@
+/*
+ * np.h — C ABI of the delta-prefetch sparse-MLP decode path for NVIDIA B200 (sm_100a).
+ *
+ * One decode step of the method (Section 3.1 of the paper, steps 2-4, in the
+ * form the synthetic MLP-stack workload fixes):
+ *
+ *   np_predict     one predictor pass scores every FFN neuron of every layer and
+ *                  keeps the top-k per layer as an active-neuron bitmap
+ *   np_delta       compares the predicted sets with the resident rows (Eq. 2-3),
+ *                  assigns freed slots to incoming rows, updates the slot map S
+ *   np_install     moves only the incoming rows from the neuron-centric record
+ *                  store (pinned host memory stands in for the NVMe file) and
+ *                  scatters them into the three resident row buffers (Section 3.5)
+ *   np_sparse_mlp  SwiGLU MLP over the active resident rows through the slot map
+ *   np_step        the four above for one token, with the install of later layers
+ *                  overlapped with the MLP of earlier ones
+ *
+ * Symbols: L layers, D model width, M FFN width, H predictor width, k rows kept
+ * per layer per sequence, C resident capacity in rows per layer (the paper's
+ * K_max), B sequences, W = M/32 bitmap words per layer, REC = 3*D*2 bytes.
+ *
+ * Conventions
+ *   - Every call returns an int: 0 = NP_OK, < 0 error, > 0 warning (work done).
+ *   - "dev" pointers are device global memory, "host" pointers host memory;
+ *     "pinned" means page-locked and reachable from the device.
+ *   - Streams are passed as void* holding a cudaStream_t (NULL = default stream).
+ *     Work is enqueued, not waited for, unless a function says it synchronises.
+ *   - The caller owns every large buffer (np_buffers) and keeps it alive and
+ *     unchanged in size until np_destroy.  The library owns only its residency
+ *     tables, list buffers, events and the context.
+ *   - A context is used from one host thread at a time.
+ *   - Bitmaps: uint32 words, bit j of word w is neuron 32*w + j.
+ *   - bf16 arrays are raw 16-bit patterns; row-major, innermost dimension last.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails
+ *     with NP_E_CUDA.
+ */
+#ifndef NP_H_
+#define NP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NP_VERSION 1
+
+/* return codes */
+#define NP_OK           0
+#define NP_E_INVAL     -1   /* bad argument or configuration */
+#define NP_E_STATE     -2   /* call out of order (e.g. install before delta) */
+#define NP_E_CUDA      -3   /* a CUDA runtime call failed; see np_last_error */
+#define NP_E_NOMEM     -4   /* allocation of library-owned state failed */
+#define NP_E_DEVICE    -5   /* a kernel's own bounds check tripped; state is suspect */
+#define NP_W_OVERFLOW   1   /* some layer's predicted set did not fit capacity */
+#define NP_W_CHUNKED    2   /* some layer's delta exceeded staging and was split */
+
+/* eviction policies (np_config.evict_policy) */
+#define NP_EVICT_EXACT  0   /* Eq. 3: every row leaving the predicted set frees its slot */
+#define NP_EVICT_LRU    1   /* keep rows while capacity allows; evict least recently predicted,
+                               ties by lower neuron index (not in the paper) */
+
+/* how np_install moves records (np_config.transfer_mode) */
+#define NP_XFER_MEMCPY_RUNS  0  /* one cudaMemcpyAsync per run of adjacent neuron IDs into
+                                   device staging, then the scatter kernel */
+#define NP_XFER_HOST_GATHER  1  /* host threads pack records into pinned staging, one
+                                   cudaMemcpyAsync per chunk, then the scatter kernel */
+#define NP_XFER_ZERO_COPY    2  /* the scatter kernel reads the pinned store directly by
+                                   neuron ID (the paper's mapped-staging idea); no host sync */
+
+/* np_config.flags */
+#define NP_F_CHECK_BOUNDS    1  /* kernels validate every slot / neuron index and report
+                                   through NP_E_DEVICE instead of touching memory */
+
+/* per-layer counters written by np_delta (np_read_counters) */
+#define NP_CNT_PRED      0  /* |P|                      */
+#define NP_CNT_KEPT      1  /* |P and R_prev|           */
+#define NP_CNT_DELTA     2  /* incoming rows given a slot */
+#define NP_CNT_EVICT     3  /* rows that released a slot */
+#define NP_CNT_OVERFLOW  4  /* incoming rows left without a slot */
+#define NP_CNT_ACTIVE    5  /* |P and R| after the update */
+#define NP_CNT_RESIDENT  6  /* |R| after the update     */
+#define NP_CNT_STEP      7  /* decode step index t of this update */
+#define NP_N_COUNTERS    8
+
+typedef struct np_ctx np_ctx;
+
+typedef struct np_config {
+  int32_t n_layers;       /* L >= 1 */
+  int32_t d_model;        /* D, multiple of 8 */
+  int32_t d_ffn;          /* M, multiple of 32 */
+  int32_t d_pred;         /* H, multiple of 8 */
+  int32_t top_k;          /* k, 0 <= k <= C */
+  int32_t capacity;       /* C, 1 <= C <= M */
+  int32_t max_batch;      /* largest B any call will pass, 1..16 */
+  int32_t evict_policy;   /* NP_EVICT_* */
+  int32_t staging_rows;   /* records the staging buffer holds (>= 1); larger deltas are
+                             split into chunks (Section 3.5, bounded staging) */
+  int32_t transfer_mode;  /* NP_XFER_* */
+  int32_t flags;          /* NP_F_* */
+  int32_t host_threads;   /* worker threads for NP_XFER_HOST_GATHER (0 = pick) */
+  int32_t reserved[4];    /* must be 0 */
+} np_config;
+
+/* Byte counts of the caller-owned buffers for a configuration. */
+typedef struct np_sizes {
+  uint64_t w1_bytes;          /* bf16 [H][D] */
+  uint64_t w2_bytes;          /* bf16 [L*M][H] */
+  uint64_t backing_bytes;     /* bf16 [L][M][3][D] */
+  uint64_t row_buffer_bytes;  /* bf16 [L][C][D], each of gate / up / downT */
+  uint64_t staging_bytes;     /* staging_rows * REC (device; pinned host too for HOST_GATHER) */
+  uint64_t workspace_bytes;   /* device scratch */
+  uint64_t host_lists_bytes;  /* pinned host area the delta lists are mirrored into */
+  uint64_t logits_bytes;      /* fp32 [max_batch][L][M] */
+  uint64_t bitmap_bytes;      /* uint32 [L][W] */
+  uint64_t record_bytes;      /* REC */
+} np_sizes;
+
+typedef struct np_buffers {
+  const void* w1;          /* dev  */
+  const void* w2;          /* dev  */
+  const void* backing;     /* pinned host (cudaHostAlloc or cudaHostRegister) */
+  void* gate_buf;          /* dev  */
+  void* up_buf;            /* dev  */
+  void* downT_buf;         /* dev  */
+  void* staging;           /* dev; unused (may be NULL) with NP_XFER_ZERO_COPY */
+  void* host_staging;      /* pinned host, staging_bytes; only for NP_XFER_HOST_GATHER */
+  void* workspace;         /* dev, 256-byte aligned */
+  void* host_lists;        /* pinned host */
+} np_buffers;
+
+/* Device views of one layer's lists from the last np_delta (valid until the next). */
+typedef struct np_delta_view {
+  const int32_t* delta_ids;     /* dev [n_delta]    incoming neurons, ascending */
+  const int32_t* delta_slots;   /* dev [n_delta]    their slots */
+  const int32_t* evict_ids;     /* dev [n_evict]    neurons that released their slot, ascending */
+  const int32_t* overflow_ids;  /* dev [n_overflow] incoming neurons left non-resident, ascending */
+  const int32_t* active_ids;    /* dev [n_active]   predicted and resident, ascending */
+  const int32_t* active_slots;  /* dev [n_active] */
+  const int32_t* counters;      /* dev [NP_N_COUNTERS] */
+} np_delta_view;
+
+/* Library version (NP_VERSION of the build). */
+int np_version(void);
+
+/* Fills *out with the buffer sizes `cfg` needs.  Pure host arithmetic (record
+ * size: Section 3.5; buffer size: Section 4.3).  NP_E_INVAL on a bad config. */
+int np_query_sizes(const np_config* cfg, np_sizes* out);
+
+/* Creates a context with empty residency (the cold-start state of Section 3.4:
+ * no row resident, every slot free).  Copies cfg; keeps the pointers in bufs.
+ * Allocates the library's tables on the current device and synchronises.
+ * Errors: NP_E_INVAL (config, NULL/misaligned/unpinned buffers), NP_E_NOMEM, NP_E_CUDA. */
+int np_init(np_ctx** out, const np_config* cfg, const np_buffers* bufs);
+
+/* Waits for the context's outstanding work, frees library-owned memory. */
+int np_destroy(np_ctx* ctx);
+
+/* Back to the cold-start state (tables cleared, step counter 0); the row
+ * buffers are left as they are.  Enqueued on `stream`. */
+int np_reset(np_ctx* ctx, void* stream);
+
+/* Text of the last error of this context (or of the last failed np_init /
+ * np_query_sizes when ctx is NULL).  Never NULL; valid until the next call. */
+const char* np_last_error(const np_ctx* ctx);
+
+/* Stage 1 + 2: predictor forward and per-layer top-k (Section 3.1 step 2; the
+ * workload's predictor is logits = W2 * relu(W1 * x), no biases).
+ *   x_bf16       dev bf16 [B][D]   layer-0 hidden states
+ *   logits_out   dev fp32 [B][L][M] or NULL (kept internally either way)
+ *   bitmap_out   dev uint32 [L][W] or NULL: union over the B sequences of each
+ *                sequence's k highest logits per layer; order = fp32 value
+ *                descending (+0 above -0), ties to the lower neuron index
+ * The bitmap is also kept inside the context for np_delta(ctx, NULL, ...).
+ * Errors: NP_E_INVAL (NULL x, B outside 1..max_batch), NP_E_CUDA. */
+int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out,
+               uint32_t* bitmap_out, void* stream);
+
+/* Stage 2 alone on caller-supplied logits (dev fp32 [B][L][M]) -> bitmap_out
+ * (dev uint32 [L][W], required).  Does not touch the context's own bitmap. */
+int np_topk(np_ctx* ctx, const float* logits, int32_t B, uint32_t* bitmap_out, void* stream);
+
+/* Stage 3a: delta and residency update for all layers (Section 3.4, Eq. 2-3).
+ *   pred_bitmap  dev uint32 [L][W], or NULL to use the last np_predict's result.
+ * Per layer: incoming = P \ R (ascending), victims per the eviction policy,
+ * victims' slots cleared in S/owner, i-th incoming row gets the i-th free slot
+ * (ascending slot index); rows beyond the free slots are listed as overflow and
+ * stay non-resident.  Tables are updated here, before the rows arrive; use
+ * np_install before np_sparse_mlp.  Advances the step counter.
+ * Does not synchronise.  Warnings are reported by np_install / np_read_counters. */
+int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream);
+
+/* Stage 3b + 3c for layers [layer_begin, layer_end): copy each incoming record
+ * (L, n) = bytes [(l*M + n)*REC, +REC) of the store to slot S[n] of the three
+ * row buffers, on `copy_stream`, and mark each layer installed (np_sparse_mlp
+ * orders itself after that mark).  The copy stream is first ordered after the
+ * delta step.  With NP_XFER_MEMCPY_RUNS / NP_XFER_HOST_GATHER this call blocks
+ * the host until the delta lists of the last np_delta are readable; with
+ * NP_XFER_ZERO_COPY it never blocks.  Deltas larger than staging_rows are split
+ * into chunks in list order (result unchanged).
+ * Returns NP_W_OVERFLOW / NP_W_CHUNKED (OVERFLOW wins) where it can know.
+ * Errors: NP_E_STATE (no np_delta since init/reset), NP_E_INVAL, NP_E_CUDA. */
+int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_stream);
+
+/* Stage 4 for one layer (Section 3.4): over act = P and R of the last np_delta,
+ *   y[b] = sum_{i in act} silu(gate[S[i]].x[b]) * (up[S[i]].x[b]) * downT[S[i]]
+ *   x  dev fp32 [B][D],  y  dev fp32 [B][D] (overwritten)
+ * bf16 rows, fp32 accumulation; partial sums are combined with floating-point
+ * atomics, so the last bits of y can differ between runs.
+ * `stream` is first ordered after the layer's install mark.
+ * Errors: NP_E_STATE, NP_E_INVAL, NP_E_CUDA. */
+int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* y, void* stream);
+
+/* One whole decode step: np_predict, np_delta, np_install of every layer on
+ * `copy_stream`, and the residual MLP chain x_{l+1} = x_l + MLP_l(x_l) on
+ * `stream`, x_0 = x_bf16 widened to fp32.
+ *   x_out  dev fp32 [B][D]  x_L
+ * Host-blocking exactly as np_install.  Returns warnings like np_install. */
+int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream,
+            void* copy_stream);
+
+/* Device pointers to one layer's lists and counters from the last np_delta. */
+int np_get_delta(np_ctx* ctx, int32_t layer, np_delta_view* out);
+
+/* Copies all layers' counters to host int32 [L][NP_N_COUNTERS]; synchronises `stream`. */
+int np_read_counters(np_ctx* ctx, int32_t* out_host, void* stream);
+
+/* Copies one layer's residency tables to host arrays (any may be NULL) and
+ * synchronises `stream`:  slot_map int32 [M] (-1 = not resident), owner int32 [C]
+ * (-1 = free), resident uint32 [W], stamp int32 [M] (step of last prediction, -1 never). */
+int np_export_state(np_ctx* ctx, int32_t layer, int32_t* slot_map, int32_t* owner,
+                    uint32_t* resident, int32_t* stamp, void* stream);
+
+/* Overwrites one layer's tables from host arrays (all required) and sets the
+ * step counter; the caller vouches for their consistency.  Synchronises. */
+int np_import_state(np_ctx* ctx, int32_t layer, const int32_t* slot_map, const int32_t* owner,
+                    const uint32_t* resident, const int32_t* stamp, int32_t step, void* stream);
+
+/* Timing of the last np_step in microseconds, host float [4]: predict+top-k,
+ * delta, install (copy stream, first enqueue to last mark), MLP chain.
+ * Synchronises both streams of that step.  NP_E_STATE if no step ran. */
+int np_last_step_times(np_ctx* ctx, float* out_us);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* NP_H_ */

@@ -1,0 +1,334 @@
+"""Thin ctypes binding of ``libnp.so``: argument marshalling only.
+
+Every function has the name and meaning of the C entry point it wraps (see
+``include/np.h``).  Tensors are passed as raw pointers; nothing is computed in
+Python.  ``Engine`` is a convenience owner of the caller-side buffers (device
+memory, pinned host memory and streams come from PyTorch).
+
+There is no fallback: if the compiled library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnp.so")
+
+NP_OK, NP_E_INVAL, NP_E_STATE, NP_E_CUDA, NP_E_NOMEM, NP_E_DEVICE = 0, -1, -2, -3, -4, -5
+NP_W_OVERFLOW, NP_W_CHUNKED = 1, 2
+NP_EVICT_EXACT, NP_EVICT_LRU = 0, 1
+NP_XFER_MEMCPY_RUNS, NP_XFER_HOST_GATHER, NP_XFER_ZERO_COPY = 0, 1, 2
+NP_F_CHECK_BOUNDS = 1
+(NP_CNT_PRED, NP_CNT_KEPT, NP_CNT_DELTA, NP_CNT_EVICT, NP_CNT_OVERFLOW, NP_CNT_ACTIVE,
+ NP_CNT_RESIDENT, NP_CNT_STEP) = range(8)
+NP_N_COUNTERS = 8
+
+EXPORTED = [
+    "np_version", "np_query_sizes", "np_init", "np_destroy", "np_reset", "np_last_error",
+    "np_predict", "np_topk", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
+    "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times",
+]
+
+
+class np_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
+        "staging_rows", "transfer_mode", "flags", "host_threads")] + [("reserved", C.c_int32 * 4)]
+
+
+class np_sizes(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in (
+        "w1_bytes", "w2_bytes", "backing_bytes", "row_buffer_bytes", "staging_bytes", "workspace_bytes",
+        "host_lists_bytes", "logits_bytes", "bitmap_bytes", "record_bytes")]
+
+
+class np_buffers(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "w1", "w2", "backing", "gate_buf", "up_buf", "downT_buf", "staging", "host_staging", "workspace",
+        "host_lists")]
+
+
+class np_delta_view(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "delta_ids", "delta_slots", "evict_ids", "overflow_ids", "active_ids", "active_slots", "counters")]
+
+
+class NpError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"libnp error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load ``libnp.so`` (once) and declare the signatures."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2608_22643_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32 = C.c_void_p, C.c_int32
+    lib.np_version.restype = C.c_int
+    lib.np_last_error.restype = C.c_char_p
+    lib.np_last_error.argtypes = [vp]
+    sigs = {
+        "np_query_sizes": [C.POINTER(np_config), C.POINTER(np_sizes)],
+        "np_init": [C.POINTER(vp), C.POINTER(np_config), C.POINTER(np_buffers)],
+        "np_destroy": [vp],
+        "np_reset": [vp, vp],
+        "np_predict": [vp, vp, i32, vp, vp, vp],
+        "np_topk": [vp, vp, i32, vp, vp],
+        "np_delta": [vp, vp, vp],
+        "np_install": [vp, i32, i32, vp],
+        "np_sparse_mlp": [vp, i32, vp, i32, vp, vp],
+        "np_step": [vp, vp, i32, vp, vp, vp],
+        "np_get_delta": [vp, i32, C.POINTER(np_delta_view)],
+        "np_read_counters": [vp, vp, vp],
+        "np_export_state": [vp, i32, vp, vp, vp, vp, vp],
+        "np_import_state": [vp, i32, vp, vp, vp, vp, i32, vp],
+        "np_last_step_times": [vp, vp],
+    }
+    for name, args in sigs.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t) -> Optional[int]:
+    """Raw address of a tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        assert t.is_contiguous()
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"]
+        return t.ctypes.data
+    return int(t)
+
+
+def _stream(s) -> Optional[int]:
+    if s is None:
+        return None
+    if isinstance(s, torch.cuda.Stream):
+        return s.cuda_stream
+    return int(s)
+
+
+def _check(ctx, rc: int) -> int:
+    if rc < 0:
+        raise NpError(rc, load().np_last_error(ctx).decode())
+    return rc
+
+
+# ---- one Python function per C entry point --------------------------------------------
+def np_version() -> int:
+    return load().np_version()
+
+
+def np_last_error(ctx=None) -> str:
+    return load().np_last_error(ctx).decode()
+
+
+def np_query_sizes(cfg: np_config) -> np_sizes:
+    out = np_sizes()
+    _check(None, load().np_query_sizes(C.byref(cfg), C.byref(out)))
+    return out
+
+
+def np_init(cfg: np_config, bufs: np_buffers) -> int:
+    ctx = C.c_void_p()
+    _check(None, load().np_init(C.byref(ctx), C.byref(cfg), C.byref(bufs)))
+    return ctx.value
+
+
+def np_destroy(ctx) -> int:
+    return load().np_destroy(ctx)
+
+
+def np_reset(ctx, stream=None) -> int:
+    return _check(ctx, load().np_reset(ctx, _stream(stream)))
+
+
+def np_predict(ctx, x_bf16, B: int, logits_out=None, bitmap_out=None, stream=None) -> int:
+    return _check(ctx, load().np_predict(ctx, _ptr(x_bf16), B, _ptr(logits_out), _ptr(bitmap_out),
+                                         _stream(stream)))
+
+
+def np_topk(ctx, logits, B: int, bitmap_out, stream=None) -> int:
+    return _check(ctx, load().np_topk(ctx, _ptr(logits), B, _ptr(bitmap_out), _stream(stream)))
+
+
+def np_delta(ctx, pred_bitmap=None, stream=None) -> int:
+    return _check(ctx, load().np_delta(ctx, _ptr(pred_bitmap), _stream(stream)))
+
+
+def np_install(ctx, layer_begin: int, layer_end: int, copy_stream=None) -> int:
+    return _check(ctx, load().np_install(ctx, layer_begin, layer_end, _stream(copy_stream)))
+
+
+def np_sparse_mlp(ctx, layer: int, x, B: int, y, stream=None) -> int:
+    return _check(ctx, load().np_sparse_mlp(ctx, layer, _ptr(x), B, _ptr(y), _stream(stream)))
+
+
+def np_step(ctx, x_bf16, B: int, x_out, stream, copy_stream) -> int:
+    return _check(ctx, load().np_step(ctx, _ptr(x_bf16), B, _ptr(x_out), _stream(stream),
+                                      _stream(copy_stream)))
+
+
+def np_get_delta(ctx, layer: int) -> np_delta_view:
+    out = np_delta_view()
+    _check(ctx, load().np_get_delta(ctx, layer, C.byref(out)))
+    return out
+
+
+def np_read_counters(ctx, out_host: np.ndarray, stream=None) -> int:
+    return _check(ctx, load().np_read_counters(ctx, _ptr(out_host), _stream(stream)))
+
+
+def np_export_state(ctx, layer: int, slot_map=None, owner=None, resident=None, stamp=None, stream=None) -> int:
+    return _check(ctx, load().np_export_state(ctx, layer, _ptr(slot_map), _ptr(owner), _ptr(resident),
+                                              _ptr(stamp), _stream(stream)))
+
+
+def np_import_state(ctx, layer: int, slot_map, owner, resident, stamp, step: int, stream=None) -> int:
+    return _check(ctx, load().np_import_state(ctx, layer, _ptr(slot_map), _ptr(owner), _ptr(resident),
+                                              _ptr(stamp), step, _stream(stream)))
+
+
+def np_last_step_times(ctx) -> np.ndarray:
+    out = np.zeros(4, dtype=np.float32)
+    _check(ctx, load().np_last_step_times(ctx, _ptr(out)))
+    return out
+
+
+# ---- buffer owner ----------------------------------------------------------------------
+def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
+                transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0) -> np_config:
+    cfg = np_config()
+    cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
+    cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
+    cfg.evict_policy, cfg.transfer_mode, cfg.flags, cfg.host_threads = evict_policy, transfer_mode, flags, host_threads
+    cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
+    return cfg
+
+
+def pin_host_tensor(t: torch.Tensor) -> None:
+    """Page-lock an existing CPU tensor in place (exact size, no pool rounding)."""
+    rc = torch.cuda.cudart().cudaHostRegister(t.data_ptr(), t.numel() * t.element_size(), 0)
+    if int(rc) != 0:
+        raise RuntimeError(f"cudaHostRegister failed with {rc}")
+
+
+def unpin_host_tensor(t: torch.Tensor) -> None:
+    torch.cuda.cudart().cudaHostUnregister(t.data_ptr())
+
+
+class _DeviceInts:
+    """int32 view of raw device memory, for torch.as_tensor."""
+
+    def __init__(self, addr: int, n: int):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (addr, True), "version": 2}
+
+
+class Engine:
+    """Owns the caller-side buffers of one context and forwards to the C calls.
+
+    ``w1``/``w2`` are bf16 device tensors, ``backing`` a bf16 CPU tensor
+    ``[L, M, 3, D]`` (it is page-locked here if it is not already)."""
+
+    def __init__(self, cfg: np_config, w1: torch.Tensor, w2: torch.Tensor, backing: torch.Tensor,
+                 device: str = "cuda:0"):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.sizes = np_query_sizes(cfg)
+        L, D, M, Cap = cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.capacity
+        assert w1.is_cuda and w2.is_cuda and not backing.is_cuda
+        assert w1.numel() * 2 == self.sizes.w1_bytes and w2.numel() * 2 == self.sizes.w2_bytes
+        assert backing.numel() * 2 == self.sizes.backing_bytes and backing.is_contiguous()
+        self.w1, self.w2, self.backing = w1.contiguous(), w2.contiguous(), backing
+        self._registered = False
+        if not backing.is_pinned():
+            pin_host_tensor(backing)
+            self._registered = True
+        dev = self.device
+        self.gate = torch.zeros((L, Cap, D), dtype=torch.bfloat16, device=dev)
+        self.up = torch.zeros((L, Cap, D), dtype=torch.bfloat16, device=dev)
+        self.downT = torch.zeros((L, Cap, D), dtype=torch.bfloat16, device=dev)
+        self.staging = torch.empty(int(self.sizes.staging_bytes), dtype=torch.uint8, device=dev)
+        self.host_staging = None
+        if cfg.transfer_mode == NP_XFER_HOST_GATHER:
+            self.host_staging = torch.empty(int(self.sizes.staging_bytes), dtype=torch.uint8).pin_memory()
+        self.workspace = torch.empty(int(self.sizes.workspace_bytes) + 256, dtype=torch.uint8, device=dev)
+        ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.host_lists = torch.zeros(int(self.sizes.host_lists_bytes) // 4, dtype=torch.int32).pin_memory()
+        b = np_buffers()
+        b.w1, b.w2, b.backing = self.w1.data_ptr(), self.w2.data_ptr(), backing.data_ptr()
+        b.gate_buf, b.up_buf, b.downT_buf = self.gate.data_ptr(), self.up.data_ptr(), self.downT.data_ptr()
+        b.staging = self.staging.data_ptr()
+        b.host_staging = self.host_staging.data_ptr() if self.host_staging is not None else None
+        b.workspace, b.host_lists = ws_ptr, self.host_lists.data_ptr()
+        self.bufs = b
+        self.ctx = np_init(cfg, b)
+        self.stream = torch.cuda.Stream(device=dev)
+        self.copy_stream = torch.cuda.Stream(device=dev)
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            np_destroy(self.ctx)
+            self.ctx = None
+        if self._registered:
+            unpin_host_tensor(self.backing)
+            self._registered = False
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers that read device lists back for tests and reports --
+    def counters(self) -> np.ndarray:
+        out = np.zeros((self.cfg.n_layers, NP_N_COUNTERS), dtype=np.int32)
+        np_read_counters(self.ctx, out, self.stream)
+        return out
+
+    def _read_i32(self, addr: int, n: int) -> np.ndarray:
+        if n == 0:
+            return np.zeros(0, dtype=np.int32)
+        return torch.as_tensor(_DeviceInts(addr, n), device=self.device).cpu().numpy()
+
+    def delta_lists(self, layer: int, counters_row: np.ndarray) -> dict:
+        self.stream.synchronize()
+        v = np_get_delta(self.ctx, layer)
+        c = counters_row
+        return {
+            "delta_ids": self._read_i32(v.delta_ids, int(c[NP_CNT_DELTA])),
+            "delta_slots": self._read_i32(v.delta_slots, int(c[NP_CNT_DELTA])),
+            "evict_ids": self._read_i32(v.evict_ids, int(c[NP_CNT_EVICT])),
+            "overflow_ids": self._read_i32(v.overflow_ids, int(c[NP_CNT_OVERFLOW])),
+            "active_ids": self._read_i32(v.active_ids, int(c[NP_CNT_ACTIVE])),
+            "active_slots": self._read_i32(v.active_slots, int(c[NP_CNT_ACTIVE])),
+        }
+
+    def export_state(self, layer: int) -> dict:
+        M, Cap, W = self.cfg.d_ffn, self.cfg.capacity, self.cfg.d_ffn // 32
+        S = np.empty(M, np.int32)
+        owner = np.empty(Cap, np.int32)
+        R = np.empty(W, np.uint32)
+        stamp = np.empty(M, np.int32)
+        np_export_state(self.ctx, layer, S, owner, R, stamp, self.stream)
+        return {"slot_map": S, "owner": owner, "resident": R, "stamp": stamp}

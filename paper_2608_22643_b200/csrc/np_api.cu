@@ -1,0 +1,701 @@
+// C ABI of libnp.so: context, argument checking, stream/event ordering and the
+// host side of the install path (run coalescing, chunking, staging).  Every
+// arithmetic step runs in the kernels of the sibling .cu files.
+#include <algorithm>
+#include <atomic>
+#include <condition_variable>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <functional>
+#include <mutex>
+#include <new>
+#include <thread>
+
+#include "np_internal.h"
+
+using namespace npi;
+
+namespace {
+
+thread_local std::string g_last_error = "";
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Small fork-join pool for packing records into pinned staging.
+class Pool {
+ public:
+  explicit Pool(int n) : stop_(false), gen_(0), pending_(0) {
+    for (int i = 0; i < n; ++i) threads_.emplace_back([this] { run(); });
+  }
+  ~Pool() {
+    {
+      std::lock_guard<std::mutex> lk(m_);
+      stop_ = true;
+      ++gen_;
+    }
+    cv_.notify_all();
+    for (auto& t : threads_) t.join();
+  }
+  // Calls fn(i) for i in [0, count) on the workers and the caller; returns when all are done.
+  void parallel_for(int count, const std::function<void(int)>& fn) {
+    if (count <= 0) return;
+    if (threads_.empty() || count == 1) {
+      for (int i = 0; i < count; ++i) fn(i);
+      return;
+    }
+    {
+      std::lock_guard<std::mutex> lk(m_);
+      fn_ = &fn;
+      count_ = count;
+      next_.store(0);
+      pending_ = (int)threads_.size();
+      ++gen_;
+    }
+    cv_.notify_all();
+    work();
+    std::unique_lock<std::mutex> lk(m_);
+    done_cv_.wait(lk, [this] { return pending_ == 0; });
+    fn_ = nullptr;
+  }
+  int size() const { return (int)threads_.size(); }
+
+ private:
+  void work() {
+    for (;;) {
+      const int i = next_.fetch_add(1);
+      if (i >= count_) break;
+      (*fn_)(i);
+    }
+  }
+  void run() {
+    unsigned long seen = 0;
+    for (;;) {
+      {
+        std::unique_lock<std::mutex> lk(m_);
+        cv_.wait(lk, [&] { return gen_ != seen; });
+        seen = gen_;
+        if (stop_) return;
+      }
+      work();
+      {
+        std::lock_guard<std::mutex> lk(m_);
+        if (--pending_ == 0) done_cv_.notify_all();
+      }
+    }
+  }
+  std::vector<std::thread> threads_;
+  std::mutex m_;
+  std::condition_variable cv_, done_cv_;
+  bool stop_;
+  unsigned long gen_;
+  int pending_;
+  const std::function<void(int)>* fn_ = nullptr;
+  int count_ = 0;
+  std::atomic<int> next_{0};
+};
+
+}  // namespace
+
+struct np_ctx {
+  np_config cfg;
+  np_buffers bufs;
+  Dims d;
+  Tables t;
+  Workspace ws;
+  void* slab = nullptr;
+  int device = 0;
+  int sm_count = 0;
+  int32_t* host_lists = nullptr;      // host address
+  int32_t* host_lists_dev = nullptr;  // device alias
+  const char* backing_dev = nullptr;  // device alias of the record store
+  cudaEvent_t ev_delta = nullptr;
+  std::vector<cudaEvent_t> ev_installed;
+  std::vector<char> install_pending;
+  cudaEvent_t ev_half[2] = {nullptr, nullptr};  // host staging halves in flight
+  bool half_pending[2] = {false, false};
+  int next_half = 0;
+  cudaEvent_t ev_t[4] = {nullptr, nullptr, nullptr, nullptr};  // compute-stream step timing
+  cudaEvent_t ev_c[2] = {nullptr, nullptr};                    // copy-stream step timing
+  bool have_delta = false;
+  bool have_pred = false;
+  bool have_step = false;
+  int step = 0;
+  Pool* pool = nullptr;
+  std::string err;
+};
+
+namespace {
+
+int fail(np_ctx* ctx, int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (ctx) ctx->err = buf;
+  g_last_error = buf;
+  return code;
+}
+
+#define NP_CUDA(ctx, call)                                                                  \
+  do {                                                                                      \
+    cudaError_t e__ = (call);                                                               \
+    if (e__ != cudaSuccess)                                                                 \
+      return fail(ctx, NP_E_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e__),  \
+                  __FILE__, __LINE__);                                                      \
+  } while (0)
+
+int check_config(const np_config* c, np_ctx* ctx) {
+  if (!c) return fail(ctx, NP_E_INVAL, "config is NULL");
+  if (c->n_layers < 1) return fail(ctx, NP_E_INVAL, "n_layers must be >= 1");
+  if (c->d_model < 8 || c->d_model % 8 || c->d_model > 16384)
+    return fail(ctx, NP_E_INVAL, "d_model must be a multiple of 8 in [8, 16384]");
+  if (c->d_ffn < 32 || c->d_ffn % 32 || c->d_ffn > 40960)
+    return fail(ctx, NP_E_INVAL, "d_ffn must be a multiple of 32 in [32, 40960]");
+  if (c->d_pred < 8 || c->d_pred % 8 || c->d_pred > 4096)
+    return fail(ctx, NP_E_INVAL, "d_pred must be a multiple of 8 in [8, 4096]");
+  if (c->capacity < 1 || c->capacity > c->d_ffn) return fail(ctx, NP_E_INVAL, "capacity must be in [1, d_ffn]");
+  if (c->top_k < 0 || c->top_k > c->capacity) return fail(ctx, NP_E_INVAL, "top_k must be in [0, capacity]");
+  if (c->max_batch < 1 || c->max_batch > kMaxBatch) return fail(ctx, NP_E_INVAL, "max_batch must be in [1, 16]");
+  if (c->evict_policy != NP_EVICT_EXACT && c->evict_policy != NP_EVICT_LRU)
+    return fail(ctx, NP_E_INVAL, "unknown evict_policy");
+  if (c->transfer_mode < NP_XFER_MEMCPY_RUNS || c->transfer_mode > NP_XFER_ZERO_COPY)
+    return fail(ctx, NP_E_INVAL, "unknown transfer_mode");
+  if (c->staging_rows < 1) return fail(ctx, NP_E_INVAL, "staging_rows must be >= 1");
+  if (c->transfer_mode == NP_XFER_HOST_GATHER && c->staging_rows < 2)
+    return fail(ctx, NP_E_INVAL, "host gather needs staging_rows >= 2 (two halves)");
+  if (c->flags & ~NP_F_CHECK_BOUNDS) return fail(ctx, NP_E_INVAL, "unknown flag bits");
+  if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
+  for (int i = 0; i < 4; ++i)
+    if (c->reserved[i]) return fail(ctx, NP_E_INVAL, "reserved fields must be 0");
+  return NP_OK;
+}
+
+struct WsLayout {
+  size_t hidden, logits, xbuf, zbuf, total;
+};
+
+WsLayout ws_layout(const np_config& c) {
+  WsLayout w;
+  size_t off = 0;
+  w.hidden = off;
+  off = align_up(off + (size_t)c.max_batch * c.d_pred * 4, 256);
+  w.logits = off;
+  off = align_up(off + (size_t)c.max_batch * c.n_layers * c.d_ffn * 4, 256);
+  const size_t vec = align_up((size_t)c.max_batch * c.d_model * 4, 256);
+  w.xbuf = off;
+  off += 2 * vec;
+  w.zbuf = off;
+  off += 3 * vec;
+  w.total = off;
+  return w;
+}
+
+size_t host_lists_ints(const np_config& c) {
+  return kHostHeaderInts + (size_t)c.n_layers * (NP_N_COUNTERS + 2 * (size_t)c.capacity);
+}
+
+cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+int check_device_status(np_ctx* ctx, cudaStream_t s) {
+  int32_t st[4];
+  NP_CUDA(ctx, cudaMemcpyAsync(st, ctx->t.status, sizeof st, cudaMemcpyDeviceToHost, s));
+  NP_CUDA(ctx, cudaStreamSynchronize(s));
+  if (st[0]) return fail(ctx, NP_E_DEVICE, "kernel bounds check tripped (status bits 0x%x)", st[0]);
+  return NP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int np_version(void) { return NP_VERSION; }
+
+const char* np_last_error(const np_ctx* ctx) { return ctx ? ctx->err.c_str() : g_last_error.c_str(); }
+
+int np_query_sizes(const np_config* cfg, np_sizes* out) {
+  if (!out) return fail(nullptr, NP_E_INVAL, "out is NULL");
+  int rc = check_config(cfg, nullptr);
+  if (rc) return rc;
+  const np_config& c = *cfg;
+  const uint64_t rec = 3ull * c.d_model * 2;
+  out->record_bytes = rec;
+  out->w1_bytes = 2ull * c.d_pred * c.d_model;
+  out->w2_bytes = 2ull * c.n_layers * c.d_ffn * c.d_pred;
+  out->backing_bytes = rec * c.n_layers * c.d_ffn;
+  out->row_buffer_bytes = 2ull * c.n_layers * c.capacity * c.d_model;
+  out->staging_bytes = rec * c.staging_rows;
+  out->workspace_bytes = ws_layout(c).total;
+  out->host_lists_bytes = host_lists_ints(c) * 4;
+  out->logits_bytes = 4ull * c.max_batch * c.n_layers * c.d_ffn;
+  out->bitmap_bytes = 4ull * c.n_layers * (c.d_ffn / 32);
+  return NP_OK;
+}
+
+int np_destroy(np_ctx* ctx) {
+  if (!ctx) return NP_OK;
+  cudaDeviceSynchronize();
+  delete ctx->pool;
+  if (ctx->slab) cudaFree(ctx->slab);
+  if (ctx->ev_delta) cudaEventDestroy(ctx->ev_delta);
+  for (auto e : ctx->ev_installed)
+    if (e) cudaEventDestroy(e);
+  for (auto e : ctx->ev_half)
+    if (e) cudaEventDestroy(e);
+  for (auto e : ctx->ev_t)
+    if (e) cudaEventDestroy(e);
+  for (auto e : ctx->ev_c)
+    if (e) cudaEventDestroy(e);
+  delete ctx;
+  return NP_OK;
+}
+
+int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
+  if (!out) return fail(nullptr, NP_E_INVAL, "out is NULL");
+  *out = nullptr;
+  int rc = check_config(cfg, nullptr);
+  if (rc) return rc;
+  if (!b) return fail(nullptr, NP_E_INVAL, "buffers is NULL");
+  const bool need_staging = cfg->transfer_mode != NP_XFER_ZERO_COPY;
+  if (!b->w1 || !b->w2 || !b->backing || !b->gate_buf || !b->up_buf || !b->downT_buf || !b->workspace ||
+      !b->host_lists || (need_staging && !b->staging) ||
+      (cfg->transfer_mode == NP_XFER_HOST_GATHER && !b->host_staging))
+    return fail(nullptr, NP_E_INVAL, "a required buffer pointer is NULL");
+  const void* aligned16[] = {b->w1, b->w2, b->backing, b->gate_buf, b->up_buf, b->downT_buf, b->staging,
+                             b->host_staging};
+  for (const void* p : aligned16)
+    if ((uintptr_t)p % 16) return fail(nullptr, NP_E_INVAL, "weight, row and staging buffers must be 16-byte aligned");
+  if ((uintptr_t)b->workspace % 256) return fail(nullptr, NP_E_INVAL, "workspace must be 256-byte aligned");
+  if ((uintptr_t)b->host_lists % 16) return fail(nullptr, NP_E_INVAL, "host_lists must be 16-byte aligned");
+
+  np_ctx* ctx = new (std::nothrow) np_ctx();
+  if (!ctx) return fail(nullptr, NP_E_NOMEM, "out of host memory");
+  ctx->cfg = *cfg;
+  ctx->bufs = *b;
+  Dims& d = ctx->d;
+  d.L = cfg->n_layers;
+  d.D = cfg->d_model;
+  d.M = cfg->d_ffn;
+  d.H = cfg->d_pred;
+  d.k = cfg->top_k;
+  d.C = cfg->capacity;
+  d.W = cfg->d_ffn / 32;
+  d.Bmax = cfg->max_batch;
+  d.rec_bytes = 3ull * d.D * 2;
+
+#define NP_INIT_CUDA(call)                                                                   \
+  do {                                                                                       \
+    cudaError_t e__ = (call);                                                                \
+    if (e__ != cudaSuccess) {                                                                \
+      int rc__ = fail(nullptr, e__ == cudaErrorMemoryAllocation ? NP_E_NOMEM : NP_E_CUDA,    \
+                      "%s failed: %s", #call, cudaGetErrorString(e__));                      \
+      np_destroy(ctx);                                                                       \
+      return rc__;                                                                           \
+    }                                                                                        \
+  } while (0)
+
+  NP_INIT_CUDA(cudaGetDevice(&ctx->device));
+  NP_INIT_CUDA(cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device));
+
+  // pinned host areas must be reachable from the device
+  void* dev_alias = nullptr;
+  if (cudaHostGetDevicePointer(&dev_alias, b->host_lists, 0) != cudaSuccess) {
+    cudaGetLastError();
+    np_destroy(ctx);
+    return fail(nullptr, NP_E_INVAL, "host_lists is not pinned, device-mapped host memory");
+  }
+  ctx->host_lists = static_cast<int32_t*>(b->host_lists);
+  ctx->host_lists_dev = static_cast<int32_t*>(dev_alias);
+  if (cudaHostGetDevicePointer(&dev_alias, const_cast<void*>(b->backing), 0) != cudaSuccess) {
+    cudaGetLastError();
+    np_destroy(ctx);
+    return fail(nullptr, NP_E_INVAL, "backing store is not pinned, device-mapped host memory");
+  }
+  ctx->backing_dev = static_cast<const char*>(dev_alias);
+
+  // library-owned slab: residency tables, lists, scratch
+  const size_t LM = (size_t)d.L * d.M, LC = (size_t)d.L * d.C, LW = (size_t)d.L * d.W;
+  size_t off = 0;
+  auto take = [&](size_t ints) {
+    size_t o = off;
+    off = align_up(off + ints * 4, 256);
+    return o;
+  };
+  const size_t o_res = take(LW), o_slot = take(LM), o_owner = take(LC), o_stamp = take(LM);
+  const size_t o_did = take(LC), o_dsl = take(LC), o_eid = take(LC), o_aid = take(LC), o_asl = take(LC);
+  const size_t o_ovf = take(LM), o_cnt = take((size_t)d.L * NP_N_COUNTERS), o_free = take(LC);
+  const size_t o_cid = take(LC), o_ckey = take(LC), o_pred = take(LW), o_stat = take(4);
+  NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
+  char* base = static_cast<char*>(ctx->slab);
+  Tables& t = ctx->t;
+  t.resident = reinterpret_cast<uint32_t*>(base + o_res);
+  t.slot_map = reinterpret_cast<int32_t*>(base + o_slot);
+  t.owner = reinterpret_cast<int32_t*>(base + o_owner);
+  t.stamp = reinterpret_cast<int32_t*>(base + o_stamp);
+  t.delta_ids = reinterpret_cast<int32_t*>(base + o_did);
+  t.delta_slots = reinterpret_cast<int32_t*>(base + o_dsl);
+  t.evict_ids = reinterpret_cast<int32_t*>(base + o_eid);
+  t.active_ids = reinterpret_cast<int32_t*>(base + o_aid);
+  t.active_slots = reinterpret_cast<int32_t*>(base + o_asl);
+  t.overflow_ids = reinterpret_cast<int32_t*>(base + o_ovf);
+  t.counters = reinterpret_cast<int32_t*>(base + o_cnt);
+  t.free_slots = reinterpret_cast<int32_t*>(base + o_free);
+  t.cand_ids = reinterpret_cast<int32_t*>(base + o_cid);
+  t.cand_keys = reinterpret_cast<uint32_t*>(base + o_ckey);
+  t.pred = reinterpret_cast<uint32_t*>(base + o_pred);
+  t.status = reinterpret_cast<int32_t*>(base + o_stat);
+
+  const WsLayout wl = ws_layout(*cfg);
+  char* wsb = static_cast<char*>(b->workspace);
+  const size_t vec = align_up((size_t)d.Bmax * d.D * 4, 256);
+  ctx->ws.hidden = reinterpret_cast<float*>(wsb + wl.hidden);
+  ctx->ws.logits = reinterpret_cast<float*>(wsb + wl.logits);
+  for (int i = 0; i < 2; ++i) ctx->ws.xbuf[i] = reinterpret_cast<float*>(wsb + wl.xbuf + i * vec);
+  for (int i = 0; i < 3; ++i) ctx->ws.zbuf[i] = reinterpret_cast<float*>(wsb + wl.zbuf + i * vec);
+
+  NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_delta, cudaEventDisableTiming));
+  ctx->ev_installed.assign(d.L, nullptr);
+  ctx->install_pending.assign(d.L, 0);
+  for (int l = 0; l < d.L; ++l)
+    NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_installed[l], cudaEventDisableTiming));
+  for (auto& e : ctx->ev_half) NP_INIT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  for (auto& e : ctx->ev_t) NP_INIT_CUDA(cudaEventCreate(&e));
+  for (auto& e : ctx->ev_c) NP_INIT_CUDA(cudaEventCreate(&e));
+
+  memset(ctx->host_lists, 0, host_lists_ints(*cfg) * 4);
+  NP_INIT_CUDA(launch_tables_reset(d, t, nullptr));
+  NP_INIT_CUDA(cudaDeviceSynchronize());
+#undef NP_INIT_CUDA
+
+  if (cfg->transfer_mode == NP_XFER_HOST_GATHER) {
+    int n = cfg->host_threads;
+    if (n == 0) n = std::max(1u, std::min(8u, std::thread::hardware_concurrency()));
+    ctx->pool = new (std::nothrow) Pool(n - 1);  // the caller's thread works too
+  }
+  *out = ctx;
+  return NP_OK;
+}
+
+int np_reset(np_ctx* ctx, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  NP_CUDA(ctx, launch_tables_reset(ctx->d, ctx->t, as_stream(stream)));
+  ctx->have_delta = ctx->have_pred = ctx->have_step = false;
+  std::fill(ctx->install_pending.begin(), ctx->install_pending.end(), 0);
+  ctx->step = 0;
+  return NP_OK;
+}
+
+int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, uint32_t* bitmap_out,
+               void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!x_bf16) return fail(ctx, NP_E_INVAL, "x is NULL");
+  if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
+  if ((uintptr_t)x_bf16 % 16) return fail(ctx, NP_E_INVAL, "x must be 16-byte aligned");
+  cudaStream_t s = as_stream(stream);
+  const Dims& d = ctx->d;
+  NP_CUDA(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
+  NP_CUDA(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, s, ctx->sm_count));
+  NP_CUDA(ctx, launch_topk(d, ctx->ws.logits, B, ctx->t.pred, s));
+  const size_t nlog = (size_t)B * d.L * d.M * 4, nbm = (size_t)d.L * d.W * 4;
+  if (logits_out) NP_CUDA(ctx, cudaMemcpyAsync(logits_out, ctx->ws.logits, nlog, cudaMemcpyDeviceToDevice, s));
+  if (bitmap_out) NP_CUDA(ctx, cudaMemcpyAsync(bitmap_out, ctx->t.pred, nbm, cudaMemcpyDeviceToDevice, s));
+  ctx->have_pred = true;
+  return NP_OK;
+}
+
+int np_topk(np_ctx* ctx, const float* logits, int32_t B, uint32_t* bitmap_out, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!logits || !bitmap_out) return fail(ctx, NP_E_INVAL, "logits or bitmap_out is NULL");
+  if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
+  NP_CUDA(ctx, launch_topk(ctx->d, logits, B, bitmap_out, as_stream(stream)));
+  return NP_OK;
+}
+
+int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!pred_bitmap) {
+    if (!ctx->have_pred) return fail(ctx, NP_E_STATE, "np_delta(NULL) needs a prior np_predict");
+    pred_bitmap = ctx->t.pred;
+  }
+  cudaStream_t s = as_stream(stream);
+  // the previous step's installs must have landed before tables and slots are reused
+  for (int l = 0; l < ctx->d.L; ++l) {
+    if (ctx->install_pending[l]) {
+      NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[l], 0));
+      ctx->install_pending[l] = 0;
+    }
+  }
+  NP_CUDA(ctx, launch_delta(ctx->d, ctx->t, pred_bitmap, ctx->cfg.evict_policy, ctx->step, ctx->host_lists_dev,
+                            ctx->cfg.flags & NP_F_CHECK_BOUNDS, s));
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_delta, s));
+  ctx->step += 1;
+  ctx->have_delta = true;
+  return NP_OK;
+}
+
+int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  const Dims& d = ctx->d;
+  if (layer_begin < 0 || layer_end > d.L || layer_begin > layer_end)
+    return fail(ctx, NP_E_INVAL, "layer range [%d, %d) outside [0, %d)", layer_begin, layer_end, d.L);
+  if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_install needs a prior np_delta");
+  cudaStream_t cs = as_stream(copy_stream);
+  const int check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+  const int mode = ctx->cfg.transfer_mode;
+  const size_t rec = d.rec_bytes;
+  const size_t row_bytes = (size_t)d.D * 2;
+  NP_CUDA(ctx, cudaStreamWaitEvent(cs, ctx->ev_delta, 0));
+  int warn = NP_OK;
+
+  if (mode == NP_XFER_ZERO_COPY) {
+    const int max_rows = d.C;
+    for (int l = layer_begin; l < layer_end; ++l) {
+      const char* store_l = ctx->backing_dev + (size_t)l * d.M * rec;
+      NP_CUDA(ctx, launch_scatter(d, store_l, true, ctx->t.delta_ids + (size_t)l * d.C,
+                                  ctx->t.delta_slots + (size_t)l * d.C,
+                                  ctx->t.counters + (size_t)l * NP_N_COUNTERS + NP_CNT_DELTA, 0, max_rows,
+                                  static_cast<char*>(ctx->bufs.gate_buf) + (size_t)l * d.C * row_bytes,
+                                  static_cast<char*>(ctx->bufs.up_buf) + (size_t)l * d.C * row_bytes,
+                                  static_cast<char*>(ctx->bufs.downT_buf) + (size_t)l * d.C * row_bytes,
+                                  ctx->t.status, check, cs, ctx->sm_count));
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], cs));
+      ctx->install_pending[l] = 1;
+    }
+    return NP_OK;
+  }
+
+  // the host plans the copies: wait until the delta lists are readable
+  NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_delta));
+  const char* store = static_cast<const char*>(ctx->bufs.backing);
+  char* staging = static_cast<char*>(ctx->bufs.staging);
+  const size_t per_layer = NP_N_COUNTERS + 2 * (size_t)d.C;
+  for (int l = layer_begin; l < layer_end; ++l) {
+    const int32_t* cnt = ctx->host_lists + kHostHeaderInts + (size_t)l * per_layer;
+    const int32_t* ids = cnt + NP_N_COUNTERS;
+    const int n = cnt[NP_CNT_DELTA];
+    if (n < 0 || n > d.C) return fail(ctx, NP_E_DEVICE, "layer %d: delta count %d outside [0, %d]", l, n, d.C);
+    if (cnt[NP_CNT_OVERFLOW] > 0) warn = NP_W_OVERFLOW;
+    const char* store_l = store + (size_t)l * d.M * rec;
+    char* gate_l = static_cast<char*>(ctx->bufs.gate_buf) + (size_t)l * d.C * row_bytes;
+    char* up_l = static_cast<char*>(ctx->bufs.up_buf) + (size_t)l * d.C * row_bytes;
+    char* down_l = static_cast<char*>(ctx->bufs.downT_buf) + (size_t)l * d.C * row_bytes;
+    const int32_t* slots_dev = ctx->t.delta_slots + (size_t)l * d.C;
+    const int32_t* count_dev = ctx->t.counters + (size_t)l * NP_N_COUNTERS + NP_CNT_DELTA;
+
+    if (mode == NP_XFER_MEMCPY_RUNS) {
+      const int cap = ctx->cfg.staging_rows;
+      if (n > cap && warn == NP_OK) warn = NP_W_CHUNKED;
+      for (int first = 0; first < n; first += cap) {
+        const int rows = std::min(cap, n - first);
+        // ascending IDs: adjacent IDs are adjacent records of the store -> one copy per run
+        int r = 0;
+        while (r < rows) {
+          int len = 1;
+          while (r + len < rows && ids[first + r + len] == ids[first + r] + len) ++len;
+          const int id = ids[first + r];
+          if (id < 0 || id + len > d.M) return fail(ctx, NP_E_DEVICE, "layer %d: neuron id %d out of range", l, id);
+          NP_CUDA(ctx, cudaMemcpyAsync(staging + (size_t)r * rec, store_l + (size_t)id * rec, (size_t)len * rec,
+                                       cudaMemcpyHostToDevice, cs));
+          r += len;
+        }
+        NP_CUDA(ctx, launch_scatter(d, staging, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
+                                    down_l, ctx->t.status, check, cs, ctx->sm_count));
+      }
+    } else {  // NP_XFER_HOST_GATHER: two halves of pinned staging, packed by the pool
+      const int half_rows = ctx->cfg.staging_rows / 2;
+      char* hstage = static_cast<char*>(ctx->bufs.host_staging);
+      if (n > half_rows && warn == NP_OK) warn = NP_W_CHUNKED;
+      for (int first = 0; first < n; first += half_rows) {
+        const int rows = std::min(half_rows, n - first);
+        const int h = ctx->next_half;
+        ctx->next_half ^= 1;
+        if (ctx->half_pending[h]) {
+          NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_half[h]));
+          ctx->half_pending[h] = false;
+        }
+        char* hbuf = hstage + (size_t)h * half_rows * rec;
+        char* dbuf = staging + (size_t)h * half_rows * rec;
+        bool bad = false;
+        const int nthreads = ctx->pool ? ctx->pool->size() + 1 : 1;
+        const int parts = std::min(rows, nthreads * 4);
+        auto body = [&](int part) {
+          const int lo = (int)((long long)rows * part / parts), hi = (int)((long long)rows * (part + 1) / parts);
+          for (int r = lo; r < hi; ++r) {
+            const int id = ids[first + r];
+            if (id < 0 || id >= d.M) {
+              bad = true;
+              continue;
+            }
+            memcpy(hbuf + (size_t)r * rec, store_l + (size_t)id * rec, rec);
+          }
+        };
+        if (ctx->pool) ctx->pool->parallel_for(parts, body);
+        else for (int part = 0; part < parts; ++part) body(part);
+        if (bad) return fail(ctx, NP_E_DEVICE, "layer %d: neuron id out of range", l);
+        NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)rows * rec, cudaMemcpyHostToDevice, cs));
+        NP_CUDA(ctx, cudaEventRecord(ctx->ev_half[h], cs));
+        ctx->half_pending[h] = true;
+        NP_CUDA(ctx, launch_scatter(d, dbuf, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
+                                    down_l, ctx->t.status, check, cs, ctx->sm_count));
+      }
+    }
+    NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], cs));
+    ctx->install_pending[l] = 1;
+  }
+  return warn;
+}
+
+static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, float* yacc, float* x_store,
+                     float* zero_out, int B, cudaStream_t s) {
+  const Dims& d = ctx->d;
+  const size_t row_bytes = (size_t)d.D * 2;
+  MlpArgs a;
+  a.gate_l = static_cast<const char*>(ctx->bufs.gate_buf) + (size_t)layer * d.C * row_bytes;
+  a.up_l = static_cast<const char*>(ctx->bufs.up_buf) + (size_t)layer * d.C * row_bytes;
+  a.downT_l = static_cast<const char*>(ctx->bufs.downT_buf) + (size_t)layer * d.C * row_bytes;
+  a.active_slots = ctx->t.active_slots + (size_t)layer * d.C;
+  a.n_active_ptr = ctx->t.counters + (size_t)layer * NP_N_COUNTERS + NP_CNT_ACTIVE;
+  a.xa = xa;
+  a.xb = xb;
+  a.yacc = yacc;
+  a.x_store = x_store;
+  a.zero_out = zero_out;
+  a.B = B;
+  a.C = d.C;
+  a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+  a.status = ctx->t.status;
+  if (ctx->install_pending[layer]) NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0));
+  NP_CUDA(ctx, launch_sparse_mlp(d, a, s, ctx->sm_count));
+  return NP_OK;
+}
+
+int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* y, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  const Dims& d = ctx->d;
+  if (layer < 0 || layer >= d.L) return fail(ctx, NP_E_INVAL, "layer %d outside [0, %d)", layer, d.L);
+  if (!x || !y) return fail(ctx, NP_E_INVAL, "x or y is NULL");
+  if ((uintptr_t)x % 16 || (uintptr_t)y % 16) return fail(ctx, NP_E_INVAL, "x and y must be 16-byte aligned");
+  if (B < 1 || B > d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, d.Bmax);
+  if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_sparse_mlp needs a prior np_delta");
+  cudaStream_t s = as_stream(stream);
+  NP_CUDA(ctx, cudaMemsetAsync(y, 0, (size_t)B * d.D * 4, s));
+  return mlp_layer(ctx, layer, x, nullptr, y, nullptr, nullptr, B, s);
+}
+
+int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream, void* copy_stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!x_out) return fail(ctx, NP_E_INVAL, "x_out is NULL");
+  if ((uintptr_t)x_out % 16) return fail(ctx, NP_E_INVAL, "x_out must be 16-byte aligned");
+  if (stream == copy_stream) return fail(ctx, NP_E_INVAL, "np_step needs two different streams");
+  const Dims& d = ctx->d;
+  cudaStream_t s = as_stream(stream), cs = as_stream(copy_stream);
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[0], s));
+  int rc = np_predict(ctx, x_bf16, B, nullptr, nullptr, stream);
+  if (rc < 0) return rc;
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[1], s));
+  rc = np_delta(ctx, nullptr, stream);
+  if (rc < 0) return rc;
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[2], s));
+  // the copy stream is ordered after the delta step inside np_install
+  NP_CUDA(ctx, cudaStreamWaitEvent(cs, ctx->ev_delta, 0));
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_c[0], cs));
+  const int warn = np_install(ctx, 0, d.L, copy_stream);
+  if (warn < 0) return warn;
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_c[1], cs));
+
+  // residual chain: x_l = xbuf[(l+1)&1] + zbuf[(l-1)%3]; layer l accumulates MLP_l(x_l) into
+  // zbuf[l%3], stores x_l to xbuf[l&1] and clears zbuf[(l+1)%3] for the next layer
+  const size_t n = (size_t)B * d.D;
+  NP_CUDA(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, n * 4, s));
+  for (int l = 0; l < d.L; ++l) {
+    rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
+                   ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, s);
+    if (rc < 0) return rc;
+  }
+  NP_CUDA(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], x_out, n, s));
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[3], s));
+  ctx->have_step = true;
+  return warn;
+}
+
+int np_last_step_times(np_ctx* ctx, float* out_us) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!out_us) return fail(ctx, NP_E_INVAL, "out is NULL");
+  if (!ctx->have_step) return fail(ctx, NP_E_STATE, "no np_step has run");
+  NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_t[3]));
+  NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_c[1]));
+  float ms[4];
+  NP_CUDA(ctx, cudaEventElapsedTime(&ms[0], ctx->ev_t[0], ctx->ev_t[1]));
+  NP_CUDA(ctx, cudaEventElapsedTime(&ms[1], ctx->ev_t[1], ctx->ev_t[2]));
+  NP_CUDA(ctx, cudaEventElapsedTime(&ms[2], ctx->ev_c[0], ctx->ev_c[1]));
+  NP_CUDA(ctx, cudaEventElapsedTime(&ms[3], ctx->ev_t[2], ctx->ev_t[3]));
+  for (int i = 0; i < 4; ++i) out_us[i] = ms[i] * 1000.f;
+  return NP_OK;
+}
+
+int np_get_delta(np_ctx* ctx, int32_t layer, np_delta_view* out) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!out) return fail(ctx, NP_E_INVAL, "out is NULL");
+  const Dims& d = ctx->d;
+  if (layer < 0 || layer >= d.L) return fail(ctx, NP_E_INVAL, "layer %d outside [0, %d)", layer, d.L);
+  if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_get_delta needs a prior np_delta");
+  out->delta_ids = ctx->t.delta_ids + (size_t)layer * d.C;
+  out->delta_slots = ctx->t.delta_slots + (size_t)layer * d.C;
+  out->evict_ids = ctx->t.evict_ids + (size_t)layer * d.C;
+  out->overflow_ids = ctx->t.overflow_ids + (size_t)layer * d.M;
+  out->active_ids = ctx->t.active_ids + (size_t)layer * d.C;
+  out->active_slots = ctx->t.active_slots + (size_t)layer * d.C;
+  out->counters = ctx->t.counters + (size_t)layer * NP_N_COUNTERS;
+  return NP_OK;
+}
+
+int np_read_counters(np_ctx* ctx, int32_t* out_host, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!out_host) return fail(ctx, NP_E_INVAL, "out is NULL");
+  cudaStream_t s = as_stream(stream);
+  NP_CUDA(ctx, cudaMemcpyAsync(out_host, ctx->t.counters, (size_t)ctx->d.L * NP_N_COUNTERS * 4,
+                               cudaMemcpyDeviceToHost, s));
+  return check_device_status(ctx, s);
+}
+
+int np_export_state(np_ctx* ctx, int32_t layer, int32_t* slot_map, int32_t* owner, uint32_t* resident,
+                    int32_t* stamp, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  const Dims& d = ctx->d;
+  if (layer < 0 || layer >= d.L) return fail(ctx, NP_E_INVAL, "layer %d outside [0, %d)", layer, d.L);
+  cudaStream_t s = as_stream(stream);
+  if (slot_map)
+    NP_CUDA(ctx, cudaMemcpyAsync(slot_map, ctx->t.slot_map + (size_t)layer * d.M, (size_t)d.M * 4,
+                                 cudaMemcpyDeviceToHost, s));
+  if (owner)
+    NP_CUDA(ctx, cudaMemcpyAsync(owner, ctx->t.owner + (size_t)layer * d.C, (size_t)d.C * 4, cudaMemcpyDeviceToHost, s));
+  if (resident)
+    NP_CUDA(ctx, cudaMemcpyAsync(resident, ctx->t.resident + (size_t)layer * d.W, (size_t)d.W * 4,
+                                 cudaMemcpyDeviceToHost, s));
+  if (stamp)
+    NP_CUDA(ctx, cudaMemcpyAsync(stamp, ctx->t.stamp + (size_t)layer * d.M, (size_t)d.M * 4, cudaMemcpyDeviceToHost, s));
+  return check_device_status(ctx, s);
+}
+
+int np_import_state(np_ctx* ctx, int32_t layer, const int32_t* slot_map, const int32_t* owner,
+                    const uint32_t* resident, const int32_t* stamp, int32_t step, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  const Dims& d = ctx->d;
+  if (layer < 0 || layer >= d.L) return fail(ctx, NP_E_INVAL, "layer %d outside [0, %d)", layer, d.L);
+  if (!slot_map || !owner || !resident || !stamp) return fail(ctx, NP_E_INVAL, "a state array is NULL");
+  if (step < 0) return fail(ctx, NP_E_INVAL, "step must be >= 0");
+  cudaStream_t s = as_stream(stream);
+  NP_CUDA(ctx, cudaMemcpyAsync(ctx->t.slot_map + (size_t)layer * d.M, slot_map, (size_t)d.M * 4,
+                               cudaMemcpyHostToDevice, s));
+  NP_CUDA(ctx, cudaMemcpyAsync(ctx->t.owner + (size_t)layer * d.C, owner, (size_t)d.C * 4, cudaMemcpyHostToDevice, s));
+  NP_CUDA(ctx, cudaMemcpyAsync(ctx->t.resident + (size_t)layer * d.W, resident, (size_t)d.W * 4,
+                               cudaMemcpyHostToDevice, s));
+  NP_CUDA(ctx, cudaMemcpyAsync(ctx->t.stamp + (size_t)layer * d.M, stamp, (size_t)d.M * 4, cudaMemcpyHostToDevice, s));
+  NP_CUDA(ctx, cudaStreamSynchronize(s));
+  ctx->step = step;
+  return NP_OK;
+}
+
+}  // extern "C"

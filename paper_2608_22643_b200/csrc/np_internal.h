@@ -1,0 +1,90 @@
+// Internal declarations shared by the translation units of libnp.so.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "np.h"
+
+namespace npi {
+
+constexpr int kMaxBatch = 16;
+constexpr int kHostHeaderInts = 16;  // global header of the host list mirror
+
+// Device-resident tables and lists of all layers (one slab, library-owned).
+struct Tables {
+  uint32_t* resident;     // [L][W]
+  int32_t* slot_map;      // [L][M]
+  int32_t* owner;         // [L][C]
+  int32_t* stamp;         // [L][M]
+  int32_t* delta_ids;     // [L][C]
+  int32_t* delta_slots;   // [L][C]
+  int32_t* evict_ids;     // [L][C]
+  int32_t* active_ids;    // [L][C]
+  int32_t* active_slots;  // [L][C]
+  int32_t* overflow_ids;  // [L][M]
+  int32_t* counters;      // [L][NP_N_COUNTERS]
+  int32_t* free_slots;    // [L][C]  scratch of the delta kernel
+  int32_t* cand_ids;      // [L][C]  scratch (LRU victim selection)
+  uint32_t* cand_keys;    // [L][C]
+  uint32_t* pred;         // [L][W]  bitmap of the last np_predict
+  int32_t* status;        // [4]     device-side error word(s)
+};
+
+// Carved out of the caller's workspace.
+struct Workspace {
+  float* hidden;   // [Bmax][H]
+  float* logits;   // [Bmax][L][M]
+  float* xbuf[2];  // [Bmax][D] each: x_l of the residual chain, ping-pong
+  float* zbuf[3];  // [Bmax][D] each: MLP_l(x_l) accumulators, rotating
+};
+
+struct Dims {
+  int L, D, M, H, k, C, W, Bmax;
+  size_t rec_bytes;
+};
+
+// ---- kernel launchers (each in its own .cu) -------------------------------
+cudaError_t launch_tables_reset(const Dims& d, const Tables& t, cudaStream_t s);
+
+cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, int B, float* hidden,
+                           cudaStream_t s);
+cudaError_t launch_pred_l2(const Dims& d, const void* w2, const float* hidden, int B, float* logits,
+                           cudaStream_t s, int sm_count);
+cudaError_t launch_topk(const Dims& d, const float* logits, int B, uint32_t* bitmap, cudaStream_t s);
+
+cudaError_t launch_delta(const Dims& d, const Tables& t, const uint32_t* pred, int policy, int step,
+                         int32_t* host_lists_dev, int check, cudaStream_t s);
+
+// src_is_store: records are read from the whole-layer store by neuron ID
+// (zero-copy); otherwise record r of `src` is the r-th entry of the lists.
+cudaError_t launch_scatter(const Dims& d, const void* src, bool src_is_store, const int32_t* ids,
+                           const int32_t* slots, const int32_t* count_ptr, int first, int max_rows,
+                           void* gate_l, void* up_l, void* downT_l, int32_t* status, int check,
+                           cudaStream_t s, int sm_count);
+
+struct MlpArgs {
+  const void* gate_l;
+  const void* up_l;
+  const void* downT_l;
+  const int32_t* active_slots;
+  const int32_t* n_active_ptr;  // device counter
+  const float* xa;              // x = xa (+ xb)
+  const float* xb;              // may be NULL
+  float* yacc;                  // [B][D] accumulated with atomics (must hold zeros or a base)
+  float* x_store;               // may be NULL: block 0 stores x here
+  float* zero_out;              // may be NULL: block 0 clears [B][D] here
+  int B;
+  int C;
+  int check;
+  int32_t* status;
+};
+cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count);
+
+cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s);
+cudaError_t launch_add_vec(const float* a, const float* b, float* out, size_t n, cudaStream_t s);
+
+}  // namespace npi

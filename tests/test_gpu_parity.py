@@ -1,0 +1,247 @@
+"""GPU parity: every stage of the CUDA path against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import np_oracle as O
+from paper_2608_22643_b200 import binding as nb
+from paper_2608_22643_b200 import synth
+from tests.harness import REL_L2_TOL, Pair, rel_l2, u16
+
+pytestmark = pytest.mark.gpu
+
+TINY = synth.CONFIGS["tiny"]
+SMALL = synth.CONFIGS["small"]     # ragged: M = 2080 (65 words), H = 96, 3 layers
+
+
+@pytest.mark.parametrize("cfg,B", [(TINY, 1), (SMALL, 1), (SMALL, 3), (TINY, 16)])
+def test_predict_logits_and_bitmap(cfg, B):
+    p = Pair(cfg, max_batch=B)
+    try:
+        xs = synth.hidden_states(cfg, 3, batch=B)
+        L, M, W = cfg.n_layers, cfg.d_ffn, cfg.d_ffn // 32
+        logits = torch.empty((B, L, M), dtype=torch.float32, device="cuda")
+        bitmap = torch.empty((L, W), dtype=torch.int32, device="cuda")
+        for t in range(3):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, B, logits, bitmap, p.eng.stream)
+            p.eng.stream.synchronize()
+            z = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)
+            assert rel_l2(logits.cpu().numpy(), z) < REL_L2_TOL
+            assert rel_l2(logits.cpu().numpy(), z) < 1e-5      # fp32 accumulation does far better
+            # selection is verified on the GPU's own logits: bit-exact
+            want = O.topk_bitmap(logits.cpu().numpy(), p.k)
+            got = bitmap.cpu().numpy().view(np.uint32)
+            assert (got == want).all()
+    finally:
+        p.close()
+
+
+def _topk_case(p, z):
+    B, L, M = z.shape
+    out = torch.empty((L, M // 32), dtype=torch.int32, device="cuda")
+    nb.np_topk(p.eng.ctx, torch.from_numpy(z).cuda(), B, out, p.eng.stream)
+    p.eng.stream.synchronize()
+    assert (out.cpu().numpy().view(np.uint32) == O.topk_bitmap(z, p.k)).all()
+
+
+def test_topk_edge_cases():
+    cfg = TINY
+    L, M = cfg.n_layers, cfg.d_ffn
+    rng = np.random.default_rng(0)
+    p = Pair(cfg, max_batch=4, with_oracle=False)
+    try:
+        _topk_case(p, np.zeros((1, L, M), np.float32))                       # all equal -> lowest indices
+        z = np.full((1, L, M), -0.0, np.float32); z[:, :, 500:600:7] = 0.0   # +0 above -0
+        _topk_case(p, z)
+        _topk_case(p, -np.abs(rng.standard_normal((1, L, M))).astype(np.float32))   # all negative
+        z = rng.standard_normal((1, L, M)).astype(np.float32)
+        z[:, :, ::3] = z[:, :, 1:2]                                          # a third of the keys tie
+        _topk_case(p, z)
+        z = rng.integers(-3, 4, size=(4, L, M)).astype(np.float32)           # heavy ties, batch union
+        _topk_case(p, z)
+        z = rng.standard_normal((2, L, M)).astype(np.float32) * 1e30
+        z[0, 0, 5] = np.inf; z[1, 1, 7] = -np.inf; z[0, 1, 9] = 1e-42        # inf and a denormal
+        _topk_case(p, z)
+    finally:
+        p.close()
+    for k, C in ((0, 8), (M, M), (1, 1)):                                    # degenerate k
+        p = Pair(cfg, k=k, C=C, with_oracle=False)
+        try:
+            _topk_case(p, rng.standard_normal((1, L, M)).astype(np.float32))
+        finally:
+            p.close()
+
+
+@pytest.mark.parametrize("policy", [nb.NP_EVICT_EXACT, nb.NP_EVICT_LRU])
+@pytest.mark.parametrize("cfg,n_set,C,persist", [
+    (TINY, 102, 205, 0.8), (TINY, 102, 102, 0.6), (SMALL, 208, 520, 0.83), (SMALL, 700, 520, 0.7),
+    (TINY, 1, 1, 0.0), (TINY, 0, 4, 0.5),
+])
+def test_delta_lists_and_tables_bit_exact(policy, cfg, n_set, C, persist):
+    """Injected bitmap sequences (fixed-size sets, full replacement, oversize sets that
+    overflow capacity, the empty set) against the oracle, every step."""
+    T = 10
+    p = Pair(cfg, policy=policy, k=min(n_set, C), C=C)
+    try:
+        words = synth.random_bitmaps(cfg.n_layers, cfg.d_ffn, n_set, 11, T, persist)
+        for t in range(T):
+            nb.np_delta(p.eng.ctx, words[t].cuda(), p.eng.stream)
+            deltas = p.ora.res.delta(words[t].numpy().view(np.uint32))
+            cnt = p.check_delta_against(deltas)
+            rc = nb.np_install(p.eng.ctx, 0, cfg.n_layers, p.eng.copy_stream)
+            if n_set > C:
+                assert rc == nb.NP_W_OVERFLOW and (cnt[:, nb.NP_CNT_OVERFLOW] > 0).all()
+            for l, d in enumerate(deltas):
+                O.install(p.store_u16, p.ora.gate, p.ora.up, p.ora.downT, l, d.delta_ids, d.delta_slots)
+        p.check_resident_bytes()
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("mode,staging_rows", [
+    (nb.NP_XFER_MEMCPY_RUNS, None), (nb.NP_XFER_MEMCPY_RUNS, 1), (nb.NP_XFER_MEMCPY_RUNS, 7),
+    (nb.NP_XFER_HOST_GATHER, None), (nb.NP_XFER_HOST_GATHER, 2), (nb.NP_XFER_HOST_GATHER, 9),
+    (nb.NP_XFER_ZERO_COPY, None),
+])
+def test_install_every_transfer_mode_and_chunking(mode, staging_rows):
+    """After each step every resident row holds its record's bytes, however the
+    delta was moved and however small the staging buffer is (Section 3.5)."""
+    cfg = SMALL
+    p = Pair(cfg, transfer_mode=mode, staging_rows=staging_rows)
+    try:
+        words = synth.random_bitmaps(cfg.n_layers, cfg.d_ffn, p.k, 5, 6, 0.8)
+        # make some IDs adjacent so that run coalescing has work to do
+        words[:, :, 3] = -1
+        for t in range(6):
+            nb.np_delta(p.eng.ctx, words[t].cuda(), p.eng.stream)
+            rc = nb.np_install(p.eng.ctx, 0, cfg.n_layers, p.eng.copy_stream)
+            if staging_rows is not None and mode != nb.NP_XFER_ZERO_COPY and t == 0:
+                assert rc == nb.NP_W_CHUNKED
+            p.check_resident_bytes()
+            deltas = p.ora.res.delta(words[t].numpy().view(np.uint32))
+            p.check_delta_against(deltas)
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("cfg,B", [(TINY, 1), (SMALL, 1), (SMALL, 2), (SMALL, 5)])
+def test_sparse_mlp_per_layer(cfg, B):
+    p = Pair(cfg, max_batch=B)
+    try:
+        words = synth.random_bitmaps(cfg.n_layers, cfg.d_ffn, p.k, 9, 3, 0.8)
+        rng = np.random.default_rng(4)
+        for t in range(3):
+            nb.np_delta(p.eng.ctx, words[t].cuda(), p.eng.stream)
+            nb.np_install(p.eng.ctx, 0, cfg.n_layers, p.eng.copy_stream)
+            deltas = p.ora.res.delta(words[t].numpy().view(np.uint32))
+            for l, d in enumerate(deltas):
+                O.install(p.store_u16, p.ora.gate, p.ora.up, p.ora.downT, l, d.delta_ids, d.delta_slots)
+            x = rng.standard_normal((B, cfg.d_model)).astype(np.float32)
+            xd = torch.from_numpy(x).cuda()
+            y = torch.full((B, cfg.d_model), 7.0, dtype=torch.float32, device="cuda")   # must be overwritten
+            for l, d in enumerate(deltas):
+                nb.np_sparse_mlp(p.eng.ctx, l, xd, B, y, p.eng.stream)
+                p.eng.stream.synchronize()
+                want = O.sparse_mlp(p.ora.gate, p.ora.up, p.ora.downT, l, d.active_slots, x.astype(np.float64))
+                assert rel_l2(y.cpu().numpy(), want) < REL_L2_TOL, (t, l)
+                assert rel_l2(y.cpu().numpy(), want) < 1e-5, (t, l)
+    finally:
+        p.close()
+
+
+def test_all_rows_active_is_the_dense_mlp():
+    """k = C = M: the sparse path over every row equals the dense SwiGLU MLP."""
+    cfg = TINY
+    M = cfg.d_ffn
+    p = Pair(cfg, k=M, C=M)
+    try:
+        x_bf = synth.hidden_states(cfg, 1)[0]
+        out = torch.empty((1, cfg.d_model), dtype=torch.float32, device="cuda")
+        nb.np_step(p.eng.ctx, x_bf.cuda(), 1, out, p.eng.stream, p.eng.copy_stream)
+        torch.cuda.synchronize()
+        x = x_bf.to(torch.float64)
+        for l in range(cfg.n_layers):
+            rec = p.backing[l].to(torch.float64)
+            x = x + (torch.nn.functional.silu(x @ rec[:, 0].T) * (x @ rec[:, 1].T)) @ rec[:, 2]
+        assert rel_l2(out.cpu().numpy(), x.numpy()) < REL_L2_TOL
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("policy", [nb.NP_EVICT_EXACT, nb.NP_EVICT_LRU])
+@pytest.mark.parametrize("mode", [nb.NP_XFER_MEMCPY_RUNS, nb.NP_XFER_HOST_GATHER, nb.NP_XFER_ZERO_COPY])
+@pytest.mark.parametrize("cfg,B", [(TINY, 1), (SMALL, 4)])
+def test_whole_step_trajectory(policy, mode, cfg, B):
+    """np_step over the config's token sequence: selection bit-exact on the GPU's own
+    logits, lists/tables bit-exact, chain output within tolerance, state carried."""
+    p = Pair(cfg, policy=policy, transfer_mode=mode, max_batch=B, C=cfg.capacity if B == 1 else cfg.d_ffn // 2)
+    try:
+        xs = synth.hidden_states(cfg, cfg.n_tokens, batch=B)
+        L, M, W = cfg.n_layers, cfg.d_ffn, cfg.d_ffn // 32
+        out = torch.empty((B, cfg.d_model), dtype=torch.float32, device="cuda")
+        logits = torch.empty((B, L, M), dtype=torch.float32, device="cuda")
+        for t in range(cfg.n_tokens):
+            # the predictor kernels are deterministic: this call's logits are the step's logits
+            nb.np_predict(p.eng.ctx, xs[t].cuda(), B, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, xs[t].cuda(), B, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            res = p.ora.step(u16(xs[t]), logits_f32=z32)
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < REL_L2_TOL, t
+            # informational: the oracle's own logits agree with the GPU's
+            z = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)
+            assert rel_l2(z32, z) < 1e-5
+        p.check_resident_bytes()
+        us = nb.np_last_step_times(p.eng.ctx)
+        assert (us >= 0).all()
+    finally:
+        p.close()
+
+
+def test_call_order_and_argument_errors():
+    p = Pair(TINY, with_oracle=False)
+    try:
+        ctx = p.eng.ctx
+        lib = nb.load()
+        assert lib.np_install(ctx, 0, 1, None) == nb.NP_E_STATE          # no delta yet
+        assert lib.np_delta(ctx, None, None) == nb.NP_E_STATE            # no predict yet
+        y = torch.zeros(256, device="cuda")
+        assert lib.np_sparse_mlp(ctx, 0, y.data_ptr(), 1, y.data_ptr(), None) == nb.NP_E_STATE
+        assert lib.np_sparse_mlp(ctx, 5, y.data_ptr(), 1, y.data_ptr(), None) == nb.NP_E_INVAL
+        assert lib.np_predict(ctx, y.data_ptr(), 2, None, None, None) == nb.NP_E_INVAL   # B > max_batch
+        assert lib.np_install(ctx, 1, 0, None) == nb.NP_E_INVAL
+        assert "np_install" in nb.np_last_error(ctx) or "layer" in nb.np_last_error(ctx)
+        words = synth.random_bitmaps(2, 1024, 50, 1, 1)
+        nb.np_delta(ctx, words[0].cuda(), p.eng.stream)
+        assert nb.np_install(ctx, 0, 2, p.eng.copy_stream) == nb.NP_OK
+        nb.np_reset(ctx, p.eng.stream)
+        assert lib.np_install(ctx, 0, 1, None) == nb.NP_E_STATE
+        st = p.eng.export_state(0)
+        assert (st["slot_map"] == -1).all() and (st["owner"] == -1).all() and not st["resident"].any()
+    finally:
+        p.close()
+
+
+def test_export_import_roundtrip_resumes_trajectory():
+    cfg = TINY
+    a = Pair(cfg, policy=nb.NP_EVICT_LRU)
+    b = Pair(cfg, policy=nb.NP_EVICT_LRU, with_oracle=False)
+    try:
+        words = synth.random_bitmaps(cfg.n_layers, cfg.d_ffn, a.k, 21, 8, 0.7)
+        for t in range(4):
+            nb.np_delta(a.eng.ctx, words[t].cuda(), a.eng.stream)
+            a.ora.res.delta(words[t].numpy().view(np.uint32))
+        for l in range(cfg.n_layers):
+            st = a.eng.export_state(l)
+            nb.np_import_state(b.eng.ctx, l, st["slot_map"], st["owner"], st["resident"], st["stamp"], 4,
+                               b.eng.stream)
+        for t in range(4, 8):
+            nb.np_delta(b.eng.ctx, words[t].cuda(), b.eng.stream)
+            deltas = a.ora.res.delta(words[t].numpy().view(np.uint32))
+            b.ora = a.ora
+            b.check_delta_against(deltas)
+    finally:
+        a.close()
+        b.close()
