@@ -240,7 +240,7 @@ class _DeviceInts:
     """int32 view of raw device memory, for torch.as_tensor."""
 
     def __init__(self, addr: int, n: int):
-        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (addr, True), "version": 2}
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<i4", "data": (addr, False), "version": 2}
 
 
 class Engine:
