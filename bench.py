@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Decode-step benchmark of the delta-prefetch sparse-MLP path.
+
+  python bench.py --gpus N --steps K --warmup W            # the CUDA library
+  python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+
+A step is one pass of the whole hot path (predict -> top-k -> delta -> install ->
+sparse MLP chain) over one decode token of the seeded synthetic 7B-shaped stack.
+`value` is measured with the token's hidden state already in HBM; `e2e` with the
+hidden state in pinned host memory and the result read back every step.  The
+record store lives in pinned host memory in both (it stands in for the NVMe
+file), so the install traffic crosses PCIe inside every timed step.
+
+With N > 1 (torchrun) every rank runs an independent replica of the stack on
+its own sequence: the path has no exchange step, so there is no collective.
+Prints exactly one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_22643_b200 import synth  # noqa: E402
+
+METRIC = "decode steps/s (predict+delta+install+sparse MLP, 7B shape)"
+UNIT = "steps/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=120)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--config", default="7b", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--policy", default="exact", choices=["exact", "lru"])
+    ap.add_argument("--transfer", default="gather", choices=["runs", "gather", "zerocopy"])
+    ap.add_argument("--rho", type=float, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-baseline-steps", type=int, default=3)
+    ap.add_argument("--details", action="store_true", help="print per-stage details to stderr")
+    return ap.parse_args()
+
+
+def u16(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as f:
+                return float(json.load(f)["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def make_workload(cfg, gen_device: str, pin: bool):
+    """Weights (CPU + generator device), the record store on the host, hidden states."""
+    t0 = time.time()
+    w1, w2 = synth.predictor_weights(cfg, gen_device)
+    store = torch.empty((cfg.n_layers, cfg.d_ffn, 3, cfg.d_model), dtype=torch.bfloat16)
+    if pin:
+        from paper_2608_22643_b200 import binding as nb
+        nb.pin_host_tensor(store)
+    synth.fill_backing_store(cfg, store, gen_device)
+    return w1, w2, store, time.time() - t0
+
+
+def run_oracle_steps(cfg, policy, w1, w2, store, xs, n_steps, layers=None):
+    """Times the oracle, as it stands, on steps 1..n_steps of the sequence (step 0 is
+    the cold start and is run untimed).  Returns seconds per timed step."""
+    from oracle import np_oracle as O
+    L = cfg.n_layers if layers is None else layers
+    eng = O.Engine(L, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
+                   O.EVICT_LRU if policy == "lru" else O.EVICT_EXACT, u16(w1),
+                   u16(w2)[: L * cfg.d_ffn], u16(store)[:L])
+    eng.step(u16(xs[0]))
+    times = []
+    for t in range(1, n_steps + 1):
+        t0 = time.perf_counter()
+        eng.step(u16(xs[t % xs.shape[0]]))
+        times.append(time.perf_counter() - t0)
+    return times
+
+
+def reference_arm(args):
+    """The oracle timed on the host cores, on this arm's config and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = synth.CONFIGS[args.config]
+    if args.rho is not None:
+        cfg = cfg.with_(rho=args.rho)
+    gen_device = "cuda" if torch.cuda.is_available() else "cpu"
+    w1, w2, store, _ = make_workload(cfg, gen_device, pin=False)
+    w1, w2 = w1.cpu(), w2.cpu()
+    K, W = args.steps, args.warmup
+    xs = synth.hidden_states(cfg, K + W + 2)
+    # one full step to size the sample: keep the whole run within ~150 s of oracle work
+    probe = run_oracle_steps(cfg, args.policy, w1, w2, store, xs, 1)[0]
+    budget = 150.0
+    L = cfg.n_layers
+    layers = L
+    if probe * (K + W) > budget:
+        layers = max(1, min(L, int(L * budget / (probe * (K + W)))))
+    from oracle import np_oracle as O
+    eng = O.Engine(layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
+                   O.EVICT_LRU if args.policy == "lru" else O.EVICT_EXACT, u16(w1),
+                   u16(w2)[: layers * cfg.d_ffn], u16(store)[:layers])
+    eng.step(u16(xs[0]))                       # cold start, untimed
+    for t in range(1, W + 1):
+        eng.step(u16(xs[t]))
+    t0 = time.perf_counter()
+    for t in range(W + 1, W + 1 + K):
+        eng.step(u16(xs[t]))
+    elapsed = time.perf_counter() - t0
+    scale = L / layers                         # a step over `layers` of L layers, scaled to the stack
+    ms = elapsed / K * 1000.0 * scale
+    value = 1000.0 / ms
+    cores = oracle_threads()
+    sample = (f"{K} steady-state decode steps of the {cfg.name} stack, first {layers} of {L} layers"
+              + (", time scaled by L/layers" if layers != L else ""))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: L={L} D={cfg.d_model} M={cfg.d_ffn} H={cfg.d_pred} "
+                               f"k={cfg.top_k} C={cfg.capacity} B=1 rho={cfg.rho} policy={args.policy}"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cuda_arm(args):
+    from paper_2608_22643_b200 import binding as nb
+    from paper_2608_22643_b200 import build as nbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (there is no CPU fallback; use --impl reference)")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        nbuild.build()
+    if dist:
+        dist.barrier()
+    nb.load()
+
+    cfg = synth.CONFIGS[args.config]
+    if args.rho is not None:
+        cfg = cfg.with_(rho=args.rho)
+    cfg = cfg.with_(seed=cfg.seed + 1000 * rank)      # every replica decodes its own sequence
+    K, W = args.steps, args.warmup
+    if W < 3:
+        raise SystemExit("bench.py: --warmup must be >= 3")
+    policy = nb.NP_EVICT_LRU if args.policy == "lru" else nb.NP_EVICT_EXACT
+    mode = {"runs": nb.NP_XFER_MEMCPY_RUNS, "gather": nb.NP_XFER_HOST_GATHER,
+            "zerocopy": nb.NP_XFER_ZERO_COPY}[args.transfer]
+
+    w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True)
+    ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
+                          max_batch=1, evict_policy=policy, transfer_mode=mode,
+                          staging_rows=2 * cfg.top_k)
+    eng = nb.Engine(ncfg, w1, w2, store, device=dev)
+    L, D, M = cfg.n_layers, cfg.d_model, cfg.d_ffn
+    rec = cfg.record_bytes
+    T = 1 + W + K                                      # cold start + warm-up + timed
+    xs_host = synth.hidden_states(cfg, T).pin_memory()             # [T, 1, D] bf16
+    xs_dev = xs_host.to(dev)
+    out = torch.empty((1, D), dtype=torch.float32, device=dev)
+    out_host = torch.empty((1, D), dtype=torch.float32).pin_memory()
+    x_stage = torch.empty((1, D), dtype=torch.bfloat16, device=dev)
+    s, cs = eng.stream, eng.copy_stream
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def run_resident(t_lo, t_hi, stats=None):
+        for t in range(t_lo, t_hi):
+            nb.np_step(eng.ctx, xs_dev[t], 1, out, s, cs)
+            if stats is not None:
+                stats.append(eng.counters().copy())
+
+    # ---- device-resident timing ("value") ----------------------------------------------
+    run_resident(0, 1 + W)                              # cold start + warm-up
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = nb.np_launch_count(eng.ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(s)
+    run_resident(1 + W, T)
+    e1.record(s)
+    barrier()
+    launches = nb.np_launch_count(eng.ctx) - launches0
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- end-to-end timing: hidden state from pinned host, result back to the host --------
+    nb.np_reset(eng.ctx, s)
+    def run_e2e(t_lo, t_hi):
+        for t in range(t_lo, t_hi):
+            with torch.cuda.stream(s):
+                x_stage.copy_(xs_host[t], non_blocking=True)
+            nb.np_step(eng.ctx, x_stage, 1, out, s, cs)
+            with torch.cuda.stream(s):
+                out_host.copy_(out, non_blocking=True)
+            s.synchronize()                              # the caller consumes the result every step
+    run_e2e(0, 1 + W)
+    barrier()
+    t0 = time.perf_counter()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record(s)
+    run_e2e(1 + W, T)
+    g1.record(s)
+    barrier()
+    e2e_ms_total = g0.elapsed_time(g1)
+    clocks = sampler.stop()
+
+    # ---- per-stage detail on a few more steady-state steps (untimed region) ----------------
+    stage_us, delta_rows, overlap = [], [], []
+    for i in range(min(16, K)):
+        t = 1 + W + i
+        nb.np_step(eng.ctx, xs_dev[t], 1, out, s, cs)
+        stage_us.append(nb.np_last_step_times(eng.ctx))
+        c = eng.counters()
+        delta_rows.append(float(c[:, nb.NP_CNT_DELTA].mean()))
+        overlap.append(float((c[:, nb.NP_CNT_KEPT] / np.maximum(1, c[:, nb.NP_CNT_PRED])).mean()))
+    stage_us = np.median(np.stack(stage_us), axis=0)
+    n_active = float(eng.counters()[:, nb.NP_CNT_ACTIVE].mean())
+
+    # ---- dominant kernel: the sparse MLP, timed alone on its own stream ---------------------
+    reps = 20
+    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        nb.np_mlp_chain(eng.ctx, xs_dev[T - 1], 1, out, s)
+    s.synchronize()
+    k0.record(s)
+    for _ in range(reps):
+        nb.np_mlp_chain(eng.ctx, xs_dev[T - 1], 1, out, s)
+    k1.record(s)
+    s.synchronize()
+    mlp_us = k0.elapsed_time(k1) * 1000.0 / (reps * L)            # per layer launch, gaps included
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    p0.record(s)
+    for _ in range(reps):
+        nb.np_predict(eng.ctx, xs_dev[T - 1], 1, None, None, s)
+    p1.record(s)
+    s.synchronize()
+    pred_us = p0.elapsed_time(p1) * 1000.0 / reps
+
+    # max over ranks
+    vals = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms_total = float(vals[0]), float(vals[1])
+
+    peak, peak_kind = measured_peaks()
+    mlp_bytes = n_active * rec + 4 * n_active + 8 * D            # rows + slot list + x in, y out
+    achieved = mlp_bytes / (mlp_us * 1e-6) / 1e9
+    pred_bytes = 2 * cfg.d_pred * D + 2 * L * M * cfg.d_pred + 4 * L * M
+    mean_delta = float(np.mean(delta_rows))
+    result = {
+        "metric": METRIC, "value": K * world / (ms_total / 1000.0), "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
+                        f"B=1 rho={cfg.rho} policy={args.policy} transfer={args.transfer}",
+            "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
+            "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
+            "replicas": world,
+        },
+        "e2e": {"value": K * world / (e2e_ms_total / 1000.0), "unit": UNIT,
+                "h2d_bytes_per_step": int(D * 2 + mean_delta * L * rec), "d2h_bytes_per_step": int(D * 4)},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "k_sparse_mlp", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                     "us_per_launch": mlp_us, "bytes_per_launch": mlp_bytes},
+        "stages_us": {"predict_topk": float(stage_us[0]), "delta": float(stage_us[1]),
+                      "install_copy_stream": float(stage_us[2]), "mlp_chain_incl_waits": float(stage_us[3]),
+                      "predict_alone": pred_us, "predict_gbs": pred_bytes / (pred_us * 1e-6) / 1e9,
+                      "mlp_chain_alone": mlp_us * L},
+        "setup_s": {"generate": gen_s},
+    }
+
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        n = args.cpu_baseline_steps
+        times = run_oracle_steps(cfg, args.policy, w1.cpu(), w2.cpu(), store, xs_host, n)
+        sec = float(np.mean(times))
+        result["cpu_baseline"] = {
+            "value": 1.0 / sec, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"{n} steady-state decode steps of the same stack (all {L} layers), after an untimed cold start"}
+    elif rank == 0:
+        result["cpu_baseline"] = None
+    eng.close()
+    if rank == 0:
+        print(json.dumps(result))
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        cuda_arm(args)
+
+
+if __name__ == "__main__":
+    main()

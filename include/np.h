@@ -219,6 +219,17 @@ int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* 
 int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream,
             void* copy_stream);
 
+/* Stage 4 for every layer in order, nothing else: the residual chain
+ * x_{l+1} = x_l + MLP_l(x_l) over the rows that are active and resident now
+ * (Section 3.1: the sparse suffix runs once the delta rows are in place).
+ *   x_bf16  dev bf16 [B][D]  x_0,   x_out  dev fp32 [B][D]  x_L
+ * Orders `stream` after any pending install marks.  Errors as np_sparse_mlp. */
+int np_mlp_chain(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream);
+
+/* Number of kernels this context has launched since np_init (memsets and
+ * copies are not counted).  Host counter, no synchronisation. */
+int np_launch_count(np_ctx* ctx, uint64_t* out);
+
 /* Device pointers to one layer's lists and counters from the last np_delta. */
 int np_get_delta(np_ctx* ctx, int32_t layer, np_delta_view* out);
 

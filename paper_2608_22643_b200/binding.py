@@ -31,7 +31,8 @@ NP_N_COUNTERS = 8
 EXPORTED = [
     "np_version", "np_query_sizes", "np_init", "np_destroy", "np_reset", "np_last_error",
     "np_predict", "np_topk", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
-    "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times",
+    "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
+    "np_launch_count",
 ]
 
 
@@ -97,6 +98,8 @@ def load() -> C.CDLL:
         "np_export_state": [vp, i32, vp, vp, vp, vp, vp],
         "np_import_state": [vp, i32, vp, vp, vp, vp, i32, vp],
         "np_last_step_times": [vp, vp],
+        "np_mlp_chain": [vp, vp, i32, vp, vp],
+        "np_launch_count": [vp, C.POINTER(C.c_uint64)],
     }
     for name, args in sigs.items():
         fn = getattr(lib, name)
@@ -212,6 +215,16 @@ def np_last_step_times(ctx) -> np.ndarray:
     out = np.zeros(4, dtype=np.float32)
     _check(ctx, load().np_last_step_times(ctx, _ptr(out)))
     return out
+
+
+def np_mlp_chain(ctx, x_bf16, B: int, x_out, stream=None) -> int:
+    return _check(ctx, load().np_mlp_chain(ctx, _ptr(x_bf16), B, _ptr(x_out), _stream(stream)))
+
+
+def np_launch_count(ctx) -> int:
+    out = C.c_uint64()
+    _check(ctx, load().np_launch_count(ctx, C.byref(out)))
+    return int(out.value)
 
 
 # ---- buffer owner ----------------------------------------------------------------------

@@ -121,6 +121,7 @@ struct np_ctx {
   bool have_pred = false;
   bool have_step = false;
   int step = 0;
+  uint64_t launches = 0;
   Pool* pool = nullptr;
   std::string err;
 };
@@ -144,6 +145,13 @@ int fail(np_ctx* ctx, int code, const char* fmt, ...) {
     if (e__ != cudaSuccess)                                                                 \
       return fail(ctx, NP_E_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e__),  \
                   __FILE__, __LINE__);                                                      \
+  } while (0)
+
+// a kernel launch: counted, then checked
+#define NP_LAUNCH(ctx, call) \
+  do {                       \
+    (ctx)->launches += 1;    \
+    NP_CUDA(ctx, call);      \
   } while (0)
 
 int check_config(const np_config* c, np_ctx* ctx) {
@@ -379,7 +387,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
 
 int np_reset(np_ctx* ctx, void* stream) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
-  NP_CUDA(ctx, launch_tables_reset(ctx->d, ctx->t, as_stream(stream)));
+  NP_LAUNCH(ctx, launch_tables_reset(ctx->d, ctx->t, as_stream(stream)));
   ctx->have_delta = ctx->have_pred = ctx->have_step = false;
   std::fill(ctx->install_pending.begin(), ctx->install_pending.end(), 0);
   ctx->step = 0;
@@ -394,9 +402,9 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
   if ((uintptr_t)x_bf16 % 16) return fail(ctx, NP_E_INVAL, "x must be 16-byte aligned");
   cudaStream_t s = as_stream(stream);
   const Dims& d = ctx->d;
-  NP_CUDA(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
-  NP_CUDA(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, s, ctx->sm_count));
-  NP_CUDA(ctx, launch_topk(d, ctx->ws.logits, B, ctx->t.pred, s));
+  NP_LAUNCH(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
+  NP_LAUNCH(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, s, ctx->sm_count));
+  NP_LAUNCH(ctx, launch_topk(d, ctx->ws.logits, B, ctx->t.pred, s));
   const size_t nlog = (size_t)B * d.L * d.M * 4, nbm = (size_t)d.L * d.W * 4;
   if (logits_out) NP_CUDA(ctx, cudaMemcpyAsync(logits_out, ctx->ws.logits, nlog, cudaMemcpyDeviceToDevice, s));
   if (bitmap_out) NP_CUDA(ctx, cudaMemcpyAsync(bitmap_out, ctx->t.pred, nbm, cudaMemcpyDeviceToDevice, s));
@@ -408,7 +416,7 @@ int np_topk(np_ctx* ctx, const float* logits, int32_t B, uint32_t* bitmap_out, v
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   if (!logits || !bitmap_out) return fail(ctx, NP_E_INVAL, "logits or bitmap_out is NULL");
   if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
-  NP_CUDA(ctx, launch_topk(ctx->d, logits, B, bitmap_out, as_stream(stream)));
+  NP_LAUNCH(ctx, launch_topk(ctx->d, logits, B, bitmap_out, as_stream(stream)));
   return NP_OK;
 }
 
@@ -426,7 +434,7 @@ int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream) {
       ctx->install_pending[l] = 0;
     }
   }
-  NP_CUDA(ctx, launch_delta(ctx->d, ctx->t, pred_bitmap, ctx->cfg.evict_policy, ctx->step, ctx->host_lists_dev,
+  NP_LAUNCH(ctx, launch_delta(ctx->d, ctx->t, pred_bitmap, ctx->cfg.evict_policy, ctx->step, ctx->host_lists_dev,
                             ctx->cfg.flags & NP_F_CHECK_BOUNDS, s));
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_delta, s));
   ctx->step += 1;
@@ -452,7 +460,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
     const int max_rows = d.C;
     for (int l = layer_begin; l < layer_end; ++l) {
       const char* store_l = ctx->backing_dev + (size_t)l * d.M * rec;
-      NP_CUDA(ctx, launch_scatter(d, store_l, true, ctx->t.delta_ids + (size_t)l * d.C,
+      NP_LAUNCH(ctx, launch_scatter(d, store_l, true, ctx->t.delta_ids + (size_t)l * d.C,
                                   ctx->t.delta_slots + (size_t)l * d.C,
                                   ctx->t.counters + (size_t)l * NP_N_COUNTERS + NP_CNT_DELTA, 0, max_rows,
                                   static_cast<char*>(ctx->bufs.gate_buf) + (size_t)l * d.C * row_bytes,
@@ -499,7 +507,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
                                        cudaMemcpyHostToDevice, cs));
           r += len;
         }
-        NP_CUDA(ctx, launch_scatter(d, staging, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
+        NP_LAUNCH(ctx, launch_scatter(d, staging, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
                                     down_l, ctx->t.status, check, cs, ctx->sm_count));
       }
     } else {  // NP_XFER_HOST_GATHER: two halves of pinned staging, packed by the pool
@@ -536,7 +544,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
         NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)rows * rec, cudaMemcpyHostToDevice, cs));
         NP_CUDA(ctx, cudaEventRecord(ctx->ev_half[h], cs));
         ctx->half_pending[h] = true;
-        NP_CUDA(ctx, launch_scatter(d, dbuf, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
+        NP_LAUNCH(ctx, launch_scatter(d, dbuf, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
                                     down_l, ctx->t.status, check, cs, ctx->sm_count));
       }
     }
@@ -566,7 +574,39 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
   a.status = ctx->t.status;
   if (ctx->install_pending[layer]) NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0));
-  NP_CUDA(ctx, launch_sparse_mlp(d, a, s, ctx->sm_count));
+  NP_LAUNCH(ctx, launch_sparse_mlp(d, a, s, ctx->sm_count));
+  return NP_OK;
+}
+
+// residual chain: x_l = xbuf[(l+1)&1] + zbuf[(l-1)%3]; layer l accumulates MLP_l(x_l) into
+// zbuf[l%3], stores x_l to xbuf[l&1] and clears zbuf[(l+1)%3] for the next layer
+static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaStream_t s) {
+  const Dims& d = ctx->d;
+  const size_t n = (size_t)B * d.D;
+  NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, n * 4, s));
+  for (int l = 0; l < d.L; ++l) {
+    int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
+                       ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, s);
+    if (rc < 0) return rc;
+  }
+  NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], x_out, n, s));
+  return NP_OK;
+}
+
+int np_mlp_chain(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!x_bf16 || !x_out) return fail(ctx, NP_E_INVAL, "x or x_out is NULL");
+  if ((uintptr_t)x_out % 16) return fail(ctx, NP_E_INVAL, "x_out must be 16-byte aligned");
+  if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
+  if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_mlp_chain needs a prior np_delta");
+  return mlp_chain(ctx, x_bf16, B, x_out, as_stream(stream));
+}
+
+int np_launch_count(np_ctx* ctx, uint64_t* out) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!out) return fail(ctx, NP_E_INVAL, "out is NULL");
+  *out = ctx->launches;
   return NP_OK;
 }
 
@@ -604,17 +644,8 @@ int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stre
   if (warn < 0) return warn;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_c[1], cs));
 
-  // residual chain: x_l = xbuf[(l+1)&1] + zbuf[(l-1)%3]; layer l accumulates MLP_l(x_l) into
-  // zbuf[l%3], stores x_l to xbuf[l&1] and clears zbuf[(l+1)%3] for the next layer
-  const size_t n = (size_t)B * d.D;
-  NP_CUDA(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
-  NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, n * 4, s));
-  for (int l = 0; l < d.L; ++l) {
-    rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
-                   ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, s);
-    if (rc < 0) return rc;
-  }
-  NP_CUDA(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], x_out, n, s));
+  rc = mlp_chain(ctx, x_bf16, B, x_out, s);
+  if (rc < 0) return rc;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[3], s));
   ctx->have_step = true;
   return warn;
