@@ -52,7 +52,9 @@ def parse_args():
     ap.add_argument("--rho", type=float, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-steps", type=int, default=3)
-    ap.add_argument("--details", action="store_true", help="print per-stage details to stderr")
+    ap.add_argument("--layer-launches", action="store_true", help="one MLP kernel launch per layer")
+    ap.add_argument("--direct-loads", action="store_true", help="MLP rows by plain global loads")
+    ap.add_argument("--chain-layers", type=int, default=0, help="layers per resident MLP kernel")
     return ap.parse_args()
 
 
@@ -245,7 +247,9 @@ def cuda_arm(args):
     w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True)
     ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
                           max_batch=1, evict_policy=policy, transfer_mode=mode,
-                          staging_rows=2 * cfg.top_k)
+                          staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
+                          flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
+                          | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0))
     eng = nb.Engine(ncfg, w1, w2, store, device=dev)
     L, D, M = cfg.n_layers, cfg.d_model, cfg.d_ffn
     rec = cfg.record_bytes

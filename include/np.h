@@ -71,6 +71,10 @@ extern "C" {
 /* np_config.flags */
 #define NP_F_CHECK_BOUNDS    1  /* kernels validate every slot / neuron index and report
                                    through NP_E_DEVICE instead of touching memory */
+#define NP_F_DIRECT_LOADS    2  /* sparse MLP: plain 16-byte global loads instead of the
+                                   shared-memory staged kernel (for comparison runs) */
+#define NP_F_LAYER_LAUNCHES  4  /* np_step / np_mlp_chain: one kernel launch per layer instead
+                                   of resident kernels spanning runs of layers */
 
 /* per-layer counters written by np_delta (np_read_counters) */
 #define NP_CNT_PRED      0  /* |P|                      */
@@ -99,7 +103,9 @@ typedef struct np_config {
   int32_t transfer_mode;  /* NP_XFER_* */
   int32_t flags;          /* NP_F_* */
   int32_t host_threads;   /* worker threads for NP_XFER_HOST_GATHER (0 = pick) */
-  int32_t reserved[4];    /* must be 0 */
+  int32_t chain_layers;   /* layers per resident MLP kernel in np_step / np_mlp_chain
+                             (0 = a quarter of the stack) */
+  int32_t reserved[3];    /* must be 0 */
 } np_config;
 
 /* Byte counts of the caller-owned buffers for a configuration. */

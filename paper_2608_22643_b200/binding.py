@@ -24,6 +24,8 @@ NP_W_OVERFLOW, NP_W_CHUNKED = 1, 2
 NP_EVICT_EXACT, NP_EVICT_LRU = 0, 1
 NP_XFER_MEMCPY_RUNS, NP_XFER_HOST_GATHER, NP_XFER_ZERO_COPY = 0, 1, 2
 NP_F_CHECK_BOUNDS = 1
+NP_F_DIRECT_LOADS = 2
+NP_F_LAYER_LAUNCHES = 4
 (NP_CNT_PRED, NP_CNT_KEPT, NP_CNT_DELTA, NP_CNT_EVICT, NP_CNT_OVERFLOW, NP_CNT_ACTIVE,
  NP_CNT_RESIDENT, NP_CNT_STEP) = range(8)
 NP_N_COUNTERS = 8
@@ -39,7 +41,7 @@ EXPORTED = [
 class np_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
-        "staging_rows", "transfer_mode", "flags", "host_threads")] + [("reserved", C.c_int32 * 4)]
+        "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers")] + [("reserved", C.c_int32 * 3)]
 
 
 class np_sizes(C.Structure):
@@ -229,11 +231,12 @@ def np_launch_count(ctx) -> int:
 
 # ---- buffer owner ----------------------------------------------------------------------
 def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
-                transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0) -> np_config:
+                transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0) -> np_config:
     cfg = np_config()
     cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
     cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
     cfg.evict_policy, cfg.transfer_mode, cfg.flags, cfg.host_threads = evict_policy, transfer_mode, flags, host_threads
+    cfg.chain_layers = chain_layers
     cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
     return cfg
 

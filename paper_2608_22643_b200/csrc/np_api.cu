@@ -173,9 +173,10 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->staging_rows < 1) return fail(ctx, NP_E_INVAL, "staging_rows must be >= 1");
   if (c->transfer_mode == NP_XFER_HOST_GATHER && c->staging_rows < 2)
     return fail(ctx, NP_E_INVAL, "host gather needs staging_rows >= 2 (two halves)");
-  if (c->flags & ~NP_F_CHECK_BOUNDS) return fail(ctx, NP_E_INVAL, "unknown flag bits");
+  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
-  for (int i = 0; i < 4; ++i)
+  if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
+  for (int i = 0; i < 3; ++i)
     if (c->reserved[i]) return fail(ctx, NP_E_INVAL, "reserved fields must be 0");
   return NP_OK;
 }
@@ -333,7 +334,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_res = take(LW), o_slot = take(LM), o_owner = take(LC), o_stamp = take(LM);
   const size_t o_did = take(LC), o_dsl = take(LC), o_eid = take(LC), o_aid = take(LC), o_asl = take(LC);
   const size_t o_ovf = take(LM), o_cnt = take((size_t)d.L * NP_N_COUNTERS), o_free = take(LC);
-  const size_t o_cid = take(LC), o_ckey = take(LC), o_pred = take(LW), o_stat = take(4);
+  const size_t o_cid = take(LC), o_ckey = take(LC), o_pred = take(LW), o_stat = take(4), o_bar = take(4);
   NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
   char* base = static_cast<char*>(ctx->slab);
   Tables& t = ctx->t;
@@ -353,6 +354,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   t.cand_keys = reinterpret_cast<uint32_t*>(base + o_ckey);
   t.pred = reinterpret_cast<uint32_t*>(base + o_pred);
   t.status = reinterpret_cast<int32_t*>(base + o_stat);
+  t.grid_bar = reinterpret_cast<unsigned int*>(base + o_bar);
 
   const WsLayout wl = ws_layout(*cfg);
   char* wsb = static_cast<char*>(b->workspace);
@@ -403,7 +405,7 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
   cudaStream_t s = as_stream(stream);
   const Dims& d = ctx->d;
   NP_LAUNCH(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
-  NP_LAUNCH(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, s, ctx->sm_count));
+  NP_LAUNCH(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
   NP_LAUNCH(ctx, launch_topk(d, ctx->ws.logits, B, ctx->t.pred, s));
   const size_t nlog = (size_t)B * d.L * d.M * 4, nbm = (size_t)d.L * d.W * 4;
   if (logits_out) NP_CUDA(ctx, cudaMemcpyAsync(logits_out, ctx->ws.logits, nlog, cudaMemcpyDeviceToDevice, s));
@@ -554,6 +556,15 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
   return warn;
 }
 
+// Orders `s` after a layer's install mark; marks that have already completed need no wait.
+static cudaError_t wait_install(np_ctx* ctx, int layer, cudaStream_t s) {
+  const cudaError_t q = cudaEventQuery(ctx->ev_installed[layer]);
+  if (q == cudaSuccess) return cudaSuccess;
+  if (q != cudaErrorNotReady) return q;
+  (void)cudaGetLastError();
+  return cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0);
+}
+
 static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, float* yacc, float* x_store,
                      float* zero_out, int B, cudaStream_t s) {
   const Dims& d = ctx->d;
@@ -572,6 +583,7 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   a.B = B;
   a.C = d.C;
   a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+  a.force_direct = (ctx->cfg.flags & NP_F_DIRECT_LOADS) ? 1 : 0;
   a.status = ctx->t.status;
   if (ctx->install_pending[layer]) NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0));
   NP_LAUNCH(ctx, launch_sparse_mlp(d, a, s, ctx->sm_count));
@@ -585,10 +597,37 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   const size_t n = (size_t)B * d.D;
   NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
   NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, n * 4, s));
-  for (int l = 0; l < d.L; ++l) {
-    int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
-                       ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, s);
-    if (rc < 0) return rc;
+  const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
+                          mlp_chain_supported(d, ctx->sm_count);
+  if (persistent) {
+    // runs of layers in one resident kernel each; a run starts once its layers are installed,
+    // so the install of later runs still overlaps the compute of earlier ones
+    const int run = std::max(1, ctx->cfg.chain_layers > 0 ? ctx->cfg.chain_layers : (d.L + 3) / 4);
+    for (int l0 = 0; l0 < d.L; l0 += run) {
+      const int l1 = std::min(d.L, l0 + run);
+      for (int l = l0; l < l1; ++l)
+        if (ctx->install_pending[l]) NP_CUDA(ctx, wait_install(ctx, l, s));
+      ChainArgs a;
+      a.gate = ctx->bufs.gate_buf;
+      a.up = ctx->bufs.up_buf;
+      a.downT = ctx->bufs.downT_buf;
+      a.active_slots = ctx->t.active_slots;
+      a.counters = ctx->t.counters;
+      for (int i = 0; i < 2; ++i) a.xbuf[i] = ctx->ws.xbuf[i];
+      for (int i = 0; i < 3; ++i) a.zbuf[i] = ctx->ws.zbuf[i];
+      a.grid_bar = ctx->t.grid_bar;
+      a.status = ctx->t.status;
+      a.l_begin = l0;
+      a.l_end = l1;
+      a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+      NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
+    }
+  } else {
+    for (int l = 0; l < d.L; ++l) {
+      int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
+                         ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, s);
+      if (rc < 0) return rc;
+    }
   }
   NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], x_out, n, s));
   return NP_OK;

@@ -32,6 +32,7 @@ struct Tables {
   uint32_t* cand_keys;    // [L][C]
   uint32_t* pred;         // [L][W]  bitmap of the last np_predict
   int32_t* status;        // [4]     device-side error word(s)
+  unsigned int* grid_bar; // [1]     arrival counter of the persistent MLP kernel
 };
 
 // Carved out of the caller's workspace.
@@ -53,7 +54,7 @@ cudaError_t launch_tables_reset(const Dims& d, const Tables& t, cudaStream_t s);
 cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, int B, float* hidden,
                            cudaStream_t s);
 cudaError_t launch_pred_l2(const Dims& d, const void* w2, const float* hidden, int B, float* logits,
-                           cudaStream_t s, int sm_count);
+                           int32_t* status, cudaStream_t s, int sm_count);
 cudaError_t launch_topk(const Dims& d, const float* logits, int B, uint32_t* bitmap, cudaStream_t s);
 
 cudaError_t launch_delta(const Dims& d, const Tables& t, const uint32_t* pred, int policy, int step,
@@ -80,9 +81,31 @@ struct MlpArgs {
   int B;
   int C;
   int check;
+  int force_direct;  // use the direct-load kernel even where the staged one applies
   int32_t* status;
 };
 cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count);
+
+// Persistent multi-layer form of the sparse MLP for one sequence (np_mlp_chain.cu).
+struct ChainPlan {
+  int n_stages, tile_rows, xj, cols;
+  size_t smem;
+};
+struct ChainArgs {
+  const void* gate;  // layer 0 of each row buffer
+  const void* up;
+  const void* downT;
+  const int32_t* active_slots;  // [L][C]
+  const int32_t* counters;      // [L][NP_N_COUNTERS]
+  float* xbuf[2];
+  float* zbuf[3];
+  unsigned int* grid_bar;
+  int32_t* status;
+  int l_begin, l_end, check;
+};
+bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p);
+bool mlp_chain_supported(const Dims& d, int sm_count);
+cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
 
 cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s);
 cudaError_t launch_add_vec(const float* a, const float* b, float* out, size_t n, cudaStream_t s);

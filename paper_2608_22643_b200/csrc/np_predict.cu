@@ -5,8 +5,11 @@
 // read once, so the kernels are organised around 16-byte coalesced streaming
 // loads with many loads in flight per thread, fp32 accumulation and
 // warp-shuffle reductions.
+#include <algorithm>
+
 #include "np_device.cuh"
 #include "np_internal.h"
+#include "np_pipe.cuh"
 
 namespace npi {
 using namespace npd;
@@ -19,6 +22,7 @@ template <int NB>
 __global__ void __launch_bounds__(128) k_pred_l1(const uint4* __restrict__ w1,
                                                   const uint4* __restrict__ x,  // bf16 [B][D]
                                                   float* __restrict__ hidden, int H, int D, int B) {
+  npp::pdl_launch_dependents();  // layer 2 may start prefetching its weights now
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= H) return;
@@ -74,114 +78,186 @@ cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, in
 
 // ---------------------------------------------------------------------------
 // Layer 2: logits[b][r] = sum_m W2[r][m] * hidden[b][m] for all L*M rows.
-// A row is short (H bf16), so LPR lanes share a row and a warp covers 32/LPR
-// consecutive rows per pass; each lane keeps CPL 16-byte loads in flight.  For
-// one sequence the lane's slice of `hidden` lives in registers.
+//
+// W2 is one contiguous array that is read exactly once, so each block streams
+// its contiguous share of rows through a ring of shared-memory stages filled by
+// 1-D bulk copies (one producer warp, mbarrier full/empty pairs).  Nothing but
+// the ring's size limits the bytes in flight per SM, and no register is spent
+// on loads.  Consumer warps read rows from shared memory: LPR lanes share a row
+// (a quarter-warp reads 128 contiguous bytes: conflict-free), each lane owns CPL
+// 16-byte chunks; for one sequence the lane's slice of `hidden` stays in
+// registers, for several it is read from shared memory.
 // ---------------------------------------------------------------------------
-template <int LPR, int CPL, int NB>
-__global__ void __launch_bounds__(256) k_pred_l2(const uint4* __restrict__ w2,
-                                                  const float* __restrict__ hidden,  // [B][H]
-                                                  float* __restrict__ logits,        // [B][rows]
-                                                  long long rows, int H, int B) {
-  extern __shared__ __align__(16) float sh[];  // [NB][H] when NB > 1
-  constexpr int RPW = 32 / LPR;                // rows per warp pass
-  const int chunks = H >> 3;
-  const int lane = threadIdx.x & 31;
-  const int sub = lane % LPR;  // position inside the row
-  const int rsel = lane / LPR;
+constexpr int kL2ConsumerWarps = 8;
+constexpr int kL2Threads = (kL2ConsumerWarps + 1) * 32;
+constexpr int kL2MaxStages = 8;
 
+template <int LPR, int CPL, int NB>
+__global__ void __launch_bounds__(kL2Threads, 1) k_pred_l2(const uint4* __restrict__ w2,
+                                                            const float* hidden,  // [B][H]; written by the previous kernel
+                                                            float* __restrict__ logits,        // [B][rows]
+                                                            long long rows, int H, int B, int stage_rows,
+                                                            int n_stages, int32_t* status) {
+  extern __shared__ __align__(128) unsigned char l2sm[];
+  __shared__ __align__(8) uint64_t full_bar[kL2MaxStages];
+  __shared__ __align__(8) uint64_t empty_bar[kL2MaxStages];
+  constexpr int RPW = 32 / LPR;  // rows per warp pass
+  const int chunks = H >> 3;
+  const uint32_t row_bytes = (uint32_t)H * 2u;
+  const uint32_t stage_bytes = (uint32_t)stage_rows * row_bytes;
+  unsigned char* ring = l2sm;
+  float* hs = reinterpret_cast<float*>(l2sm + (size_t)n_stages * stage_bytes);  // [NB][H] when NB > 1
+
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  // this block's contiguous share of rows
+  const long long r_begin = rows * blockIdx.x / gridDim.x;
+  const long long r_end = rows * (blockIdx.x + 1) / gridDim.x;
+  const int n_iter = (int)((r_end - r_begin + stage_rows - 1) / stage_rows);
+
+  if (tid == 0) {
+    for (int s = 0; s < n_stages; ++s) {
+      npp::mbar_init(&full_bar[s], 1);
+      npp::mbar_init(&empty_bar[s], kL2ConsumerWarps);
+    }
+    npp::fence_barrier_init();
+  }
+  __syncthreads();
+
+  if (wid == kL2ConsumerWarps) {
+    // ---------------- producer warp: one lane issues the bulk copies ----------------
+    if (lane == 0) {
+      const uint64_t pol = npp::policy_evict_first();
+      for (int it = 0; it < n_iter; ++it) {
+        const int s = it % n_stages;
+        const uint32_t ph = (uint32_t)(it / n_stages) & 1u;
+        if (!npp::mbar_wait(&empty_bar[s], ph ^ 1u)) {
+          atomicOr(status, npp::kStatTimeout);
+          break;
+        }
+        const long long r0 = r_begin + (long long)it * stage_rows;
+        const uint32_t nrows = (uint32_t)min((long long)stage_rows, r_end - r0);
+        const uint32_t bytes = nrows * row_bytes;
+        npp::mbar_expect_tx(&full_bar[s], bytes);
+        npp::bulk_g2s_stream(ring + (size_t)s * stage_bytes, reinterpret_cast<const unsigned char*>(w2) + (size_t)r0 * row_bytes,
+                             bytes, &full_bar[s], pol);
+      }
+    }
+    return;
+  }
+
+  // ---------------- consumer warps ----------------
+  // the weights above do not depend on the previous kernel; `hidden` does
+  npp::pdl_wait_prior();
+  const int sub = lane % LPR, rsel = lane / LPR;
   float hreg[NB == 1 ? CPL * 8 : 1];
   if (NB == 1) {
 #pragma unroll
     for (int i = 0; i < CPL; ++i) {
       const int c = sub + i * LPR;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) hreg[(NB == 1 ? i * 8 + e : 0)] = c < chunks ? hidden[c * 8 + e] : 0.f;
+      for (int e = 0; e < 8; ++e) hreg[NB == 1 ? i * 8 + e : 0] = c < chunks ? hidden[c * 8 + e] : 0.f;
     }
   } else {
-    for (int i = threadIdx.x; i < B * H; i += blockDim.x) sh[i] = hidden[i];
-    __syncthreads();
+    for (int i = tid; i < B * H; i += kL2ConsumerWarps * 32) hs[i] = hidden[i];
+    asm volatile("bar.sync 1, %0;" ::"n"(kL2ConsumerWarps * 32) : "memory");  // consumers only
   }
 
-  const long long warps_total = (long long)gridDim.x * (blockDim.x >> 5);
-  const long long wglobal = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long passes = (rows + RPW - 1) / RPW;
-  // contiguous range of passes per warp keeps each warp streaming through one region
-  const long long per = (passes + warps_total - 1) / warps_total;
-  const long long p0 = wglobal * per, p1 = min(passes, p0 + per);
-
-  for (long long p = p0; p < p1; ++p) {
-    const long long r = p * RPW + rsel;
-    const bool live = r < rows;
-    const uint4* row = w2 + (size_t)(live ? r : 0) * chunks;
-    uint4 w[CPL];
-#pragma unroll
-    for (int i = 0; i < CPL; ++i) {
-      const int c = sub + i * LPR;
-      w[i] = (live && c < chunks) ? ldg_stream(row + c) : make_uint4(0, 0, 0, 0);
+  for (int it = 0; it < n_iter; ++it) {
+    const int s = it % n_stages;
+    const uint32_t ph = (uint32_t)(it / n_stages) & 1u;
+    if (!npp::mbar_wait(&full_bar[s], ph)) {
+      if (lane == 0) atomicOr(status, npp::kStatTimeout);
+      break;
     }
-    float acc[NB];
+    const long long r0 = r_begin + (long long)it * stage_rows;
+    const int nrows = (int)min((long long)stage_rows, r_end - r0);
+    const unsigned char* st = ring + (size_t)s * stage_bytes;
+    for (int g = wid * RPW; g < nrows; g += kL2ConsumerWarps * RPW) {
+      const int rl = g + rsel;
+      const bool live = rl < nrows;
+      const uint4* row = reinterpret_cast<const uint4*>(st + (size_t)(live ? rl : 0) * row_bytes);
+      float acc[NB];
 #pragma unroll
-    for (int b = 0; b < NB; ++b) acc[b] = 0.f;
-    if (NB == 1) {
-#pragma unroll
-      for (int i = 0; i < CPL; ++i) {
-        const float4 ha = make_float4(hreg[i * 8 + 0], hreg[i * 8 + 1], hreg[i * 8 + 2], hreg[i * 8 + 3]);
-        const float4 hb = make_float4(hreg[i * 8 + 4], hreg[i * 8 + 5], hreg[i * 8 + 6], hreg[i * 8 + 7]);
-        acc[0] = dot8(w[i], ha, hb, acc[0]);
-      }
-    } else {
+      for (int b = 0; b < NB; ++b) acc[b] = 0.f;
 #pragma unroll
       for (int i = 0; i < CPL; ++i) {
         const int c = sub + i * LPR;
         if (c < chunks) {
+          const uint4 w = row[c];
+          if (NB == 1) {
+            const float4 ha = make_float4(hreg[NB == 1 ? i * 8 + 0 : 0], hreg[NB == 1 ? i * 8 + 1 : 0],
+                                          hreg[NB == 1 ? i * 8 + 2 : 0], hreg[NB == 1 ? i * 8 + 3 : 0]);
+            const float4 hb = make_float4(hreg[NB == 1 ? i * 8 + 4 : 0], hreg[NB == 1 ? i * 8 + 5 : 0],
+                                          hreg[NB == 1 ? i * 8 + 6 : 0], hreg[NB == 1 ? i * 8 + 7 : 0]);
+            acc[0] = dot8(w, ha, hb, acc[0]);
+          } else {
 #pragma unroll
-          for (int b = 0; b < NB; ++b) {
-            if (b < B) {
-              const float4* hp = reinterpret_cast<const float4*>(sh + (size_t)b * H + c * 8);
-              acc[b] = dot8(w[i], hp[0], hp[1], acc[b]);
+            for (int b = 0; b < NB; ++b) {
+              if (b < B) {
+                const float4* hp = reinterpret_cast<const float4*>(hs + (size_t)b * H + c * 8);
+                acc[b] = dot8(w, hp[0], hp[1], acc[b]);
+              }
             }
           }
         }
       }
-    }
 #pragma unroll
-    for (int b = 0; b < NB; ++b) {
-      float v = acc[b];
+      for (int b = 0; b < NB; ++b) {
+        float v = acc[b];
 #pragma unroll
-      for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (sub == 0 && live && b < B) logits[(size_t)b * rows + r] = v;
+        for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (sub == 0 && live && b < B) logits[(size_t)b * rows + r0 + rl] = v;
+      }
     }
+    __syncwarp();
+    if (lane == 0) npp::mbar_arrive(&empty_bar[s]);  // this warp is done reading the stage
   }
 }
 
 template <int LPR, int CPL>
 static cudaError_t l2_dispatch_nb(const uint4* w2, const float* hidden, float* logits, long long rows,
-                                  int H, int B, int blocks, cudaStream_t s) {
-  const int threads = 256;
-  if (B == 1) {
-    k_pred_l2<LPR, CPL, 1><<<blocks, threads, 0, s>>>(w2, hidden, logits, rows, H, B);
-  } else if (B <= 4) {
-    k_pred_l2<LPR, CPL, 4><<<blocks, threads, (size_t)B * H * 4, s>>>(w2, hidden, logits, rows, H, B);
-  } else {
-    const size_t sm = (size_t)B * H * 4;
-    auto kfn = k_pred_l2<LPR, CPL, 16>;
-    if (sm > 48 * 1024) {
-      cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-      if (e != cudaSuccess) return e;
-    }
-    kfn<<<blocks, threads, sm, s>>>(w2, hidden, logits, rows, H, B);
-  }
-  return cudaGetLastError();
+                                  int H, int B, int blocks, int32_t* status, cudaStream_t s) {
+  // stage: about 32 KB of whole rows, a multiple of the rows one pass of all consumer warps covers
+  const int row_bytes = H * 2;
+  const int pass_rows = kL2ConsumerWarps * (32 / LPR);
+  int stage_rows = std::max(1, 32768 / row_bytes);
+  stage_rows = std::max(pass_rows, stage_rows / pass_rows * pass_rows);
+  const size_t stage_bytes = (size_t)stage_rows * row_bytes;
+  const size_t hs_bytes = B > 1 ? (size_t)B * H * 4 : 0;
+  int n_stages = (int)std::min<size_t>(kL2MaxStages, (200 * 1024 - hs_bytes) / stage_bytes);
+  if (n_stages < 2) return cudaErrorInvalidValue;
+  const size_t sm = (size_t)n_stages * stage_bytes + hs_bytes;
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(kL2Threads);
+  cfg.dynamicSmemBytes = sm;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+#define NP_L2_LAUNCH(NBV)                                                                             \
+  do {                                                                                                \
+    auto kfn = k_pred_l2<LPR, CPL, NBV>;                                                              \
+    cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);  \
+    if (e != cudaSuccess) return e;                                                                   \
+    return cudaLaunchKernelEx(&cfg, kfn, w2, hidden, logits, rows, H, B, stage_rows, n_stages, status); \
+  } while (0)
+  if (B == 1) NP_L2_LAUNCH(1);
+  if (B <= 4) NP_L2_LAUNCH(4);
+  NP_L2_LAUNCH(16);
+#undef NP_L2_LAUNCH
 }
 
 cudaError_t launch_pred_l2(const Dims& d, const void* w2v, const float* hidden, int B, float* logits,
-                           cudaStream_t s, int sm_count) {
+                           int32_t* status, cudaStream_t s, int sm_count) {
   const uint4* w2 = static_cast<const uint4*>(w2v);
   const long long rows = (long long)d.L * d.M;
   const int chunks = d.H >> 3;
-  const int blocks = sm_count * 4;
-#define NP_L2(LPR, CPL) return l2_dispatch_nb<LPR, CPL>(w2, hidden, logits, rows, d.H, B, blocks, s)
+  const int blocks = sm_count;
+#define NP_L2(LPR, CPL) return l2_dispatch_nb<LPR, CPL>(w2, hidden, logits, rows, d.H, B, blocks, status, s)
   if (chunks <= 1) NP_L2(1, 1);
   if (chunks <= 2) NP_L2(2, 1);
   if (chunks <= 4) NP_L2(4, 1);

@@ -200,6 +200,37 @@ def test_whole_step_trajectory(policy, mode, cfg, B):
         p.close()
 
 
+@pytest.mark.parametrize("flags,chain_layers", [
+    (nb.NP_F_CHECK_BOUNDS, 1), (nb.NP_F_CHECK_BOUNDS, 2), (nb.NP_F_CHECK_BOUNDS, 0), (0, 0),
+    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0),
+    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES | nb.NP_F_DIRECT_LOADS, 0),
+])
+@pytest.mark.parametrize("cfg", [TINY, SMALL])
+def test_mlp_kernel_variants_agree_with_oracle(cfg, flags, chain_layers):
+    """The resident multi-layer kernel (any run length), the staged per-layer kernel and the
+    direct-load kernel all reproduce the oracle's residual chain."""
+    p = Pair(cfg, flags=flags, chain_layers=chain_layers)
+    try:
+        xs = synth.hidden_states(cfg, 5)
+        L, M = cfg.n_layers, cfg.d_ffn
+        out = torch.empty((1, cfg.d_model), dtype=torch.float32, device="cuda")
+        logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")
+        for t in range(5):
+            nb.np_predict(p.eng.ctx, xs[t].cuda(), 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, xs[t].cuda(), 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            res = p.ora.step(u16(xs[t]), logits_f32=logits.cpu().numpy())
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+            # the chain alone, on the state the step left behind, gives the same vector
+            out2 = torch.empty_like(out)
+            nb.np_mlp_chain(p.eng.ctx, xs[t].cuda(), 1, out2, p.eng.stream)
+            p.eng.stream.synchronize()
+            assert rel_l2(out2.cpu().numpy(), res["x_final"]) < 1e-5, t
+    finally:
+        p.close()
+
+
 def test_call_order_and_argument_errors():
     p = Pair(TINY, with_oracle=False)
     try:
