@@ -276,6 +276,7 @@ def cuda_arm(args):
     # ---- device-resident timing ("value") ----------------------------------------------
     run_resident(0, 1 + W)                              # cold start + warm-up
     barrier()
+    eng.counters()                                      # raises if a kernel reported a fault or a timed-out wait
     sampler = ClockSampler(local)
     sampler.start()
     launches0 = nb.np_launch_count(eng.ctx)
@@ -286,6 +287,7 @@ def cuda_arm(args):
     barrier()
     launches = nb.np_launch_count(eng.ctx) - launches0
     ms_total = e0.elapsed_time(e1)
+    eng.counters()
 
     # ---- end-to-end timing: hidden state from pinned host, result back to the host --------
     nb.np_reset(eng.ctx, s)

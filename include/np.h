@@ -105,7 +105,9 @@ typedef struct np_config {
   int32_t host_threads;   /* worker threads for NP_XFER_HOST_GATHER (0 = pick) */
   int32_t chain_layers;   /* layers per resident MLP kernel in np_step / np_mlp_chain
                              (0 = a quarter of the stack) */
-  int32_t reserved[3];    /* must be 0 */
+  int32_t ring_stages;    /* cap on the records the MLP kernels stage in shared memory
+                             (0 = as many as fit; >= 2 otherwise) */
+  int32_t reserved[2];    /* must be 0 */
 } np_config;
 
 /* Byte counts of the caller-owned buffers for a configuration. */

@@ -41,7 +41,7 @@ EXPORTED = [
 class np_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
-        "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers")] + [("reserved", C.c_int32 * 3)]
+        "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers", "ring_stages")] + [("reserved", C.c_int32 * 2)]
 
 
 class np_sizes(C.Structure):
@@ -231,12 +231,13 @@ def np_launch_count(ctx) -> int:
 
 # ---- buffer owner ----------------------------------------------------------------------
 def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
-                transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0) -> np_config:
+                transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0, ring_stages=0) -> np_config:
     cfg = np_config()
     cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
     cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
     cfg.evict_policy, cfg.transfer_mode, cfg.flags, cfg.host_threads = evict_policy, transfer_mode, flags, host_threads
     cfg.chain_layers = chain_layers
+    cfg.ring_stages = ring_stages
     cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
     return cfg
 

@@ -176,7 +176,8 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
-  for (int i = 0; i < 3; ++i)
+  if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
+  for (int i = 0; i < 2; ++i)
     if (c->reserved[i]) return fail(ctx, NP_E_INVAL, "reserved fields must be 0");
   return NP_OK;
 }
@@ -196,7 +197,7 @@ WsLayout ws_layout(const np_config& c) {
   w.xbuf = off;
   off += 2 * vec;
   w.zbuf = off;
-  off += 3 * vec;
+  off += 3 * kZRep * vec;
   w.total = off;
   return w;
 }
@@ -291,6 +292,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   d.C = cfg->capacity;
   d.W = cfg->d_ffn / 32;
   d.Bmax = cfg->max_batch;
+  d.ring_stages = cfg->ring_stages;
   d.rec_bytes = 3ull * d.D * 2;
 
 #define NP_INIT_CUDA(call)                                                                   \
@@ -362,7 +364,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   ctx->ws.hidden = reinterpret_cast<float*>(wsb + wl.hidden);
   ctx->ws.logits = reinterpret_cast<float*>(wsb + wl.logits);
   for (int i = 0; i < 2; ++i) ctx->ws.xbuf[i] = reinterpret_cast<float*>(wsb + wl.xbuf + i * vec);
-  for (int i = 0; i < 3; ++i) ctx->ws.zbuf[i] = reinterpret_cast<float*>(wsb + wl.zbuf + i * vec);
+  for (int i = 0; i < 3; ++i) ctx->ws.zbuf[i] = reinterpret_cast<float*>(wsb + wl.zbuf + i * kZRep * vec);
 
   NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_delta, cudaEventDisableTiming));
   ctx->ev_installed.assign(d.L, nullptr);
@@ -596,9 +598,10 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   const Dims& d = ctx->d;
   const size_t n = (size_t)B * d.D;
   NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
-  NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, n * 4, s));
   const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
                           mlp_chain_supported(d, ctx->sm_count);
+  // the accumulator of layer 0 starts at zero (later ones are cleared one layer ahead)
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, (persistent ? (size_t)kZRep * d.D : n) * 4, s));
   if (persistent) {
     // runs of layers in one resident kernel each; a run starts once its layers are installed,
     // so the install of later runs still overlaps the compute of earlier ones
@@ -629,7 +632,8 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       if (rc < 0) return rc;
     }
   }
-  NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], x_out, n, s));
+  NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], persistent ? kZRep : 1, x_out,
+                                n, s));
   return NP_OK;
 }
 

@@ -12,7 +12,8 @@
 namespace npi {
 
 constexpr int kMaxBatch = 16;
-constexpr int kHostHeaderInts = 16;  // global header of the host list mirror
+constexpr int kHostHeaderInts = 16;
+constexpr int kZRep = 4;  // copies of each MLP accumulator vector (spreads same-address adds)  // global header of the host list mirror
 
 // Device-resident tables and lists of all layers (one slab, library-owned).
 struct Tables {
@@ -40,11 +41,12 @@ struct Workspace {
   float* hidden;   // [Bmax][H]
   float* logits;   // [Bmax][L][M]
   float* xbuf[2];  // [Bmax][D] each: x_l of the residual chain, ping-pong
-  float* zbuf[3];  // [Bmax][D] each: MLP_l(x_l) accumulators, rotating
+  float* zbuf[3];  // [kZRep][Bmax][D] each: MLP_l(x_l) accumulators, rotating
 };
 
 struct Dims {
   int L, D, M, H, k, C, W, Bmax;
+  int ring_stages;  // cap on shared-memory ring stages of the MLP kernels (0 = as many as fit)
   size_t rec_bytes;
 };
 
@@ -89,6 +91,8 @@ cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, i
 // Persistent multi-layer form of the sparse MLP for one sequence (np_mlp_chain.cu).
 struct ChainPlan {
   int n_stages, tile_rows, xj, cols;
+  int run_layers;       // layers one launch can span (bounded by the slot cache)
+  int slot_cache_rows;
   size_t smem;
 };
 struct ChainArgs {
@@ -108,6 +112,7 @@ bool mlp_chain_supported(const Dims& d, int sm_count);
 cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
 
 cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s);
-cudaError_t launch_add_vec(const float* a, const float* b, float* out, size_t n, cudaStream_t s);
+// out = a + sum of `reps` consecutive copies of b (each n floats)
+cudaError_t launch_add_vec(const float* a, const float* b, int reps, float* out, size_t n, cudaStream_t s);
 
 }  // namespace npi

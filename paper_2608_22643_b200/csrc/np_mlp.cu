@@ -433,6 +433,7 @@ static bool mlp_pipe_plan(const Dims& d, int sm_count, MlpPipeArgs* pa, size_t* 
   const size_t budget = 200 * 1024;
   int n_stages = (int)std::min<size_t>(kPipeMaxStages, budget / rec);
   if (n_stages < 2) return false;
+  if (d.ring_stages >= 2) n_stages = std::min(n_stages, d.ring_stages);
   const long long expect = std::min<long long>(d.C, d.k);
   const int per_block = (int)std::max<long long>(1, (expect + sm_count - 1) / sm_count);
   // tile rows: a power of two, about half the block's share (or half the ring), so that the

@@ -18,6 +18,7 @@
 // Every wait (mbarrier, grid barrier) is bounded; on expiry the block records
 // kStatTimeout and leaves, and the other blocks follow at their next barrier.
 #include <algorithm>
+#include <cstdlib>
 
 #include "np_device.cuh"
 #include "np_internal.h"
@@ -26,8 +27,9 @@
 namespace npi {
 using namespace npd;
 
-constexpr int kChainThreads = 512;
-constexpr int kChainWarps = kChainThreads / 32;
+constexpr int kChainWarps = 16;                      // consumer warps
+constexpr int kChainThreads = kChainWarps * 32;      // consumer threads
+constexpr int kChainBlock = kChainThreads + 32;      // plus one producer warp
 constexpr int kChainMaxStages = 16;
 constexpr int kChainMaxLayers = 128;  // layers per launch (longer runs are split by the host)
 
@@ -38,22 +40,55 @@ struct ChainKernelArgs {
   const int32_t* slots;        // active_slots [L][C]
   const int32_t* counters;     // [L][NP_N_COUNTERS]
   float* xbuf[2];              // x_l is stored to xbuf[l & 1]
-  float* zbuf[3];              // MLP_l(x_l) accumulates into zbuf[l % 3]
+  float* zbuf[3];              // MLP_l(x_l) accumulates into zbuf[l % 3]: kZRep copies of [D], block g adds
+                               // into copy g % kZRep (fewer adds per address), readers sum the copies
   unsigned int* grid_bar;      // zeroed by the host before the launch
   int32_t* status;
   int l_begin, l_end, D, C, n_stages, tile_rows, check;
+  int slot_cache_rows;         // capacity of the per-block slot cache (rows)
 };
+
+#ifdef NP_TRACE
+__device__ unsigned long long np_trace_buf[4][128][16];
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define NP_TR(slot)                                                                   \
+  do {                                                                                \
+    if (threadIdx.x == 0 && (blockIdx.x & 31) == 0 && (blockIdx.x >> 5) < 4 && li < 128) \
+      np_trace_buf[blockIdx.x >> 5][li][slot] = gtime();                              \
+  } while (0)
+extern "C" int np_debug_trace(void* out) {
+  return (int)cudaMemcpyFromSymbol(out, np_trace_buf, sizeof(np_trace_buf));
+}
+#else
+#define NP_TR(slot) do { } while (0)
+#endif
 
 __device__ __forceinline__ float4 ldcg4(const float* p) {
   return __ldcg(reinterpret_cast<const float4*>(p));
 }
 
+// barrier among the consumer warps only (the producer warp never joins it)
+__device__ __forceinline__ void consumer_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kChainWarps * 32) : "memory");
+}
+
+// 16-byte floating-point reduction to global memory, no return value
+__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
+
 template <int XJ, int COLS>
-__global__ void __launch_bounds__(kChainThreads, 1) k_mlp_chain(ChainKernelArgs a) {
+__global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a) {
   extern __shared__ __align__(128) unsigned char csm[];
-  __shared__ __align__(8) uint64_t full_bar[kChainMaxStages];
-  __shared__ float part[kChainWarps][2];
-  __shared__ float act[kChainWarps];
+  __shared__ __align__(8) uint64_t full_bar[kChainMaxStages];   // a stage's record has landed
+  __shared__ __align__(8) uint64_t empty_bar[kChainMaxStages];  // every consumer warp is done with it
+  __shared__ float part[kChainWarps][2];        // (g, u) partial sums of the tile's (row, segment) items
+  __shared__ float act[kChainWarps];            // a_i of the tile's rows
   __shared__ int s_ok;
   __shared__ int lay_rb[kChainMaxLayers];       // first active-list index of this block, per layer
   __shared__ int lay_pre[kChainMaxLayers + 1];  // rows of this block before each layer (virtual row index)
@@ -66,6 +101,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_mlp_chain(ChainKernelArgs 
   const int seg_chunks = (chunks + SEG - 1) / SEG;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int G = gridDim.x, nl = a.l_end - a.l_begin;
+  float* xs = reinterpret_cast<float*>(csm + (size_t)n_stages * rec_bytes);  // x_l, fp32 [D], kept across layers
+  int* slot_cache = reinterpret_cast<int*>(xs + D);                         // this block's slots, virtual row order
 
   // ---- this block's share of every layer of the run ----
   if (tid < nl) {
@@ -80,7 +117,10 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_mlp_chain(ChainKernelArgs 
     lay_pre[tid + 1] = re - rb;  // turned into a prefix sum below
   }
   if (tid == 0) {
-    for (int s = 0; s < n_stages; ++s) npp::mbar_init(&full_bar[s], 1);
+    for (int s = 0; s < n_stages; ++s) {
+      npp::mbar_init(&full_bar[s], 1);
+      npp::mbar_init(&empty_bar[s], kChainWarps);
+    }
     npp::fence_barrier_init();
     s_ok = 1;
   }
@@ -90,46 +130,64 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_mlp_chain(ChainKernelArgs 
     for (int i = 0; i < nl; ++i) lay_pre[i + 1] += lay_pre[i];
   }
   __syncthreads();
-  const int total_rows = lay_pre[nl];
-
-  // ---- producer state (used by warp 0 only; identical in all its lanes) ----
-  int issued = 0;    // virtual rows requested so far
-  int consumed = 0;  // virtual rows whose stage has been read completely
-  int issue_layer = 0;
-  auto issue_more = [&]() {  // warp 0, all lanes
-    const int limit = min(total_rows, consumed + n_stages);
-    while (issued < limit) {
-      const int v = issued + lane;
-      if (v < limit) {
-        int ll = issue_layer;
-        while (v >= lay_pre[ll + 1]) ++ll;
-        const int i = v - lay_pre[ll];
-        int slot = a.slots[(size_t)(a.l_begin + ll) * a.C + lay_rb[ll] + i];
+  const int total_rows = min(lay_pre[nl], a.slot_cache_rows);
+  // slots of all this block's rows, so that no request waits on a global load later
+  for (int li = 0; li < nl; ++li) {
+    const int nr = lay_pre[li + 1] - lay_pre[li];
+    for (int i = tid; i < nr; i += blockDim.x) {
+      const int v = lay_pre[li] + i;
+      if (v < total_rows) {
+        int slot = a.slots[(size_t)(a.l_begin + li) * a.C + lay_rb[li] + i];
         if (a.check && (slot < 0 || slot >= a.C)) {
           atomicOr(a.status, kStatBadSlot);
           slot = 0;
         }
-        const int s = v % n_stages;
+        slot_cache[v] = slot;
+      }
+    }
+  }
+  __syncthreads();
+
+  if (wid == kChainWarps) {
+    // =========================== producer warp ===========================
+    // One lane requests the block's virtual rows strictly in order: rows are consumed in
+    // order, so stage v % n_stages is always the next one to be released.  (Lanes that wait
+    // on different barriers must not be used here: the compiler may reconverge the warp
+    // after the wait, and a lane whose stage is free would then be held back by a lane whose
+    // stage is released only after the first lane's row has been consumed.)
+    if (lane == 0) {
+      int ll = 0, s = 0;
+      uint32_t use = 0;
+      for (int v = 0; v < total_rows; ++v) {
+        if (!npp::mbar_wait(&empty_bar[s], (use & 1u) ^ 1u)) {
+          atomicOr(a.status, npp::kStatTimeout);
+          break;
+        }
+        while (v >= lay_pre[ll + 1]) ++ll;
+        const size_t off = (size_t)(a.l_begin + ll) * layer_bytes + (size_t)slot_cache[v] * row_bytes;
         unsigned char* dst = csm + (size_t)s * rec_bytes;
-        const size_t off = (size_t)(a.l_begin + ll) * layer_bytes + (size_t)slot * row_bytes;
         npp::mbar_expect_tx(&full_bar[s], rec_bytes);
         npp::bulk_g2s(dst, a.gate + off, row_bytes, &full_bar[s]);
         npp::bulk_g2s(dst + row_bytes, a.up + off, row_bytes, &full_bar[s]);
         npp::bulk_g2s(dst + 2 * row_bytes, a.downT + off, row_bytes, &full_bar[s]);
+        if (++s == n_stages) {
+          s = 0;
+          ++use;
+        }
       }
-      issued = min(limit, issued + 32);
     }
-    while (issue_layer < nl && issued >= lay_pre[issue_layer + 1]) ++issue_layer;
-    if (issue_layer >= nl) issue_layer = nl - 1;
-  };
-  if (wid == 0) issue_more();
+    return;
+  }
 
+  // =========================== consumer warps ===========================
   const int sg = wid % SEG, row_in_tile = wid / SEG;
   const int c_lo = sg * seg_chunks, c_hi = min(chunks, c_lo + seg_chunks);
+  const int l_last = a.l_end - 1;
 
   for (int li = 0; li < nl; ++li) {
     const int l = a.l_begin + li;
-    // ---- wait until every block has added its part of layer l-1 (x_l is final) ----
+    NP_TR(0);
+    // ---- wait until every block has added its part of layer l-1 ----
     if (li > 0) {
       if (tid == 0) {
         const unsigned int target = (unsigned int)li * (unsigned int)G;
@@ -147,34 +205,65 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_mlp_chain(ChainKernelArgs 
           s_ok = 0;
         }
       }
-      __syncthreads();
+      consumer_sync();
       if (!s_ok) break;
     }
-
-    // ---- x_l = xbuf[(l+1)&1] + zbuf[(l-1)%3]: this warp's slice, in registers ----
-    const float* xa = a.xbuf[(l + 1) & 1];
-    const float* xb = l > 0 ? a.zbuf[(l - 1) % 3] : nullptr;
+    NP_TR(1);
+    // ---- x_l: first layer of the run from global, afterwards x_l = x_{l-1} + MLP_{l-1} ----
+    {
+      const float* xa = a.xbuf[(l + 1) & 1];
+      const float* zb = l > 0 ? a.zbuf[(l - 1) % 3] : nullptr;
+      float* xst = a.xbuf[l & 1];
+      const int nf4 = chunks * 2;  // float4 granules of one vector
+      for (int c0 = tid; c0 < nf4; c0 += 2 * kChainThreads) {
+        // all loads of two granules (and of every accumulator copy) are issued before any is used
+        const int c1 = c0 + kChainThreads;
+        const bool has1 = c1 < nf4;
+        float4 w0[kZRep], w1[kZRep];
+        if (zb) {
+#pragma unroll
+          for (int r = 0; r < kZRep; ++r) {
+            w0[r] = ldcg4(zb + (size_t)r * D + (size_t)c0 * 4);
+            w1[r] = has1 ? ldcg4(zb + (size_t)r * D + (size_t)c1 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+        float4 v0, v1 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (li == 0) {
+          v0 = ldcg4(xa + (size_t)c0 * 4);
+          if (has1) v1 = ldcg4(xa + (size_t)c1 * 4);
+        } else {
+          v0 = reinterpret_cast<float4*>(xs)[c0];
+          if (has1) v1 = reinterpret_cast<float4*>(xs)[c1];
+        }
+        if (zb) {
+#pragma unroll
+          for (int r = 0; r < kZRep; ++r) {
+            v0.x += w0[r].x; v0.y += w0[r].y; v0.z += w0[r].z; v0.w += w0[r].w;
+            v1.x += w1[r].x; v1.y += w1[r].y; v1.z += w1[r].z; v1.w += w1[r].w;
+          }
+        }
+        reinterpret_cast<float4*>(xs)[c0] = v0;
+        if (has1) reinterpret_cast<float4*>(xs)[c1] = v1;
+        if (blockIdx.x == 0 && l == l_last) {  // x for the next launch
+          reinterpret_cast<float4*>(xst)[c0] = v0;
+          if (has1) reinterpret_cast<float4*>(xst)[c1] = v1;
+        }
+      }
+      // clear the next layer's accumulator copies: every block takes a slice
+      float4* znext = reinterpret_cast<float4*>(a.zbuf[(l + 1) % 3]);
+      const int ztotal = nf4 * kZRep;
+      const int zlo = (int)(((long long)ztotal * blockIdx.x) / G), zhi = (int)(((long long)ztotal * (blockIdx.x + 1)) / G);
+      for (int c = zlo + tid; c < zhi; c += kChainThreads) znext[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    consumer_sync();
     float xr[XJ][8];
 #pragma unroll
     for (int j = 0; j < XJ; ++j) {
       const int c = c_lo + lane + 32 * j;
       if (c < c_hi) {
-        float4 v0 = ldcg4(xa + (size_t)c * 8), v1 = ldcg4(xa + (size_t)c * 8 + 4);
-        if (xb) {
-          const float4 w0 = ldcg4(xb + (size_t)c * 8), w1 = ldcg4(xb + (size_t)c * 8 + 4);
-          v0.x += w0.x; v0.y += w0.y; v0.z += w0.z; v0.w += w0.w;
-          v1.x += w1.x; v1.y += w1.y; v1.z += w1.z; v1.w += w1.w;
-        }
+        const float4 v0 = reinterpret_cast<const float4*>(xs)[2 * c], v1 = reinterpret_cast<const float4*>(xs)[2 * c + 1];
         xr[j][0] = v0.x; xr[j][1] = v0.y; xr[j][2] = v0.z; xr[j][3] = v0.w;
         xr[j][4] = v1.x; xr[j][5] = v1.y; xr[j][6] = v1.z; xr[j][7] = v1.w;
-        if (blockIdx.x == 0 && row_in_tile == 0) {  // one warp per segment: store x_l, clear the next accumulator
-          float4* ps = reinterpret_cast<float4*>(a.xbuf[l & 1] + (size_t)c * 8);
-          ps[0] = v0;
-          ps[1] = v1;
-          float4* pz = reinterpret_cast<float4*>(a.zbuf[(l + 1) % 3] + (size_t)c * 8);
-          pz[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-          pz[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
       } else {
 #pragma unroll
         for (int e = 0; e < 8; ++e) xr[j][e] = 0.f;
@@ -187,22 +276,30 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_mlp_chain(ChainKernelArgs 
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
 
-    const int vbase = lay_pre[li], nrows = lay_pre[li + 1] - vbase;
+    const int vbase = lay_pre[li], nrows = min(lay_pre[li + 1], total_rows) - vbase;
+    NP_TR(2);
     for (int t0 = 0; t0 < nrows; t0 += TR) {
       const int rows = min(TR, nrows - t0);
+      const int s0 = (vbase + t0) % n_stages;  // stage of the tile's first row; the rest follow, wrapping
+      const uint32_t use0 = (uint32_t)((vbase + t0) / n_stages);
       // ---- phase 1: (row, segment) partial dot products from shared memory ----
       if (row_in_tile < rows) {
-        const int v = vbase + t0 + row_in_tile;
-        const int s = v % n_stages;
-        if (!npp::mbar_wait(&full_bar[s], (uint32_t)(v / n_stages) & 1u)) {
+        int s = s0 + row_in_tile;
+        uint32_t use = use0;
+        if (s >= n_stages) {
+          s -= n_stages;
+          ++use;
+        }
+        if (!npp::mbar_wait(&full_bar[s], use & 1u)) {
           if (lane == 0) {
             atomicOr(a.status, npp::kStatTimeout);
             s_ok = 0;
           }
         }
+        if (t0 == 0) NP_TR(7);
         const uint4* gp = reinterpret_cast<const uint4*>(csm + (size_t)s * rec_bytes);
         const uint4* up = gp + chunks;
-        float g = 0.f, u = 0.f;
+        float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;  // two chains each: the FMAs of a dot product are dependent
 #pragma unroll
         for (int j = 0; j < XJ; ++j) {
           const int c = c_lo + lane + 32 * j;
@@ -210,69 +307,94 @@ __global__ void __launch_bounds__(kChainThreads, 1) k_mlp_chain(ChainKernelArgs 
             const uint4 gw = gp[c], uw = up[c];
             const float4 x0 = make_float4(xr[j][0], xr[j][1], xr[j][2], xr[j][3]);
             const float4 x1 = make_float4(xr[j][4], xr[j][5], xr[j][6], xr[j][7]);
-            g = dot8(gw, x0, x1, g);
-            u = dot8(uw, x0, x1, u);
+            if (j & 1) {
+              g1 = dot8(gw, x0, x1, g1);
+              u1 = dot8(uw, x0, x1, u1);
+            } else {
+              g0 = dot8(gw, x0, x1, g0);
+              u0 = dot8(uw, x0, x1, u0);
+            }
           }
         }
-        g = warp_sum(g);
-        u = warp_sum(u);
+        float g = g0 + g1, u = u0 + u1;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          g += __shfl_xor_sync(0xffffffffu, g, o);
+          u += __shfl_xor_sync(0xffffffffu, u, o);
+        }
         if (lane == 0) {
           part[wid][0] = g;
           part[wid][1] = u;
         }
+        if (t0 == 0) NP_TR(8);
       }
-      __syncthreads();
+      consumer_sync();
+      if (t0 == 0) NP_TR(3);
       if (!s_ok) break;
       if (tid < rows) {
         float gs = 0.f, us = 0.f;
-        for (int q = 0; q < SEG; ++q) {
-          gs += part[tid * SEG + q][0];
-          us += part[tid * SEG + q][1];
+        for (int w = 0; w < SEG; ++w) {
+          gs += part[tid * SEG + w][0];
+          us += part[tid * SEG + w][1];
         }
         act[tid] = gs / (1.f + __expf(-gs)) * us;
       }
-      __syncthreads();
+      consumer_sync();
       // ---- phase 2: y[cols] += a_i * downT[s_i][cols] ----
+      {
+        int s = s0;
+        for (int q = 0; q < rows; ++q) {
+          const float av = act[q];
+          const uint4* dp = reinterpret_cast<const uint4*>(csm + (size_t)s * rec_bytes + 2 * row_bytes);
 #pragma unroll
-      for (int j = 0; j < COLS; ++j) {
-        const int c = tid + j * kChainThreads;
-        if (c < chunks) {
+          for (int j = 0; j < COLS; ++j) {
+            const int c = tid + j * kChainThreads;
+            if (c < chunks) {
+              const uint4 w = dp[c];
+              acc[j][0] = fmaf(av, bf16_lo(w.x), acc[j][0]);
+              acc[j][1] = fmaf(av, bf16_hi(w.x), acc[j][1]);
+              acc[j][2] = fmaf(av, bf16_lo(w.y), acc[j][2]);
+              acc[j][3] = fmaf(av, bf16_hi(w.y), acc[j][3]);
+              acc[j][4] = fmaf(av, bf16_lo(w.z), acc[j][4]);
+              acc[j][5] = fmaf(av, bf16_hi(w.z), acc[j][5]);
+              acc[j][6] = fmaf(av, bf16_lo(w.w), acc[j][6]);
+              acc[j][7] = fmaf(av, bf16_hi(w.w), acc[j][7]);
+            }
+          }
+          if (++s == n_stages) s = 0;
+        }
+        // this warp is done with the tile's stages.  (`part` is rewritten only after every warp
+        // has passed the barrier above, `act` only after the next tile's first barrier.)
+        __syncwarp();
+        if (lane == 0) {
+          s = s0;
           for (int q = 0; q < rows; ++q) {
-            const int s = (vbase + t0 + q) % n_stages;
-            const uint4 w = reinterpret_cast<const uint4*>(csm + (size_t)s * rec_bytes + 2 * row_bytes)[c];
-            const float av = act[q];
-            acc[j][0] = fmaf(av, bf16_lo(w.x), acc[j][0]);
-            acc[j][1] = fmaf(av, bf16_hi(w.x), acc[j][1]);
-            acc[j][2] = fmaf(av, bf16_lo(w.y), acc[j][2]);
-            acc[j][3] = fmaf(av, bf16_hi(w.y), acc[j][3]);
-            acc[j][4] = fmaf(av, bf16_lo(w.z), acc[j][4]);
-            acc[j][5] = fmaf(av, bf16_hi(w.z), acc[j][5]);
-            acc[j][6] = fmaf(av, bf16_lo(w.w), acc[j][6]);
-            acc[j][7] = fmaf(av, bf16_hi(w.w), acc[j][7]);
+            npp::mbar_arrive(&empty_bar[s]);
+            if (++s == n_stages) s = 0;
           }
         }
       }
-      __syncthreads();  // the tile's stages have been read: request the rows that come next,
-      consumed += rows; // possibly those of the following layers
-      if (wid == 0) issue_more();
+      if (t0 == 0) NP_TR(10);
     }
     if (!s_ok) break;
+    NP_TR(4);
 
     // ---- add this block's partial MLP_l(x_l) to the layer's accumulator ----
     if (nrows > 0) {
-      float* yacc = a.zbuf[l % 3];
+      float* yacc = a.zbuf[l % 3] + (size_t)(blockIdx.x % kZRep) * D;
 #pragma unroll
       for (int j = 0; j < COLS; ++j) {
         const int c = tid + j * kChainThreads;
         if (c < chunks) {
-          float4* yp = reinterpret_cast<float4*>(yacc + (size_t)c * 8);
-          atomicAdd(yp, make_float4(acc[j][0], acc[j][1], acc[j][2], acc[j][3]));
-          atomicAdd(yp + 1, make_float4(acc[j][4], acc[j][5], acc[j][6], acc[j][7]));
+          red_add_v4(yacc + (size_t)c * 8, acc[j][0], acc[j][1], acc[j][2], acc[j][3]);
+          red_add_v4(yacc + (size_t)c * 8 + 4, acc[j][4], acc[j][5], acc[j][6], acc[j][7]);
         }
       }
     }
+    NP_TR(5);
     if (li + 1 < nl) {  // publish: every thread's adds and stores precede the arrival
-      __syncthreads();
+      consumer_sync();
+      NP_TR(6);
       if (tid == 0) {
         __threadfence();
         atomicAdd(a.grid_bar, 1u);
@@ -287,12 +409,12 @@ static cudaError_t chain_launch(const ChainKernelArgs& ka, size_t sm, int grid_x
   cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
   if (e != cudaSuccess) return e;
   int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kfn, kChainThreads, sm);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kfn, kChainBlock, sm);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid_x);
-  cfg.blockDim = dim3(kChainThreads);
+  cfg.blockDim = dim3(kChainBlock);
   cfg.dynamicSmemBytes = sm;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
@@ -311,11 +433,17 @@ bool mlp_chain_supported(const Dims& d, int sm_count) {
 bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
   const int chunks = d.D >> 3;
   const size_t rec = (size_t)d.D * 6;
-  const size_t budget = 200 * 1024;
-  int n_stages = (int)std::min<size_t>(kChainMaxStages, budget / rec);
-  if (n_stages < 2) return false;
+  // shared memory: ring + x (fp32 [D]) + slot cache, under the 227 KB per-block limit
   const long long expect = std::min<long long>(d.C, d.k);
   const int per_block = (int)std::max<long long>(1, (expect + sm_count - 1) / sm_count);
+  const int max_per_block = d.C / sm_count + 2;   // whatever the active count turns out to be
+  p->run_layers = std::max(1, std::min(kChainMaxLayers, 16384 / (4 * max_per_block)));
+  p->slot_cache_rows = p->run_layers * max_per_block;
+  const size_t fixed = (size_t)d.D * 4 + (size_t)p->slot_cache_rows * 4;
+  const size_t budget = 227 * 1024 - 4096;  // static shared memory and the driver's reserve
+  if (fixed + 2 * rec > budget) return false;
+  int n_stages = (int)std::min<size_t>(kChainMaxStages, (budget - fixed) / rec);
+  if (d.ring_stages >= 2) n_stages = std::min(n_stages, d.ring_stages);
   int tr = 1;
   const int tr_cap = std::max(1, std::min(per_block, n_stages) / 2);
   while (tr * 2 <= tr_cap && tr * 2 <= kChainWarps) tr *= 2;
@@ -329,7 +457,15 @@ bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
   p->cols = need_cols <= 1 ? 1 : (need_cols <= 2 ? 2 : 4);
   p->n_stages = n_stages;
   p->tile_rows = tr;
-  p->smem = (size_t)n_stages * rec;
+#ifdef NP_TRACE
+  if (const char* e = getenv("NP_TILE_ROWS")) {
+    tr = atoi(e);
+    const int seg2 = kChainWarps / tr;
+    p->xj = ((chunks + seg2 - 1) / seg2 + 31) / 32;
+    p->tile_rows = tr;
+  }
+#endif
+  p->smem = (size_t)n_stages * rec + fixed;
   return true;
 }
 
@@ -337,7 +473,7 @@ cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, 
   ChainPlan p;
   if (!mlp_chain_plan(d, sm_count, &p)) return cudaErrorInvalidValue;
   cudaError_t e = cudaSuccess;
-  for (int l0 = a.l_begin; l0 < a.l_end; l0 += kChainMaxLayers) {
+  for (int l0 = a.l_begin; l0 < a.l_end; l0 += p.run_layers) {
     ChainKernelArgs ka;
     ka.gate = static_cast<const unsigned char*>(a.gate);
     ka.up = static_cast<const unsigned char*>(a.up);
@@ -349,7 +485,8 @@ cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, 
     ka.grid_bar = a.grid_bar;
     ka.status = a.status;
     ka.l_begin = l0;
-    ka.l_end = std::min(a.l_end, l0 + kChainMaxLayers);
+    ka.l_end = std::min(a.l_end, l0 + p.run_layers);
+    ka.slot_cache_rows = p.slot_cache_rows;
     ka.D = d.D;
     ka.C = d.C;
     ka.n_stages = p.n_stages;

@@ -13,7 +13,7 @@
 namespace npp {
 
 constexpr int kStatTimeout = 8;           // a bounded wait ran out
-constexpr uint32_t kSpinLimit = 1u << 22;  // polls; each poll may suspend for a short time
+constexpr uint32_t kSpinLimit = 1u << 20;  // polls; each poll may suspend for a short time
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -81,6 +81,11 @@ __device__ __forceinline__ void bulk_g2s_stream(void* dst_smem, const void* src_
           "r"(smem_addr(dst_smem)),
       "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
       : "memory");
+}
+
+// Asks the L2 to fetch [src, src + bytes) from DRAM; nothing is written anywhere else.
+__device__ __forceinline__ void prefetch_l2(const void* src_gmem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src_gmem), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ uint64_t policy_evict_first() {

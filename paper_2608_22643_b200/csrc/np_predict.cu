@@ -281,10 +281,14 @@ __global__ void k_widen_bf16(const uint16_t* __restrict__ x, float* __restrict__
   if (i < n) out[i] = __uint_as_float((uint32_t)x[i] << 16);
 }
 
-__global__ void k_add_vec(const float* __restrict__ a, const float* __restrict__ b,
+__global__ void k_add_vec(const float* __restrict__ a, const float* __restrict__ b, int reps,
                           float* __restrict__ out, size_t n) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = a[i] + b[i];
+  if (i < n) {
+    float v = a[i];
+    for (int r = 0; r < reps; ++r) v += b[(size_t)r * n + i];
+    out[i] = v;
+  }
 }
 
 cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s) {
@@ -292,8 +296,8 @@ cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStre
   return cudaGetLastError();
 }
 
-cudaError_t launch_add_vec(const float* a, const float* b, float* out, size_t n, cudaStream_t s) {
-  k_add_vec<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(a, b, out, n);
+cudaError_t launch_add_vec(const float* a, const float* b, int reps, float* out, size_t n, cudaStream_t s) {
+  k_add_vec<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(a, b, reps, out, n);
   return cudaGetLastError();
 }
 

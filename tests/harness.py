@@ -27,7 +27,7 @@ class Pair:
 
     def __init__(self, cfg: synth.StackConfig, policy=nb.NP_EVICT_EXACT, max_batch=1, k=None, C=None,
                  transfer_mode=nb.NP_XFER_MEMCPY_RUNS, staging_rows=None, flags=nb.NP_F_CHECK_BOUNDS,
-                 gen_device="cpu", with_oracle=True, chain_layers=0):
+                 gen_device="cpu", with_oracle=True, chain_layers=0, ring_stages=0):
         nbuild.build()
         self.cfg = cfg
         self.k = cfg.top_k if k is None else k
@@ -37,7 +37,7 @@ class Pair:
         self.backing = synth.backing_store(cfg, gen_device=gen_device)
         ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, self.k, self.C,
                               max_batch=max_batch, evict_policy=policy, staging_rows=staging_rows,
-                              transfer_mode=transfer_mode, flags=flags, chain_layers=chain_layers)
+                              transfer_mode=transfer_mode, flags=flags, chain_layers=chain_layers, ring_stages=ring_stages)
         self.eng = nb.Engine(ncfg, w1.cuda(), w2.cuda(), self.backing)
         self.store_u16 = self.backing.view(torch.int16).numpy().view(np.uint16)
         self.ora = None

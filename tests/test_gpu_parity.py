@@ -200,16 +200,24 @@ def test_whole_step_trajectory(policy, mode, cfg, B):
         p.close()
 
 
-@pytest.mark.parametrize("flags,chain_layers", [
-    (nb.NP_F_CHECK_BOUNDS, 1), (nb.NP_F_CHECK_BOUNDS, 2), (nb.NP_F_CHECK_BOUNDS, 0), (0, 0),
-    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0),
-    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES | nb.NP_F_DIRECT_LOADS, 0),
+# a stack whose per-block share (k = 900 rows over the SMs) exceeds a small ring several times
+# over, so that shared-memory stages are reused within a layer and across layers
+DENSE = synth.StackConfig("dense", 4, 512, 2048, 64, 44, 60, 5, 13, 0.9)
+
+
+@pytest.mark.parametrize("flags,chain_layers,ring_stages", [
+    (nb.NP_F_CHECK_BOUNDS, 1, 0), (nb.NP_F_CHECK_BOUNDS, 2, 0), (nb.NP_F_CHECK_BOUNDS, 0, 0), (0, 0, 0),
+    (nb.NP_F_CHECK_BOUNDS, 0, 2), (nb.NP_F_CHECK_BOUNDS, 3, 3), (nb.NP_F_CHECK_BOUNDS, 0, 4),
+    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0, 0),
+    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0, 2),
+    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0, 5),
+    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES | nb.NP_F_DIRECT_LOADS, 0, 0),
 ])
-@pytest.mark.parametrize("cfg", [TINY, SMALL])
-def test_mlp_kernel_variants_agree_with_oracle(cfg, flags, chain_layers):
+@pytest.mark.parametrize("cfg", [TINY, SMALL, DENSE])
+def test_mlp_kernel_variants_agree_with_oracle(cfg, flags, chain_layers, ring_stages):
     """The resident multi-layer kernel (any run length), the staged per-layer kernel and the
     direct-load kernel all reproduce the oracle's residual chain."""
-    p = Pair(cfg, flags=flags, chain_layers=chain_layers)
+    p = Pair(cfg, flags=flags, chain_layers=chain_layers, ring_stages=ring_stages)
     try:
         xs = synth.hidden_states(cfg, 5)
         L, M = cfg.n_layers, cfg.d_ffn
