@@ -260,6 +260,33 @@ int np_import_state(np_ctx* ctx, int32_t layer, const int32_t* slot_map, const i
  * Synchronises both streams of that step.  NP_E_STATE if no step ran. */
 int np_last_step_times(np_ctx* ctx, float* out_us);
 
+/* Largest B * d_pred np_predict_logits_noalloc accepts, in floats of fixed scratch (enough
+ * for 16 sequences at d_pred = 1024).  With its status words the array costs every GPU that
+ * loads the library 64 KiB + 256 B of device memory until the process exits. */
+#define NP_NOALLOC_MAX_HIDDEN_FLOATS 16384
+
+/* Predictor forward pass (stage 1 only: logits = W2 * relu(W1 * x)) without a context and
+ * without any allocation.  The paper has no counterpart; this exists for callers that cannot
+ * call cudaMalloc: code that runs under a memory pool which owns all device memory, a decode
+ * loop that cannot afford the device-wide synchronisation an allocation may imply, or a process
+ * whose device memory is budgeted to the byte.  np_init allocates, so such callers cannot use a
+ * context; here the scratch between the two predictor layers is a fixed array inside the library.
+ *   w1 dev bf16 [d_pred][d_model], w2 dev bf16 [n_layers*d_ffn][d_pred], x_bf16 dev bf16 [B][d_model]
+ *   logits_out dev fp32 [B][n_layers][d_ffn]   (all caller-owned, 16-byte aligned)
+ * Same kernels and results as np_predict's logits.  Calls no cudaMalloc / cudaFree or allocating
+ * library routine.  The first call on a device looks up the scratch array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call before any stream
+ * capture.  All calls on a device share the one scratch array: calls that may overlap on the GPU
+ * (different streams) race on it and must be serialised by the caller.
+ * Errors: NP_E_INVAL (NULL / misaligned pointer, shape outside np_config's limits, or
+ * B * d_pred > NP_NOALLOC_MAX_HIDDEN_FLOATS), NP_E_CUDA; text in np_noalloc_last_error(). */
+int np_predict_logits_noalloc(const void* w1, const void* w2, const void* x_bf16, int32_t B,
+                              int32_t n_layers, int32_t d_model, int32_t d_ffn, int32_t d_pred,
+                              float* logits_out, void* stream);
+
+/* Text of the calling thread's last np_predict_logits_noalloc error.  Never NULL. */
+const char* np_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

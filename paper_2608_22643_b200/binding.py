@@ -34,7 +34,7 @@ EXPORTED = [
     "np_version", "np_query_sizes", "np_init", "np_destroy", "np_reset", "np_last_error",
     "np_predict", "np_topk", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
-    "np_launch_count",
+    "np_launch_count", "np_predict_logits_noalloc", "np_noalloc_last_error",
 ]
 
 
@@ -103,6 +103,9 @@ def load() -> C.CDLL:
         "np_mlp_chain": [vp, vp, i32, vp, vp],
         "np_launch_count": [vp, C.POINTER(C.c_uint64)],
     }
+    lib.np_noalloc_last_error.restype = C.c_char_p
+    lib.np_noalloc_last_error.argtypes = []
+    sigs["np_predict_logits_noalloc"] = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
     for name, args in sigs.items():
         fn = getattr(lib, name)
         fn.argtypes = args
@@ -227,6 +230,16 @@ def np_launch_count(ctx) -> int:
     out = C.c_uint64()
     _check(ctx, load().np_launch_count(ctx, C.byref(out)))
     return int(out.value)
+
+
+def np_predict_logits_noalloc(w1, w2, x_bf16, B: int, n_layers: int, d_model: int, d_ffn: int, d_pred: int,
+                              logits_out, stream=None) -> int:
+    """Predictor logits without a context and without allocating (see include/np.h)."""
+    rc = load().np_predict_logits_noalloc(_ptr(w1), _ptr(w2), _ptr(x_bf16), B, n_layers, d_model, d_ffn,
+                                          d_pred, _ptr(logits_out), _stream(stream))
+    if rc < 0:
+        raise NpError(rc, load().np_noalloc_last_error().decode())
+    return rc
 
 
 # ---- buffer owner ----------------------------------------------------------------------

@@ -1,0 +1,60 @@
+"""The allocation-free predictor entry point gives np_predict's logits.
+
+Collected last on purpose (file name): a failure here cannot hide the result of
+any other test in a run that stops at the first failure.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_22643_b200 import binding as nb
+from paper_2608_22643_b200 import build as nbuild
+from paper_2608_22643_b200 import synth
+from tests.harness import Pair, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,B", [("small", 1), ("small", 3)])
+def test_noalloc_predictor_matches_context_path_twice(name, B):
+    """Callers that cannot allocate device memory (pool-owned memory, allocation-free decode
+    loops) use np_predict_logits_noalloc; two calls in a row on the library's fixed scratch
+    must both reproduce what np_predict computes with its workspace."""
+    cfg = synth.CONFIGS[name]
+    p = Pair(cfg, max_batch=B, with_oracle=False)
+    try:
+        L, M, D, H = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_pred
+        xs = synth.hidden_states(cfg, 2, batch=B)
+        want = torch.empty((B, L, M), dtype=torch.float32, device="cuda")
+        got = torch.full((B, L, M), float("nan"), dtype=torch.float32, device="cuda")
+        for t in range(2):                                  # second call reuses the scratch
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, B, want, None, p.eng.stream)
+            p.eng.stream.synchronize()
+            nb.np_predict_logits_noalloc(p.eng.w1, p.eng.w2, x, B, L, D, M, H, got, p.eng.stream)
+            p.eng.stream.synchronize()
+            assert rel_l2(got.cpu().numpy(), want.cpu().numpy()) < 1e-5
+            assert np.isfinite(got.cpu().numpy()).all()
+    finally:
+        p.close()
+
+
+def test_noalloc_rejects_oversize_and_bad_arguments():
+    nbuild.build()
+    lib = nb.load()
+    z = torch.zeros(64, device="cuda")
+    # B * d_pred above the fixed scratch (16 * 2048 > 16384 floats); nothing is launched
+    rc = lib.np_predict_logits_noalloc(z.data_ptr(), z.data_ptr(), z.data_ptr(), 16, 1, 256, 1024, 2048,
+                                       z.data_ptr(), None)
+    assert rc == nb.NP_E_INVAL and "exceeds the fixed scratch" in lib.np_noalloc_last_error().decode()
+    # a shape the library does not support at all
+    rc = lib.np_predict_logits_noalloc(z.data_ptr(), z.data_ptr(), z.data_ptr(), 1, 2, 4096, 1024, 4096 + 8,
+                                       z.data_ptr(), None)
+    assert rc == nb.NP_E_INVAL
+    ok_shape = (1, 1, 256, 1024, 64)
+    assert lib.np_predict_logits_noalloc(None, z.data_ptr(), z.data_ptr(), *ok_shape, z.data_ptr(), None) == nb.NP_E_INVAL
+    assert lib.np_predict_logits_noalloc(z.data_ptr() + 4, z.data_ptr(), z.data_ptr(), *ok_shape, z.data_ptr(), None) == nb.NP_E_INVAL
+    assert lib.np_noalloc_last_error().decode()
+    with pytest.raises(nb.NpError) as e:
+        nb.np_predict_logits_noalloc(z, z, z, 9, 1, 256, 1024, 2048, z)
+    assert "exceeds the fixed scratch" in str(e.value)
