@@ -93,6 +93,7 @@ struct ChainPlan {
   int n_stages, tile_rows, xj, cols;
   int run_layers;       // layers one launch can span (bounded by the slot cache)
   int slot_cache_rows;
+  int window_rows;      // records in flight per block
   size_t smem;
 };
 struct ChainArgs {

@@ -9,16 +9,17 @@
 // separate launches spend as long on launch latency and on the dependency
 // between layers as on the rows.  Here one block per SM stays resident for the
 // whole run of layers (cooperative launch).  Each block owns a ring of
-// shared-memory stages, one 3*D*2-byte record each, filled by 1-D bulk copies;
-// the rows of layer l+1 are requested as soon as a tile of layer l has been
-// read, i.e. before layer l's partial sums are reduced and before the grid-wide
-// barrier that publishes x_{l+1}.  The HBM pipe therefore stays busy across
-// layer boundaries and the only exposed latency per layer is the barrier.
+// shared-memory stages, one 3*D*2-byte record each, filled by 1-D bulk copies
+// from a producer lane; the rows of layer l+1 are requested as soon as a tile of
+// layer l has been read, i.e. before layer l's partial sums are reduced and
+// before the grid-wide barrier that publishes x_{l+1}, so the row traffic of the
+// next layer overlaps this layer's reduction.  What stays exposed per layer is
+// the all-reduce of the 4*D-byte output across the blocks (flush of the
+// reductions, barrier, re-read of the accumulators) and the two compute phases.
 //
 // Every wait (mbarrier, grid barrier) is bounded; on expiry the block records
 // kStatTimeout and leaves, and the other blocks follow at their next barrier.
 #include <algorithm>
-#include <cstdlib>
 
 #include "np_device.cuh"
 #include "np_internal.h"
@@ -46,26 +47,8 @@ struct ChainKernelArgs {
   int32_t* status;
   int l_begin, l_end, D, C, n_stages, tile_rows, check;
   int slot_cache_rows;         // capacity of the per-block slot cache (rows)
+  int window_rows;             // records in flight per block (< n_stages)
 };
-
-#ifdef NP_TRACE
-__device__ unsigned long long np_trace_buf[4][128][16];
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-#define NP_TR(slot)                                                                   \
-  do {                                                                                \
-    if (threadIdx.x == 0 && (blockIdx.x & 31) == 0 && (blockIdx.x >> 5) < 4 && li < 128) \
-      np_trace_buf[blockIdx.x >> 5][li][slot] = gtime();                              \
-  } while (0)
-extern "C" int np_debug_trace(void* out) {
-  return (int)cudaMemcpyFromSymbol(out, np_trace_buf, sizeof(np_trace_buf));
-}
-#else
-#define NP_TR(slot) do { } while (0)
-#endif
 
 __device__ __forceinline__ float4 ldcg4(const float* p) {
   return __ldcg(reinterpret_cast<const float4*>(p));
@@ -158,7 +141,18 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
     if (lane == 0) {
       int ll = 0, s = 0;
       uint32_t use = 0;
+      const int window = a.window_rows;
       for (int v = 0; v < total_rows; ++v) {
+        // pacing: at most `window` records in flight per block.  A deeper burst moves no more
+        // bytes (HBM is shared by all blocks) but queues in front of the short loads on the
+        // layer's critical path (barrier counter, accumulator vectors).
+        if (v >= window) {
+          const int vv = v - window;
+          if (!npp::mbar_wait(&full_bar[vv % n_stages], (uint32_t)(vv / n_stages) & 1u)) {
+            atomicOr(a.status, npp::kStatTimeout);
+            break;
+          }
+        }
         if (!npp::mbar_wait(&empty_bar[s], (use & 1u) ^ 1u)) {
           atomicOr(a.status, npp::kStatTimeout);
           break;
@@ -186,7 +180,6 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
 
   for (int li = 0; li < nl; ++li) {
     const int l = a.l_begin + li;
-    NP_TR(0);
     // ---- wait until every block has added its part of layer l-1 ----
     if (li > 0) {
       if (tid == 0) {
@@ -208,7 +201,6 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       consumer_sync();
       if (!s_ok) break;
     }
-    NP_TR(1);
     // ---- x_l: first layer of the run from global, afterwards x_l = x_{l-1} + MLP_{l-1} ----
     {
       const float* xa = a.xbuf[(l + 1) & 1];
@@ -277,7 +269,6 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
 
     const int vbase = lay_pre[li], nrows = min(lay_pre[li + 1], total_rows) - vbase;
-    NP_TR(2);
     for (int t0 = 0; t0 < nrows; t0 += TR) {
       const int rows = min(TR, nrows - t0);
       const int s0 = (vbase + t0) % n_stages;  // stage of the tile's first row; the rest follow, wrapping
@@ -296,7 +287,6 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
             s_ok = 0;
           }
         }
-        if (t0 == 0) NP_TR(7);
         const uint4* gp = reinterpret_cast<const uint4*>(csm + (size_t)s * rec_bytes);
         const uint4* up = gp + chunks;
         float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;  // two chains each: the FMAs of a dot product are dependent
@@ -326,10 +316,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
           part[wid][0] = g;
           part[wid][1] = u;
         }
-        if (t0 == 0) NP_TR(8);
       }
       consumer_sync();
-      if (t0 == 0) NP_TR(3);
       if (!s_ok) break;
       if (tid < rows) {
         float gs = 0.f, us = 0.f;
@@ -374,10 +362,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
           }
         }
       }
-      if (t0 == 0) NP_TR(10);
     }
     if (!s_ok) break;
-    NP_TR(4);
 
     // ---- add this block's partial MLP_l(x_l) to the layer's accumulator ----
     if (nrows > 0) {
@@ -391,10 +377,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
         }
       }
     }
-    NP_TR(5);
     if (li + 1 < nl) {  // publish: every thread's adds and stores precede the arrival
       consumer_sync();
-      NP_TR(6);
       if (tid == 0) {
         __threadfence();
         atomicAdd(a.grid_bar, 1u);
@@ -457,14 +441,7 @@ bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
   p->cols = need_cols <= 1 ? 1 : (need_cols <= 2 ? 2 : 4);
   p->n_stages = n_stages;
   p->tile_rows = tr;
-#ifdef NP_TRACE
-  if (const char* e = getenv("NP_TILE_ROWS")) {
-    tr = atoi(e);
-    const int seg2 = kChainWarps / tr;
-    p->xj = ((chunks + seg2 - 1) / seg2 + 31) / 32;
-    p->tile_rows = tr;
-  }
-#endif
+  p->window_rows = 2;
   p->smem = (size_t)n_stages * rec + fixed;
   return true;
 }
@@ -487,6 +464,7 @@ cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, 
     ka.l_begin = l0;
     ka.l_end = std::min(a.l_end, l0 + p.run_layers);
     ka.slot_cache_rows = p.slot_cache_rows;
+    ka.window_rows = std::max(1, std::min(p.n_stages - 1, p.window_rows));
     ka.D = d.D;
     ka.C = d.C;
     ka.n_stages = p.n_stages;

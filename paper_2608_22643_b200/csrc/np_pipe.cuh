@@ -83,11 +83,6 @@ __device__ __forceinline__ void bulk_g2s_stream(void* dst_smem, const void* src_
       : "memory");
 }
 
-// Asks the L2 to fetch [src, src + bytes) from DRAM; nothing is written anywhere else.
-__device__ __forceinline__ void prefetch_l2(const void* src_gmem, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src_gmem), "r"(bytes) : "memory");
-}
-
 __device__ __forceinline__ uint64_t policy_evict_first() {
   uint64_t p;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
