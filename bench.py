@@ -211,6 +211,37 @@ def reference_arm(args):
     }))
 
 
+def init_replicas(backend: str, device=None):
+    """torch.distributed for N > 1 (None for a single process).  Ranks are independent
+    replicas: the only traffic is the barrier and the max-reduction of the timings."""
+    if int(os.environ.get("WORLD_SIZE", "1")) <= 1:
+        return None
+    import torch.distributed as dist
+    if device is not None:
+        dist.init_process_group(backend, device_id=device)
+    else:
+        dist.init_process_group(backend)
+    return dist
+
+
+def replica_config(cfg, rank: int):
+    """Every replica decodes its own sequence over its own stack."""
+    return cfg.with_(seed=cfg.seed + 1000 * rank)
+
+
+def max_over_ranks(dist, values, device):
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def finish_replicas(dist):
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def cuda_arm(args):
     from paper_2608_22643_b200 import binding as nb
     from paper_2608_22643_b200 import build as nbuild
@@ -222,11 +253,7 @@ def cuda_arm(args):
         raise SystemExit("bench.py: no CUDA device (there is no CPU fallback; use --impl reference)")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    dist = init_replicas("nccl", torch.device(dev))
     if rank == 0:
         nbuild.build()
     if dist:
@@ -236,7 +263,7 @@ def cuda_arm(args):
     cfg = synth.CONFIGS[args.config]
     if args.rho is not None:
         cfg = cfg.with_(rho=args.rho)
-    cfg = cfg.with_(seed=cfg.seed + 1000 * rank)      # every replica decodes its own sequence
+    cfg = replica_config(cfg, rank)
     K, W = args.steps, args.warmup
     if W < 3:
         raise SystemExit("bench.py: --warmup must be >= 3")
@@ -343,10 +370,7 @@ def cuda_arm(args):
     pred_us = p0.elapsed_time(p1) * 1000.0 / reps
 
     # max over ranks
-    vals = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms_total = float(vals[0]), float(vals[1])
+    ms_total, e2e_ms_total = max_over_ranks(dist, [ms_total, e2e_ms_total], dev)
 
     peak, peak_kind = measured_peaks()
     mlp_bytes = n_active * rec + 4 * n_active + 8 * D            # rows + slot list + x in, y out
@@ -390,9 +414,7 @@ def cuda_arm(args):
     eng.close()
     if rank == 0:
         print(json.dumps(result))
-    if dist:
-        dist.barrier()
-        dist.destroy_process_group()
+    finish_replicas(dist)
 
 
 def main():

@@ -220,15 +220,17 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
 int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* y, void* stream);
 
 /* One whole decode step: np_predict, np_delta, np_install of every layer on
- * `copy_stream`, and the residual MLP chain x_{l+1} = x_l + MLP_l(x_l) on
- * `stream`, x_0 = x_bf16 widened to fp32.
+ * `copy_stream`, and the pre-normalised residual MLP chain
+ *   x_{l+1} = x_l + MLP_l(n_l),  n_l = x_l / sqrt(mean(x_l^2) + 1e-6)
+ * on `stream`, x_0 = x_bf16 widened to fp32 (the RMS normalisation with unit gain stands
+ * for the per-layer norm in front of every MLP block of the paper's models).
  *   x_out  dev fp32 [B][D]  x_L
  * Host-blocking exactly as np_install.  Returns warnings like np_install. */
 int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream,
             void* copy_stream);
 
-/* Stage 4 for every layer in order, nothing else: the residual chain
- * x_{l+1} = x_l + MLP_l(x_l) over the rows that are active and resident now
+/* Stage 4 for every layer in order, nothing else: the chain of np_step,
+ * x_{l+1} = x_l + MLP_l(x_l / rms(x_l)), over the rows that are active and resident now
  * (Section 3.1: the sparse suffix runs once the delta rows are in place).
  *   x_bf16  dev bf16 [B][D]  x_0,   x_out  dev fp32 [B][D]  x_L
  * Orders `stream` after any pending install marks.  Errors as np_sparse_mlp. */

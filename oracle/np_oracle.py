@@ -18,7 +18,8 @@ degenerate k for ``topk_bitmap``; the set identities of Eq. 2-3, slot-map
 bijection invariants and a set-based brute force for ``Residency.delta``;
 byte identity for ``install``; the dense SwiGLU library form when every row is
 active, linearity over disjoint sets and a scalar loop for ``sparse_mlp``; the
-paper's buffer-size arithmetic (Section 4.3) for ``record_bytes``.
+paper's buffer-size arithmetic (Section 4.3) for ``record_bytes``; unit output
+RMS, scale invariance and a hand value for ``rms_normalize``.
 
 Parity unpinned against the paper (the paper is silent; these are this build's
 definitions, pinned only by invariants and determinism): the victim order of
@@ -290,8 +291,21 @@ def sparse_mlp_from_store(backing_u16: np.ndarray, layer: int, ids: np.ndarray, 
 
 
 # --------------------------------------------------------------------------
-# one whole decode step of the stack (residual chain x_{l+1} = x_l + MLP_l(x_l))
+# one whole decode step of the stack.  The layers form a pre-normalised residual
+# chain, x_{l+1} = x_l + MLP_l(rms_normalize(x_l)), as the MLP blocks of the
+# paper's models do (their per-layer normalisation parameters stay resident,
+# Section 3.1); the gain is 1.  Without the normalisation a chain of random
+# N(0, 0.02) SwiGLU layers of width 4096 overflows within a dozen layers.
 # --------------------------------------------------------------------------
+RMS_EPS = 1e-6
+
+
+def rms_normalize(x: np.ndarray) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) along the last axis."""
+    x = np.asarray(x, dtype=np.float64)
+    return x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + RMS_EPS)
+
+
 class Engine:
     """State carried across decode steps: residency tables and resident buffers."""
 
@@ -326,7 +340,7 @@ class Engine:
         ys = []
         xs = [x]
         for l, d in enumerate(deltas):
-            y = sparse_mlp(self.gate, self.up, self.downT, l, d.active_slots, x)
+            y = sparse_mlp(self.gate, self.up, self.downT, l, d.active_slots, rms_normalize(x))
             ys.append(y)
             x = x + y
             xs.append(x)

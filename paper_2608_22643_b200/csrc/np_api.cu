@@ -568,7 +568,7 @@ static cudaError_t wait_install(np_ctx* ctx, int layer, cudaStream_t s) {
 }
 
 static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, float* yacc, float* x_store,
-                     float* zero_out, int B, cudaStream_t s) {
+                     float* zero_out, int B, int normalize, cudaStream_t s) {
   const Dims& d = ctx->d;
   const size_t row_bytes = (size_t)d.D * 2;
   MlpArgs a;
@@ -585,6 +585,7 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   a.B = B;
   a.C = d.C;
   a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+  a.normalize = normalize;
   a.force_direct = (ctx->cfg.flags & NP_F_DIRECT_LOADS) ? 1 : 0;
   a.status = ctx->t.status;
   if (ctx->install_pending[layer]) NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0));
@@ -628,7 +629,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   } else {
     for (int l = 0; l < d.L; ++l) {
       int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
-                         ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, s);
+                         ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, 1, s);
       if (rc < 0) return rc;
     }
   }
@@ -663,7 +664,7 @@ int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* 
   if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_sparse_mlp needs a prior np_delta");
   cudaStream_t s = as_stream(stream);
   NP_CUDA(ctx, cudaMemsetAsync(y, 0, (size_t)B * d.D * 4, s));
-  return mlp_layer(ctx, layer, x, nullptr, y, nullptr, nullptr, B, s);
+  return mlp_layer(ctx, layer, x, nullptr, y, nullptr, nullptr, B, 0, s);
 }
 
 int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream, void* copy_stream) {

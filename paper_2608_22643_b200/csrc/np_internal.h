@@ -13,6 +13,7 @@ namespace npi {
 
 constexpr int kMaxBatch = 16;
 constexpr int kHostHeaderInts = 16;
+constexpr float kRmsEps = 1e-6f;  // x / sqrt(mean(x^2) + eps) in front of every MLP of the chain
 constexpr int kZRep = 4;  // copies of each MLP accumulator vector (spreads same-address adds)  // global header of the host list mirror
 
 // Device-resident tables and lists of all layers (one slab, library-owned).
@@ -83,6 +84,7 @@ struct MlpArgs {
   int B;
   int C;
   int check;
+  int normalize;     // scale x to unit RMS before the dot products (the chain's pre-MLP norm)
   int force_direct;  // use the direct-load kernel even where the staged one applies
   int32_t* status;
 };

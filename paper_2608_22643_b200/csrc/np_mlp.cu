@@ -37,7 +37,7 @@ struct MlpKernelArgs {
   float* x_store;
   float* zero_out;
   int32_t* status;
-  int B, D, C, seg, check;
+  int B, D, C, seg, check, normalize;
 };
 
 template <int NB, int kMaxCols>  // kMaxCols: column rounds per thread, D <= 8 * kMlpThreads * kMaxCols
@@ -83,6 +83,29 @@ __global__ void __launch_bounds__(kMlpThreads, 1) k_sparse_mlp(MlpKernelArgs a) 
     for (int j = 0; j < kMaxCols; ++j)
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[b][j][e] = 0.f;
+  __syncthreads();
+  // optional pre-MLP RMS normalisation: the dot products are linear in x, so only their
+  // sums are scaled
+  __shared__ float s_ssq[NB][kMlpWarps];
+  __shared__ float s_inv[NB];
+  if (a.normalize) {
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+      float ss = 0.f;
+      if (b < nb)
+        for (int i = tid; i < D; i += kMlpThreads) ss += xs[(size_t)b * D + i] * xs[(size_t)b * D + i];
+      ss = warp_sum(ss);
+      if (lane == 0) s_ssq[b][wid] = ss;
+    }
+    __syncthreads();
+    if (tid < NB) {
+      float ss = 0.f;
+      for (int w = 0; w < kMlpWarps; ++w) ss += s_ssq[tid][w];
+      s_inv[tid] = rsqrtf(ss / (float)D + kRmsEps);
+    }
+  } else if (tid < NB) {
+    s_inv[tid] = 1.f;
+  }
   __syncthreads();
 
   for (int t0 = r_begin; t0 < r_end; t0 += kTileRows) {
@@ -148,6 +171,8 @@ __global__ void __launch_bounds__(kMlpThreads, 1) k_sparse_mlp(MlpKernelArgs a) 
         gs += pp[0];
         us += pp[1];
       }
+      gs *= s_inv[b];
+      us *= s_inv[b];
       act[b * kTileRows + i] = gs / (1.f + __expf(-gs)) * us;
     }
     __syncthreads();
@@ -235,6 +260,7 @@ __global__ void __launch_bounds__(kMlpThreads, 1) k_sparse_mlp_pipe(MlpPipeArgs 
   __shared__ float part[kMlpWarps][2];
   __shared__ float act[kMlpWarps];
   __shared__ int s_ok;
+  __shared__ float ssq_part[kMlpWarps];  // sums of x^2 per segment (optional RMS normalisation)
 
   const int D = a.D, chunks = D >> 3;
   const uint32_t row_bytes = (uint32_t)D * 2u;
@@ -323,7 +349,16 @@ __global__ void __launch_bounds__(kMlpThreads, 1) k_sparse_mlp_pipe(MlpPipeArgs 
   for (int j = 0; j < COLS; ++j)
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
-  __syncthreads();  // barrier init and s_ok visible to all
+  if (row_in_tile == 0) {  // one warp per segment covers x exactly once
+    float ss = 0.f;
+#pragma unroll
+    for (int j = 0; j < XJ; ++j)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) ss += xr[j][e] * xr[j][e];
+    ss = warp_sum(ss);
+    if (lane == 0) ssq_part[sg] = ss;
+  }
+  __syncthreads();  // barrier init, s_ok and ssq_part visible to all
 
   for (int t0 = 0; t0 < nrows; t0 += TR) {
     const int rows = min(TR, nrows - t0);
@@ -365,6 +400,13 @@ __global__ void __launch_bounds__(kMlpThreads, 1) k_sparse_mlp_pipe(MlpPipeArgs 
       for (int q = 0; q < SEG; ++q) {
         gs += part[tid * SEG + q][0];
         us += part[tid * SEG + q][1];
+      }
+      if (a.normalize) {
+        float ss = 0.f;
+        for (int q = 0; q < SEG; ++q) ss += ssq_part[q];
+        const float inv_rms = rsqrtf(ss / (float)D + kRmsEps);
+        gs *= inv_rms;
+        us *= inv_rms;
       }
       act[tid] = gs / (1.f + __expf(-gs)) * us;
     }
@@ -518,6 +560,7 @@ cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, i
   ka.D = d.D;
   ka.C = a.C;
   ka.check = a.check;
+  ka.normalize = a.normalize;
   // warps per row in phase 1: spread the block's expected share of rows over its warps,
   // but keep at least one 16-byte chunk per lane in a segment
   const int chunks = d.D >> 3;

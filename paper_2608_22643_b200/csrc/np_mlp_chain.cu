@@ -1,6 +1,7 @@
 // Stage 4 over a run of consecutive layers in ONE persistent kernel (B = 1).
 //
-//   x_{l+1} = x_l + sum_{i in act_l} silu(gate_l[s_i].x_l) * (up_l[s_i].x_l) * downT_l[s_i]
+//   x_{l+1} = x_l + sum_{i in act_l} silu(gate_l[s_i].n_l) * (up_l[s_i].n_l) * downT_l[s_i],
+//   n_l = x_l / sqrt(mean(x_l^2) + 1e-6)   (pre-MLP RMS normalisation, unit gain)
 //
 // (Section 3.4: the sparse MLP reads each active row through the slot map;
 // Section 3.1: the sparse suffix runs once its delta rows are in place.)
@@ -72,6 +73,7 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   __shared__ __align__(8) uint64_t empty_bar[kChainMaxStages];  // every consumer warp is done with it
   __shared__ float part[kChainWarps][2];        // (g, u) partial sums of the tile's (row, segment) items
   __shared__ float act[kChainWarps];            // a_i of the tile's rows
+  __shared__ float ssq_part[kChainWarps];       // per-warp sums of x_l^2 (for the RMS normalisation)
   __shared__ int s_ok;
   __shared__ int lay_rb[kChainMaxLayers];       // first active-list index of this block, per layer
   __shared__ int lay_pre[kChainMaxLayers + 1];  // rows of this block before each layer (virtual row index)
@@ -207,6 +209,7 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       const float* zb = l > 0 ? a.zbuf[(l - 1) % 3] : nullptr;
       float* xst = a.xbuf[l & 1];
       const int nf4 = chunks * 2;  // float4 granules of one vector
+      float ssq = 0.f;
       for (int c0 = tid; c0 < nf4; c0 += 2 * kChainThreads) {
         // all loads of two granules (and of every accumulator copy) are issued before any is used
         const int c1 = c0 + kChainThreads;
@@ -236,11 +239,15 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
         }
         reinterpret_cast<float4*>(xs)[c0] = v0;
         if (has1) reinterpret_cast<float4*>(xs)[c1] = v1;
+        ssq += v0.x * v0.x + v0.y * v0.y + v0.z * v0.z + v0.w * v0.w;
+        ssq += v1.x * v1.x + v1.y * v1.y + v1.z * v1.z + v1.w * v1.w;  // zeros when there is no second granule
         if (blockIdx.x == 0 && l == l_last) {  // x for the next launch
           reinterpret_cast<float4*>(xst)[c0] = v0;
           if (has1) reinterpret_cast<float4*>(xst)[c1] = v1;
         }
       }
+      ssq = warp_sum(ssq);
+      if (lane == 0) ssq_part[wid] = ssq;
       // clear the next layer's accumulator copies: every block takes a slice
       float4* znext = reinterpret_cast<float4*>(a.zbuf[(l + 1) % 3]);
       const int ztotal = nf4 * kZRep;
@@ -325,6 +332,12 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
           gs += part[tid * SEG + w][0];
           us += part[tid * SEG + w][1];
         }
+        // the MLP's input is x_l scaled to unit RMS; the dot products are linear in it
+        float ss = 0.f;
+        for (int w = 0; w < kChainWarps; ++w) ss += ssq_part[w];
+        const float inv_rms = rsqrtf(ss / (float)D + kRmsEps);
+        gs *= inv_rms;
+        us *= inv_rms;
         act[tid] = gs / (1.f + __expf(-gs)) * us;
       }
       consumer_sync();

@@ -1,0 +1,65 @@
+"""Parity at the benchmark's full 7B-shaped size, in the launch configuration bench.py times
+(host-gather transfer, resident multi-layer MLP kernel, default run length)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import np_oracle as O
+from paper_2608_22643_b200 import binding as nb
+from paper_2608_22643_b200 import synth
+from tests.harness import REL_L2_TOL, Pair, rel_l2, u16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("policy", [nb.NP_EVICT_EXACT, nb.NP_EVICT_LRU])
+def test_7b_shape_steps_match_oracle(policy):
+    cfg = synth.CONFIGS["7b"]
+    L, M, D, W = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_ffn // 32
+    free, _ = torch.cuda.mem_get_info()
+    if free < 8 * 2**30:
+        pytest.skip("needs 8 GB of device memory")
+    p = Pair(cfg, policy=policy, transfer_mode=nb.NP_XFER_HOST_GATHER, staging_rows=2 * cfg.top_k,
+             flags=0, gen_device="cuda")
+    try:
+        n_steps = 3
+        xs = synth.hidden_states(cfg, n_steps)
+        logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")
+        bitmap = torch.empty((L, W), dtype=torch.int32, device="cuda")
+        out = torch.empty((1, D), dtype=torch.float32, device="cuda")
+        rng = np.random.default_rng(0)
+        w1 = O.bf16_to_f64(u16(p.w1_cpu))
+        w2_u16 = u16(p.w2_cpu)
+        for t in range(n_steps):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, 1, logits, bitmap, p.eng.stream)
+            rc = nb.np_step(p.eng.ctx, x, 1, out, p.eng.stream, p.eng.copy_stream)
+            assert rc in (nb.NP_OK, nb.NP_W_CHUNKED)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            # stage 1: sampled logits, each against its own fp64 dot product
+            h = np.maximum(0.0, O.bf16_to_f64(u16(xs[t])) @ w1.T)[0]
+            rows = rng.integers(0, L * M, size=400)
+            want = np.array([O.bf16_to_f64(w2_u16[r]) @ h for r in rows])
+            got = z32.reshape(-1)[rows]
+            assert np.linalg.norm(got - want) / np.linalg.norm(want) < REL_L2_TOL
+            assert np.max(np.abs(got - want)) < 1e-4 * np.max(np.abs(want))
+            # stage 2: the whole selection, bit-exact on the GPU's own logits
+            assert (bitmap.cpu().numpy().view(np.uint32) == O.topk_bitmap(z32, p.k)).all()
+            # stages 3-4 through the oracle engine (its own tables, buffers and chain)
+            res = p.ora.step(u16(xs[t]), logits_f32=z32)
+            cnt = p.check_delta_against(res["deltas"])
+            assert (cnt[:, nb.NP_CNT_ACTIVE] == p.k).all() and (cnt[:, nb.NP_CNT_OVERFLOW] == 0).all()
+            if policy == nb.NP_EVICT_EXACT:
+                assert (cnt[:, nb.NP_CNT_RESIDENT] == p.k).all()
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < REL_L2_TOL, t
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+            # install: sampled resident rows of every layer hold their record's bytes
+            for l in range(L):
+                ids = np.flatnonzero(p.ora.res.R[l])
+                pick = rng.choice(ids, size=min(48, ids.size), replace=False)
+                slots = torch.from_numpy(p.ora.res.S[l][pick].astype(np.int64)).cuda()
+                for part, buf in enumerate((p.eng.gate, p.eng.up, p.eng.downT)):
+                    assert (u16(buf[l][slots]) == p.store_u16[l, pick, part]).all(), (t, l, part)
+    finally:
+        p.close()

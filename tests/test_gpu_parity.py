@@ -163,7 +163,8 @@ def test_all_rows_active_is_the_dense_mlp():
         x = x_bf.to(torch.float64)
         for l in range(cfg.n_layers):
             rec = p.backing[l].to(torch.float64)
-            x = x + (torch.nn.functional.silu(x @ rec[:, 0].T) * (x @ rec[:, 1].T)) @ rec[:, 2]
+            n = x / torch.sqrt((x * x).mean(dim=-1, keepdim=True) + 1e-6)     # pre-MLP RMS norm, unit gain
+            x = x + (torch.nn.functional.silu(n @ rec[:, 0].T) * (n @ rec[:, 1].T)) @ rec[:, 2]
         assert rel_l2(out.cpu().numpy(), x.numpy()) < REL_L2_TOL
     finally:
         p.close()

@@ -93,6 +93,18 @@ def test_linearity_over_disjoint_sets_and_buffer_vs_store():
     assert not O.sparse_mlp(g, u, dn, 0, np.zeros(0, np.int32), x).any()
 
 
+def test_rms_normalize_pins():
+    x = np.array([[3.0, -4.0, 0.0, 0.0]])
+    # mean square = 25/4, so the scale is 1/2.5 (up to the 1e-6 epsilon)
+    assert np.allclose(O.rms_normalize(x), x / 2.5, rtol=1e-6, atol=0)
+    r = np.random.default_rng(5).standard_normal((3, 64)) * 7.0
+    n = O.rms_normalize(r)
+    assert np.allclose(np.sqrt((n * n).mean(axis=1)), 1.0, rtol=1e-6)
+    assert np.allclose(O.rms_normalize(5.0 * r), n, rtol=1e-6)          # scale invariant
+    assert np.allclose(n * np.sqrt((r * r).mean(axis=1, keepdims=True) + 1e-6), r, rtol=1e-12)
+    assert not O.rms_normalize(np.zeros((1, 8))).any()                   # epsilon keeps 0/0 away
+
+
 def test_engine_trajectory_consistency():
     """Whole-step driver: buffers always hold the right bytes for every resident
     row, and the chain through slots equals the chain from the store."""
@@ -117,7 +129,7 @@ def test_engine_trajectory_consistency():
                 assert (eng.downT[l, S] == st[l, R, 2]).all()
             x = O.bf16_to_f64(as_u16(xs[t]))
             for l, d in enumerate(out["deltas"]):
-                x = x + O.sparse_mlp_from_store(st, l, d.active_ids, x)
+                x = x + O.sparse_mlp_from_store(st, l, d.active_ids, O.rms_normalize(x))
             assert np.allclose(x, out["x_final"], rtol=1e-12, atol=1e-15)
             if prev is not None:
                 overlaps.append((P & prev).sum() / P.sum())

@@ -1,0 +1,42 @@
+"""The N > 1 plumbing of bench.py (independent replicas, max-over-ranks timing, rank-0 report)
+on two CPU processes over gloo."""
+import json
+import os
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_two_replicas_reduce_to_the_slowest_rank(tmp_path):
+    script = tmp_path / "ranks.py"
+    script.write_text(
+        "import json, os, sys\n"
+        f"sys.path.insert(0, {ROOT!r})\n"
+        "import bench\n"
+        "from paper_2608_22643_b200 import synth\n"
+        "dist = bench.init_replicas('gloo')\n"
+        "rank = int(os.environ['RANK'])\n"
+        "cfg = bench.replica_config(synth.CONFIGS['tiny'], rank)\n"
+        "ms = bench.max_over_ranks(dist, [10.0 + 5.0 * rank, 3.0 - rank], 'cpu')\n"
+        "x = synth.hidden_states(cfg, 2)\n"
+        "print(json.dumps({'rank': rank, 'seed': cfg.seed, 'ms': ms, 'x0': float(x.float().sum())}))\n"
+        "bench.finish_replicas(dist)\n")
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29611", WORLD_SIZE="2")
+    procs = [subprocess.Popen([sys.executable, str(script)], env=dict(env, RANK=str(r), LOCAL_RANK=str(r)),
+                              stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True) for r in range(2)]
+    outs = []
+    for pr in procs:
+        o, e = pr.communicate(timeout=120)
+        assert pr.returncode == 0, e
+        outs.append(json.loads(o.strip().splitlines()[-1]))
+    outs.sort(key=lambda d: d["rank"])
+    assert outs[0]["ms"] == outs[1]["ms"] == [15.0, 3.0]          # every rank sees the slowest rank's time
+    assert outs[0]["seed"] != outs[1]["seed"] and outs[0]["x0"] != outs[1]["x0"]   # own sequence per replica
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
+                       env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0 and r.stdout.strip() == ""
