@@ -55,6 +55,7 @@ def parse_args():
     ap.add_argument("--layer-launches", action="store_true", help="one MLP kernel launch per layer")
     ap.add_argument("--direct-loads", action="store_true", help="MLP rows by plain global loads")
     ap.add_argument("--chain-layers", type=int, default=0, help="layers per resident MLP kernel")
+    ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
     return ap.parse_args()
 
 
@@ -275,13 +276,15 @@ def cuda_arm(args):
     ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
                           max_batch=1, evict_policy=policy, transfer_mode=mode,
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
+                          host_threads=args.host_threads,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0))
     eng = nb.Engine(ncfg, w1, w2, store, device=dev)
     L, D, M = cfg.n_layers, cfg.d_model, cfg.d_ffn
     rec = cfg.record_bytes
     T = 1 + W + K                                      # cold start + warm-up + timed
-    xs_host = synth.hidden_states(cfg, T).pin_memory()             # [T, 1, D] bf16
+    n_detail = 16
+    xs_host = synth.hidden_states(cfg, T + n_detail).pin_memory()  # [T + n_detail, 1, D] bf16
     xs_dev = xs_host.to(dev)
     out = torch.empty((1, D), dtype=torch.float32, device=dev)
     out_host = torch.empty((1, D), dtype=torch.float32).pin_memory()
@@ -316,6 +319,18 @@ def cuda_arm(args):
     ms_total = e0.elapsed_time(e1)
     eng.counters()
 
+    # ---- per-stage detail on a few more steady-state steps (untimed region) ----------------
+    stage_us, delta_rows, overlap = [], [], []
+    for i in range(n_detail):
+        t = T + i                                       # the sequence simply continues
+        nb.np_step(eng.ctx, xs_dev[t], 1, out, s, cs)
+        stage_us.append(nb.np_last_step_times(eng.ctx))
+        c = eng.counters()
+        delta_rows.append(float(c[:, nb.NP_CNT_DELTA].mean()))
+        overlap.append(float((c[:, nb.NP_CNT_KEPT] / np.maximum(1, c[:, nb.NP_CNT_PRED])).mean()))
+    stage_us = np.median(np.stack(stage_us), axis=0)
+    n_active = float(eng.counters()[:, nb.NP_CNT_ACTIVE].mean())
+
     # ---- end-to-end timing: hidden state from pinned host, result back to the host --------
     nb.np_reset(eng.ctx, s)
     def run_e2e(t_lo, t_hi):
@@ -336,18 +351,6 @@ def cuda_arm(args):
     barrier()
     e2e_ms_total = g0.elapsed_time(g1)
     clocks = sampler.stop()
-
-    # ---- per-stage detail on a few more steady-state steps (untimed region) ----------------
-    stage_us, delta_rows, overlap = [], [], []
-    for i in range(min(16, K)):
-        t = 1 + W + i
-        nb.np_step(eng.ctx, xs_dev[t], 1, out, s, cs)
-        stage_us.append(nb.np_last_step_times(eng.ctx))
-        c = eng.counters()
-        delta_rows.append(float(c[:, nb.NP_CNT_DELTA].mean()))
-        overlap.append(float((c[:, nb.NP_CNT_KEPT] / np.maximum(1, c[:, nb.NP_CNT_PRED])).mean()))
-    stage_us = np.median(np.stack(stage_us), axis=0)
-    n_active = float(eng.counters()[:, nb.NP_CNT_ACTIVE].mean())
 
     # ---- dominant kernel: the sparse MLP, timed alone on its own stream ---------------------
     reps = 20

@@ -3,6 +3,7 @@
 // arithmetic step runs in the kernels of the sibling .cu files.
 #include <algorithm>
 #include <atomic>
+#include <chrono>
 #include <condition_variable>
 #include <cstdarg>
 #include <cstdio>
@@ -22,17 +23,20 @@ thread_local std::string g_last_error = "";
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Small fork-join pool for packing records into pinned staging.
+// Small fork-join pool for packing records into pinned staging.  A step issues one short
+// job per layer, tens of microseconds apart, so idle workers spin on the job counter for a
+// while before they go to sleep on the condition variable (a sleeping thread takes longer
+// to wake than a layer's records take to pack).
 class Pool {
  public:
-  explicit Pool(int n) : stop_(false), gen_(0), pending_(0) {
+  explicit Pool(int n) {
     for (int i = 0; i < n; ++i) threads_.emplace_back([this] { run(); });
   }
   ~Pool() {
     {
       std::lock_guard<std::mutex> lk(m_);
-      stop_ = true;
-      ++gen_;
+      stop_.store(true);
+      ticket_.fetch_add(1ull << 32);
     }
     cv_.notify_all();
     for (auto& t : threads_) t.join();
@@ -44,55 +48,84 @@ class Pool {
       for (int i = 0; i < count; ++i) fn(i);
       return;
     }
+    // Index claims carry the job's generation, so a worker that is late leaving one job can
+    // never claim (or count) an index of the next.
+    const uint64_t g = (ticket_.load() >> 32) + 1;
+    Job& job = jobs_[g & 1];
+    job.fn.store(&fn);
+    job.count.store(count);
+    job.done.store(0);
     {
-      std::lock_guard<std::mutex> lk(m_);
-      fn_ = &fn;
-      count_ = count;
-      next_.store(0);
-      pending_ = (int)threads_.size();
-      ++gen_;
+      std::lock_guard<std::mutex> lk(m_);  // pairs with the sleepers' predicate check
+      ticket_.store(g << 32);
     }
-    cv_.notify_all();
-    work();
-    std::unique_lock<std::mutex> lk(m_);
-    done_cv_.wait(lk, [this] { return pending_ == 0; });
-    fn_ = nullptr;
+    if (sleepers_.load() > 0) cv_.notify_all();
+    work(g);
+    while (job.done.load(std::memory_order_acquire) < count) cpu_relax();
   }
   int size() const { return (int)threads_.size(); }
 
  private:
-  void work() {
+  struct Job {
+    std::atomic<const std::function<void(int)>*> fn{nullptr};
+    std::atomic<int> count{0};
+    std::atomic<int> done{0};
+  };
+  static void cpu_relax() {
+#if defined(__x86_64__) || defined(__i386__)
+    __builtin_ia32_pause();
+#else
+    std::this_thread::yield();
+#endif
+  }
+  void work(uint64_t g) {
+    Job& job = jobs_[g & 1];
+    const std::function<void(int)>* fn = job.fn.load();
+    const int count = job.count.load();
     for (;;) {
-      const int i = next_.fetch_add(1);
-      if (i >= count_) break;
-      (*fn_)(i);
+      uint64_t t = ticket_.load();
+      if ((t >> 32) != g) return;  // the job is over (and fn / count may belong to a later one)
+      const int i = (int)(t & 0xffffffffu);
+      if (i >= count) return;
+      if (!ticket_.compare_exchange_weak(t, t + 1)) continue;
+      (*fn)(i);
+      job.done.fetch_add(1, std::memory_order_release);
     }
   }
   void run() {
-    unsigned long seen = 0;
+    uint64_t seen = 0;
     for (;;) {
-      {
+      // spin for roughly a quarter of a millisecond, then sleep
+      bool got = false;
+      const auto t0 = std::chrono::steady_clock::now();
+      for (int spin = 0;; ++spin) {
+        if ((ticket_.load(std::memory_order_acquire) >> 32) != seen) {
+          got = true;
+          break;
+        }
+        cpu_relax();
+        if ((spin & 1023) == 1023 &&
+            std::chrono::steady_clock::now() - t0 > std::chrono::microseconds(250))
+          break;
+      }
+      if (!got) {
         std::unique_lock<std::mutex> lk(m_);
-        cv_.wait(lk, [&] { return gen_ != seen; });
-        seen = gen_;
-        if (stop_) return;
+        sleepers_.fetch_add(1);
+        cv_.wait(lk, [&] { return (ticket_.load() >> 32) != seen; });
+        sleepers_.fetch_sub(1);
       }
-      work();
-      {
-        std::lock_guard<std::mutex> lk(m_);
-        if (--pending_ == 0) done_cv_.notify_all();
-      }
+      seen = ticket_.load(std::memory_order_acquire) >> 32;
+      if (stop_.load()) return;
+      work(seen);
     }
   }
   std::vector<std::thread> threads_;
   std::mutex m_;
-  std::condition_variable cv_, done_cv_;
-  bool stop_;
-  unsigned long gen_;
-  int pending_;
-  const std::function<void(int)>* fn_ = nullptr;
-  int count_ = 0;
-  std::atomic<int> next_{0};
+  std::condition_variable cv_;
+  std::atomic<bool> stop_{false};
+  std::atomic<uint64_t> ticket_{0};  // generation << 32 | next index of that generation's job
+  std::atomic<int> sleepers_{0};
+  Job jobs_[2];
 };
 
 }  // namespace
@@ -382,7 +415,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
 
   if (cfg->transfer_mode == NP_XFER_HOST_GATHER) {
     int n = cfg->host_threads;
-    if (n == 0) n = std::max(1u, std::min(8u, std::thread::hardware_concurrency()));
+    if (n == 0) n = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
     ctx->pool = new (std::nothrow) Pool(n - 1);  // the caller's thread works too
   }
   *out = ctx;
