@@ -73,6 +73,8 @@ extern "C" {
                                    through NP_E_DEVICE instead of touching memory */
 #define NP_F_DIRECT_LOADS    2  /* sparse MLP: plain 16-byte global loads instead of the
                                    shared-memory staged kernel (for comparison runs) */
+#define NP_F_NO_TENSOR_CORES 8  /* np_predict with B > 4: ALU kernel instead of the tcgen05 GEMM
+                                   (for comparison runs) */
 #define NP_F_LAYER_LAUNCHES  4  /* np_step / np_mlp_chain: one kernel launch per layer instead
                                    of resident kernels spanning runs of layers */
 

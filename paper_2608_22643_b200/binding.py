@@ -26,6 +26,7 @@ NP_XFER_MEMCPY_RUNS, NP_XFER_HOST_GATHER, NP_XFER_ZERO_COPY = 0, 1, 2
 NP_F_CHECK_BOUNDS = 1
 NP_F_DIRECT_LOADS = 2
 NP_F_LAYER_LAUNCHES = 4
+NP_F_NO_TENSOR_CORES = 8
 (NP_CNT_PRED, NP_CNT_KEPT, NP_CNT_DELTA, NP_CNT_EVICT, NP_CNT_OVERFLOW, NP_CNT_ACTIVE,
  NP_CNT_RESIDENT, NP_CNT_STEP) = range(8)
 NP_N_COUNTERS = 8

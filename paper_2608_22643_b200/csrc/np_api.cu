@@ -156,6 +156,7 @@ struct np_ctx {
   int step = 0;
   uint64_t launches = 0;
   Pool* pool = nullptr;
+  PredTcState tc = {};
   std::string err;
 };
 
@@ -206,7 +207,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->staging_rows < 1) return fail(ctx, NP_E_INVAL, "staging_rows must be >= 1");
   if (c->transfer_mode == NP_XFER_HOST_GATHER && c->staging_rows < 2)
     return fail(ctx, NP_E_INVAL, "host gather needs staging_rows >= 2 (two halves)");
-  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
+  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
   if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
@@ -216,7 +217,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
 }
 
 struct WsLayout {
-  size_t hidden, logits, xbuf, zbuf, total;
+  size_t hidden, hsplit, logits, xbuf, zbuf, total;
 };
 
 WsLayout ws_layout(const np_config& c) {
@@ -224,6 +225,8 @@ WsLayout ws_layout(const np_config& c) {
   size_t off = 0;
   w.hidden = off;
   off = align_up(off + (size_t)c.max_batch * c.d_pred * 4, 256);
+  w.hsplit = off;
+  off = align_up(off + (size_t)48 * c.d_pred * 2, 256);
   w.logits = off;
   off = align_up(off + (size_t)c.max_batch * c.n_layers * c.d_ffn * 4, 256);
   const size_t vec = align_up((size_t)c.max_batch * c.d_model * 4, 256);
@@ -395,6 +398,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   char* wsb = static_cast<char*>(b->workspace);
   const size_t vec = align_up((size_t)d.Bmax * d.D * 4, 256);
   ctx->ws.hidden = reinterpret_cast<float*>(wsb + wl.hidden);
+  ctx->ws.hsplit = wsb + wl.hsplit;
   ctx->ws.logits = reinterpret_cast<float*>(wsb + wl.logits);
   for (int i = 0; i < 2; ++i) ctx->ws.xbuf[i] = reinterpret_cast<float*>(wsb + wl.xbuf + i * vec);
   for (int i = 0; i < 3; ++i) ctx->ws.zbuf[i] = reinterpret_cast<float*>(wsb + wl.zbuf + i * kZRep * vec);
@@ -408,6 +412,8 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   for (auto& e : ctx->ev_t) NP_INIT_CUDA(cudaEventCreate(&e));
   for (auto& e : ctx->ev_c) NP_INIT_CUDA(cudaEventCreate(&e));
 
+  // tensor-core predictor for batches: tensor maps over W2 and the split hidden terms
+  if (cfg->max_batch > 4 && !(cfg->flags & NP_F_NO_TENSOR_CORES)) pred_tc_prepare(d, b->w2, ctx->ws.hsplit, &ctx->tc);
   memset(ctx->host_lists, 0, host_lists_ints(*cfg) * 4);
   NP_INIT_CUDA(launch_tables_reset(d, t, nullptr));
   NP_INIT_CUDA(cudaDeviceSynchronize());
@@ -440,7 +446,12 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
   cudaStream_t s = as_stream(stream);
   const Dims& d = ctx->d;
   NP_LAUNCH(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
-  NP_LAUNCH(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
+  if (B > 4 && ctx->tc.ready) {
+    ctx->launches += 1;  // split kernel + GEMM kernel
+    NP_LAUNCH(ctx, launch_pred_l2_tc(d, ctx->tc, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
+  } else {
+    NP_LAUNCH(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
+  }
   NP_LAUNCH(ctx, launch_topk(d, ctx->ws.logits, B, ctx->t.pred, s));
   const size_t nlog = (size_t)B * d.L * d.M * 4, nbm = (size_t)d.L * d.W * 4;
   if (logits_out) NP_CUDA(ctx, cudaMemcpyAsync(logits_out, ctx->ws.logits, nlog, cudaMemcpyDeviceToDevice, s));

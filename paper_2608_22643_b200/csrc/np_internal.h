@@ -40,6 +40,7 @@ struct Tables {
 // Carved out of the caller's workspace.
 struct Workspace {
   float* hidden;   // [Bmax][H]
+  void* hsplit;    // bf16 [48][H]: hidden split into three bf16 terms (tensor-core predictor)
   float* logits;   // [Bmax][L][M]
   float* xbuf[2];  // [Bmax][D] each: x_l of the residual chain, ping-pong
   float* zbuf[3];  // [kZRep][Bmax][D] each: MLP_l(x_l) accumulators, rotating
@@ -58,6 +59,20 @@ cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, in
                            cudaStream_t s);
 cudaError_t launch_pred_l2(const Dims& d, const void* w2, const float* hidden, int B, float* logits,
                            int32_t* status, cudaStream_t s, int sm_count);
+// Tensor-core form of predictor layer 2 for batches (np_predict_tc.cu).
+struct PredTcState {
+  alignas(64) unsigned char map_w2[128];  // CUtensorMap of W2 [L*M][H]
+  alignas(64) unsigned char map_h[128];   // CUtensorMap of the split hidden terms [48][H]
+  void* hsplit;                           // device bf16 [48][H] (workspace)
+  int n_stages;
+  size_t smem;
+  int ready;
+};
+bool pred_tc_supported(const Dims& d);
+bool pred_tc_prepare(const Dims& d, const void* w2, void* hsplit, PredTcState* st);
+cudaError_t launch_pred_l2_tc(const Dims& d, const PredTcState& st, const float* hidden, int B, float* logits,
+                              int32_t* status, cudaStream_t s, int sm_count);
+
 cudaError_t launch_topk(const Dims& d, const float* logits, int B, uint32_t* bitmap, cudaStream_t s);
 
 cudaError_t launch_delta(const Dims& d, const Tables& t, const uint32_t* pred, int policy, int step,

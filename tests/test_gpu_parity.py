@@ -14,9 +14,17 @@ TINY = synth.CONFIGS["tiny"]
 SMALL = synth.CONFIGS["small"]     # ragged: M = 2080 (65 words), H = 96, 3 layers
 
 
-@pytest.mark.parametrize("cfg,B", [(TINY, 1), (SMALL, 1), (SMALL, 3), (TINY, 16)])
-def test_predict_logits_and_bitmap(cfg, B):
-    p = Pair(cfg, max_batch=B)
+# predictor width a multiple of 64 (three k-blocks) and a row count that is not a multiple of
+# the 128-row MMA tile: the batch path runs on the tensor cores with a ragged last tile
+TCW = synth.StackConfig("tcw", 3, 512, 2080, 192, 10, 25, 4, 21, 0.9)
+
+
+@pytest.mark.parametrize("cfg,B,flags", [
+    (TINY, 1, 0), (SMALL, 1, 0), (SMALL, 3, 0), (TINY, 16, 0), (TCW, 16, 0), (TCW, 7, 0), (TCW, 5, 0),
+    (TCW, 16, nb.NP_F_NO_TENSOR_CORES), (SMALL, 9, 0),
+])
+def test_predict_logits_and_bitmap(cfg, B, flags):
+    p = Pair(cfg, max_batch=B, flags=flags | nb.NP_F_CHECK_BOUNDS)
     try:
         xs = synth.hidden_states(cfg, 3, batch=B)
         L, M, W = cfg.n_layers, cfg.d_ffn, cfg.d_ffn // 32
