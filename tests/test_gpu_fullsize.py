@@ -63,3 +63,32 @@ def test_7b_shape_steps_match_oracle(policy):
                     assert (u16(buf[l][slots]) == p.store_u16[l, pick, part]).all(), (t, l, part)
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("name,n_layers,mode", [
+    ("13b", 3, nb.NP_XFER_HOST_GATHER), ("70b", 2, nb.NP_XFER_ZERO_COPY), ("70b", 2, nb.NP_XFER_MEMCPY_RUNS),
+])
+def test_larger_shapes_few_layers(name, n_layers, mode):
+    """The 13B- and 70B-shaped rows (D = 5120 / 8192, M = 13824 / 28672) on a few layers:
+    other ring depths, column rounds and segment splits than the 7B shape."""
+    cfg = synth.CONFIGS[name].with_(n_layers=n_layers)
+    L, M, D, W = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_ffn // 32
+    p = Pair(cfg, transfer_mode=mode, flags=nb.NP_F_CHECK_BOUNDS, gen_device="cuda")
+    try:
+        xs = synth.hidden_states(cfg, 3)
+        logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")
+        out = torch.empty((1, D), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, x, 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            z = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)
+            assert rel_l2(z32, z) < 1e-5
+            res = p.ora.step(u16(xs[t]), logits_f32=z32)
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+        p.check_resident_bytes()
+    finally:
+        p.close()
