@@ -33,6 +33,7 @@ constexpr int kChainWarps = 16;                      // consumer warps
 constexpr int kChainThreads = kChainWarps * 32;      // consumer threads
 constexpr int kChainBlock = kChainThreads + 32;      // plus one producer warp
 constexpr int kChainMaxStages = 16;
+constexpr int kChainMaxRpw = 2;   // rows a warp may take per tile in phase 1
 constexpr int kChainMaxLayers = 128;  // layers per launch (longer runs are split by the host)
 
 struct ChainKernelArgs {
@@ -46,7 +47,7 @@ struct ChainKernelArgs {
                                // into copy g % kZRep (fewer adds per address), readers sum the copies
   unsigned int* grid_bar;      // zeroed by the host before the launch
   int32_t* status;
-  int l_begin, l_end, D, C, n_stages, tile_rows, check;
+  int l_begin, l_end, D, C, n_stages, tile_rows, rows_per_warp, check;
   int slot_cache_rows;         // capacity of the per-block slot cache (rows)
   int window_rows;             // records in flight per block (< n_stages)
 };
@@ -71,8 +72,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   extern __shared__ __align__(128) unsigned char csm[];
   __shared__ __align__(8) uint64_t full_bar[kChainMaxStages];   // a stage's record has landed
   __shared__ __align__(8) uint64_t empty_bar[kChainMaxStages];  // every consumer warp is done with it
-  __shared__ float part[kChainWarps][2];        // (g, u) partial sums of the tile's (row, segment) items
-  __shared__ float act[kChainWarps];            // a_i of the tile's rows
+  __shared__ float part[kChainMaxRpw * kChainWarps][2];  // (g, u) partial sums of the tile's (row, segment) items
+  __shared__ float act[kChainMaxRpw * kChainWarps];      // a_i of the tile's rows
   __shared__ float ssq_part[kChainWarps];       // per-warp sums of x_l^2 (for the RMS normalisation)
   __shared__ int s_ok;
   __shared__ int lay_rb[kChainMaxLayers];       // first active-list index of this block, per layer
@@ -82,7 +83,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   const uint32_t row_bytes = (uint32_t)D * 2u;
   const uint32_t rec_bytes = 3u * row_bytes;
   const size_t layer_bytes = (size_t)a.C * row_bytes;
-  const int n_stages = a.n_stages, TR = a.tile_rows, SEG = kChainWarps / TR;
+  // a tile is TR = RPW * (16 / SEG) rows: phase 1 gives every warp RPW (row, segment) items
+  const int n_stages = a.n_stages, RPW = a.rows_per_warp, TR = a.tile_rows, SEG = kChainWarps * RPW / TR;
   const int seg_chunks = (chunks + SEG - 1) / SEG;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int G = gridDim.x, nl = a.l_end - a.l_begin;
@@ -281,8 +283,10 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       const int s0 = (vbase + t0) % n_stages;  // stage of the tile's first row; the rest follow, wrapping
       const uint32_t use0 = (uint32_t)((vbase + t0) / n_stages);
       // ---- phase 1: (row, segment) partial dot products from shared memory ----
-      if (row_in_tile < rows) {
-        int s = s0 + row_in_tile;
+      for (int rr = 0; rr < RPW; ++rr) {
+        const int row = row_in_tile + rr * (TR / RPW);
+        if (row >= rows) break;
+        int s = s0 + row;
         uint32_t use = use0;
         if (s >= n_stages) {
           s -= n_stages;
@@ -320,8 +324,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
           u += __shfl_xor_sync(0xffffffffu, u, o);
         }
         if (lane == 0) {
-          part[wid][0] = g;
-          part[wid][1] = u;
+          part[row * SEG + sg][0] = g;
+          part[row * SEG + sg][1] = u;
         }
       }
       consumer_sync();
@@ -452,6 +456,13 @@ bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
   const int need_cols = (chunks + kChainThreads - 1) / kChainThreads;
   if (p->xj > 8 || need_cols > 4) return false;
   p->cols = need_cols <= 1 ? 1 : (need_cols <= 2 ? 2 : 4);
+  // when the whole share of a layer fits the ring, take it as one tile: two rows per warp
+  // in phase 1, half the block-wide barriers
+  p->rows_per_warp = 1;
+  if (d.chain_rpw != 1 && 2 * tr <= n_stages && 2 * tr >= per_block) {
+    p->rows_per_warp = 2;
+    tr *= 2;
+  }
   p->n_stages = n_stages;
   p->tile_rows = tr;
   p->window_rows = 2;
@@ -482,6 +493,7 @@ cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, 
     ka.C = d.C;
     ka.n_stages = p.n_stages;
     ka.tile_rows = p.tile_rows;
+    ka.rows_per_warp = p.rows_per_warp;
     ka.check = a.check;
     e = cudaMemsetAsync(a.grid_bar, 0, sizeof(unsigned int), s);
     if (e != cudaSuccess) return e;
