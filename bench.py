@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--layer-launches", action="store_true", help="one MLP kernel launch per layer")
     ap.add_argument("--direct-loads", action="store_true", help="MLP rows by plain global loads")
     ap.add_argument("--chain-layers", type=int, default=0, help="layers per resident MLP kernel")
+    ap.add_argument("--batch", type=int, default=1, help="sequences per step (the metric's workload is 1)")
+    ap.add_argument("--gamma", type=float, default=0.9, help="shared-driver weight of batched hidden states")
     ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
     return ap.parse_args()
 
@@ -274,7 +276,7 @@ def cuda_arm(args):
 
     w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True)
     ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
-                          max_batch=1, evict_policy=policy, transfer_mode=mode,
+                          max_batch=args.batch, evict_policy=policy, transfer_mode=mode,
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
                           host_threads=args.host_threads,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
@@ -284,11 +286,12 @@ def cuda_arm(args):
     rec = cfg.record_bytes
     T = 1 + W + K                                      # cold start + warm-up + timed
     n_detail = 16
-    xs_host = synth.hidden_states(cfg, T + n_detail).pin_memory()  # [T + n_detail, 1, D] bf16
+    Bq = args.batch
+    xs_host = synth.hidden_states(cfg, T + n_detail, batch=Bq, gamma=args.gamma).pin_memory()  # [T + n_detail, B, D] bf16
     xs_dev = xs_host.to(dev)
-    out = torch.empty((1, D), dtype=torch.float32, device=dev)
-    out_host = torch.empty((1, D), dtype=torch.float32).pin_memory()
-    x_stage = torch.empty((1, D), dtype=torch.bfloat16, device=dev)
+    out = torch.empty((Bq, D), dtype=torch.float32, device=dev)
+    out_host = torch.empty((Bq, D), dtype=torch.float32).pin_memory()
+    x_stage = torch.empty((Bq, D), dtype=torch.bfloat16, device=dev)
     s, cs = eng.stream, eng.copy_stream
 
     def barrier():
@@ -299,7 +302,7 @@ def cuda_arm(args):
 
     def run_resident(t_lo, t_hi, stats=None):
         for t in range(t_lo, t_hi):
-            nb.np_step(eng.ctx, xs_dev[t], 1, out, s, cs)
+            nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
             if stats is not None:
                 stats.append(eng.counters().copy())
 
@@ -320,13 +323,14 @@ def cuda_arm(args):
     eng.counters()
 
     # ---- per-stage detail on a few more steady-state steps (untimed region) ----------------
-    stage_us, delta_rows, overlap = [], [], []
+    stage_us, delta_rows, overlap, overflow_steps = [], [], [], 0
     for i in range(n_detail):
         t = T + i                                       # the sequence simply continues
-        nb.np_step(eng.ctx, xs_dev[t], 1, out, s, cs)
+        nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
         stage_us.append(nb.np_last_step_times(eng.ctx))
         c = eng.counters()
         delta_rows.append(float(c[:, nb.NP_CNT_DELTA].mean()))
+        overflow_steps += int((c[:, nb.NP_CNT_OVERFLOW] > 0).any())
         overlap.append(float((c[:, nb.NP_CNT_KEPT] / np.maximum(1, c[:, nb.NP_CNT_PRED])).mean()))
     stage_us = np.median(np.stack(stage_us), axis=0)
     n_active = float(eng.counters()[:, nb.NP_CNT_ACTIVE].mean())
@@ -337,7 +341,7 @@ def cuda_arm(args):
         for t in range(t_lo, t_hi):
             with torch.cuda.stream(s):
                 x_stage.copy_(xs_host[t], non_blocking=True)
-            nb.np_step(eng.ctx, x_stage, 1, out, s, cs)
+            nb.np_step(eng.ctx, x_stage, Bq, out, s, cs)
             with torch.cuda.stream(s):
                 out_host.copy_(out, non_blocking=True)
             s.synchronize()                              # the caller consumes the result every step
@@ -356,18 +360,22 @@ def cuda_arm(args):
     reps = 20
     k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for _ in range(3):
-        nb.np_mlp_chain(eng.ctx, xs_dev[T - 1], 1, out, s)
+        nb.np_mlp_chain(eng.ctx, xs_dev[T - 1], Bq, out, s)
     s.synchronize()
     k0.record(s)
     for _ in range(reps):
-        nb.np_mlp_chain(eng.ctx, xs_dev[T - 1], 1, out, s)
+        nb.np_mlp_chain(eng.ctx, xs_dev[T - 1], Bq, out, s)
     k1.record(s)
     s.synchronize()
-    mlp_us = k0.elapsed_time(k1) * 1000.0 / (reps * L)            # per layer launch, gaps included
+    chain_layers = args.chain_layers if args.chain_layers > 0 else (L + 3) // 4
+    if args.layer_launches or args.direct_loads or Bq > 1:
+        chain_layers = 1
+    n_launch = -(-L // chain_layers)                                # MLP kernel launches per chain
+    mlp_us = k0.elapsed_time(k1) * 1000.0 / (reps * n_launch)      # per launch, gaps included
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record(s)
     for _ in range(reps):
-        nb.np_predict(eng.ctx, xs_dev[T - 1], 1, None, None, s)
+        nb.np_predict(eng.ctx, xs_dev[T - 1], Bq, None, None, s)
     p1.record(s)
     s.synchronize()
     pred_us = p0.elapsed_time(p1) * 1000.0 / reps
@@ -376,8 +384,12 @@ def cuda_arm(args):
     ms_total, e2e_ms_total = max_over_ranks(dist, [ms_total, e2e_ms_total], dev)
 
     peak, peak_kind = measured_peaks()
-    mlp_bytes = n_active * rec + 4 * n_active + 8 * D            # rows + slot list + x in, y out
+    layer_bytes = n_active * rec + 4 * n_active + 8 * D          # rows + slot list + x in, y out
+    mlp_bytes = layer_bytes * L / n_launch                       # one launch spans L / n_launch layers
     achieved = mlp_bytes / (mlp_us * 1e-6) / 1e9
+    # DRAM bytes of one layer from the ncu capture in profiles/k_mlp_chain_7b.md (7B shape):
+    # (216.63 MB read + 3.82 MB written) / 8 layers; scaled by the layers a launch spans
+    traffic = 27.56e6 * L / n_launch if cfg.name == "7b" else None
     pred_bytes = 2 * cfg.d_pred * D + 2 * L * M * cfg.d_pred + 4 * L * M
     mean_delta = float(np.mean(delta_rows))
     result = {
@@ -386,26 +398,28 @@ def cuda_arm(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
-                        f"B=1 rho={cfg.rho} policy={args.policy} transfer={args.transfer}",
+                        f"B={Bq} rho={cfg.rho} policy={args.policy} transfer={args.transfer}",
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
             "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
+            "active_rows_per_layer": n_active, "overflow_steps": int(overflow_steps),
             "replicas": world,
         },
         "e2e": {"value": K * world / (e2e_ms_total / 1000.0), "unit": UNIT,
-                "h2d_bytes_per_step": int(D * 2 + mean_delta * L * rec), "d2h_bytes_per_step": int(D * 4)},
+                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * L * rec), "d2h_bytes_per_step": int(Bq * D * 4)},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "k_sparse_mlp", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
-                     "us_per_launch": mlp_us, "bytes_per_launch": mlp_bytes},
+        "roofline": {"bound": "hbm", "kernel": "k_mlp_chain" if chain_layers > 1 else "k_sparse_mlp_pipe", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth (burst)",
+                     "traffic": traffic, "us_per_launch": mlp_us, "bytes_per_launch": mlp_bytes,
+                     "layers_per_launch": L / n_launch},
         "stages_us": {"predict_topk": float(stage_us[0]), "delta": float(stage_us[1]),
                       "install_copy_stream": float(stage_us[2]), "mlp_chain_incl_waits": float(stage_us[3]),
                       "predict_alone": pred_us, "predict_gbs": pred_bytes / (pred_us * 1e-6) / 1e9,
-                      "mlp_chain_alone": mlp_us * L},
+                      "mlp_chain_alone": mlp_us * n_launch},
         "setup_s": {"generate": gen_s},
     }
 
-    if rank == 0 and not args.no_cpu_baseline and world == 1:
+    if rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1:
         n = args.cpu_baseline_steps
         times = run_oracle_steps(cfg, args.policy, w1.cpu(), w2.cpu(), store, xs_host, n)
         sec = float(np.mean(times))
