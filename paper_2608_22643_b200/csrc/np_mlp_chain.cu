@@ -33,7 +33,7 @@ constexpr int kChainWarps = 16;                      // consumer warps
 constexpr int kChainThreads = kChainWarps * 32;      // consumer threads
 constexpr int kChainBlock = kChainThreads + 32;      // plus one producer warp
 constexpr int kChainMaxStages = 16;
-constexpr int kChainMaxRpw = 2;   // rows a warp may take per tile in phase 1
+constexpr int kChainTileRows = 8;  // rows per tile: with their gate and up rows, the 16 rows of one MMA
 constexpr int kChainMaxLayers = 128;  // layers per launch (longer runs are split by the host)
 
 struct ChainKernelArgs {
@@ -47,7 +47,7 @@ struct ChainKernelArgs {
                                // into copy g % kZRep (fewer adds per address), readers sum the copies
   unsigned int* grid_bar;      // zeroed by the host before the launch
   int32_t* status;
-  int l_begin, l_end, D, C, n_stages, tile_rows, rows_per_warp, check;
+  int l_begin, l_end, D, C, n_stages, tile_rows, check;
   int slot_cache_rows;         // capacity of the per-block slot cache (rows)
   int window_rows;             // records in flight per block (< n_stages)
 };
@@ -67,13 +67,41 @@ __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, 
                : "memory");
 }
 
-template <int XJ, int COLS>
+// mma.sync m16n8k16, bf16 x bf16 -> fp32 (the 16 x 16 A tile holds 8 gate rows and 8 up rows)
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(npp::smem_addr(smem_row)));
+}
+
+// fp32 -> three bf16 terms by truncation: v = t0 + t1 + t2 up to 2^-24 |v|; returns the terms
+// as fp32 values whose low 16 bits are zero
+__device__ __forceinline__ void split3(float v, uint32_t& t0, uint32_t& t1, uint32_t& t2) {
+  t0 = __float_as_uint(v) & 0xffff0000u;
+  const float r1 = v - __uint_as_float(t0);
+  t1 = __float_as_uint(r1) & 0xffff0000u;
+  const float r2 = r1 - __uint_as_float(t1);
+  t2 = __float_as_uint(r2) & 0xffff0000u;
+}
+// two truncated terms -> one packed bf16x2 word (first element in the low half)
+__device__ __forceinline__ uint32_t pack_hi16(uint32_t first, uint32_t second) {
+  return __byte_perm(first, second, 0x7632);
+}
+
+template <int COLS>
 __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a) {
   extern __shared__ __align__(128) unsigned char csm[];
   __shared__ __align__(8) uint64_t full_bar[kChainMaxStages];   // a stage's record has landed
   __shared__ __align__(8) uint64_t empty_bar[kChainMaxStages];  // every consumer warp is done with it
-  __shared__ float part[kChainMaxRpw * kChainWarps][2];  // (g, u) partial sums of the tile's (row, segment) items
-  __shared__ float act[kChainMaxRpw * kChainWarps];      // a_i of the tile's rows
+  __shared__ float part[kChainWarps][16];       // per warp: partial gate (0-7) and up (8-15) sums of the tile's rows
+  __shared__ float act[kChainTileRows];         // a_i of the tile's rows
   __shared__ float ssq_part[kChainWarps];       // per-warp sums of x_l^2 (for the RMS normalisation)
   __shared__ int s_ok;
   __shared__ int lay_rb[kChainMaxLayers];       // first active-list index of this block, per layer
@@ -82,14 +110,16 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   const int D = a.D, chunks = D >> 3;
   const uint32_t row_bytes = (uint32_t)D * 2u;
   const uint32_t rec_bytes = 3u * row_bytes;
+  // stages are 16 bytes further apart than a record, so that the same column of the rows of
+  // consecutive stages falls into different shared-memory banks (ldmatrix reads 8 rows at once)
+  const uint32_t stage_stride = rec_bytes + 16u;
+  const uint32_t term_stride = row_bytes + 16u;  // the three bf16 terms of x, staggered the same way
   const size_t layer_bytes = (size_t)a.C * row_bytes;
-  // a tile is TR = RPW * (16 / SEG) rows: phase 1 gives every warp RPW (row, segment) items
-  const int n_stages = a.n_stages, RPW = a.rows_per_warp, TR = a.tile_rows, SEG = kChainWarps * RPW / TR;
-  const int seg_chunks = (chunks + SEG - 1) / SEG;
+  const int n_stages = a.n_stages, TR = a.tile_rows;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int G = gridDim.x, nl = a.l_end - a.l_begin;
-  float* xs = reinterpret_cast<float*>(csm + (size_t)n_stages * rec_bytes);  // x_l, fp32 [D], kept across layers
-  int* slot_cache = reinterpret_cast<int*>(xs + D);                         // this block's slots, virtual row order
+  unsigned char* xsp = csm + (size_t)n_stages * stage_stride;               // x_l as 3 bf16 terms, [3][D] (+ stagger)
+  int* slot_cache = reinterpret_cast<int*>(xsp + 3 * (size_t)term_stride);  // this block's slots, virtual row order
 
   // ---- this block's share of every layer of the run ----
   if (tid < nl) {
@@ -163,7 +193,7 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
         }
         while (v >= lay_pre[ll + 1]) ++ll;
         const size_t off = (size_t)(a.l_begin + ll) * layer_bytes + (size_t)slot_cache[v] * row_bytes;
-        unsigned char* dst = csm + (size_t)s * rec_bytes;
+        unsigned char* dst = csm + (size_t)s * stage_stride;
         npp::mbar_expect_tx(&full_bar[s], rec_bytes);
         npp::bulk_g2s(dst, a.gate + off, row_bytes, &full_bar[s]);
         npp::bulk_g2s(dst + row_bytes, a.up + off, row_bytes, &full_bar[s]);
@@ -178,9 +208,13 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   }
 
   // =========================== consumer warps ===========================
-  const int sg = wid % SEG, row_in_tile = wid / SEG;
-  const int c_lo = sg * seg_chunks, c_hi = min(chunks, c_lo + seg_chunks);
   const int l_last = a.l_end - 1;
+  const int g8 = lane >> 2, t4 = lane & 3;  // mma fragment coordinates of this lane
+  // phase 1 splits the K dimension (D, in blocks of 16) evenly over the consumer warps
+  const int kblocks = D >> 4;
+  const int kb_lo = (int)(((long long)kblocks * wid) / kChainWarps), kb_hi = (int)(((long long)kblocks * (wid + 1)) / kChainWarps);
+  // x_l lives in registers: this thread owns float4 granules tid, tid + 512, ... for the whole run
+  float4 xown[2 * COLS];
 
   for (int li = 0; li < nl; ++li) {
     const int l = a.l_begin + li;
@@ -205,47 +239,55 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       consumer_sync();
       if (!s_ok) break;
     }
-    // ---- x_l: first layer of the run from global, afterwards x_l = x_{l-1} + MLP_{l-1} ----
+    // ---- x_l: first layer of the run from global, afterwards x_l = x_{l-1} + MLP_{l-1};
+    //      each thread updates its own granules and publishes them as three bf16 terms ----
     {
       const float* xa = a.xbuf[(l + 1) & 1];
       const float* zb = l > 0 ? a.zbuf[(l - 1) % 3] : nullptr;
       float* xst = a.xbuf[l & 1];
       const int nf4 = chunks * 2;  // float4 granules of one vector
       float ssq = 0.f;
-      for (int c0 = tid; c0 < nf4; c0 += 2 * kChainThreads) {
-        // all loads of two granules (and of every accumulator copy) are issued before any is used
-        const int c1 = c0 + kChainThreads;
-        const bool has1 = c1 < nf4;
-        float4 w0[kZRep], w1[kZRep];
-        if (zb) {
+      float4 w[2 * COLS][kZRep];
+      // every load of the pass is issued before any is used
 #pragma unroll
-          for (int r = 0; r < kZRep; ++r) {
-            w0[r] = ldcg4(zb + (size_t)r * D + (size_t)c0 * 4);
-            w1[r] = has1 ? ldcg4(zb + (size_t)r * D + (size_t)c1 * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int i = 0; i < 2 * COLS; ++i) {
+        const int c = tid + i * kChainThreads;
+        if (c < nf4) {
+          if (li == 0) xown[i] = ldcg4(xa + (size_t)c * 4);
+          if (zb) {
+#pragma unroll
+            for (int r = 0; r < kZRep; ++r) w[i][r] = ldcg4(zb + (size_t)r * D + (size_t)c * 4);
           }
-        }
-        float4 v0, v1 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (li == 0) {
-          v0 = ldcg4(xa + (size_t)c0 * 4);
-          if (has1) v1 = ldcg4(xa + (size_t)c1 * 4);
         } else {
-          v0 = reinterpret_cast<float4*>(xs)[c0];
-          if (has1) v1 = reinterpret_cast<float4*>(xs)[c1];
+          xown[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        if (zb) {
+      }
 #pragma unroll
-          for (int r = 0; r < kZRep; ++r) {
-            v0.x += w0[r].x; v0.y += w0[r].y; v0.z += w0[r].z; v0.w += w0[r].w;
-            v1.x += w1[r].x; v1.y += w1[r].y; v1.z += w1[r].z; v1.w += w1[r].w;
+      for (int i = 0; i < 2 * COLS; ++i) {
+        const int c = tid + i * kChainThreads;
+        if (c < nf4) {
+          float4 v = xown[i];
+          if (zb) {
+#pragma unroll
+            for (int r = 0; r < kZRep; ++r) {
+              v.x += w[i][r].x; v.y += w[i][r].y; v.z += w[i][r].z; v.w += w[i][r].w;
+            }
           }
-        }
-        reinterpret_cast<float4*>(xs)[c0] = v0;
-        if (has1) reinterpret_cast<float4*>(xs)[c1] = v1;
-        ssq += v0.x * v0.x + v0.y * v0.y + v0.z * v0.z + v0.w * v0.w;
-        ssq += v1.x * v1.x + v1.y * v1.y + v1.z * v1.z + v1.w * v1.w;  // zeros when there is no second granule
-        if (blockIdx.x == 0 && l == l_last) {  // x for the next launch
-          reinterpret_cast<float4*>(xst)[c0] = v0;
-          if (has1) reinterpret_cast<float4*>(xst)[c1] = v1;
+          xown[i] = v;
+          ssq += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+          uint32_t p0[3], p1[3], p2[3], p3[3];
+          split3(v.x, p0[0], p0[1], p0[2]);
+          split3(v.y, p1[0], p1[1], p1[2]);
+          split3(v.z, p2[0], p2[1], p2[2]);
+          split3(v.w, p3[0], p3[1], p3[2]);
+#pragma unroll
+          for (int term = 0; term < 3; ++term) {
+            uint2 packed;
+            packed.x = pack_hi16(p0[term], p1[term]);
+            packed.y = pack_hi16(p2[term], p3[term]);
+            *reinterpret_cast<uint2*>(xsp + (size_t)term * term_stride + (size_t)c * 8) = packed;
+          }
+          if (blockIdx.x == 0 && l == l_last) reinterpret_cast<float4*>(xst)[c] = v;  // x for the next launch
         }
       }
       ssq = warp_sum(ssq);
@@ -257,19 +299,6 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       for (int c = zlo + tid; c < zhi; c += kChainThreads) znext[c] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     consumer_sync();
-    float xr[XJ][8];
-#pragma unroll
-    for (int j = 0; j < XJ; ++j) {
-      const int c = c_lo + lane + 32 * j;
-      if (c < c_hi) {
-        const float4 v0 = reinterpret_cast<const float4*>(xs)[2 * c], v1 = reinterpret_cast<const float4*>(xs)[2 * c + 1];
-        xr[j][0] = v0.x; xr[j][1] = v0.y; xr[j][2] = v0.z; xr[j][3] = v0.w;
-        xr[j][4] = v1.x; xr[j][5] = v1.y; xr[j][6] = v1.z; xr[j][7] = v1.w;
-      } else {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) xr[j][e] = 0.f;
-      }
-    }
 
     float acc[COLS][8];
 #pragma unroll
@@ -282,62 +311,69 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       const int rows = min(TR, nrows - t0);
       const int s0 = (vbase + t0) % n_stages;  // stage of the tile's first row; the rest follow, wrapping
       const uint32_t use0 = (uint32_t)((vbase + t0) / n_stages);
-      // ---- phase 1: (row, segment) partial dot products from shared memory ----
-      for (int rr = 0; rr < RPW; ++rr) {
-        const int row = row_in_tile + rr * (TR / RPW);
-        if (row >= rows) break;
-        int s = s0 + row;
+      // ---- phase 1 on the tensor cores: [8 gate rows; 8 up rows] x [x as 3 bf16 terms] over this
+      //      warp's K range.  Every warp reads all rows of the tile, so it waits for all of them. ----
+      {
+        int s = s0;
         uint32_t use = use0;
-        if (s >= n_stages) {
-          s -= n_stages;
-          ++use;
-        }
-        if (!npp::mbar_wait(&full_bar[s], use & 1u)) {
-          if (lane == 0) {
-            atomicOr(a.status, npp::kStatTimeout);
-            s_ok = 0;
-          }
-        }
-        const uint4* gp = reinterpret_cast<const uint4*>(csm + (size_t)s * rec_bytes);
-        const uint4* up = gp + chunks;
-        float g0 = 0.f, g1 = 0.f, u0 = 0.f, u1 = 0.f;  // two chains each: the FMAs of a dot product are dependent
-#pragma unroll
-        for (int j = 0; j < XJ; ++j) {
-          const int c = c_lo + lane + 32 * j;
-          if (c < c_hi) {
-            const uint4 gw = gp[c], uw = up[c];
-            const float4 x0 = make_float4(xr[j][0], xr[j][1], xr[j][2], xr[j][3]);
-            const float4 x1 = make_float4(xr[j][4], xr[j][5], xr[j][6], xr[j][7]);
-            if (j & 1) {
-              g1 = dot8(gw, x0, x1, g1);
-              u1 = dot8(uw, x0, x1, u1);
-            } else {
-              g0 = dot8(gw, x0, x1, g0);
-              u0 = dot8(uw, x0, x1, u0);
+        for (int q = 0; q < rows; ++q) {
+          if (!npp::mbar_wait(&full_bar[s], use & 1u)) {
+            if (lane == 0) {
+              atomicOr(a.status, npp::kStatTimeout);
+              s_ok = 0;
             }
           }
+          if (++s == n_stages) {
+            s = 0;
+            ++use;
+          }
         }
-        float g = g0 + g1, u = u0 + u1;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          g += __shfl_xor_sync(0xffffffffu, g, o);
-          u += __shfl_xor_sync(0xffffffffu, u, o);
+      }
+      {
+        // ldmatrix: lanes 8m..8m+7 give the row addresses of 8x8 matrix m; m & 1 picks up
+        // (rows 8-15 of A) over gate, m >> 1 the second 8 columns of the 16-wide K block
+        const int m = lane >> 3;
+        int r = lane & 7;
+        if (r >= rows) r = 0;  // rows past the tile's end: any valid address, results unused
+        int sr = s0 + r;
+        if (sr >= n_stages) sr -= n_stages;
+        const unsigned char* arow = csm + (size_t)sr * stage_stride + (size_t)(m & 1) * row_bytes + (size_t)(m >> 1) * 16;
+        const unsigned char* brow = xsp + (size_t)(g8 < 3 ? g8 : 0) * term_stride + (size_t)t4 * 4;
+        float c4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
+          uint32_t af[4];
+          ldmatrix_x4(af, arow + (size_t)kb * 32);
+          uint32_t b0 = 0u, b1 = 0u;
+          if (g8 < 3) {  // column n of B is term n of x; columns 3-7 are zero
+            b0 = *reinterpret_cast<const uint32_t*>(brow + (size_t)kb * 32);
+            b1 = *reinterpret_cast<const uint32_t*>(brow + (size_t)kb * 32 + 16);
+          }
+          mma_bf16_16816(c4, af, b0, b1);
         }
-        if (lane == 0) {
-          part[row * SEG + sg][0] = g;
-          part[row * SEG + sg][1] = u;
+        // C: c4[0], c4[1] = (row g8, columns 2*t4, 2*t4+1); c4[2], c4[3] = (row g8 + 8, same columns).
+        // The three terms sit in columns 0, 1 (lane t4 = 0) and 2 (lane t4 = 1).
+        float lo = t4 == 0 ? c4[0] + c4[1] : (t4 == 1 ? c4[0] : 0.f);
+        float hi = t4 == 0 ? c4[2] + c4[3] : (t4 == 1 ? c4[2] : 0.f);
+        lo += __shfl_xor_sync(0xffffffffu, lo, 1);
+        hi += __shfl_xor_sync(0xffffffffu, hi, 1);
+        if (t4 == 0) {
+          part[wid][g8] = lo;      // gate . x over this warp's K range, tile row g8
+          part[wid][8 + g8] = hi;  // up . x
         }
       }
       consumer_sync();
       if (!s_ok) break;
       if (tid < rows) {
         float gs = 0.f, us = 0.f;
-        for (int w = 0; w < SEG; ++w) {
-          gs += part[tid * SEG + w][0];
-          us += part[tid * SEG + w][1];
+#pragma unroll
+        for (int w = 0; w < kChainWarps; ++w) {
+          gs += part[w][tid];
+          us += part[w][8 + tid];
         }
         // the MLP's input is x_l scaled to unit RMS; the dot products are linear in it
         float ss = 0.f;
+#pragma unroll
         for (int w = 0; w < kChainWarps; ++w) ss += ssq_part[w];
         const float inv_rms = rsqrtf(ss / (float)D + kRmsEps);
         gs *= inv_rms;
@@ -350,7 +386,7 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
         int s = s0;
         for (int q = 0; q < rows; ++q) {
           const float av = act[q];
-          const uint4* dp = reinterpret_cast<const uint4*>(csm + (size_t)s * rec_bytes + 2 * row_bytes);
+          const uint4* dp = reinterpret_cast<const uint4*>(csm + (size_t)s * stage_stride + 2 * row_bytes);
 #pragma unroll
           for (int j = 0; j < COLS; ++j) {
             const int c = tid + j * kChainThreads;
@@ -404,9 +440,9 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   }
 }
 
-template <int XJ, int COLS>
+template <int COLS>
 static cudaError_t chain_launch(const ChainKernelArgs& ka, size_t sm, int grid_x, cudaStream_t s) {
-  auto kfn = k_mlp_chain<XJ, COLS>;
+  auto kfn = k_mlp_chain<COLS>;
   cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
   if (e != cudaSuccess) return e;
   int per_sm = 0;
@@ -432,41 +468,33 @@ bool mlp_chain_supported(const Dims& d, int sm_count) {
 }
 
 bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
+  if (d.D % 16) return false;  // phase 1 walks D in MMA K blocks of 16
   const int chunks = d.D >> 3;
-  const size_t rec = (size_t)d.D * 6;
-  // shared memory: ring + x (fp32 [D]) + slot cache, under the 227 KB per-block limit
+  const size_t stage = (size_t)d.D * 6 + 16;      // record + stagger
+  const size_t terms = 3 * ((size_t)d.D * 2 + 16);  // x as three bf16 terms
   const long long expect = std::min<long long>(d.C, d.k);
   const int per_block = (int)std::max<long long>(1, (expect + sm_count - 1) / sm_count);
-  const int max_per_block = d.C / sm_count + 2;   // whatever the active count turns out to be
-  p->run_layers = std::max(1, std::min(kChainMaxLayers, 16384 / (4 * max_per_block)));
+  const int max_per_block = d.C / sm_count + 2;  // whatever the active count turns out to be
+  // slot cache: up to 4 KB of it, which bounds the layers one launch can span
+  p->run_layers = std::max(1, std::min(kChainMaxLayers, 4096 / (4 * max_per_block)));
   p->slot_cache_rows = p->run_layers * max_per_block;
-  const size_t fixed = (size_t)d.D * 4 + (size_t)p->slot_cache_rows * 4;
-  const size_t budget = 227 * 1024 - 4096;  // static shared memory and the driver's reserve
-  if (fixed + 2 * rec > budget) return false;
-  int n_stages = (int)std::min<size_t>(kChainMaxStages, (budget - fixed) / rec);
+  const size_t fixed = terms + (size_t)p->slot_cache_rows * 4;
+  const size_t budget = 227 * 1024 - 3072;  // static shared memory of the kernel
+  if (fixed + 2 * stage > budget) return false;
+  int n_stages = (int)std::min<size_t>(kChainMaxStages, (budget - fixed) / stage);
   if (d.ring_stages >= 2) n_stages = std::min(n_stages, d.ring_stages);
-  int tr = 1;
-  const int tr_cap = std::max(1, std::min(per_block, n_stages) / 2);
-  while (tr * 2 <= tr_cap && tr * 2 <= kChainWarps) tr *= 2;
-  while (tr < kChainWarps && chunks / (kChainWarps / tr) < 32) tr *= 2;
-  if (tr > n_stages) return false;
-  const int seg = kChainWarps / tr;
-  const int seg_chunks = (chunks + seg - 1) / seg;
-  p->xj = (seg_chunks + 31) / 32;
+  // one tile per layer when the block's share fits the ring, else half-ring tiles so that the
+  // next tile's rows arrive while this one is computed
+  int tr = per_block <= n_stages ? std::min(n_stages, kChainTileRows) : std::max(1, std::min(kChainTileRows, n_stages / 2));
   const int need_cols = (chunks + kChainThreads - 1) / kChainThreads;
-  if (p->xj > 8 || need_cols > 4) return false;
+  if (need_cols > 4) return false;
   p->cols = need_cols <= 1 ? 1 : (need_cols <= 2 ? 2 : 4);
-  // when the whole share of a layer fits the ring, take it as one tile: two rows per warp
-  // in phase 1, half the block-wide barriers
+  p->xj = 0;
   p->rows_per_warp = 1;
-  if (d.chain_rpw != 1 && 2 * tr <= n_stages && 2 * tr >= per_block) {
-    p->rows_per_warp = 2;
-    tr *= 2;
-  }
   p->n_stages = n_stages;
   p->tile_rows = tr;
   p->window_rows = 2;
-  p->smem = (size_t)n_stages * rec + fixed;
+  p->smem = (size_t)n_stages * stage + fixed;
   return true;
 }
 
@@ -493,26 +521,12 @@ cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, 
     ka.C = d.C;
     ka.n_stages = p.n_stages;
     ka.tile_rows = p.tile_rows;
-    ka.rows_per_warp = p.rows_per_warp;
     ka.check = a.check;
     e = cudaMemsetAsync(a.grid_bar, 0, sizeof(unsigned int), s);
     if (e != cudaSuccess) return e;
-#define NP_CHAIN(XJV)                                                        \
-  do {                                                                       \
-    if (p.cols == 1) e = chain_launch<XJV, 1>(ka, p.smem, sm_count, s);      \
-    else if (p.cols == 2) e = chain_launch<XJV, 2>(ka, p.smem, sm_count, s); \
-    else e = chain_launch<XJV, 4>(ka, p.smem, sm_count, s);                  \
-  } while (0)
-    switch (p.xj) {
-      case 1: NP_CHAIN(1); break;
-      case 2: NP_CHAIN(2); break;
-      case 3: NP_CHAIN(3); break;
-      case 4: NP_CHAIN(4); break;
-      case 5: NP_CHAIN(5); break;
-      case 6: NP_CHAIN(6); break;
-      default: NP_CHAIN(8); break;
-    }
-#undef NP_CHAIN
+    if (p.cols == 1) e = chain_launch<1>(ka, p.smem, sm_count, s);
+    else if (p.cols == 2) e = chain_launch<2>(ka, p.smem, sm_count, s);
+    else e = chain_launch<4>(ka, p.smem, sm_count, s);
     if (e != cudaSuccess) return e;
   }
   return e;
