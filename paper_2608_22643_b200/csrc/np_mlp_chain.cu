@@ -99,7 +99,7 @@ template <int COLS>
 __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a) {
   extern __shared__ __align__(128) unsigned char csm[];
   __shared__ __align__(8) uint64_t full_bar[kChainMaxStages];   // a stage's record has landed
-  __shared__ __align__(8) uint64_t empty_bar[kChainMaxStages];  // every consumer warp is done with it
+  __shared__ __align__(8) uint64_t empty_bar[kChainMaxStages];  // the consumers are done with it
   __shared__ float part[kChainWarps][16];       // per warp: partial gate (0-7) and up (8-15) sums of the tile's rows
   __shared__ float act[kChainTileRows];         // a_i of the tile's rows
   __shared__ float ssq_part[kChainWarps];       // per-warp sums of x_l^2 (for the RMS normalisation)
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   if (tid == 0) {
     for (int s = 0; s < n_stages; ++s) {
       npp::mbar_init(&full_bar[s], 1);
-      npp::mbar_init(&empty_bar[s], kChainWarps);
+      npp::mbar_init(&empty_bar[s], 1);
     }
     npp::fence_barrier_init();
     s_ok = 1;
@@ -314,20 +314,23 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       // ---- phase 1 on the tensor cores: [8 gate rows; 8 up rows] x [x as 3 bf16 terms] over this
       //      warp's K range.  Every warp reads all rows of the tile, so it waits for all of them. ----
       {
-        int s = s0;
+        // every warp reads all rows of the tile, but each polls only one row's barrier (an
+        // mbarrier poll costs ~0.1 us even when the phase is complete); the block-wide
+        // barrier then publishes all of them
+        const int q = wid % rows;
+        int s = s0 + q;
         uint32_t use = use0;
-        for (int q = 0; q < rows; ++q) {
-          if (!npp::mbar_wait(&full_bar[s], use & 1u)) {
-            if (lane == 0) {
-              atomicOr(a.status, npp::kStatTimeout);
-              s_ok = 0;
-            }
-          }
-          if (++s == n_stages) {
-            s = 0;
-            ++use;
+        if (s >= n_stages) {
+          s -= n_stages;
+          ++use;
+        }
+        if (!npp::mbar_wait(&full_bar[s], use & 1u)) {
+          if (lane == 0) {
+            atomicOr(a.status, npp::kStatTimeout);
+            s_ok = 0;
           }
         }
+        consumer_sync();
       }
       {
         // ldmatrix: lanes 8m..8m+7 give the row addresses of 8x8 matrix m; m & 1 picks up
@@ -404,16 +407,14 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
           }
           if (++s == n_stages) s = 0;
         }
-        // this warp is done with the tile's stages.  (`part` is rewritten only after every warp
-        // has passed the barrier above, `act` only after the next tile's first barrier.)
-        __syncwarp();
-        if (lane == 0) {
-          s = s0;
-          for (int q = 0; q < rows; ++q) {
-            npp::mbar_arrive(&empty_bar[s]);
-            if (++s == n_stages) s = 0;
-          }
-        }
+      }
+      // every warp is done with the tile's stages: one thread per row releases its stage (a single
+      // arrival per stage instead of one per warp keeps the barrier unit out of the way)
+      consumer_sync();
+      if (tid < rows) {
+        int s = s0 + tid;
+        if (s >= n_stages) s -= n_stages;
+        npp::mbar_arrive(&empty_bar[s]);
       }
     }
     if (!s_ok) break;
