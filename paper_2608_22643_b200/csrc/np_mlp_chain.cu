@@ -298,6 +298,20 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
       const int zlo = (int)(((long long)ztotal * blockIdx.x) / G), zhi = (int)(((long long)ztotal * (blockIdx.x + 1)) / G);
       for (int c = zlo + tid; c < zhi; c += kChainThreads) znext[c] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    // this warp's share of the wait for the layer's first tile rides on the same barrier
+    const int vbase = lay_pre[li], nrows = min(lay_pre[li + 1], total_rows) - vbase;
+    auto poll_tile_row = [&](int t0, int rows) {
+      // every warp reads all rows of a tile, but each polls only one row's barrier (an mbarrier
+      // poll costs ~0.1 us even when the phase is complete); a block-wide barrier publishes them
+      const int v = vbase + t0 + wid % rows;
+      if (!npp::mbar_wait(&full_bar[v % n_stages], (uint32_t)(v / n_stages) & 1u)) {
+        if (lane == 0) {
+          atomicOr(a.status, npp::kStatTimeout);
+          s_ok = 0;
+        }
+      }
+    };
+    if (nrows > 0) poll_tile_row(0, min(TR, nrows));
     consumer_sync();
 
     float acc[COLS][8];
@@ -306,30 +320,13 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
 
-    const int vbase = lay_pre[li], nrows = min(lay_pre[li + 1], total_rows) - vbase;
     for (int t0 = 0; t0 < nrows; t0 += TR) {
       const int rows = min(TR, nrows - t0);
       const int s0 = (vbase + t0) % n_stages;  // stage of the tile's first row; the rest follow, wrapping
-      const uint32_t use0 = (uint32_t)((vbase + t0) / n_stages);
       // ---- phase 1 on the tensor cores: [8 gate rows; 8 up rows] x [x as 3 bf16 terms] over this
       //      warp's K range.  Every warp reads all rows of the tile, so it waits for all of them. ----
-      {
-        // every warp reads all rows of the tile, but each polls only one row's barrier (an
-        // mbarrier poll costs ~0.1 us even when the phase is complete); the block-wide
-        // barrier then publishes all of them
-        const int q = wid % rows;
-        int s = s0 + q;
-        uint32_t use = use0;
-        if (s >= n_stages) {
-          s -= n_stages;
-          ++use;
-        }
-        if (!npp::mbar_wait(&full_bar[s], use & 1u)) {
-          if (lane == 0) {
-            atomicOr(a.status, npp::kStatTimeout);
-            s_ok = 0;
-          }
-        }
+      if (t0 > 0) {
+        poll_tile_row(t0, rows);
         consumer_sync();
       }
       {
@@ -409,12 +406,15 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
         }
       }
       // every warp is done with the tile's stages: one thread per row releases its stage (a single
-      // arrival per stage instead of one per warp keeps the barrier unit out of the way)
-      consumer_sync();
-      if (tid < rows) {
-        int s = s0 + tid;
-        if (s >= n_stages) s -= n_stages;
-        npp::mbar_arrive(&empty_bar[s]);
+      // arrival per stage instead of one per warp keeps the barrier unit out of the way).  The
+      // layer's last tile is released after the reductions below, on their barrier.
+      if (t0 + TR < nrows) {
+        consumer_sync();
+        if (tid < rows) {
+          int s = s0 + tid;
+          if (s >= n_stages) s -= n_stages;
+          npp::mbar_arrive(&empty_bar[s]);
+        }
       }
     }
     if (!s_ok) break;
@@ -433,6 +433,10 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
     }
     if (li + 1 < nl) {  // publish: every thread's adds and stores precede the arrival
       consumer_sync();
+      if (nrows > 0) {  // release the stages of the layer's last tile
+        const int t_last = ((nrows - 1) / TR) * TR;
+        if (tid < nrows - t_last) npp::mbar_arrive(&empty_bar[(vbase + t_last + tid) % n_stages]);
+      }
       if (tid == 0) {
         __threadfence();
         atomicAdd(a.grid_bar, 1u);
