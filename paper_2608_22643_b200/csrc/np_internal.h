@@ -49,7 +49,6 @@ struct Workspace {
 struct Dims {
   int L, D, M, H, k, C, W, Bmax;
   int ring_stages;  // cap on shared-memory ring stages of the MLP kernels (0 = as many as fit)
-  int chain_rpw;    // 1: never give a warp two rows per tile in the resident MLP kernel (tuning)
   size_t rec_bytes;
 };
 
@@ -108,10 +107,10 @@ cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, i
 
 // Persistent multi-layer form of the sparse MLP for one sequence (np_mlp_chain.cu).
 struct ChainPlan {
-  int n_stages, tile_rows, rows_per_warp, xj, cols;
+  int n_stages, tile_rows, cols;
   int run_layers;       // layers one launch can span (bounded by the slot cache)
   int slot_cache_rows;
-  int window_rows;      // records in flight per block
+  int window_rows;      // records in flight per block (producer pacing)
   size_t smem;
 };
 struct ChainArgs {

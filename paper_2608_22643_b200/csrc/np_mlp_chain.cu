@@ -18,6 +18,13 @@
 // the all-reduce of the 4*D-byte output across the blocks (flush of the
 // reductions, barrier, re-read of the accumulators) and the two compute phases.
 //
+// Phase 1 (gate and up dot products of the tile's rows) is on the layer's critical path and
+// was issue-bound on the ALUs (an unpack and an FMA per bf16 element), so it runs as
+// mma.sync m16n8k16: A = 8 gate rows + 8 up rows read with ldmatrix from the ring (stages are
+// staggered by 16 bytes against bank conflicts), B = x_l as three truncated bf16 terms
+// (exact to 2^-24), K split over the 16 consumer warps.  Phase 2 (down rows) stays on the
+// ALUs: thread c owns 8 output columns.  x_l itself lives in registers, 8 floats per thread.
+//
 // Every wait (mbarrier, grid barrier) is bounded; on expiry the block records
 // kStatTimeout and leaves, and the other blocks follow at their next barrier.
 #include <algorithm>
@@ -494,8 +501,6 @@ bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
   const int need_cols = (chunks + kChainThreads - 1) / kChainThreads;
   if (need_cols > 4) return false;
   p->cols = need_cols <= 1 ? 1 : (need_cols <= 2 ? 2 : 4);
-  p->xj = 0;
-  p->rows_per_warp = 1;
   p->n_stages = n_stages;
   p->tile_rows = tr;
   p->window_rows = 2;
