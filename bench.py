@@ -388,8 +388,8 @@ def cuda_arm(args):
     mlp_bytes = layer_bytes * L / n_launch                       # one launch spans L / n_launch layers
     achieved = mlp_bytes / (mlp_us * 1e-6) / 1e9
     # DRAM bytes of one layer from the ncu capture in profiles/k_mlp_chain_7b.md (7B shape):
-    # (216.63 MB read + 3.82 MB written) / 8 layers; scaled by the layers a launch spans
-    traffic = 27.56e6 * L / n_launch if cfg.name == "7b" else None
+    # (216.63 MB read + 3.51 MB written) / 8 layers; scaled by the layers a launch spans
+    traffic = 27.52e6 * L / n_launch if cfg.name == "7b" else None
     pred_bytes = 2 * cfg.d_pred * D + 2 * L * M * cfg.d_pred + 4 * L * M
     mean_delta = float(np.mean(delta_rows))
     result = {
