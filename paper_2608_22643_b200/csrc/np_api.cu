@@ -12,6 +12,10 @@
 #include <mutex>
 #include <new>
 #include <thread>
+#if defined(__SSE2__)
+#include <emmintrin.h>
+#include <xmmintrin.h>
+#endif
 
 #include "np_internal.h"
 
@@ -22,6 +26,31 @@ namespace {
 thread_local std::string g_last_error = "";
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Packs one record into pinned staging.  The staging lines are written once and read next by
+// the copy engine, never by this core: non-temporal stores skip the read-for-ownership a
+// cached store would cost (both pointers are 16-byte aligned, n a multiple of 16).
+void copy_record_streaming(void* dst, const void* src, size_t n) {
+#if defined(__SSE2__)
+  const __m128i* s = static_cast<const __m128i*>(src);
+  __m128i* d = static_cast<__m128i*>(dst);
+  const size_t m = n / 16;
+  size_t i = 0;
+  for (; i + 4 <= m; i += 4) {
+    _mm_prefetch(reinterpret_cast<const char*>(s + i) + 512, _MM_HINT_NTA);
+    const __m128i a = _mm_load_si128(s + i), b = _mm_load_si128(s + i + 1);
+    const __m128i c = _mm_load_si128(s + i + 2), e = _mm_load_si128(s + i + 3);
+    _mm_stream_si128(d + i, a);
+    _mm_stream_si128(d + i + 1, b);
+    _mm_stream_si128(d + i + 2, c);
+    _mm_stream_si128(d + i + 3, e);
+  }
+  for (; i < m; ++i) _mm_stream_si128(d + i, _mm_load_si128(s + i));
+  _mm_sfence();
+#else
+  memcpy(dst, src, n);
+#endif
+}
 
 // Small fork-join pool for packing records into pinned staging.  A step issues one short
 // job per layer, tens of microseconds apart, so idle workers spin on the job counter for a
@@ -421,7 +450,11 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
 
   if (cfg->transfer_mode == NP_XFER_HOST_GATHER) {
     int n = cfg->host_threads;
-    if (n == 0) n = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
+    if (n == 0) {
+      // leave a few cores to the caller's thread, the driver and the copy engine's interrupts
+      const unsigned hc = std::thread::hardware_concurrency();
+      n = (int)std::max(1u, std::min(16u, hc > 8 ? hc - 4 : hc));
+    }
     ctx->pool = new (std::nothrow) Pool(n - 1);  // the caller's thread works too
   }
   *out = ctx;
@@ -583,7 +616,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
               bad = true;
               continue;
             }
-            memcpy(hbuf + (size_t)r * rec, store_l + (size_t)id * rec, rec);
+            copy_record_streaming(hbuf + (size_t)r * rec, store_l + (size_t)id * rec, rec);
           }
         };
         if (ctx->pool) ctx->pool->parallel_for(parts, body);
