@@ -61,6 +61,46 @@ __global__ void __launch_bounds__(128) k_pred_l1(const uint4* __restrict__ w1,
   }
 }
 
+// Batched form (B > 4): the B input vectors are staged once per block in shared memory (as
+// bf16), so that a weight chunk is multiplied with all sequences without going back to L1/L2
+// for x; one warp per output row.
+__global__ void __launch_bounds__(128) k_pred_l1_batch(const uint4* __restrict__ w1, const uint4* __restrict__ x,
+                                                        float* __restrict__ hidden, int H, int D, int B) {
+  extern __shared__ __align__(16) uint4 xsm[];  // [B][D/8]
+  npp::pdl_launch_dependents();
+  const int chunks = D >> 3;
+  for (int i = threadIdx.x; i < B * chunks; i += blockDim.x) xsm[i] = __ldg(x + i);
+  __syncthreads();
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= H) return;
+  const uint4* row = w1 + (size_t)warp * chunks;
+  float acc[kMaxBatch];
+#pragma unroll
+  for (int b = 0; b < kMaxBatch; ++b) acc[b] = 0.f;
+  for (int c0 = lane; c0 < chunks; c0 += 64) {
+    const int c1 = c0 + 32;
+    const uint4 wa = ldg_stream(row + c0);
+    const uint4 wb = c1 < chunks ? ldg_stream(row + c1) : make_uint4(0, 0, 0, 0);
+    const float4 wa0 = make_float4(bf16_lo(wa.x), bf16_hi(wa.x), bf16_lo(wa.y), bf16_hi(wa.y));
+    const float4 wa1 = make_float4(bf16_lo(wa.z), bf16_hi(wa.z), bf16_lo(wa.w), bf16_hi(wa.w));
+    const float4 wb0 = make_float4(bf16_lo(wb.x), bf16_hi(wb.x), bf16_lo(wb.y), bf16_hi(wb.y));
+    const float4 wb1 = make_float4(bf16_lo(wb.z), bf16_hi(wb.z), bf16_lo(wb.w), bf16_hi(wb.w));
+#pragma unroll
+    for (int b = 0; b < kMaxBatch; ++b) {
+      if (b < B) {
+        acc[b] = dot8(xsm[(size_t)b * chunks + c0], wa0, wa1, acc[b]);
+        if (c1 < chunks) acc[b] = dot8(xsm[(size_t)b * chunks + c1], wb0, wb1, acc[b]);
+      }
+    }
+  }
+#pragma unroll
+  for (int b = 0; b < kMaxBatch; ++b) {
+    const float v = warp_sum(acc[b]);
+    if (lane == 0 && b < B) hidden[(size_t)b * H + warp] = fmaxf(v, 0.f);
+  }
+}
+
 cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, int B, float* hidden,
                            cudaStream_t s) {
   const int threads = 128;
@@ -71,8 +111,16 @@ cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, in
     k_pred_l1<1><<<blocks, threads, 0, s>>>(w, x, hidden, d.H, d.D, B);
   else if (B <= 4)
     k_pred_l1<4><<<blocks, threads, 0, s>>>(w, x, hidden, d.H, d.D, B);
-  else
-    k_pred_l1<16><<<blocks, threads, 0, s>>>(w, x, hidden, d.H, d.D, B);
+  else {
+    const size_t sm = (size_t)B * d.D * 2;
+    if (sm <= 200 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(k_pred_l1_batch, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+      if (e != cudaSuccess) return e;
+      k_pred_l1_batch<<<blocks, threads, sm, s>>>(w, x, hidden, d.H, d.D, B);
+    } else {
+      k_pred_l1<16><<<blocks, threads, 0, s>>>(w, x, hidden, d.H, d.D, B);
+    }
+  }
   return cudaGetLastError();
 }
 
