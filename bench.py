@@ -55,6 +55,7 @@ def parse_args():
     ap.add_argument("--layer-launches", action="store_true", help="one MLP kernel launch per layer")
     ap.add_argument("--direct-loads", action="store_true", help="MLP rows by plain global loads")
     ap.add_argument("--chain-layers", type=int, default=0, help="layers per resident MLP kernel")
+    ap.add_argument("--capacity-pct", type=int, default=None, help="resident capacity in percent of FFN rows")
     ap.add_argument("--batch", type=int, default=1, help="sequences per step (the metric's workload is 1)")
     ap.add_argument("--gamma", type=float, default=0.9, help="shared-driver weight of batched hidden states")
     ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
@@ -266,6 +267,8 @@ def cuda_arm(args):
     cfg = synth.CONFIGS[args.config]
     if args.rho is not None:
         cfg = cfg.with_(rho=args.rho)
+    if args.capacity_pct is not None:
+        cfg = cfg.with_(capacity_pct=args.capacity_pct)
     cfg = replica_config(cfg, rank)
     K, W = args.steps, args.warmup
     if W < 3:

@@ -108,6 +108,7 @@ cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, i
 // Persistent multi-layer form of the sparse MLP for one sequence (np_mlp_chain.cu).
 struct ChainPlan {
   int n_stages, tile_rows, cols;
+  int single_tile;      // the block's expected share of a layer fits the ring as one tile
   int run_layers;       // layers one launch can span (bounded by the slot cache)
   int slot_cache_rows;
   int window_rows;      // records in flight per block (producer pacing)
@@ -128,6 +129,10 @@ struct ChainArgs {
 bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p);
 bool mlp_chain_supported(const Dims& d, int sm_count);
 cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
+namespace chain_alu {  // ALU form of phase 1, for shares that do not fit the ring as one tile (np_mlp_chain_alu.cu)
+bool supported(const Dims& d, int sm_count);
+cudaError_t launch(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
+}  // namespace chain_alu
 
 cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s);
 // out = a + sum of `reps` consecutive copies of b (each n floats)

@@ -476,7 +476,7 @@ static cudaError_t chain_launch(const ChainKernelArgs& ka, size_t sm, int grid_x
 
 bool mlp_chain_supported(const Dims& d, int sm_count) {
   ChainPlan p;
-  return mlp_chain_plan(d, sm_count, &p);
+  return mlp_chain_plan(d, sm_count, &p) || chain_alu::supported(d, sm_count);
 }
 
 bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
@@ -501,6 +501,7 @@ bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
   const int need_cols = (chunks + kChainThreads - 1) / kChainThreads;
   if (need_cols > 4) return false;
   p->cols = need_cols <= 1 ? 1 : (need_cols <= 2 ? 2 : 4);
+  p->single_tile = per_block <= std::min(n_stages, kChainTileRows) ? 1 : 0;
   p->n_stages = n_stages;
   p->tile_rows = tr;
   p->window_rows = 2;
@@ -510,7 +511,10 @@ bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p) {
 
 cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count) {
   ChainPlan p;
-  if (!mlp_chain_plan(d, sm_count, &p)) return cudaErrorInvalidValue;
+  const bool mma_ok = mlp_chain_plan(d, sm_count, &p);
+  // the tensor-core form pays a fixed price per tile: keep it for shares that are one tile
+  if ((!mma_ok || !p.single_tile) && chain_alu::supported(d, sm_count)) return chain_alu::launch(d, a, s, sm_count);
+  if (!mma_ok) return cudaErrorInvalidValue;
   cudaError_t e = cudaSuccess;
   for (int l0 = a.l_begin; l0 < a.l_end; l0 += p.run_layers) {
     ChainKernelArgs ka;
