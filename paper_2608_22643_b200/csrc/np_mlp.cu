@@ -576,8 +576,10 @@ cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, i
     int xj = 0, cols = 0;
     if (mlp_pipe_plan(d, sm_count, &pa, &sm, &xj, &cols)) return mlp_pipe_dispatch(pa, sm, xj, cols, sm_count, s);
   }
-  if (a.B == 1) return mlp_launch_nb<1>(ka, 1, sm_count, s);
-  if (a.B == 2) return mlp_launch_nb<2>(ka, 1, sm_count, s);
+  // sequences per block: as many as keep their fp32 x vectors in shared memory (<= 200 KB)
+  const size_t x_bytes = (size_t)d.D * 4;
+  if (a.B == 1 || 2 * x_bytes > 200 * 1024) return mlp_launch_nb<1>(ka, a.B, sm_count, s);
+  if (a.B == 2 || 4 * x_bytes > 200 * 1024) return mlp_launch_nb<2>(ka, (a.B + 1) / 2, sm_count, s);
   return mlp_launch_nb<4>(ka, (a.B + 3) / 4, sm_count, s);
 }
 

@@ -293,3 +293,34 @@ def test_export_import_roundtrip_resumes_trajectory():
     finally:
         a.close()
         b.close()
+
+
+@pytest.mark.parametrize("shape", [
+    # name, L, D, M, H, density %, capacity %
+    ("max_ffn", 1, 64, 40960, 8, 10, 20),        # widest FFN the library accepts (top-k keys fill shared memory)
+    ("max_model", 2, 16384, 64, 64, 25, 50),     # widest model: 96 KB records, four column rounds
+    ("max_pred", 2, 64, 64, 4096, 25, 50),       # widest predictor: 8 KB rows of W2
+    ("min_all", 1, 8, 32, 8, 10, 20),            # smallest legal sizes
+])
+@pytest.mark.parametrize("B", [1, 3])
+def test_limit_shapes(shape, B):
+    """The extreme sizes np_init accepts run the whole path and match the oracle."""
+    name, L, D, M, H, dens, cap = shape
+    cfg = synth.StackConfig(name, L, D, M, H, dens, cap, 3, 31, 0.9)
+    p = Pair(cfg, max_batch=B, k=max(1, cfg.top_k), C=max(2, cfg.capacity))
+    try:
+        xs = synth.hidden_states(cfg, 3, batch=B)
+        out = torch.empty((B, D), dtype=torch.float32, device="cuda")
+        logits = torch.empty((B, L, M), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            nb.np_predict(p.eng.ctx, xs[t].cuda(), B, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, xs[t].cuda(), B, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            assert rel_l2(z32, O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)) < 1e-5
+            res = p.ora.step(u16(xs[t]), logits_f32=z32)
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+        p.check_resident_bytes()
+    finally:
+        p.close()
