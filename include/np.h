@@ -242,6 +242,14 @@ int np_mlp_chain(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void*
  * copies are not counted).  Host counter, no synchronisation. */
 int np_launch_count(np_ctx* ctx, uint64_t* out);
 
+/* Failure-detection self-test.  Every device-side wait of this library (mbarrier, grid
+ * barrier) is bounded: after a fixed number of polls the kernel records a time-out in the
+ * context's device status word and returns, and the next synchronising call reports
+ * NP_E_DEVICE.  This call launches a kernel whose wait can never be satisfied (about 25 ms),
+ * synchronises `stream` and returns NP_E_DEVICE if the time-out was recorded as it should
+ * be (NP_E_STATE if it was not).  The status word stays set until np_reset. */
+int np_selftest_bounded_wait(np_ctx* ctx, void* stream);
+
 /* Device pointers to one layer's lists and counters from the last np_delta. */
 int np_get_delta(np_ctx* ctx, int32_t layer, np_delta_view* out);
 

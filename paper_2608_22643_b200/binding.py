@@ -35,7 +35,7 @@ EXPORTED = [
     "np_version", "np_query_sizes", "np_init", "np_destroy", "np_reset", "np_last_error",
     "np_predict", "np_topk", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
-    "np_launch_count", "np_predict_logits_noalloc", "np_noalloc_last_error",
+    "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_last_error",
 ]
 
 
@@ -102,6 +102,7 @@ def load() -> C.CDLL:
         "np_import_state": [vp, i32, vp, vp, vp, vp, i32, vp],
         "np_last_step_times": [vp, vp],
         "np_mlp_chain": [vp, vp, i32, vp, vp],
+        "np_selftest_bounded_wait": [vp, vp],
         "np_launch_count": [vp, C.POINTER(C.c_uint64)],
     }
     lib.np_noalloc_last_error.restype = C.c_char_p
@@ -225,6 +226,11 @@ def np_last_step_times(ctx) -> np.ndarray:
 
 def np_mlp_chain(ctx, x_bf16, B: int, x_out, stream=None) -> int:
     return _check(ctx, load().np_mlp_chain(ctx, _ptr(x_bf16), B, _ptr(x_out), _stream(stream)))
+
+
+def np_selftest_bounded_wait(ctx, stream=None) -> int:
+    """Returns the raw code (NP_E_DEVICE when the bounded wait timed out as designed)."""
+    return load().np_selftest_bounded_wait(ctx, _stream(stream))
 
 
 def np_launch_count(ctx) -> int:

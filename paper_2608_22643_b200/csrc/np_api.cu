@@ -724,6 +724,14 @@ int np_mlp_chain(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void*
   return mlp_chain(ctx, x_bf16, B, x_out, as_stream(stream));
 }
 
+int np_selftest_bounded_wait(np_ctx* ctx, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  cudaStream_t s = as_stream(stream);
+  NP_LAUNCH(ctx, launch_selftest_wait(ctx->t.status, s));
+  const int rc = check_device_status(ctx, s);
+  return rc == NP_E_DEVICE ? NP_E_DEVICE : (rc < 0 ? rc : fail(ctx, NP_E_STATE, "the wait did not time out"));
+}
+
 int np_launch_count(np_ctx* ctx, uint64_t* out) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   if (!out) return fail(ctx, NP_E_INVAL, "out is NULL");

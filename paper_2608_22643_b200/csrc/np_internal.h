@@ -134,6 +134,7 @@ bool supported(const Dims& d, int sm_count);
 cudaError_t launch(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
 }  // namespace chain_alu
 
+cudaError_t launch_selftest_wait(int32_t* status, cudaStream_t s);
 cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s);
 // out = a + sum of `reps` consecutive copies of b (each n floats)
 cudaError_t launch_add_vec(const float* a, const float* b, int reps, float* out, size_t n, cudaStream_t s);

@@ -322,6 +322,25 @@ cudaError_t launch_pred_l2(const Dims& d, const void* w2v, const float* hidden, 
 }
 
 // ---------------------------------------------------------------------------
+// Self-test of the bounded waits: one thread waits on an mbarrier that nothing
+// ever arrives at.  The wait gives up after kSpinLimit polls and records
+// kStatTimeout; the kernel returns normally.
+// ---------------------------------------------------------------------------
+__global__ void k_selftest_wait(int32_t* status) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    npp::mbar_init(&bar, 1);
+    npp::fence_barrier_init();
+    if (!npp::mbar_wait(&bar, 0)) atomicOr(status, npp::kStatTimeout);
+  }
+}
+
+cudaError_t launch_selftest_wait(int32_t* status, cudaStream_t s) {
+  k_selftest_wait<<<1, 32, 0, s>>>(status);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
 // small elementwise helpers of the residual chain
 // ---------------------------------------------------------------------------
 __global__ void k_widen_bf16(const uint16_t* __restrict__ x, float* __restrict__ out, size_t n) {

@@ -324,3 +324,27 @@ def test_limit_shapes(shape, B):
         p.check_resident_bytes()
     finally:
         p.close()
+
+
+def test_bounded_wait_times_out_and_context_survives():
+    """A wait that nothing satisfies gives up, is reported as NP_E_DEVICE, and after np_reset
+    the context computes correctly again (no hang, no trap)."""
+    p = Pair(TINY)
+    try:
+        assert nb.np_selftest_bounded_wait(p.eng.ctx, p.eng.stream) == nb.NP_E_DEVICE
+        assert "bounds check" in nb.np_last_error(p.eng.ctx) or "status" in nb.np_last_error(p.eng.ctx)
+        with pytest.raises(nb.NpError):
+            p.eng.counters()                      # the status word stays set ...
+        nb.np_reset(p.eng.ctx, p.eng.stream)      # ... until the context is reset
+        xs = synth.hidden_states(TINY, 2)
+        out = torch.empty((1, TINY.d_model), dtype=torch.float32, device="cuda")
+        logits = torch.empty((1, TINY.n_layers, TINY.d_ffn), dtype=torch.float32, device="cuda")
+        for t in range(2):
+            nb.np_predict(p.eng.ctx, xs[t].cuda(), 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, xs[t].cuda(), 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            res = p.ora.step(u16(xs[t]), logits_f32=logits.cpu().numpy())
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5
+    finally:
+        p.close()
