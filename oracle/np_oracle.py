@@ -14,7 +14,8 @@ Conventions (same symbols as the C header):
 
 Pins (see tests/test_oracle_*.py): exact rational brute force and structured
 closed forms for ``predict``; full-sort brute force, constructed ties and
-degenerate k for ``topk_bitmap``; the set identities of Eq. 2-3, slot-map
+degenerate k for ``topk_bitmap``; a per-bit scalar loop, constructed ties and
+the one-hot/identity-bank special cases for ``centroid_select``; the set identities of Eq. 2-3, slot-map
 bijection invariants and a set-based brute force for ``Residency.delta``;
 byte identity for ``install``; the dense SwiGLU library form when every row is
 active, linearity over disjoint sets and a scalar loop for ``sparse_mlp``; the
@@ -131,6 +132,37 @@ def topk_bitmap(logits_f32: np.ndarray, k: int) -> np.ndarray:
             order = np.argsort(-key, kind="stable")     # ties keep ascending index
             bits[l, order[:k]] = True
     return bool_to_bitmap(bits)
+
+
+def centroid_select(logits_f32: np.ndarray, bank_words: np.ndarray):
+    """Selection through centroid heads (Section 3.3, third stage of the
+    predictor; Section 3.4: the active set is the intersection of the gate and
+    the up centroid masks).
+
+    ``logits_f32`` is ``[B, L, 2, K]`` float32: for every sequence and layer
+    one row of logits over the centroid vocabulary for the gate head (index 0)
+    and one for the up head (index 1).  Each head takes its arg-max centroid
+    (ties: the lower centroid ID; order = the fp32 total order used by
+    ``topk_bitmap``).  ``bank_words`` is the bit-packed centroid bank
+    ``[L, 2, K, W]`` uint32.  The layer's active set for one sequence is
+    gate_mask AND up_mask; sequences are ORed.
+
+    Returns ``(ids, words)``: int32 ``[B, L, 2]`` chosen centroid IDs and the
+    uint32 bitmap ``[L, W]``."""
+    z = np.ascontiguousarray(logits_f32, dtype=np.float32)
+    bank = np.ascontiguousarray(bank_words).view(np.uint32)
+    B, L, two, K = z.shape
+    assert two == 2 and bank.shape[:3] == (L, 2, K)
+    W = bank.shape[3]
+    ids = np.zeros((B, L, 2), dtype=np.int32)
+    words = np.zeros((L, W), dtype=np.uint32)
+    for b in range(B):
+        for l in range(L):
+            for h in range(2):
+                key = fp32_order_key(z[b, l, h]).astype(np.int64)
+                ids[b, l, h] = int(np.argmax(key))      # first maximum = lowest ID
+            words[l] |= bank[l, 0, ids[b, l, 0]] & bank[l, 1, ids[b, l, 1]]
+    return ids, words
 
 
 # --------------------------------------------------------------------------
