@@ -59,7 +59,16 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=1, help="sequences per step (the metric's workload is 1)")
     ap.add_argument("--gamma", type=float, default=0.9, help="shared-driver weight of batched hidden states")
     ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
+    ap.add_argument("--selection", default="topk", choices=["topk", "centroid"],
+                    help="topk: the metric's selection; centroid: centroid heads + bank lookup + gate AND up")
+    ap.add_argument("--centroids", type=int, default=512, help="centroid vocabulary per head (centroid selection)")
     return ap.parse_args()
+
+
+def fnum(v):
+    """float for the JSON line; None where a stage was not timed."""
+    v = float(v)
+    return None if v != v else v
 
 
 def u16(t: torch.Tensor) -> np.ndarray:
@@ -296,6 +305,24 @@ def cuda_arm(args):
     out_host = torch.empty((Bq, D), dtype=torch.float32).pin_memory()
     x_stage = torch.empty((Bq, D), dtype=torch.bfloat16, device=dev)
     s, cs = eng.stream, eng.copy_stream
+    centroid = args.selection == "centroid"
+    if centroid:
+        Kc = args.centroids
+        w2c = synth.centroid_head_weights(cfg, Kc, "cuda")
+        bank = synth.centroid_bank(cfg, Kc).to(dev)
+        head_logits = torch.empty((Bq, L, 2, Kc), dtype=torch.float32, device=dev)
+        sel_words = torch.empty((L, M // 32), dtype=torch.int32, device=dev)
+
+    def step(x):
+        if not centroid:
+            return nb.np_step(eng.ctx, x, Bq, out, s, cs)
+        # the same path with the selection stage swapped: head logits -> arg-max centroids ->
+        # bank lookup -> gate AND up -> delta -> install -> MLP chain, all through the C ABI
+        nb.np_predict_logits_noalloc(eng.w1, w2c, x, Bq, L, D, 2 * Kc, cfg.d_pred, head_logits, s)
+        nb.np_centroid_select(eng.ctx, head_logits, Bq, Kc, bank, None, sel_words, s)
+        nb.np_delta(eng.ctx, sel_words, s)
+        nb.np_install(eng.ctx, 0, L, cs)
+        return nb.np_mlp_chain(eng.ctx, x, Bq, out, s)
 
     def barrier():
         torch.cuda.synchronize()
@@ -305,7 +332,7 @@ def cuda_arm(args):
 
     def run_resident(t_lo, t_hi, stats=None):
         for t in range(t_lo, t_hi):
-            nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
+            step(xs_dev[t])
             if stats is not None:
                 stats.append(eng.counters().copy())
 
@@ -329,8 +356,8 @@ def cuda_arm(args):
     stage_us, delta_rows, overlap, overflow_steps = [], [], [], 0
     for i in range(n_detail):
         t = T + i                                       # the sequence simply continues
-        nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
-        stage_us.append(nb.np_last_step_times(eng.ctx))
+        step(xs_dev[t])
+        stage_us.append(np.full(4, np.nan, np.float32) if centroid else nb.np_last_step_times(eng.ctx))
         c = eng.counters()
         delta_rows.append(float(c[:, nb.NP_CNT_DELTA].mean()))
         overflow_steps += int((c[:, nb.NP_CNT_OVERFLOW] > 0).any())
@@ -344,7 +371,7 @@ def cuda_arm(args):
         for t in range(t_lo, t_hi):
             with torch.cuda.stream(s):
                 x_stage.copy_(xs_host[t], non_blocking=True)
-            nb.np_step(eng.ctx, x_stage, Bq, out, s, cs)
+            step(x_stage)
             with torch.cuda.stream(s):
                 out_host.copy_(out, non_blocking=True)
             s.synchronize()                              # the caller consumes the result every step
@@ -378,7 +405,11 @@ def cuda_arm(args):
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record(s)
     for _ in range(reps):
-        nb.np_predict(eng.ctx, xs_dev[T - 1], Bq, None, None, s)
+        if centroid:
+            nb.np_predict_logits_noalloc(eng.w1, w2c, xs_dev[T - 1], Bq, L, D, 2 * Kc, cfg.d_pred, head_logits, s)
+            nb.np_centroid_select(eng.ctx, head_logits, Bq, Kc, bank, None, sel_words, s)
+        else:
+            nb.np_predict(eng.ctx, xs_dev[T - 1], Bq, None, None, s)
     p1.record(s)
     s.synchronize()
     pred_us = p0.elapsed_time(p1) * 1000.0 / reps
@@ -393,7 +424,8 @@ def cuda_arm(args):
     # DRAM bytes of one layer from the ncu capture in profiles/k_mlp_chain_7b.md (7B shape):
     # (216.63 MB read + 3.51 MB written) / 8 layers; scaled by the layers a launch spans
     traffic = 27.52e6 * L / n_launch if cfg.name == "7b" else None
-    pred_bytes = 2 * cfg.d_pred * D + 2 * L * M * cfg.d_pred + 4 * L * M
+    pred_rows = L * 2 * args.centroids if centroid else L * M
+    pred_bytes = 2 * cfg.d_pred * D + 2 * pred_rows * cfg.d_pred + 4 * pred_rows
     mean_delta = float(np.mean(delta_rows))
     result = {
         "metric": METRIC, "value": K * world / (ms_total / 1000.0), "unit": UNIT, "n_gpus": world,
@@ -401,7 +433,8 @@ def cuda_arm(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
-                        f"B={Bq} rho={cfg.rho} policy={args.policy} transfer={args.transfer}",
+                        f"B={Bq} rho={cfg.rho} policy={args.policy} transfer={args.transfer}"
+                        + (f" selection=centroid K={args.centroids}" if centroid else ""),
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
             "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
             "active_rows_per_layer": n_active, "overflow_steps": int(overflow_steps),
@@ -415,14 +448,14 @@ def cuda_arm(args):
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth (burst)",
                      "traffic": traffic, "us_per_launch": mlp_us, "bytes_per_launch": mlp_bytes,
                      "layers_per_launch": L / n_launch},
-        "stages_us": {"predict_topk": float(stage_us[0]), "delta": float(stage_us[1]),
-                      "install_copy_stream": float(stage_us[2]), "mlp_chain_incl_waits": float(stage_us[3]),
+        "stages_us": {"predict_topk": fnum(stage_us[0]), "delta": fnum(stage_us[1]),
+                      "install_copy_stream": fnum(stage_us[2]), "mlp_chain_incl_waits": fnum(stage_us[3]),
                       "predict_alone": pred_us, "predict_gbs": pred_bytes / (pred_us * 1e-6) / 1e9,
                       "mlp_chain_alone": mlp_us * n_launch},
         "setup_s": {"generate": gen_s},
     }
 
-    if rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1:
+    if rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid:
         n = args.cpu_baseline_steps
         times = run_oracle_steps(cfg, args.policy, w1.cpu(), w2.cpu(), store, xs_host, n)
         sec = float(np.mean(times))

@@ -190,6 +190,22 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out,
  * (dev uint32 [L][W], required).  Does not touch the context's own bitmap. */
 int np_topk(np_ctx* ctx, const float* logits, int32_t B, uint32_t* bitmap_out, void* stream);
 
+/* Stage 2 in the paper's own form (Section 3.3, the heads of the predictor;
+ * Section 3.4, the gate/up intersection): per sequence and layer two heads
+ * score a vocabulary of K centroids, each head takes its highest-scoring
+ * centroid (ties: the lower ID; order as in np_predict), and the layer's
+ * active set is gate_mask[id_gate] AND up_mask[id_up], ORed over sequences.
+ *   logits      dev fp32 [B][L][2][K]   head 0 = gate, head 1 = up
+ *   bank        dev uint32 [L][2][K][W] bit-packed centroid masks (caller-owned,
+ *               read only); the sets it yields may have any size up to M
+ *   ids_out     dev int32 [B][L][2] chosen centroid IDs, or NULL
+ *   bitmap_out  dev uint32 [L][W], required; pass it to np_delta
+ * Does not touch the context's own bitmap.  Logits of this shape come from
+ * np_predict_logits_noalloc with d_ffn = 2*K, or from any other producer.
+ * Errors: NP_E_INVAL (NULL pointer, B outside 1..max_batch, K < 1), NP_E_CUDA. */
+int np_centroid_select(np_ctx* ctx, const float* logits, int32_t B, int32_t K, const uint32_t* bank,
+                       int32_t* ids_out, uint32_t* bitmap_out, void* stream);
+
 /* Stage 3a: delta and residency update for all layers (Section 3.4, Eq. 2-3).
  *   pred_bitmap  dev uint32 [L][W], or NULL to use the last np_predict's result.
  * Per layer: incoming = P \ R (ascending), victims per the eviction policy,

@@ -33,7 +33,7 @@ NP_N_COUNTERS = 8
 
 EXPORTED = [
     "np_version", "np_query_sizes", "np_init", "np_destroy", "np_reset", "np_last_error",
-    "np_predict", "np_topk", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
+    "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
     "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_last_error",
 ]
@@ -92,6 +92,7 @@ def load() -> C.CDLL:
         "np_reset": [vp, vp],
         "np_predict": [vp, vp, i32, vp, vp, vp],
         "np_topk": [vp, vp, i32, vp, vp],
+        "np_centroid_select": [vp, vp, i32, i32, vp, vp, vp, vp],
         "np_delta": [vp, vp, vp],
         "np_install": [vp, i32, i32, vp],
         "np_sparse_mlp": [vp, i32, vp, i32, vp, vp],
@@ -179,6 +180,11 @@ def np_predict(ctx, x_bf16, B: int, logits_out=None, bitmap_out=None, stream=Non
 
 def np_topk(ctx, logits, B: int, bitmap_out, stream=None) -> int:
     return _check(ctx, load().np_topk(ctx, _ptr(logits), B, _ptr(bitmap_out), _stream(stream)))
+
+
+def np_centroid_select(ctx, logits, B: int, K: int, bank, ids_out, bitmap_out, stream=None) -> int:
+    return _check(ctx, load().np_centroid_select(ctx, _ptr(logits), B, K, _ptr(bank), _ptr(ids_out),
+                                                 _ptr(bitmap_out), _stream(stream)))
 
 
 def np_delta(ctx, pred_bitmap=None, stream=None) -> int:

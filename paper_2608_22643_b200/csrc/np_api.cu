@@ -501,6 +501,16 @@ int np_topk(np_ctx* ctx, const float* logits, int32_t B, uint32_t* bitmap_out, v
   return NP_OK;
 }
 
+int np_centroid_select(np_ctx* ctx, const float* logits, int32_t B, int32_t K, const uint32_t* bank,
+                       int32_t* ids_out, uint32_t* bitmap_out, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!logits || !bank || !bitmap_out) return fail(ctx, NP_E_INVAL, "logits, bank or bitmap_out is NULL");
+  if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
+  if (K < 1) return fail(ctx, NP_E_INVAL, "K=%d must be positive", K);
+  NP_LAUNCH(ctx, launch_centroid_select(ctx->d, logits, B, K, bank, ids_out, bitmap_out, as_stream(stream)));
+  return NP_OK;
+}
+
 int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   if (!pred_bitmap) {

@@ -75,6 +75,10 @@ cudaError_t launch_pred_l2_tc(const Dims& d, const PredTcState& st, const float*
 
 cudaError_t launch_topk(const Dims& d, const float* logits, int B, uint32_t* bitmap, cudaStream_t s);
 
+// Centroid heads -> arg-max -> bank lookup -> gate AND up (np_centroid.cu).
+cudaError_t launch_centroid_select(const Dims& d, const float* logits, int B, int K, const uint32_t* bank,
+                                   int32_t* ids_out, uint32_t* bitmap, cudaStream_t s);
+
 cudaError_t launch_delta(const Dims& d, const Tables& t, const uint32_t* pred, int policy, int step,
                          int32_t* host_lists_dev, int check, cudaStream_t s);
 

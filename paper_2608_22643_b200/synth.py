@@ -190,3 +190,43 @@ def random_bitmaps(n_layers: int, d_ffn: int, n_set: int, seed: int, n_steps: in
     # store as the uint32 bit pattern inside int32
     out = torch.where(out >= (1 << 31), out - (1 << 32), out)
     return out.to(torch.int32)
+
+
+def centroid_head_weights(cfg: StackConfig, n_centroids: int, device: str = "cpu") -> torch.Tensor:
+    """Head weights of the centroid selection stage, bf16 ``[L * 2 * K, H]``: for each layer the
+    K rows of the gate head, then the K rows of the up head (same draw recipe as the other
+    predictor weights)."""
+    return _randn_bf16((cfg.n_layers * 2 * n_centroids, cfg.d_pred), cfg.seed, 2, device)
+
+
+def centroid_bank(cfg: StackConfig, n_centroids: int, mask_rows: Optional[int] = None,
+                  layers: Optional[int] = None) -> torch.Tensor:
+    """A synthetic centroid bank, int32-typed uint32 words ``[L, 2, K, M/32]``.
+
+    Stands in for the bank the method builds offline by clustering thresholded activation masks
+    (no trained model is available here).  Every layer has one popularity score per neuron (hot
+    neurons recur across centroids, as clustered masks do); centroid ``c`` of head ``h`` is the
+    ``mask_rows`` neurons with the highest ``popularity + noise[h, c]``, so every mask has exactly
+    the target size, gate and up masks of a layer overlap well above chance, and their
+    intersection has a size that varies from pair to pair and never exceeds the mask size.
+    ``mask_rows`` defaults to ``top_k``, the target sparsity every centroid is pruned to.  Bit
+    ``j`` of word ``w`` stands for neuron ``32 * w + j``.
+    """
+    L = cfg.n_layers if layers is None else layers
+    M, K = cfg.d_ffn, n_centroids
+    assert M % 32 == 0
+    n_mask = cfg.top_k if mask_rows is None else mask_rows
+    g = torch.Generator(device="cpu")
+    g.manual_seed(cfg.seed * _SEED_MUL + 4242)
+    weights = (1 << torch.arange(32, dtype=torch.int64))
+    out = torch.empty((L, 2, K, M // 32), dtype=torch.int32)
+    for l in range(L):
+        pop = torch.randn(M, generator=g)
+        for h in range(2):
+            score = pop[None, :] + torch.randn(K, M, generator=g)
+            idx = score.topk(n_mask, dim=1).indices
+            bits = torch.zeros((K, M), dtype=torch.int64)
+            bits.scatter_(1, idx, 1)
+            words = (bits.view(K, M // 32, 32) * weights).sum(dim=2)          # < 2**32
+            out[l, h] = torch.where(words >= (1 << 31), words - (1 << 32), words).to(torch.int32)
+    return out
