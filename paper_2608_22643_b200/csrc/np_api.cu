@@ -186,6 +186,8 @@ struct np_ctx {
   uint64_t launches = 0;
   Pool* pool = nullptr;
   PredTcState tc = {};
+  size_t gu_bytes = 0;   // both dot-product accumulators of the batch MLP, contiguous
+  bool mlp_tc = false;   // batches run the tensor-core MLP kernels
   std::string err;
 };
 
@@ -246,7 +248,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
 }
 
 struct WsLayout {
-  size_t hidden, hsplit, logits, xbuf, zbuf, total;
+  size_t hidden, hsplit, logits, xbuf, zbuf, gu, gu_each, total;
 };
 
 WsLayout ws_layout(const np_config& c) {
@@ -263,6 +265,10 @@ WsLayout ws_layout(const np_config& c) {
   off += 2 * vec;
   w.zbuf = off;
   off += 3 * kZRep * vec;
+  // batch MLP: two dot-product accumulators, each followed by its per-sequence sums of squares
+  w.gu = off;
+  w.gu_each = align_up(((size_t)c.capacity * 2 * kMaxBatch + kMaxBatch) * 4, 256);
+  off += 2 * w.gu_each;
   w.total = off;
   return w;
 }
@@ -431,6 +437,11 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   ctx->ws.logits = reinterpret_cast<float*>(wsb + wl.logits);
   for (int i = 0; i < 2; ++i) ctx->ws.xbuf[i] = reinterpret_cast<float*>(wsb + wl.xbuf + i * vec);
   for (int i = 0; i < 3; ++i) ctx->ws.zbuf[i] = reinterpret_cast<float*>(wsb + wl.zbuf + i * kZRep * vec);
+  for (int i = 0; i < 2; ++i) {
+    ctx->ws.gu[i] = reinterpret_cast<float*>(wsb + wl.gu + i * wl.gu_each);
+    ctx->ws.ssq[i] = ctx->ws.gu[i] + (size_t)cfg->capacity * 2 * kMaxBatch;
+  }
+  ctx->gu_bytes = 2 * wl.gu_each;
 
   NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_delta, cudaEventDisableTiming));
   ctx->ev_installed.assign(d.L, nullptr);
@@ -442,6 +453,8 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   for (auto& e : ctx->ev_c) NP_INIT_CUDA(cudaEventCreate(&e));
 
   // tensor-core predictor for batches: tensor maps over W2 and the split hidden terms
+  ctx->mlp_tc = cfg->max_batch >= kTcMinBatch && !(cfg->flags & (NP_F_NO_TENSOR_CORES | NP_F_DIRECT_LOADS)) &&
+                mlp_tc_supported(d, ctx->sm_count);
   if (cfg->max_batch > 4 && !(cfg->flags & NP_F_NO_TENSOR_CORES)) pred_tc_prepare(d, b->w2, ctx->ws.hsplit, &ctx->tc);
   memset(ctx->host_lists, 0, host_lists_ints(*cfg) * 4);
   NP_INIT_CUDA(launch_tables_reset(d, t, nullptr));
@@ -654,8 +667,10 @@ static cudaError_t wait_install(np_ctx* ctx, int layer, cudaStream_t s) {
   return cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0);
 }
 
+// gu_sel: which of the two dot-product accumulators this layer uses (the batch kernels clear the
+// other one for the next layer); -1 = a single layer outside a chain
 static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, float* yacc, float* x_store,
-                     float* zero_out, int B, int normalize, cudaStream_t s) {
+                     float* zero_out, int B, int normalize, int gu_sel, cudaStream_t s) {
   const Dims& d = ctx->d;
   const size_t row_bytes = (size_t)d.D * 2;
   MlpArgs a;
@@ -675,7 +690,20 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   a.normalize = normalize;
   a.force_direct = (ctx->cfg.flags & NP_F_DIRECT_LOADS) ? 1 : 0;
   a.status = ctx->t.status;
+  a.gu = a.gu_next = a.ssq = a.ssq_next = nullptr;
   if (ctx->install_pending[layer]) NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0));
+  if (ctx->mlp_tc && B >= kTcMinBatch && !a.force_direct) {
+    const int cur = gu_sel < 0 ? 0 : gu_sel;
+    a.gu = ctx->ws.gu[cur];
+    a.ssq = ctx->ws.ssq[cur];
+    if (gu_sel >= 0) {
+      a.gu_next = ctx->ws.gu[cur ^ 1];
+      a.ssq_next = ctx->ws.ssq[cur ^ 1];
+    }
+    ctx->launches += 1;  // two kernels per layer
+    NP_LAUNCH(ctx, launch_sparse_mlp_tc(d, a, s, ctx->sm_count));
+    return NP_OK;
+  }
   NP_LAUNCH(ctx, launch_sparse_mlp(d, a, s, ctx->sm_count));
   return NP_OK;
 }
@@ -714,9 +742,10 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
     }
   } else {
+    if (ctx->mlp_tc && B >= kTcMinBatch) NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.gu[0], 0, ctx->gu_bytes, s));
     for (int l = 0; l < d.L; ++l) {
       int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
-                         ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, 1, s);
+                         ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, 1, l & 1, s);
       if (rc < 0) return rc;
     }
   }
@@ -759,7 +788,8 @@ int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* 
   if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_sparse_mlp needs a prior np_delta");
   cudaStream_t s = as_stream(stream);
   NP_CUDA(ctx, cudaMemsetAsync(y, 0, (size_t)B * d.D * 4, s));
-  return mlp_layer(ctx, layer, x, nullptr, y, nullptr, nullptr, B, 0, s);
+  if (ctx->mlp_tc && B >= kTcMinBatch) NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.gu[0], 0, ctx->gu_bytes / 2, s));
+  return mlp_layer(ctx, layer, x, nullptr, y, nullptr, nullptr, B, 0, -1, s);
 }
 
 int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream, void* copy_stream) {

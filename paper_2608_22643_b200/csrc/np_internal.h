@@ -44,6 +44,8 @@ struct Workspace {
   float* logits;   // [Bmax][L][M]
   float* xbuf[2];  // [Bmax][D] each: x_l of the residual chain, ping-pong
   float* zbuf[3];  // [kZRep][Bmax][D] each: MLP_l(x_l) accumulators, rotating
+  float* gu[2];    // [C][2][kMaxBatch] each: gate/up dot products of a layer (batch MLP), alternating
+  float* ssq[2];   // [kMaxBatch] each: sum of x_l^2 per sequence
 };
 
 struct Dims {
@@ -106,8 +108,18 @@ struct MlpArgs {
   int normalize;     // scale x to unit RMS before the dot products (the chain's pre-MLP norm)
   int force_direct;  // use the direct-load kernel even where the staged one applies
   int32_t* status;
+  // tensor-core batch path only (np_mlp_tc.cu); NULL gu keeps the layer on the other kernels
+  float* gu;        // [C][2][kMaxBatch] dot-product accumulators of this layer, zero on entry
+  float* gu_next;   // the next layer's, cleared by this layer (may be NULL)
+  float* ssq;       // [kMaxBatch] sum of x^2 per sequence, zero on entry (needed with normalize)
+  float* ssq_next;  // may be NULL
 };
 cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count);
+// Batches on tensor cores: two launches per layer (np_mlp_tc.cu).
+constexpr int kTcMinBatch = 2;
+bool mlp_tc_supported(const Dims& d, int sm_count);
+size_t mlp_tc_gu_floats(const Dims& d);
+cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count);
 
 // Persistent multi-layer form of the sparse MLP for one sequence (np_mlp_chain.cu).
 struct ChainPlan {
