@@ -1,29 +1,28 @@
-// Stage 4 for batches: the sparse SwiGLU MLP of one layer on tensor cores.
+// Stage 4 on tensor cores: the sparse SwiGLU MLP through the slot map,
 //
 //   y[b] = sum_{i in act} silu(gate[s_i] . x[b]) * (up[s_i] . x[b]) * downT[s_i]      (Section 3.4)
 //
-// With several sequences every weight row is used once per sequence, so the
-// dot products are small matrix products: bf16 weights times activations that
-// are kept in fp32 and split, on the fly, into three truncated bf16 terms
-// (x = t0 + t1 + t2 up to 2^-24 |x|; one MMA per term, fp32 accumulation).
+// for one to sixteen sequences.  The dot products are small matrix products of bf16 weights
+// with activations that stay in fp32 and are split into three truncated bf16 terms
+// (v = t0 + t1 + t2 up to 2^-24 |v|; one MMA per term, fp32 accumulation).
 //
-// Two kernels per layer, no block ever waits for another block:
+// The work of a layer is cut twice, and no step needs a vector-wide all-reduce:
 //
-//   k_mlp_tc_up    grid (row blocks, K slices).  A block streams the K slice of
-//                  its rows' gate and up vectors through a ring of bulk copies
-//                  and adds its partial dot products (for all sequences) into
-//                  GU[row][gate|up][sequence] in global memory.  Slicing K keeps
-//                  the block's piece of x small (16 sequences x 1024 columns),
-//                  so shared memory goes to rows in flight.
-//   k_mlp_tc_down  grid (row blocks, column slices).  A block turns the finished
-//                  dot products of its rows into activations h, streams the
-//                  column slice of the rows' down vectors and accumulates
-//                  y[:, slice] += h^T . down in registers; one vector reduction
-//                  per output element and block at the end.
+//   phase "up"    grid (row blocks, K slices).  A block streams the K slice of its rows' gate
+//                 and up vectors through a ring of bulk copies and adds its partial dot
+//                 products, for all sequences, into GU[row][gate|up][sequence] in global
+//                 memory.  Slicing K keeps the block's piece of x small, so shared memory
+//                 goes to rows in flight; the split of x is done once per block and layer.
+//   phase "down"  grid (row blocks, column slices).  A block turns the finished dot products of
+//                 its rows into activations h, streams the column slice of the rows' down
+//                 vectors and accumulates y[:, slice] += h^T . down in registers; one 16-byte
+//                 reduction per four output elements and block at the end.
 //
-// Every weight byte is read once.  The kernels are chained by programmatic
-// dependent launch: weight copies are issued before the wait for the previous
-// kernel, everything that depends on it after.
+// Every weight byte is read once.  The two kernels of a layer (k_mlp_tc_up, k_mlp_tc_down) are
+// chained by programmatic dependent launch: weight copies are issued before the wait for the
+// previous kernel, everything that depends on it after.  (A resident form with two grid
+// barriers per layer was measured and was slower at every batch size: the barriers cost as
+// much as the kernel boundaries they replace.)
 #include <algorithm>
 
 #include "np_device.cuh"
@@ -39,38 +38,43 @@ namespace {
 constexpr int kSeq = 16;  // sequence columns of the MMA tiles (= kMaxBatch)
 static_assert(kSeq == kMaxBatch, "tile width follows the batch limit");
 
-constexpr int kUpWarps = 16;  // consumer warps: four per tile slot (all sixteen build the B fragments)
-constexpr int kUpSlots = 4;   // tiles in flight, at most
-constexpr int kUpBatch = 8;  // prologue items whose loads a thread keeps in flight
-constexpr int kUpTile = 8;    // records per tile: 8 gate rows + 8 up rows = the 16 rows of one MMA
-constexpr int kUpThreads = (kUpWarps + 1) * 32;
+constexpr int kWarps = 16;                   // consumer warps of every kernel here
+constexpr int kC = kWarps * 32;              // consumer threads
+constexpr int kThreads = kC + 32;            // plus one producer warp
+constexpr int kQ = 4;                        // warps that share one up tile (they interleave its K steps)
+constexpr int kMaxSlots = 8;                 // tiles in flight, at most
+constexpr int kTileRows = 16;                // rows of a ring slot: 8 gate + 8 up rows, or 16 down rows
+constexpr int kUpTile = 8;                   // records per up tile
+constexpr int kDownTile = 16;                // records per down tile = the K extent of one MMA
+constexpr int kDownChunk = 128;              // rows whose activations sit in shared memory at a time
+constexpr int kSlotCache = 512;              // slot indices of a block's first rows, fetched in one batch
+constexpr int kHsStride = kDownChunk + 8;    // floats per sequence in hs: conflict-free fragment reads
+constexpr size_t kHsBytes = (size_t)kSeq * kHsStride * 4;
 
-constexpr int kDownWarps = 16;  // consumer warps: each owns up to 8 n-tiles (64 columns) of the slice
-constexpr int kDownTile = 16;   // records per tile = the K extent of one MMA
-constexpr int kDownMaxSlots = 8;
-constexpr int kDownChunk = 128;  // rows whose activations sit in shared memory at a time
-constexpr int kDownThreads = (kDownWarps + 1) * 32;
-constexpr int kSlotCache = 512;  // slot indices of a block's first rows, fetched in one batch
-constexpr int kXPad = 8;  // floats between sequences / activation rows: conflict-free fragment reads
-
-struct TcArgs {
-  const unsigned char* gate;  // this layer's row buffers
-  const unsigned char* up;
-  const unsigned char* downT;
-  const int32_t* slots;
-  const int32_t* n_ptr;
-  const float* xa;
-  const float* xb;
-  float* yacc;
-  float* x_store;
-  float* zero_out;
-  float* gu;        // [C][2][kSeq] dot products of this layer, zero on entry
-  float* gu_next;   // cleared for the next layer by the down kernel (may be NULL)
-  float* ssq;       // [kSeq] sum of x^2 per sequence, zero on entry
-  float* ssq_next;  // may be NULL
+// Block geometry and the few scalars every helper needs.
+struct Blk {
+  int D, SW, B, NJ, n_ksteps, C, check;
+  uint32_t slice_bytes;  // SW * 2
+  uint32_t row_stride;   // slice_bytes + 16: consecutive rows of a tile fall into different banks
+  uint32_t slot_bytes;   // kTileRows * row_stride
+  size_t slice_off;      // byte offset of this block's slice within a row
   int32_t* status;
-  int B, D, C, SW, check, normalize, up_slots, down_slots;
 };
+
+__device__ __forceinline__ Blk make_blk(int B, int D, int C, int SW, int slice, int check, int32_t* status) {
+  Blk k;
+  k.D = D, k.SW = SW, k.B = B, k.C = C, k.check = check;
+  k.NJ = B > 8 ? 2 : 1;
+  k.n_ksteps = SW >> 4;
+  k.slice_bytes = (uint32_t)SW * 2u;
+  k.row_stride = k.slice_bytes + 16u;
+  k.slot_bytes = (uint32_t)kTileRows * k.row_stride;
+  k.slice_off = (size_t)slice * k.slice_bytes;
+  k.status = status;
+  return k;
+}
+
+__device__ __forceinline__ size_t xf_bytes(const Blk& k) { return (size_t)k.n_ksteps * k.NJ * 3 * 32 * 8; }
 
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
@@ -110,54 +114,369 @@ __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, 
                : "memory");
 }
 
-template <int kThreads>
-__device__ __forceinline__ void consumer_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
-}
+// barrier among the consumer warps only (the producer warp never joins it)
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kC) : "memory"); }
 
-__device__ __forceinline__ int checked_slot(const TcArgs& a, int r) {
-  int s = a.slots[r];
-  if (a.check && (s < 0 || s >= a.C)) {
-    atomicOr(a.status, kStatBadSlot);
+__device__ __forceinline__ int checked_slot(const Blk& k, const int32_t* slots, int r) {
+  int s = slots[r];
+  if (k.check && (s < 0 || s >= k.C)) {
+    atomicOr(k.status, kStatBadSlot);
     s = 0;
   }
   return s;
 }
 
-__device__ __forceinline__ int checked_count(const TcArgs& a) {
-  int n = *a.n_ptr;
-  if (a.check && (n < 0 || n > a.C)) {
-    if (threadIdx.x == 0) atomicOr(a.status, kStatBadCount);
+__device__ __forceinline__ int checked_count(const Blk& k, const int32_t* n_ptr) {
+  int n = *n_ptr;
+  if (k.check && (n < 0 || n > k.C)) {
+    if (threadIdx.x == 0) atomicOr(k.status, kStatBadCount);
     n = 0;
   }
   return n;
 }
 
 // ---------------------------------------------------------------------------
-// Phase 1: GU[r][0][b] += gate[s_r][slice] . x[b][slice], GU[r][1][b] likewise for up.
+// Producer side (one warp): slot indices of the block's rows, then one bulk copy per row.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void fill_slot_cache(const Blk& k, const int32_t* slots, int* s_slots, int r_begin,
+                                                int r_end, int lane) {
+  for (int i = lane; i < min(r_end - r_begin, kSlotCache); i += 32) s_slots[i] = checked_slot(k, slots, r_begin + i);
+  __syncwarp();
+}
+
+__device__ __forceinline__ int slot_of(const Blk& k, const int32_t* slots, const int* s_slots, int r_begin, int r) {
+  const int ri = r - r_begin;
+  return ri < kSlotCache ? s_slots[ri] : checked_slot(k, slots, r);
+}
+
+// gate rows into tile rows 0-7, up rows into 8-15
+__device__ __forceinline__ void issue_up_tile(const Blk& k, const unsigned char* gate, const unsigned char* up,
+                                              const int32_t* slots, const int* s_slots, int r_begin, int r0,
+                                              int rows, unsigned char* tile, uint64_t* full, int lane) {
+  if (lane == 0) mbar_expect_tx(full, (uint32_t)rows * 2u * k.slice_bytes);
+  __syncwarp();
+  if (lane < rows) {
+    const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r0 + lane) * k.D * 2 + k.slice_off;
+    unsigned char* dst = tile + (size_t)lane * k.row_stride;
+    bulk_g2s(dst, gate + src, k.slice_bytes, full);
+    bulk_g2s(dst + (size_t)kUpTile * k.row_stride, up + src, k.slice_bytes, full);
+  }
+}
+
+// A short last tile repeats its last record: those rows meet h = 0, and the shared memory
+// they would otherwise leave stale could hold anything (0 * NaN).
+__device__ __forceinline__ void issue_down_tile(const Blk& k, const unsigned char* downT, const int32_t* slots,
+                                                const int* s_slots, int r_begin, int r0, int rows,
+                                                unsigned char* tile, uint64_t* full, int lane) {
+  if (lane == 0) mbar_expect_tx(full, (uint32_t)kDownTile * k.slice_bytes);
+  __syncwarp();
+  if (lane < kDownTile) {
+    const int r = r0 + min(lane, rows - 1);
+    const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r) * k.D * 2 + k.slice_off;
+    bulk_g2s(tile + (size_t)lane * k.row_stride, downT + src, k.slice_bytes, full);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Up phase, consumer side.
 //
 // MMA shape: rows = 8 gate rows + 8 up rows of a tile, K = 16 columns of the slice, columns =
 // 8 sequences; one MMA per term of x and per group of 8 sequences.  The split of x is the
-// same for every tile, so it is done once per block: the prologue leaves the B fragments of
-// every K step in shared memory in register layout (a lane's b0/b1 words side by side).
+// same for every tile, so it is done once: build_x_fragments leaves the B fragments of every
+// K step in shared memory in register layout (a lane's b0/b1 words side by side).
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(kUpThreads, 1) k_mlp_tc_up(TcArgs a) {
+
+// x = xa (+ xb) of this block's slice -> xf[K step][sequence group][term][lane].  The block
+// with `side` set also keeps the chain's side effects for its slice: x is stored, the
+// accumulator one layer ahead is cleared, and the slice's share of sum(x^2) is added to ssq.
+template <int kBatch>  // items whose loads a thread keeps in flight
+__device__ __forceinline__ void build_x_fragments(const Blk& k, int slice, const float* xa, const float* xb,
+                                                  float* x_store, float* zero_out, float* ssq, bool side,
+                                                  uint2* xf, int tid) {
+  // item = (K step, sequence group, lane): the four x values behind that lane's b0/b1.
+  // A thread's items all belong to one sequence (kC / 32 is a multiple of NJ).
+  const int lane = tid & 31, wid = tid >> 5;
+  const int g = lane >> 2, q = lane & 3;
+  const int items = k.n_ksteps * k.NJ * 32;
+  const bool has_b = xb != nullptr;
+  float ss = 0.f;
+  for (int base = tid; base < items; base += kC * kBatch) {
+    float2 va[kBatch][2], vb[kBatch][2];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int it = base + u * kC, pair = it >> 5;
+      const int b = 8 * (pair % k.NJ) + g;
+      va[u][0] = va[u][1] = vb[u][0] = vb[u][1] = make_float2(0.f, 0.f);
+      if (it < items && b < k.B) {
+        const size_t gi = (size_t)b * k.D + (size_t)slice * k.SW + (size_t)(pair / k.NJ) * 16 + 2 * q;
+        va[u][0] = __ldcg(reinterpret_cast<const float2*>(xa + gi));
+        va[u][1] = __ldcg(reinterpret_cast<const float2*>(xa + gi + 8));
+        if (has_b) {
+          vb[u][0] = __ldcg(reinterpret_cast<const float2*>(xb + gi));
+          vb[u][1] = __ldcg(reinterpret_cast<const float2*>(xb + gi + 8));
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int it = base + u * kC, pair = it >> 5;
+      if (it < items) {
+        const float2 lo = make_float2(va[u][0].x + vb[u][0].x, va[u][0].y + vb[u][0].y);
+        const float2 hi = make_float2(va[u][1].x + vb[u][1].x, va[u][1].y + vb[u][1].y);
+        uint32_t l0[3], l1[3], h0[3], h1[3];
+        split3(lo.x, l0[0], l0[1], l0[2]);
+        split3(lo.y, l1[0], l1[1], l1[2]);
+        split3(hi.x, h0[0], h0[1], h0[2]);
+        split3(hi.y, h1[0], h1[1], h1[2]);
+#pragma unroll
+        for (int e = 0; e < 3; ++e)
+          xf[((size_t)pair * 3 + e) * 32 + lane] = make_uint2(pack2(l0[e], l1[e]), pack2(h0[e], h1[e]));
+        ss += lo.x * lo.x + lo.y * lo.y + hi.x * hi.x + hi.y * hi.y;
+        const int b = 8 * (pair % k.NJ) + g;
+        if (side && b < k.B) {
+          const size_t gi = (size_t)b * k.D + (size_t)slice * k.SW + (size_t)(pair / k.NJ) * 16 + 2 * q;
+          if (x_store) {
+            *reinterpret_cast<float2*>(x_store + gi) = lo;
+            *reinterpret_cast<float2*>(x_store + gi + 8) = hi;
+          }
+          if (zero_out) {
+            *reinterpret_cast<float2*>(zero_out + gi) = make_float2(0.f, 0.f);
+            *reinterpret_cast<float2*>(zero_out + gi + 8) = make_float2(0.f, 0.f);
+          }
+        }
+      }
+    }
+  }
+  if (side && ssq) {
+    // lanes 4g..4g+3 hold parts of the same sequence
+    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+    const int b = 8 * (wid % k.NJ) + g;
+    if (q == 0 && b < k.B) atomicAdd(ssq + b, ss);
+  }
+}
+
+// One warp's part of an up tile: K steps kq, kq + nw, ... of the tile at shared address
+// `tile`; afterwards the partial dot products go to GU.  Rows g (gate of record g) and g + 8
+// (up of record g) of the accumulator; columns = sequences 8j + 2q, +1.  Lane pairs trade
+// halves so that even-q lanes add four consecutive sequences of the gate row and odd-q lanes
+// the same four of the up row: every reduction is 16 bytes wide.
+template <int NJ>
+__device__ __forceinline__ void up_tile_mma_n(const Blk& k, const uint2* xf, uint32_t tile, int kq, int nw,
+                                              int lane, float (&acc)[NJ][3][4]) {
+#pragma unroll
+  for (int j = 0; j < NJ; ++j)
+#pragma unroll
+    for (int e = 0; e < 3; ++e)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[j][e][i] = 0.f;
+  const uint32_t a_base = tile + (uint32_t)(lane & 15) * k.row_stride + (uint32_t)(lane >> 4) * 16u;
+  const uint2* xf_lane = xf + lane;
+  constexpr int kstep_stride = NJ * 3 * 32;  // uint2 units
+#pragma unroll 2
+  for (int kstep = kq; kstep < k.n_ksteps; kstep += nw) {
+    uint32_t af[4];
+    ldsm_x4(af, a_base + (uint32_t)kstep * 32u);
+    const uint2* xp = xf_lane + (size_t)kstep * kstep_stride;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+#pragma unroll
+      for (int e = 0; e < 3; ++e) {
+        const uint2 b = xp[(j * 3 + e) * 32];
+        mma_16816(acc[j][e], af[0], af[1], af[2], af[3], b.x, b.y);
+      }
+    }
+  }
+}
+
+template <int NJ>
+__device__ __forceinline__ void up_tile_reds(const Blk& k, const float (&acc)[NJ][3][4], float* gu, int r0,
+                                             int rows, int lane) {
+  const int g = lane >> 2, q = lane & 3;
+  const bool odd = q & 1;
+  const bool row_ok = g < rows;
+  float* dst = gu + ((size_t)(r0 + g) * 2 + (odd ? 1 : 0)) * kSeq + (q & ~1) * 2;
+#pragma unroll
+  for (int j = 0; j < NJ; ++j) {
+    {
+      const float g0 = acc[j][0][0] + acc[j][1][0] + acc[j][2][0], g1 = acc[j][0][1] + acc[j][1][1] + acc[j][2][1];
+      const float u0 = acc[j][0][2] + acc[j][1][2] + acc[j][2][2], u1 = acc[j][0][3] + acc[j][1][3] + acc[j][2][3];
+      const float ra = __shfl_xor_sync(0xffffffffu, odd ? g0 : u0, 1);
+      const float rb = __shfl_xor_sync(0xffffffffu, odd ? g1 : u1, 1);
+      if (row_ok && 8 * j + (q & ~1) * 2 < k.B) {
+        if (odd)
+          red_add_v4(dst + 8 * j, ra, rb, u0, u1);
+        else
+          red_add_v4(dst + 8 * j, g0, g1, ra, rb);
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Down phase, consumer side.
+//
+// MMA shape: rows = sequences, K = 16 records, columns = 8 output columns.  The three terms of
+// h share one accumulator: a first MMA carries t0 in rows 0-7 and t1 in rows 8-15 (both of
+// sequence g), a second one t2 in rows 0-7; rows g and g + 8 are added at the end.
+// ---------------------------------------------------------------------------
+
+// h[b][rec] = silu(inv_b * GU[rec][0][b]) * inv_b * GU[rec][1][b] for the chunk's rows; rows up
+// to the next multiple of the tile get h = 0.
+__device__ __forceinline__ void down_activations(const Blk& k, const float* gu, const float* s_inv, float* hs,
+                                                 int c0, int rows_c, int tid) {
+  const int rows_pad = (rows_c + kDownTile - 1) / kDownTile * kDownTile;
+  for (int i = tid; i < rows_pad * kSeq; i += kC) {
+    const int rec = i / kSeq, b = i % kSeq;
+    float h = 0.f;
+    if (rec < rows_c && b < k.B) {
+      const float* p = gu + (size_t)(c0 + rec) * 2 * kSeq + b;
+      const float gs = __ldcg(p) * s_inv[b], us = __ldcg(p + kSeq) * s_inv[b];
+      h = gs / (1.f + __expf(-gs)) * us;
+    }
+    hs[(size_t)b * kHsStride + rec] = h;
+  }
+}
+
+// One warp's part of a down tile: its n-tiles [nt0, nt0 + my_nt) of the slice, records
+// rl .. rl + 15 of the chunk.
+template <int NJ>
+__device__ __forceinline__ void down_tile_mma(const Blk& k, const float* hs, int rl, uint32_t tile, int nt0,
+                                              int my_nt, int lane, float (&acc)[NJ][8][4]) {
+  const int g = lane >> 2, q = lane & 3;
+  // A fragments: the three terms of h[8m + g][rl + 2q, +1, +8, +9]
+  uint32_t a1[NJ][4], a2[NJ][2];
+#pragma unroll
+  for (int m = 0; m < NJ; ++m) {
+    {
+      const float* hp = hs + (size_t)(8 * m + g) * kHsStride + rl + 2 * q;
+      const float2 lo = *reinterpret_cast<const float2*>(hp);
+      const float2 hi = *reinterpret_cast<const float2*>(hp + 8);
+      uint32_t l0[3], l1[3], h0[3], h1[3];
+      split3(lo.x, l0[0], l0[1], l0[2]);
+      split3(lo.y, l1[0], l1[1], l1[2]);
+      split3(hi.x, h0[0], h0[1], h0[2]);
+      split3(hi.y, h1[0], h1[1], h1[2]);
+      a1[m][0] = pack2(l0[0], l1[0]);  // row g:     t0, records 2q, 2q+1
+      a1[m][1] = pack2(l0[1], l1[1]);  // row g + 8: t1
+      a1[m][2] = pack2(h0[0], h1[0]);  // row g:     t0, records 2q+8, 2q+9
+      a1[m][3] = pack2(h0[1], h1[1]);  // row g + 8: t1
+      a2[m][0] = pack2(l0[2], l1[2]);  // row g:     t2
+      a2[m][1] = pack2(h0[2], h1[2]);
+    }
+  }
+  // ldmatrix.trans lane address: matrices 0/1 = records 0-7 / 8-15 of n-tile j, 2/3 = the same of n-tile j + 1
+  const uint32_t b_base = tile + (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * k.row_stride +
+                          (uint32_t)(nt0 + (lane >> 4)) * 16u;
+  // two halves of four n-tiles: fragment loads first, then a round of MMAs with (t0 | t1)
+  // and a round with t2, eight independent accumulators per round
+#pragma unroll
+  for (int hf = 0; hf < 2; ++hf) {
+    if (4 * hf < my_nt) {
+      uint32_t bf[2][4];
+#pragma unroll
+      for (int p2 = 0; p2 < 2; ++p2)
+        if (4 * hf + 2 * p2 < my_nt) ldsm_x4_trans(bf[p2], b_base + (uint32_t)(2 * hf + p2) * 32u);
+#pragma unroll
+      for (int p2 = 0; p2 < 2; ++p2) {
+        if (4 * hf + 2 * p2 < my_nt) {
+          const int j = 4 * hf + 2 * p2;
+#pragma unroll
+          for (int m = 0; m < NJ; ++m) {
+            mma_16816(acc[m][j], a1[m][0], a1[m][1], a1[m][2], a1[m][3], bf[p2][0], bf[p2][1]);
+            mma_16816(acc[m][j + 1], a1[m][0], a1[m][1], a1[m][2], a1[m][3], bf[p2][2], bf[p2][3]);
+          }
+        }
+      }
+#pragma unroll
+      for (int p2 = 0; p2 < 2; ++p2) {
+        if (4 * hf + 2 * p2 < my_nt) {
+          const int j = 4 * hf + 2 * p2;
+#pragma unroll
+          for (int m = 0; m < NJ; ++m) {
+            mma_16816(acc[m][j], a2[m][0], 0u, a2[m][1], 0u, bf[p2][0], bf[p2][1]);
+            mma_16816(acc[m][j + 1], a2[m][0], 0u, a2[m][1], 0u, bf[p2][2], bf[p2][3]);
+          }
+        }
+      }
+    }
+  }
+}
+
+// y[seq][slice columns] += acc.  Rows g and g + 8 of an accumulator belong to the same
+// sequence.  Even-q lanes end up with four consecutive columns of sequence g, odd-q lanes with
+// the same four columns of sequence 8 + g, so every reduction is 16 bytes wide.
+template <int NJ>
+__device__ __forceinline__ void down_reds(const Blk& k, const float (&acc)[NJ][8][4], float* y_slice, int nt0,
+                                          int my_nt, int lane) {
+  const int g = lane >> 2, q = lane & 3;
+  const bool odd = q & 1;
+  const int seq = odd ? 8 + g : g;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    if (j < my_nt) {
+      const float m0a = acc[0][j][0] + acc[0][j][2], m0b = acc[0][j][1] + acc[0][j][3];
+      const float m1a = NJ == 2 ? acc[NJ - 1][j][0] + acc[NJ - 1][j][2] : 0.f;
+      const float m1b = NJ == 2 ? acc[NJ - 1][j][1] + acc[NJ - 1][j][3] : 0.f;
+      const float ra = __shfl_xor_sync(0xffffffffu, odd ? m0a : m1a, 1);
+      const float rb = __shfl_xor_sync(0xffffffffu, odd ? m0b : m1b, 1);
+      if (seq < k.B) {
+        float* dst = y_slice + (size_t)seq * k.D + (size_t)(nt0 + j) * 8 + (q & ~1) * 2;
+        if (odd)
+          red_add_v4(dst, ra, rb, m1a, m1b);
+        else
+          red_add_v4(dst, m0a, m0b, ra, rb);
+      }
+    }
+  }
+}
+
+// every block clears its share of the next layer's accumulators
+__device__ __forceinline__ void clear_next(float* gu_next, float* ssq_next, int C, int bid, int nblk, int tid) {
+  if (gu_next) {
+    const size_t total = (size_t)C * 2 * kSeq / 4;  // float4 units
+    const size_t lo = total * bid / nblk, hi = total * (bid + 1) / nblk;
+    float4* p = reinterpret_cast<float4*>(gu_next);
+    for (size_t i = lo + tid; i < hi; i += kC) p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (ssq_next && bid == 0 && tid < kSeq) ssq_next[tid] = 0.f;
+}
+
+// ---------------------------------------------------------------------------
+// Per-layer form: two kernels, chained by programmatic dependent launch.
+// ---------------------------------------------------------------------------
+struct TcArgs {
+  const unsigned char* gate;  // this layer's row buffers
+  const unsigned char* up;
+  const unsigned char* downT;
+  const int32_t* slots;
+  const int32_t* n_ptr;
+  const float* xa;
+  const float* xb;
+  float* yacc;
+  float* x_store;
+  float* zero_out;
+  float* gu;        // [C][2][kSeq] dot products of this layer, zero on entry
+  float* gu_next;   // cleared for the next layer by the down kernel (may be NULL)
+  float* ssq;       // [kSeq] sum of x^2 per sequence, zero on entry
+  float* ssq_next;  // may be NULL
+  int32_t* status;
+  int B, D, C, SW, check, normalize, up_slots, down_slots;
+};
+
+template <int NJ>
+__global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_up(TcArgs a) {
   extern __shared__ __align__(128) unsigned char tsm[];
-  __shared__ __align__(8) uint64_t full_bar[kUpSlots];
-  __shared__ __align__(8) uint64_t empty_bar[kUpSlots];
+  __shared__ __align__(8) uint64_t full_bar[kMaxSlots];
+  __shared__ __align__(8) uint64_t empty_bar[kMaxSlots];
   __shared__ int s_slots[kSlotCache];
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int rb = blockIdx.x, RB = gridDim.x, ks = blockIdx.y;
-  const int D = a.D, SW = a.SW, NS = a.up_slots;
-  const int NJ = a.B > 8 ? 2 : 1;                          // groups of 8 sequences
-  const int n_ksteps = SW >> 4;
-  const uint32_t slice_bytes = (uint32_t)SW * 2u;
-  const uint32_t row_stride = slice_bytes + 16u;          // consecutive rows fall into different banks
-  uint2* xf = reinterpret_cast<uint2*>(tsm);              // [n_ksteps][NJ][3 terms][32 lanes]
-  unsigned char* ring = tsm + (size_t)n_ksteps * NJ * 3 * 32 * 8;  // [NS][16 rows][row_stride]
-  const uint32_t slot_bytes = 16u * row_stride;
-  constexpr int kQ = 4;                                    // warps per tile; they interleave the K steps
+  const int NS = a.up_slots;
+  const Blk k = make_blk(a.B, a.D, a.C, a.SW, ks, a.check, a.status);
+  uint2* xf = reinterpret_cast<uint2*>(tsm);  // [n_ksteps][NJ][3 terms][32 lanes]
+  unsigned char* ring = tsm + xf_bytes(k);    // [NS][kTileRows][row_stride]
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) {
@@ -169,16 +488,14 @@ __global__ void __launch_bounds__(kUpThreads, 1) k_mlp_tc_up(TcArgs a) {
   __syncthreads();
   pdl_launch_dependents();
 
-  const int n = checked_count(a);
+  const int n = checked_count(k, a.n_ptr);
   const int r_begin = (int)(((long long)n * rb) / RB);
   const int r_end = (int)(((long long)n * (rb + 1)) / RB);
   const int n_tiles = (r_end - r_begin + kUpTile - 1) / kUpTile;
 
-  if (wid == kUpWarps) {
+  if (wid == kWarps) {
     // ---- producer warp: weight rows do not depend on the previous kernel ----
-    const size_t slice_off = (size_t)ks * slice_bytes;
-    for (int i = lane; i < min(r_end - r_begin, kSlotCache); i += 32) s_slots[i] = checked_slot(a, r_begin + i);
-    __syncwarp();
+    fill_slot_cache(k, a.slots, s_slots, r_begin, r_end, lane);
     for (int t = 0; t < n_tiles; ++t) {
       const int slot = t % NS;
       if (t >= NS && !mbar_wait(&empty_bar[slot], (uint32_t)((t / NS - 1) & 1))) {
@@ -186,197 +503,66 @@ __global__ void __launch_bounds__(kUpThreads, 1) k_mlp_tc_up(TcArgs a) {
         break;
       }
       const int r0 = r_begin + t * kUpTile;
-      const int rows = min(kUpTile, r_end - r0);
-      if (lane == 0) mbar_expect_tx(&full_bar[slot], (uint32_t)rows * 2u * slice_bytes);
-      __syncwarp();
-      if (lane < rows) {
-        const int ri = r0 - r_begin + lane;
-        const size_t src = (size_t)(ri < kSlotCache ? s_slots[ri] : checked_slot(a, r0 + lane)) * D * 2 + slice_off;
-        unsigned char* dst = ring + (size_t)slot * slot_bytes + (size_t)lane * row_stride;
-        bulk_g2s(dst, a.gate + src, slice_bytes, &full_bar[slot]);
-        bulk_g2s(dst + (size_t)kUpTile * row_stride, a.up + src, slice_bytes, &full_bar[slot]);
-      }
+      issue_up_tile(k, a.gate, a.up, a.slots, s_slots, r_begin, r0, min(kUpTile, r_end - r0),
+                    ring + (size_t)slot * k.slot_bytes, &full_bar[slot], lane);
     }
     return;
   }
 
-  // ---- consumers: B fragments of the x slice (depends on the previous kernel) ----
+  // ---- consumers: everything that depends on the previous kernel ----
   pdl_wait_prior();
-  constexpr int kC = kUpWarps * 32;
-  {
-    // item = (K step, sequence group, lane): the four x values behind that lane's b0/b1.
-    // A thread's items all belong to one sequence (kC / 32 is a multiple of NJ).
-    const int items = n_ksteps * NJ * 32;
-    const bool has_b = a.xb != nullptr;
-    const int g = lane >> 2, q = lane & 3;
-    float ss = 0.f;
-    for (int base = tid; base < items; base += kC * kUpBatch) {
-      float2 va[kUpBatch][2], vb[kUpBatch][2];
-#pragma unroll
-      for (int u = 0; u < kUpBatch; ++u) {
-        const int it = base + u * kC, pair = it >> 5;
-        const int b = 8 * (pair % NJ) + g;
-        va[u][0] = va[u][1] = vb[u][0] = vb[u][1] = make_float2(0.f, 0.f);
-        if (it < items && b < a.B) {
-          const size_t gi = (size_t)b * D + (size_t)ks * SW + (size_t)(pair / NJ) * 16 + 2 * q;
-          va[u][0] = __ldcg(reinterpret_cast<const float2*>(a.xa + gi));
-          va[u][1] = __ldcg(reinterpret_cast<const float2*>(a.xa + gi + 8));
-          if (has_b) {
-            vb[u][0] = __ldcg(reinterpret_cast<const float2*>(a.xb + gi));
-            vb[u][1] = __ldcg(reinterpret_cast<const float2*>(a.xb + gi + 8));
-          }
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < kUpBatch; ++u) {
-        const int it = base + u * kC, pair = it >> 5;
-        if (it < items) {
-          const float2 lo = make_float2(va[u][0].x + vb[u][0].x, va[u][0].y + vb[u][0].y);
-          const float2 hi = make_float2(va[u][1].x + vb[u][1].x, va[u][1].y + vb[u][1].y);
-          uint32_t l0[3], l1[3], h0[3], h1[3];
-          split3(lo.x, l0[0], l0[1], l0[2]);
-          split3(lo.y, l1[0], l1[1], l1[2]);
-          split3(hi.x, h0[0], h0[1], h0[2]);
-          split3(hi.y, h1[0], h1[1], h1[2]);
-#pragma unroll
-          for (int e = 0; e < 3; ++e)
-            xf[((size_t)pair * 3 + e) * 32 + lane] = make_uint2(pack2(l0[e], l1[e]), pack2(h0[e], h1[e]));
-          ss += lo.x * lo.x + lo.y * lo.y + hi.x * hi.x + hi.y * hi.y;
-          const int b = 8 * (pair % NJ) + g;
-          if (rb == 0 && b < a.B) {
-            const size_t gi = (size_t)b * D + (size_t)ks * SW + (size_t)(pair / NJ) * 16 + 2 * q;
-            if (a.x_store) {
-              *reinterpret_cast<float2*>(a.x_store + gi) = lo;
-              *reinterpret_cast<float2*>(a.x_store + gi + 8) = hi;
-            }
-            if (a.zero_out) {
-              *reinterpret_cast<float2*>(a.zero_out + gi) = make_float2(0.f, 0.f);
-              *reinterpret_cast<float2*>(a.zero_out + gi + 8) = make_float2(0.f, 0.f);
-            }
-          }
-        }
-      }
-    }
-    if (rb == 0 && a.normalize) {
-      // this slice's share of sum(x^2): lanes 4g..4g+3 hold parts of the same sequence
-      ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-      ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-      const int b = 8 * (wid % NJ) + g;
-      if (q == 0 && b < a.B) atomicAdd(a.ssq + b, ss);
-    }
-  }
-  consumer_sync<kC>();
-  if (wid >= kQ * NS) return;  // warps beyond the tile slots only helped with the prologue
+  build_x_fragments<4 * NJ>(k, ks, a.xa, a.xb, a.x_store, a.zero_out, a.normalize ? a.ssq : nullptr, rb == 0, xf, tid);
+  consumer_sync();
+  if (wid >= kQ * NS) return;  // warps beyond the tile slots only helped with the fragments
 
   const int slot = wid % NS, kq = wid / NS;
-  const int g = lane >> 2, q = lane & 3;
-  const bool two = NJ == 2;
-  const uint32_t a_lane = (uint32_t)(lane & 15) * row_stride + (uint32_t)(lane >> 4) * 16u;
   const uint32_t ring_addr = smem_addr(ring);
-  const uint2* xf_lane = xf + lane;
-  const int kstep_stride = NJ * 3 * 32;  // uint2 units
-
   for (int t = slot; t < n_tiles; t += NS) {
     if (!__all_sync(0xffffffffu, mbar_wait(&full_bar[slot], (uint32_t)((t / NS) & 1)))) {
       if (lane == 0) atomicOr(a.status, kStatTimeout);
       break;
     }
-    float acc[2][3][4];
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-      for (int e = 0; e < 3; ++e)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[j][e][i] = 0.f;
-    const uint32_t a_base = ring_addr + (uint32_t)slot * slot_bytes + a_lane;
-#pragma unroll 2
-    for (int kstep = kq; kstep < n_ksteps; kstep += kQ) {
-      uint32_t af[4];
-      ldsm_x4(af, a_base + (uint32_t)kstep * 32u);
-      const uint2* xp = xf_lane + (size_t)kstep * kstep_stride;
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        if (j == 0 || two) {
-#pragma unroll
-          for (int e = 0; e < 3; ++e) {
-            const uint2 b = xp[(j * 3 + e) * 32];
-            mma_16816(acc[j][e], af[0], af[1], af[2], af[3], b.x, b.y);
-          }
-        }
-      }
-    }
+    float acc[NJ][3][4];
+    up_tile_mma_n<NJ>(k, xf, ring_addr + (uint32_t)slot * k.slot_bytes, kq, kQ, lane, acc);
     __syncwarp();
     if (lane == 0) mbar_arrive(&empty_bar[slot]);  // this warp is done with the tile's rows
-
-    // Rows g (gate of record g) and g + 8 (up of record g); columns = sequences 8j + 2q, +1.
-    // Lane pairs trade halves so that even-q lanes add four consecutive sequences of the gate
-    // row and odd-q lanes the same four of the up row: every reduction is 16 bytes wide.
     const int r0 = r_begin + t * kUpTile;
-    const bool odd = q & 1;
-    const bool row_ok = g < min(kUpTile, r_end - r0);
-    float* dst = a.gu + ((size_t)(r0 + g) * 2 + (odd ? 1 : 0)) * kSeq + (q & ~1) * 2;
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      if (j == 0 || two) {
-        const float g0 = acc[j][0][0] + acc[j][1][0] + acc[j][2][0], g1 = acc[j][0][1] + acc[j][1][1] + acc[j][2][1];
-        const float u0 = acc[j][0][2] + acc[j][1][2] + acc[j][2][2], u1 = acc[j][0][3] + acc[j][1][3] + acc[j][2][3];
-        const float ra = __shfl_xor_sync(0xffffffffu, odd ? g0 : u0, 1);
-        const float rbv = __shfl_xor_sync(0xffffffffu, odd ? g1 : u1, 1);
-        if (row_ok && 8 * j + (q & ~1) * 2 < a.B) {
-          if (odd)
-            red_add_v4(dst + 8 * j, ra, rbv, u0, u1);
-          else
-            red_add_v4(dst + 8 * j, g0, g1, ra, rbv);
-        }
-      }
-    }
+    up_tile_reds<NJ>(k, acc, a.gu, r0, min(kUpTile, r_end - r0), lane);
   }
 }
 
-// ---------------------------------------------------------------------------
-// Phase 2: h[b][r] = silu(inv_b * GU[r][0][b]) * inv_b * GU[r][1][b];
-//          y[b][slice] += sum_r h[b][r] * downT[s_r][slice].
-// MMA shape: rows = sequences, K = 16 records, columns = 8 output columns.  The three terms of
-// h share one accumulator: a first MMA carries t0 in rows 0-7 and t1 in rows 8-15 (both of
-// sequence g), a second one t2 in rows 0-7; rows g and g + 8 are added at the end.
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(kDownThreads, 1) k_mlp_tc_down(TcArgs a) {
+template <int NJ>
+__global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_down(TcArgs a) {
   extern __shared__ __align__(128) unsigned char tsm[];
-  __shared__ __align__(8) uint64_t full_bar[kDownMaxSlots];
-  __shared__ __align__(8) uint64_t empty_bar[kDownMaxSlots];
+  __shared__ __align__(8) uint64_t full_bar[kMaxSlots];
+  __shared__ __align__(8) uint64_t empty_bar[kMaxSlots];
   __shared__ float s_inv[kSeq];
   __shared__ int s_slots[kSlotCache];
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int rb = blockIdx.x, RB = gridDim.x, cs = blockIdx.y;
-  const int D = a.D, SW = a.SW, NS = a.down_slots;
-  constexpr int hs_stride = kDownChunk + kXPad;             // floats per sequence
-  const uint32_t slice_bytes = (uint32_t)SW * 2u;
-  const uint32_t row_stride = slice_bytes + 16u;
-  float* hs = reinterpret_cast<float*>(tsm);                // [kSeq][kDownChunk + kXPad]
-  unsigned char* ring = tsm + (size_t)kSeq * hs_stride * 4;  // [NS][16 rows][row_stride]
-  const uint32_t slot_bytes = (uint32_t)kDownTile * row_stride;
+  const int NS = a.down_slots;
+  const Blk k = make_blk(a.B, a.D, a.C, a.SW, cs, a.check, a.status);
+  float* hs = reinterpret_cast<float*>(tsm);  // [kSeq][kHsStride]
+  unsigned char* ring = tsm + kHsBytes;       // [NS][kTileRows][row_stride]
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) {
       mbar_init(&full_bar[i], 1);
-      mbar_init(&empty_bar[i], kDownWarps);
+      mbar_init(&empty_bar[i], kWarps);
     }
     fence_barrier_init();
   }
   __syncthreads();
   pdl_launch_dependents();
 
-  const int n = checked_count(a);
+  const int n = checked_count(k, a.n_ptr);
   const int r_begin = (int)(((long long)n * rb) / RB);
   const int r_end = (int)(((long long)n * (rb + 1)) / RB);
   const int n_tiles = (r_end - r_begin + kDownTile - 1) / kDownTile;
 
-  if (wid == kDownWarps) {
-    // ---- producer warp ----
-    const size_t slice_off = (size_t)cs * slice_bytes;
-    for (int i = lane; i < min(r_end - r_begin, kSlotCache); i += 32) s_slots[i] = checked_slot(a, r_begin + i);
-    __syncwarp();
+  if (wid == kWarps) {
+    fill_slot_cache(k, a.slots, s_slots, r_begin, r_end, lane);
     for (int t = 0; t < n_tiles; ++t) {
       const int slot = t % NS;
       if (t >= NS && !mbar_wait(&empty_bar[slot], (uint32_t)((t / NS - 1) & 1))) {
@@ -384,71 +570,33 @@ __global__ void __launch_bounds__(kDownThreads, 1) k_mlp_tc_down(TcArgs a) {
         break;
       }
       const int r0 = r_begin + t * kDownTile;
-      const int rows = min(kDownTile, r_end - r0);
-      if (lane == 0) mbar_expect_tx(&full_bar[slot], (uint32_t)kDownTile * slice_bytes);
-      __syncwarp();
-      if (lane < kDownTile) {
-        // a short last tile repeats its last record: those rows meet h = 0, and the shared
-        // memory they would otherwise leave stale could hold anything
-        const int r = r0 + min(lane, rows - 1);
-        const int ri = r - r_begin;
-        const size_t src = (size_t)(ri < kSlotCache ? s_slots[ri] : checked_slot(a, r)) * D * 2 + slice_off;
-        bulk_g2s(ring + (size_t)slot * slot_bytes + (size_t)lane * row_stride, a.downT + src, slice_bytes,
-                 &full_bar[slot]);
-      }
+      issue_down_tile(k, a.downT, a.slots, s_slots, r_begin, r0, min(kDownTile, r_end - r0),
+                      ring + (size_t)slot * k.slot_bytes, &full_bar[slot], lane);
     }
     return;
   }
 
-  // ---- consumers ----
   pdl_wait_prior();
-  constexpr int kC = kDownWarps * 32;
-  if (tid < kSeq) s_inv[tid] = a.normalize ? rsqrtf(__ldcg(a.ssq + tid) / (float)D + kRmsEps) : 1.f;
-  {
-    // clear the next layer's accumulators (every block a share)
-    const int nblk = RB * gridDim.y, bid = cs * RB + rb;
-    if (a.gu_next) {
-      const size_t total = (size_t)a.C * 2 * kSeq / 4;  // float4 units
-      const size_t lo = total * bid / nblk, hi = total * (bid + 1) / nblk;
-      float4* p = reinterpret_cast<float4*>(a.gu_next);
-      for (size_t i = lo + tid; i < hi; i += kC) p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    if (a.ssq_next && bid == 0 && tid < kSeq) a.ssq_next[tid] = 0.f;
-  }
-  consumer_sync<kC>();
+  if (tid < kSeq) s_inv[tid] = a.normalize ? rsqrtf(__ldcg(a.ssq + tid) / (float)a.D + kRmsEps) : 1.f;
+  clear_next(a.gu_next, a.ssq_next, a.C, cs * RB + rb, RB * gridDim.y, tid);
+  consumer_sync();
 
-  const int g = lane >> 2, q = lane & 3;
-  const int n_mt = a.B > 8 ? 2 : 1;
-  const int nt0 = wid * 8;                        // this warp's first n-tile of the slice
-  const int my_nt = max(0, min(8, SW / 8 - nt0));  // n-tiles it owns (even: SW % 16 == 0)
-  float acc[2][8][4];
+  const int nt0 = wid * 8;                           // this warp's first n-tile of the slice
+  const int my_nt = max(0, min(8, a.SW / 8 - nt0));  // n-tiles it owns (even: SW % 16 == 0)
+  float acc[NJ][8][4];
 #pragma unroll
-  for (int m = 0; m < 2; ++m)
+  for (int m = 0; m < NJ; ++m)
 #pragma unroll
     for (int j = 0; j < 8; ++j)
 #pragma unroll
       for (int i = 0; i < 4; ++i) acc[m][j][i] = 0.f;
-  // ldmatrix.trans lane address: matrices 0/1 = records 0-7 / 8-15 of n-tile j, 2/3 = the same of n-tile j + 1
-  const uint32_t b_lane = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * row_stride +
-                          (uint32_t)(nt0 + (lane >> 4)) * 16u;
   const uint32_t ring_addr = smem_addr(ring);
   bool ok = true;
 
   for (int c0 = r_begin; c0 < r_end; c0 += kDownChunk) {
     const int rows_c = min(kDownChunk, r_end - c0);
-    const int rows_pad = (rows_c + kDownTile - 1) / kDownTile * kDownTile;
-    for (int i = tid; i < rows_pad * kSeq; i += kC) {
-      const int rec = i / kSeq, b = i % kSeq;
-      float h = 0.f;
-      if (rec < rows_c && b < a.B) {
-        const float* p = a.gu + (size_t)(c0 + rec) * 2 * kSeq + b;
-        const float gs = __ldcg(p) * s_inv[b], us = __ldcg(p + kSeq) * s_inv[b];
-        h = gs / (1.f + __expf(-gs)) * us;
-      }
-      hs[(size_t)b * hs_stride + rec] = h;
-    }
-    consumer_sync<kC>();
-
+    down_activations(k, a.gu, s_inv, hs, c0, rows_c, tid);
+    consumer_sync();
     for (int rl = 0; rl < rows_c; rl += kDownTile) {
       const int t = (c0 - r_begin + rl) / kDownTile;
       const int slot = t % NS;
@@ -459,98 +607,18 @@ __global__ void __launch_bounds__(kDownThreads, 1) k_mlp_tc_down(TcArgs a) {
         ok = false;
       }
       if (!ok) continue;
-      // A fragments: the three terms of h[8m + g][rl + 2q, +1, +8, +9]
-      uint32_t a1[2][4], a2[2][2];
-#pragma unroll
-      for (int m = 0; m < 2; ++m) {
-        if (m < n_mt) {
-          const float* hp = hs + (size_t)(8 * m + g) * hs_stride + rl + 2 * q;
-          const float2 lo = *reinterpret_cast<const float2*>(hp);
-          const float2 hi = *reinterpret_cast<const float2*>(hp + 8);
-          uint32_t l0[3], l1[3], h0[3], h1[3];
-          split3(lo.x, l0[0], l0[1], l0[2]);
-          split3(lo.y, l1[0], l1[1], l1[2]);
-          split3(hi.x, h0[0], h0[1], h0[2]);
-          split3(hi.y, h1[0], h1[1], h1[2]);
-          a1[m][0] = pack2(l0[0], l1[0]);  // row g:     t0, records 2q, 2q+1
-          a1[m][1] = pack2(l0[1], l1[1]);  // row g + 8: t1
-          a1[m][2] = pack2(h0[0], h1[0]);  // row g:     t0, records 2q+8, 2q+9
-          a1[m][3] = pack2(h0[1], h1[1]);  // row g + 8: t1
-          a2[m][0] = pack2(l0[2], l1[2]);  // row g:     t2
-          a2[m][1] = pack2(h0[2], h1[2]);
-        }
-      }
-      const uint32_t b_base = ring_addr + (uint32_t)slot * slot_bytes + b_lane;
-      // two halves of four n-tiles: fragment loads first, then a round of MMAs with (t0 | t1)
-      // and a round with t2, eight independent accumulators per round
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        if (4 * hf < my_nt) {
-          uint32_t bf[2][4];
-#pragma unroll
-          for (int p2 = 0; p2 < 2; ++p2)
-            if (4 * hf + 2 * p2 < my_nt) ldsm_x4_trans(bf[p2], b_base + (uint32_t)(2 * hf + p2) * 32u);
-#pragma unroll
-          for (int p2 = 0; p2 < 2; ++p2) {
-            if (4 * hf + 2 * p2 < my_nt) {
-              const int j = 4 * hf + 2 * p2;
-#pragma unroll
-              for (int m = 0; m < 2; ++m) {
-                if (m < n_mt) {
-                  mma_16816(acc[m][j], a1[m][0], a1[m][1], a1[m][2], a1[m][3], bf[p2][0], bf[p2][1]);
-                  mma_16816(acc[m][j + 1], a1[m][0], a1[m][1], a1[m][2], a1[m][3], bf[p2][2], bf[p2][3]);
-                }
-              }
-            }
-          }
-#pragma unroll
-          for (int p2 = 0; p2 < 2; ++p2) {
-            if (4 * hf + 2 * p2 < my_nt) {
-              const int j = 4 * hf + 2 * p2;
-#pragma unroll
-              for (int m = 0; m < 2; ++m) {
-                if (m < n_mt) {
-                  mma_16816(acc[m][j], a2[m][0], 0u, a2[m][1], 0u, bf[p2][0], bf[p2][1]);
-                  mma_16816(acc[m][j + 1], a2[m][0], 0u, a2[m][1], 0u, bf[p2][2], bf[p2][3]);
-                }
-              }
-            }
-          }
-        }
-      }
+      down_tile_mma<NJ>(k, hs, rl, ring_addr + (uint32_t)slot * k.slot_bytes, nt0, my_nt, lane, acc);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[slot]);
     }
-    consumer_sync<kC>();  // hs is rewritten by the next chunk
+    consumer_sync();  // hs is rewritten by the next chunk
   }
-
-  // y[seq][slice columns]: rows g and g + 8 of an accumulator belong to the same sequence.
-  // Even-q lanes end up with four consecutive columns of sequence g, odd-q lanes with the
-  // same four columns of sequence 8 + g, so every reduction is 16 bytes wide.
-  if (r_end > r_begin && ok) {
-    const bool odd = q & 1;
-    const int seq = odd ? 8 + g : g;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if (j < my_nt) {
-        const float m0a = acc[0][j][0] + acc[0][j][2], m0b = acc[0][j][1] + acc[0][j][3];
-        const float m1a = acc[1][j][0] + acc[1][j][2], m1b = acc[1][j][1] + acc[1][j][3];
-        const float ra = __shfl_xor_sync(0xffffffffu, odd ? m0a : m1a, 1);
-        const float rbv = __shfl_xor_sync(0xffffffffu, odd ? m0b : m1b, 1);
-        if (seq < a.B) {
-          float* dst = a.yacc + (size_t)seq * D + (size_t)cs * SW + (size_t)(nt0 + j) * 8 + (q & ~1) * 2;
-          if (odd)
-            red_add_v4(dst, ra, rbv, m1a, m1b);
-          else
-            red_add_v4(dst, m0a, m0b, ra, rbv);
-        }
-      }
-    }
-  }
+  if (r_end > r_begin && ok) down_reds<NJ>(k, acc, a.yacc + (size_t)cs * a.SW, nt0, my_nt, lane);
 }
 
 struct TcPlan {
-  int KS, SW, RB, up_slots, down_slots;
+  int KS, SW, RB;
+  int up_slots, down_slots;
   size_t smem_up, smem_down;
 };
 
@@ -567,29 +635,25 @@ bool tc_plan(const Dims& d, int sm_count, int B, TcPlan* p) {
   p->KS = ks;
   p->SW = d.D / ks;
   p->RB = std::max(1, sm_count / ks);
-  const size_t row_stride = (size_t)p->SW * 2 + 16;
+  const size_t slot_bytes = (size_t)kTileRows * ((size_t)p->SW * 2 + 16);
   const size_t budget = 220 * 1024;
-  const size_t xf_bytes = (size_t)(p->SW / 16) * (B > 8 ? 2 : 1) * 3 * 32 * 8;
-  if (xf_bytes + 16 * row_stride > budget) return false;
-  p->up_slots = (int)std::min<size_t>(kUpSlots, (budget - xf_bytes) / (16 * row_stride));
-  if (d.ring_stages > 0) p->up_slots = std::min(p->up_slots, d.ring_stages);
-  p->smem_up = xf_bytes + (size_t)p->up_slots * 16 * row_stride;
-  const size_t hs_bytes = (size_t)kSeq * (kDownChunk + kXPad) * 4;
-  int ns = (int)std::min<size_t>(kDownMaxSlots, (budget - hs_bytes) / (kDownTile * row_stride));
-  if (d.ring_stages > 0) ns = std::min(ns, std::max(2, d.ring_stages));
-  if (ns < 1) return false;
-  p->down_slots = ns;
-  p->smem_down = hs_bytes + (size_t)ns * kDownTile * row_stride;
+  const size_t xf = (size_t)(p->SW / 16) * (B > 8 ? 2 : 1) * 3 * 32 * 8;
+  if (std::max(xf, kHsBytes) + slot_bytes > budget) return false;
+  const int cap = d.ring_stages > 0 ? std::min(kMaxSlots, d.ring_stages) : kMaxSlots;
+  p->up_slots = (int)std::min<size_t>(std::min(cap, kWarps / kQ), (budget - xf) / slot_bytes);
+  p->down_slots = (int)std::min<size_t>(cap, (budget - kHsBytes) / slot_bytes);
+  p->smem_up = xf + (size_t)p->up_slots * slot_bytes;
+  p->smem_down = kHsBytes + (size_t)p->down_slots * slot_bytes;
   return true;
 }
 
 template <typename K>
-cudaError_t tc_launch(K kfn, dim3 grid, int threads, size_t smem, const TcArgs& ka, cudaStream_t s) {
+cudaError_t tc_launch(K kfn, dim3 grid, size_t smem, const TcArgs& ka, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(threads);
+  cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
@@ -637,9 +701,12 @@ cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s
   ka.up_slots = p.up_slots;
   ka.down_slots = p.down_slots;
   const dim3 grid(p.RB, p.KS);
-  cudaError_t e = tc_launch(k_mlp_tc_up, grid, kUpThreads, p.smem_up, ka, s);
-  if (e != cudaSuccess) return e;
-  return tc_launch(k_mlp_tc_down, grid, kDownThreads, p.smem_down, ka, s);
+  if (a.B > 8) {
+    cudaError_t e = tc_launch(k_mlp_tc_up<2>, grid, p.smem_up, ka, s);
+    return e != cudaSuccess ? e : tc_launch(k_mlp_tc_down<2>, grid, p.smem_down, ka, s);
+  }
+  cudaError_t e = tc_launch(k_mlp_tc_up<1>, grid, p.smem_up, ka, s);
+  return e != cudaSuccess ? e : tc_launch(k_mlp_tc_down<1>, grid, p.smem_down, ka, s);
 }
 
 }  // namespace npi
