@@ -401,6 +401,14 @@ def cuda_arm(args):
     if args.layer_launches or args.direct_loads or Bq > 1:
         chain_layers = 1
     n_launch = -(-L // chain_layers)                                # MLP kernel launches per chain
+    if chain_layers > 1:
+        mlp_kernel = "k_mlp_chain"
+    elif args.direct_loads:
+        mlp_kernel = "k_sparse_mlp"
+    elif Bq > 1:
+        mlp_kernel = "k_mlp_tc_up + k_mlp_tc_down (the two launches of one layer)"
+    else:
+        mlp_kernel = "k_sparse_mlp_pipe"
     mlp_us = k0.elapsed_time(k1) * 1000.0 / (reps * n_launch)      # per launch, gaps included
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record(s)
@@ -444,7 +452,7 @@ def cuda_arm(args):
                 "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * L * rec), "d2h_bytes_per_step": int(Bq * D * 4)},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "k_mlp_chain" if chain_layers > 1 else "k_sparse_mlp_pipe", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": mlp_kernel, "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth (burst)",
                      "traffic": traffic, "us_per_launch": mlp_us, "bytes_per_launch": mlp_bytes,
                      "layers_per_launch": L / n_launch},
