@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=1, help="sequences per step (the metric's workload is 1)")
     ap.add_argument("--gamma", type=float, default=0.9, help="shared-driver weight of batched hidden states")
     ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
+    ap.add_argument("--no-variants", action="store_true",
+                    help="skip the extra measurement of the zero-copy transfer mode (default run only)")
     ap.add_argument("--selection", default="topk", choices=["topk", "centroid"],
                     help="topk: the metric's selection; centroid: centroid heads + bank lookup + gate AND up")
     ap.add_argument("--centroids", type=int, default=512, help="centroid vocabulary per head (centroid selection)")
@@ -462,6 +464,30 @@ def cuda_arm(args):
                       "mlp_chain_alone": mlp_us * n_launch},
         "setup_s": {"generate": gen_s},
     }
+
+    # ---- the same step with the other pinned-host transfer mode (reported beside, not as, the value) ----
+    if (args.transfer == "gather" and not args.no_variants and not centroid and Bq == 1
+            and args.config == "7b" and not (args.layer_launches or args.direct_loads)):
+        eng.close()
+        zcfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
+                              max_batch=Bq, evict_policy=policy, transfer_mode=nb.NP_XFER_ZERO_COPY,
+                              chain_layers=args.chain_layers)
+        eng = nb.Engine(zcfg, w1, w2, store, device=dev)
+        s, cs = eng.stream, eng.copy_stream
+        for t in range(0, 1 + W):
+            nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
+        barrier()
+        z0, z1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        z0.record(s)
+        for t in range(1 + W, T):
+            nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
+        z1.record(s)
+        barrier()
+        eng.counters()
+        (z_ms,) = max_over_ranks(dist, [z0.elapsed_time(z1)], dev)
+        result["variants"] = {"transfer=zerocopy": {
+            "value": K * world / (z_ms / 1000.0), "unit": UNIT, "ms_per_step": z_ms / K,
+            "note": "scatter kernel reads the pinned store over PCIe by neuron ID; no host packing, no staging copy"}}
 
     if rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid:
         n = args.cpu_baseline_steps
