@@ -175,6 +175,10 @@ struct np_ctx {
   std::vector<cudaEvent_t> ev_installed;
   std::vector<char> install_pending;
   cudaEvent_t ev_half[2] = {nullptr, nullptr};  // host staging halves in flight
+  // library-owned side streams of the install path: [0] runs the scatter kernels behind the
+  // staged copies; in zero-copy mode consecutive layers alternate between the two
+  cudaStream_t aux[2] = {nullptr, nullptr};
+  cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr}, ev_copied[2] = {nullptr, nullptr};
   bool half_pending[2] = {false, false};
   int next_half = 0;
   cudaEvent_t ev_t[4] = {nullptr, nullptr, nullptr, nullptr};  // compute-stream step timing
@@ -324,6 +328,12 @@ int np_destroy(np_ctx* ctx) {
     if (e) cudaEventDestroy(e);
   for (auto e : ctx->ev_half)
     if (e) cudaEventDestroy(e);
+  for (int i = 0; i < 2; ++i) {
+    if (ctx->ev_join[i]) cudaEventDestroy(ctx->ev_join[i]);
+    if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
+    if (ctx->aux[i]) cudaStreamDestroy(ctx->aux[i]);
+  }
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
   for (auto e : ctx->ev_t)
     if (e) cudaEventDestroy(e);
   for (auto e : ctx->ev_c)
@@ -449,6 +459,12 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   for (int l = 0; l < d.L; ++l)
     NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_installed[l], cudaEventDisableTiming));
   for (auto& e : ctx->ev_half) NP_INIT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  for (int i = 0; i < 2; ++i) {
+    NP_INIT_CUDA(cudaStreamCreateWithFlags(&ctx->aux[i], cudaStreamNonBlocking));
+    NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming));
+    NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming));
+  }
+  NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
   for (auto& e : ctx->ev_t) NP_INIT_CUDA(cudaEventCreate(&e));
   for (auto& e : ctx->ev_c) NP_INIT_CUDA(cudaEventCreate(&e));
 
@@ -559,10 +575,28 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
   const size_t row_bytes = (size_t)d.D * 2;
   NP_CUDA(ctx, cudaStreamWaitEvent(cs, ctx->ev_delta, 0));
   int warn = NP_OK;
+  // Side streams: ordered after everything the caller's copy stream holds so far, and joined
+  // back into it at the end, so the caller sees one stream's worth of ordering.
+  const bool forked = mode != NP_XFER_MEMCPY_RUNS;
+  if (forked) {
+    NP_CUDA(ctx, cudaEventRecord(ctx->ev_fork, cs));
+    for (int i = 0; i < 2; ++i) NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[i], ctx->ev_fork, 0));
+  }
+  auto join = [&]() -> cudaError_t {
+    for (int i = 0; i < 2; ++i) {
+      cudaError_t e = cudaEventRecord(ctx->ev_join[i], ctx->aux[i]);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, ctx->ev_join[i], 0);
+      if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+  };
 
   if (mode == NP_XFER_ZERO_COPY) {
+    // consecutive layers alternate between the two side streams: one kernel's tail (its last
+    // reads are still crossing PCIe) overlaps the next kernel's start
     const int max_rows = d.C;
     for (int l = layer_begin; l < layer_end; ++l) {
+      cudaStream_t zs = ctx->aux[l & 1];
       const char* store_l = ctx->backing_dev + (size_t)l * d.M * rec;
       NP_LAUNCH(ctx, launch_scatter(d, store_l, true, ctx->t.delta_ids + (size_t)l * d.C,
                                   ctx->t.delta_slots + (size_t)l * d.C,
@@ -570,10 +604,11 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
                                   static_cast<char*>(ctx->bufs.gate_buf) + (size_t)l * d.C * row_bytes,
                                   static_cast<char*>(ctx->bufs.up_buf) + (size_t)l * d.C * row_bytes,
                                   static_cast<char*>(ctx->bufs.downT_buf) + (size_t)l * d.C * row_bytes,
-                                  ctx->t.status, check, cs, ctx->sm_count));
-      NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], cs));
+                                  ctx->t.status, check, zs, ctx->sm_count));
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], zs));
       ctx->install_pending[l] = 1;
     }
+    NP_CUDA(ctx, join());
     return NP_OK;
   }
 
@@ -645,16 +680,24 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
         if (ctx->pool) ctx->pool->parallel_for(parts, body);
         else for (int part = 0; part < parts; ++part) body(part);
         if (bad) return fail(ctx, NP_E_DEVICE, "layer %d: neuron id out of range", l);
+        // the copies queue back to back on the caller's stream; the scatter kernels follow them
+        // on a side stream, so a copy never waits for the previous layer's kernel
         NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)rows * rec, cudaMemcpyHostToDevice, cs));
-        NP_CUDA(ctx, cudaEventRecord(ctx->ev_half[h], cs));
-        ctx->half_pending[h] = true;
+        NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[h], cs));
+        NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[h], 0));
         NP_LAUNCH(ctx, launch_scatter(d, dbuf, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
-                                    down_l, ctx->t.status, check, cs, ctx->sm_count));
+                                    down_l, ctx->t.status, check, ctx->aux[0], ctx->sm_count));
+        NP_CUDA(ctx, cudaEventRecord(ctx->ev_half[h], ctx->aux[0]));  // both copies of the half are free again
+        ctx->half_pending[h] = true;
       }
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], ctx->aux[0]));
+      ctx->install_pending[l] = 1;
+      continue;
     }
     NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], cs));
     ctx->install_pending[l] = 1;
   }
+  if (forked) NP_CUDA(ctx, join());
   return warn;
 }
 
