@@ -220,7 +220,10 @@ int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream);
  * (L, n) = bytes [(l*M + n)*REC, +REC) of the store to slot S[n] of the three
  * row buffers, on `copy_stream`, and mark each layer installed (np_sparse_mlp
  * orders itself after that mark).  The copy stream is first ordered after the
- * delta step.  With NP_XFER_MEMCPY_RUNS / NP_XFER_HOST_GATHER this call blocks
+ * delta step.  Scatter kernels may run on streams the library owns; those are
+ * ordered after the work `copy_stream` held on entry and joined back into it
+ * before the call returns, so work queued on `copy_stream` afterwards sees
+ * every row installed.  With NP_XFER_MEMCPY_RUNS / NP_XFER_HOST_GATHER this call blocks
  * the host until the delta lists of the last np_delta are readable; with
  * NP_XFER_ZERO_COPY it never blocks.  Deltas larger than staging_rows are split
  * into chunks in list order (result unchanged).
