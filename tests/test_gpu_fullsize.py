@@ -92,3 +92,35 @@ def test_larger_shapes_few_layers(name, n_layers, mode):
         p.check_resident_bytes()
     finally:
         p.close()
+
+
+def test_stress_shape_batch16_few_layers():
+    """Sixteen sequences at the 7B row shape (the delta-stress workload) on four layers: the
+    tensor-core predictor and the tensor-core batch MLP in the configuration bench.py --batch 16
+    times; unions of the per-sequence sets, tables bit-exact, chain within tolerance."""
+    cfg = synth.CONFIGS["stress"].with_(n_layers=4)
+    L, M, D, B = cfg.n_layers, cfg.d_ffn, cfg.d_model, 16
+    p = Pair(cfg, max_batch=B, transfer_mode=nb.NP_XFER_HOST_GATHER, staging_rows=2 * cfg.top_k, flags=0,
+             gen_device="cuda")
+    try:
+        xs = synth.hidden_states(cfg, 3, batch=B, gamma=0.9)
+        logits = torch.empty((B, L, M), dtype=torch.float32, device="cuda")
+        out = torch.empty((B, D), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, B, logits, None, p.eng.stream)
+            rc = nb.np_step(p.eng.ctx, x, B, out, p.eng.stream, p.eng.copy_stream)
+            assert rc in (nb.NP_OK, nb.NP_W_CHUNKED)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            z = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)
+            assert rel_l2(z32, z) < 1e-5
+            res = p.ora.step(u16(xs[t]), logits_f32=z32)
+            cnt = p.check_delta_against(res["deltas"])
+            assert (cnt[:, nb.NP_CNT_PRED] > 1.5 * p.k).all() and (cnt[:, nb.NP_CNT_OVERFLOW] == 0).all()
+            got = out.cpu().numpy()
+            for b in range(B):
+                assert rel_l2(got[b], res["x_final"][b]) < 1e-5, (t, b)
+        p.check_resident_bytes()
+    finally:
+        p.close()
