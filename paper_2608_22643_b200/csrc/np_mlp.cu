@@ -523,11 +523,11 @@ template <int NB, int COLS>
 static cudaError_t mlp_launch_cols(const MlpKernelArgs& ka, int groups, int grid_x, cudaStream_t s) {
   const size_t sm = ((size_t)NB * ka.D + (size_t)NB * kTileRows * kMaxSeg * 2 + NB * kTileRows) * 4;
   auto kfn = k_sparse_mlp<NB, COLS>;
-  static size_t configured = 0;
-  if (sm > 48 * 1024 && sm > configured) {
+  // set on every launch: the attribute belongs to the current device's context, and a cache in
+  // this function would be shared by all devices and threads of the process
+  if (sm > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    configured = sm;
   }
   dim3 grid(grid_x, groups);
   kfn<<<grid, kMlpThreads, sm, s>>>(ka);

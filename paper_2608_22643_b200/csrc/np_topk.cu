@@ -143,11 +143,10 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
 cudaError_t launch_topk(const Dims& d, const float* logits, int B, uint32_t* bitmap, cudaStream_t s) {
   const int W = d.W;
   const size_t sm = (size_t)d.M * 4 + (size_t)W * 4 + 32 * 256 * 4 + 256 * 4 + 40 * 4;
-  static size_t configured = 0;
-  if (sm > 48 * 1024 && sm > configured) {
+  // set on every launch: the attribute belongs to the current device's context
+  if (sm > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k_topk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    configured = sm;
   }
   const int use_atomic = B > 1 ? 1 : 0;
   if (use_atomic) {
