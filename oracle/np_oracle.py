@@ -24,7 +24,9 @@ RMS, scale invariance and a hand value for ``rms_normalize``.
 
 Parity unpinned against the paper (the paper is silent; these are this build's
 definitions, pinned only by invariants and determinism): the victim order of
-the LRU policy, and the truncation rule when a predicted set exceeds capacity.
+the LRU policy, the truncation rule when a predicted set exceeds capacity, and
+``dense_prefix_plan`` against the paper's own operating points (found there by
+a throughput sweep on its device, not by a formula).
 """
 from __future__ import annotations
 
@@ -45,6 +47,21 @@ def record_bytes(D: int, elem_bytes: int = 2) -> int:
 def resident_buffer_bytes(C: int, D: int, elem_bytes: int = 2) -> int:
     """Bytes of one layer's resident row buffers (three projections, C rows each)."""
     return C * record_bytes(D, elem_bytes)
+
+
+def dense_prefix_plan(L: int, M: int, D: int, C: int, budget_bytes: int, fixed_bytes: int = 0,
+                      elem_bytes: int = 2) -> int:
+    """Largest dense prefix d (Section 3.1: "the largest dense prefix that fits within the
+    memory budget"): d dense layers hold all M records, the other L - d layers a resident
+    buffer of C records each, next to ``fixed_bytes`` of other resident state.  Returns -1 when
+    not even d = 0 fits.  (The paper finds its operating point by a throughput sweep on its
+    device; this is the memory rule that sweep is described by.)"""
+    rec = record_bytes(D, elem_bytes)
+    best = -1
+    for d in range(L + 1):
+        if d * M * rec + (L - d) * C * rec + fixed_bytes <= budget_bytes:
+            best = d
+    return best
 
 
 def record_offset_bytes(layer: int, neuron: int, M: int, D: int) -> int:
@@ -341,8 +358,13 @@ def rms_normalize(x: np.ndarray) -> np.ndarray:
 class Engine:
     """State carried across decode steps: residency tables and resident buffers."""
 
-    def __init__(self, L, D, M, H, k, C, policy, w1_u16, w2_u16, backing_u16):
+    def __init__(self, L, D, M, H, k, C, policy, w1_u16, w2_u16, backing_u16, dense_layers: int = 0):
+        """``dense_layers`` = d: the first d layers are dense (Section 3.1): all their rows are
+        resident and used, they are never predicted, diffed or installed; their entries of the
+        predicted bitmap are empty and their tables stay empty."""
+        assert 0 <= dense_layers <= L
         self.L, self.D, self.M, self.H, self.k, self.C = L, D, M, H, k, C
+        self.dense_layers = dense_layers
         self.w1, self.w2, self.backing = w1_u16, w2_u16, backing_u16
         self.res = Residency(L, M, C, policy)
         self.gate = np.zeros((L, C, D), dtype=np.uint16)
@@ -361,6 +383,9 @@ class Engine:
                 out["logits"] = z
                 logits_f32 = z.astype(np.float32)
             pred_words = topk_bitmap(logits_f32, self.k)
+        if self.dense_layers:
+            pred_words = np.array(pred_words, copy=True)
+            pred_words[:self.dense_layers] = 0
         out["pred"] = pred_words
         deltas = self.res.delta(pred_words)
         out["deltas"] = deltas
@@ -371,8 +396,12 @@ class Engine:
         x = bf16_to_f64(x_u16)
         ys = []
         xs = [x]
+        all_rows = np.arange(self.M)
         for l, d in enumerate(deltas):
-            y = sparse_mlp(self.gate, self.up, self.downT, l, d.active_slots, rms_normalize(x))
+            if l < self.dense_layers:
+                y = sparse_mlp_from_store(self.backing, l, all_rows, rms_normalize(x))
+            else:
+                y = sparse_mlp(self.gate, self.up, self.downT, l, d.active_slots, rms_normalize(x))
             ys.append(y)
             x = x + y
             xs.append(x)
