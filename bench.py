@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=1, help="sequences per step (the metric's workload is 1)")
     ap.add_argument("--gamma", type=float, default=0.9, help="shared-driver weight of batched hidden states")
     ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
+    ap.add_argument("--dense-layers", type=int, default=0,
+                    help="dense prefix: the first d layers stay whole on the GPU and take no part in selection or install")
     ap.add_argument("--no-variants", action="store_true",
                     help="skip the extra measurement of the zero-copy transfer mode (default run only)")
     ap.add_argument("--selection", default="topk", choices=["topk", "centroid"],
@@ -292,7 +294,7 @@ def cuda_arm(args):
     ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
                           max_batch=args.batch, evict_policy=policy, transfer_mode=mode,
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
-                          host_threads=args.host_threads,
+                          host_threads=args.host_threads, dense_layers=args.dense_layers,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0))
     eng = nb.Engine(ncfg, w1, w2, store, device=dev)
@@ -354,6 +356,7 @@ def cuda_arm(args):
     ms_total = e0.elapsed_time(e1)
     eng.counters()
 
+    nd = args.dense_layers
     # ---- per-stage detail on a few more steady-state steps (untimed region) ----------------
     stage_us, delta_rows, overlap, overflow_steps = [], [], [], 0
     for i in range(n_detail):
@@ -361,11 +364,11 @@ def cuda_arm(args):
         step(xs_dev[t])
         stage_us.append(np.full(4, np.nan, np.float32) if centroid else nb.np_last_step_times(eng.ctx))
         c = eng.counters()
-        delta_rows.append(float(c[:, nb.NP_CNT_DELTA].mean()))
+        delta_rows.append(float(c[nd:, nb.NP_CNT_DELTA].mean()) if nd < L else 0.0)
         overflow_steps += int((c[:, nb.NP_CNT_OVERFLOW] > 0).any())
-        overlap.append(float((c[:, nb.NP_CNT_KEPT] / np.maximum(1, c[:, nb.NP_CNT_PRED])).mean()))
+        overlap.append(float((c[nd:, nb.NP_CNT_KEPT] / np.maximum(1, c[nd:, nb.NP_CNT_PRED])).mean()) if nd < L else 1.0)
     stage_us = np.median(np.stack(stage_us), axis=0)
-    n_active = float(eng.counters()[:, nb.NP_CNT_ACTIVE].mean())
+    n_active = float(eng.counters()[nd:, nb.NP_CNT_ACTIVE].mean()) if nd < L else 0.0
 
     # ---- end-to-end timing: hidden state from pinned host, result back to the host --------
     nb.np_reset(eng.ctx, s)
@@ -430,10 +433,16 @@ def cuda_arm(args):
     peak, peak_kind = measured_peaks()
     layer_bytes = n_active * rec + 4 * n_active + 8 * D          # rows + slot list + x in, y out
     mlp_bytes = layer_bytes * L / n_launch                       # one launch spans L / n_launch layers
+    if nd:
+        # with a dense prefix the figure covers the whole chain: d whole layers + the sparse rest
+        n_launch = 1
+        mlp_us = k0.elapsed_time(k1) * 1000.0 / reps
+        mlp_bytes = nd * (M * rec + 8 * D) + (L - nd) * layer_bytes
+        mlp_kernel = "whole MLP chain (dense prefix + sparse layers)"
     achieved = mlp_bytes / (mlp_us * 1e-6) / 1e9
     # DRAM bytes of one layer from the ncu capture in profiles/k_mlp_chain_7b.md (7B shape):
     # (216.63 MB read + 3.51 MB written) / 8 layers; scaled by the layers a launch spans
-    traffic = 27.52e6 * L / n_launch if cfg.name == "7b" else None
+    traffic = 27.52e6 * L / n_launch if cfg.name == "7b" and not nd else None
     pred_rows = L * 2 * args.centroids if centroid else L * M
     pred_bytes = 2 * cfg.d_pred * D + 2 * pred_rows * cfg.d_pred + 4 * pred_rows
     mean_delta = float(np.mean(delta_rows))
@@ -444,14 +453,15 @@ def cuda_arm(args):
         "config": {
             "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
                         f"B={Bq} rho={cfg.rho} policy={args.policy} transfer={args.transfer}"
-                        + (f" selection=centroid K={args.centroids}" if centroid else ""),
+                        + (f" selection=centroid K={args.centroids}" if centroid else "")
+                        + (f" dense_layers={args.dense_layers}" if args.dense_layers else ""),
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
             "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
             "active_rows_per_layer": n_active, "overflow_steps": int(overflow_steps),
             "replicas": world,
         },
         "e2e": {"value": K * world / (e2e_ms_total / 1000.0), "unit": UNIT,
-                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * L * rec), "d2h_bytes_per_step": int(Bq * D * 4)},
+                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * (L - nd) * rec), "d2h_bytes_per_step": int(Bq * D * 4)},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": mlp_kernel, "achieved": achieved, "peak": peak,
@@ -467,7 +477,7 @@ def cuda_arm(args):
 
     # ---- the same step with the other pinned-host transfer mode (reported beside, not as, the value) ----
     if (args.transfer == "gather" and not args.no_variants and not centroid and Bq == 1
-            and args.config == "7b" and not (args.layer_launches or args.direct_loads)):
+            and args.config == "7b" and not (args.layer_launches or args.direct_loads) and not args.dense_layers):
         eng.close()
         zcfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
                               max_batch=Bq, evict_policy=policy, transfer_mode=nb.NP_XFER_ZERO_COPY,
@@ -489,7 +499,7 @@ def cuda_arm(args):
             "value": K * world / (z_ms / 1000.0), "unit": UNIT, "ms_per_step": z_ms / K,
             "note": "scatter kernel reads the pinned store over PCIe by neuron ID; no host packing, no staging copy"}}
 
-    if rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid:
+    if rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid and not args.dense_layers:
         n = args.cpu_baseline_steps
         times = run_oracle_steps(cfg, args.policy, w1.cpu(), w2.cpu(), store, xs_host, n)
         sec = float(np.mean(times))

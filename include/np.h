@@ -43,7 +43,7 @@
 extern "C" {
 #endif
 
-#define NP_VERSION 1
+#define NP_VERSION 2
 
 /* return codes */
 #define NP_OK           0
@@ -109,7 +109,13 @@ typedef struct np_config {
                              (0 = a quarter of the stack) */
   int32_t ring_stages;    /* cap on the records the MLP kernels stage in shared memory
                              (0 = as many as fit; >= 2 otherwise) */
-  int32_t reserved[2];    /* must be 0 */
+  int32_t dense_layers;   /* d, 0 <= d <= L: the first d layers are dense (Section 3.1): all M
+                             records of each sit in dense_buf (copied from the store by
+                             np_init), every row is used, and the layers take no part in
+                             selection, delta or install: their rows of every bitmap read as
+                             empty and their tables stay empty.  d > 0 needs max_batch = 1 and
+                             neither NP_F_LAYER_LAUNCHES nor NP_F_DIRECT_LOADS */
+  int32_t reserved[1];    /* must be 0 */
 } np_config;
 
 /* Byte counts of the caller-owned buffers for a configuration. */
@@ -117,13 +123,14 @@ typedef struct np_sizes {
   uint64_t w1_bytes;          /* bf16 [H][D] */
   uint64_t w2_bytes;          /* bf16 [L*M][H] */
   uint64_t backing_bytes;     /* bf16 [L][M][3][D] */
-  uint64_t row_buffer_bytes;  /* bf16 [L][C][D], each of gate / up / downT */
+  uint64_t row_buffer_bytes;  /* bf16 [L - d][C][D], each of gate / up / downT (sparse layers only) */
   uint64_t staging_bytes;     /* staging_rows * REC (device; pinned host too for HOST_GATHER) */
   uint64_t workspace_bytes;   /* device scratch */
   uint64_t host_lists_bytes;  /* pinned host area the delta lists are mirrored into */
   uint64_t logits_bytes;      /* fp32 [max_batch][L][M] */
   uint64_t bitmap_bytes;      /* uint32 [L][W] */
   uint64_t record_bytes;      /* REC */
+  uint64_t dense_bytes;       /* bf16 [d][M][3][D]: the dense layers' records (0 when d = 0) */
 } np_sizes;
 
 typedef struct np_buffers {
@@ -137,6 +144,7 @@ typedef struct np_buffers {
   void* host_staging;      /* pinned host, staging_bytes; only for NP_XFER_HOST_GATHER */
   void* workspace;         /* dev, 256-byte aligned */
   void* host_lists;        /* pinned host */
+  void* dense_buf;         /* dev, dense_bytes; NULL when dense_layers = 0.  Filled by np_init */
 } np_buffers;
 
 /* Device views of one layer's lists from the last np_delta (valid until the next). */
@@ -156,6 +164,16 @@ int np_version(void);
 /* Fills *out with the buffer sizes `cfg` needs.  Pure host arithmetic (record
  * size: Section 3.5; buffer size: Section 4.3).  NP_E_INVAL on a bad config. */
 int np_query_sizes(const np_config* cfg, np_sizes* out);
+
+/* The dense/sparse split's memory rule (Section 3.1: "the largest dense prefix
+ * that fits within the memory budget"): the largest d in [0, L] with
+ *   d * M * REC + (L - d) * C * REC + fixed_bytes <= budget_bytes,
+ * i.e. d dense layers, resident buffers of C records for the rest, next to
+ * fixed_bytes of other resident state.  cfg->dense_layers is ignored.
+ * *d_out = -1 when not even d = 0 fits.  Pure host arithmetic.  (The paper
+ * finds its operating point by a throughput sweep on its device; this is the
+ * rule that sweep is described by.)  NP_E_INVAL on a bad config or NULL. */
+int np_plan_dense_prefix(const np_config* cfg, uint64_t budget_bytes, uint64_t fixed_bytes, int32_t* d_out);
 
 /* Creates a context with empty residency (the cold-start state of Section 3.4:
  * no row resident, every slot free).  Copies cfg; keeps the pointers in bufs.
@@ -182,6 +200,8 @@ const char* np_last_error(const np_ctx* ctx);
  *                sequence's k highest logits per layer; order = fp32 value
  *                descending (+0 above -0), ties to the lower neuron index
  * The bitmap is also kept inside the context for np_delta(ctx, NULL, ...).
+ * Dense layers (dense_layers > 0) are not scored: their logits are left
+ * untouched and their bitmap rows are zero.
  * Errors: NP_E_INVAL (NULL x, B outside 1..max_batch), NP_E_CUDA. */
 int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out,
                uint32_t* bitmap_out, void* stream);
@@ -237,6 +257,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
  * bf16 rows, fp32 accumulation; partial sums are combined with floating-point
  * atomics, so the last bits of y can differ between runs.
  * `stream` is first ordered after the layer's install mark.
+ * Dense layers run only inside np_mlp_chain / np_step (NP_E_INVAL here).
  * Errors: NP_E_STATE, NP_E_INVAL, NP_E_CUDA. */
 int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* y, void* stream);
 

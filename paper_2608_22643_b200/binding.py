@@ -32,7 +32,7 @@ NP_F_NO_TENSOR_CORES = 8
 NP_N_COUNTERS = 8
 
 EXPORTED = [
-    "np_version", "np_query_sizes", "np_init", "np_destroy", "np_reset", "np_last_error",
+    "np_version", "np_query_sizes", "np_plan_dense_prefix", "np_init", "np_destroy", "np_reset", "np_last_error",
     "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
     "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_last_error",
@@ -42,19 +42,20 @@ EXPORTED = [
 class np_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
-        "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers", "ring_stages")] + [("reserved", C.c_int32 * 2)]
+        "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers", "ring_stages",
+        "dense_layers")] + [("reserved", C.c_int32 * 1)]
 
 
 class np_sizes(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "w1_bytes", "w2_bytes", "backing_bytes", "row_buffer_bytes", "staging_bytes", "workspace_bytes",
-        "host_lists_bytes", "logits_bytes", "bitmap_bytes", "record_bytes")]
+        "host_lists_bytes", "logits_bytes", "bitmap_bytes", "record_bytes", "dense_bytes")]
 
 
 class np_buffers(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "w1", "w2", "backing", "gate_buf", "up_buf", "downT_buf", "staging", "host_staging", "workspace",
-        "host_lists")]
+        "host_lists", "dense_buf")]
 
 
 class np_delta_view(C.Structure):
@@ -87,6 +88,7 @@ def load() -> C.CDLL:
     lib.np_last_error.argtypes = [vp]
     sigs = {
         "np_query_sizes": [C.POINTER(np_config), C.POINTER(np_sizes)],
+        "np_plan_dense_prefix": [C.POINTER(np_config), C.c_uint64, C.c_uint64, C.POINTER(C.c_int32)],
         "np_init": [C.POINTER(vp), C.POINTER(np_config), C.POINTER(np_buffers)],
         "np_destroy": [vp],
         "np_reset": [vp, vp],
@@ -157,6 +159,13 @@ def np_query_sizes(cfg: np_config) -> np_sizes:
     out = np_sizes()
     _check(None, load().np_query_sizes(C.byref(cfg), C.byref(out)))
     return out
+
+
+def np_plan_dense_prefix(cfg: np_config, budget_bytes: int, fixed_bytes: int = 0) -> int:
+    """Largest dense prefix that fits the budget (-1: not even none); see include/np.h."""
+    out = C.c_int32()
+    _check(None, load().np_plan_dense_prefix(C.byref(cfg), budget_bytes, fixed_bytes, C.byref(out)))
+    return out.value
 
 
 def np_init(cfg: np_config, bufs: np_buffers) -> int:
@@ -257,13 +266,15 @@ def np_predict_logits_noalloc(w1, w2, x_bf16, B: int, n_layers: int, d_model: in
 
 # ---- buffer owner ----------------------------------------------------------------------
 def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
-                transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0, ring_stages=0) -> np_config:
+                transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0, ring_stages=0,
+                dense_layers=0) -> np_config:
     cfg = np_config()
     cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
     cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
     cfg.evict_policy, cfg.transfer_mode, cfg.flags, cfg.host_threads = evict_policy, transfer_mode, flags, host_threads
     cfg.chain_layers = chain_layers
     cfg.ring_stages = ring_stages
+    cfg.dense_layers = dense_layers
     cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
     return cfg
 
@@ -308,9 +319,11 @@ class Engine:
             pin_host_tensor(backing)
             self._registered = True
         dev = self.device
-        self.gate = torch.zeros((L, Cap, D), dtype=torch.bfloat16, device=dev)
-        self.up = torch.zeros((L, Cap, D), dtype=torch.bfloat16, device=dev)
-        self.downT = torch.zeros((L, Cap, D), dtype=torch.bfloat16, device=dev)
+        nd = cfg.dense_layers                       # leading dense layers: no slot buffers, one record buffer
+        self.gate = torch.zeros((L - nd, Cap, D), dtype=torch.bfloat16, device=dev)
+        self.up = torch.zeros((L - nd, Cap, D), dtype=torch.bfloat16, device=dev)
+        self.downT = torch.zeros((L - nd, Cap, D), dtype=torch.bfloat16, device=dev)
+        self.dense = torch.empty((nd, M, 3, D), dtype=torch.bfloat16, device=dev) if nd else None
         self.staging = torch.empty(int(self.sizes.staging_bytes), dtype=torch.uint8, device=dev)
         self.host_staging = None
         if cfg.transfer_mode == NP_XFER_HOST_GATHER:
@@ -320,10 +333,12 @@ class Engine:
         self.host_lists = torch.zeros(int(self.sizes.host_lists_bytes) // 4, dtype=torch.int32).pin_memory()
         b = np_buffers()
         b.w1, b.w2, b.backing = self.w1.data_ptr(), self.w2.data_ptr(), backing.data_ptr()
-        b.gate_buf, b.up_buf, b.downT_buf = self.gate.data_ptr(), self.up.data_ptr(), self.downT.data_ptr()
+        if L - nd > 0:
+            b.gate_buf, b.up_buf, b.downT_buf = self.gate.data_ptr(), self.up.data_ptr(), self.downT.data_ptr()
         b.staging = self.staging.data_ptr()
         b.host_staging = self.host_staging.data_ptr() if self.host_staging is not None else None
         b.workspace, b.host_lists = ws_ptr, self.host_lists.data_ptr()
+        b.dense_buf = self.dense.data_ptr() if self.dense is not None else None
         self.bufs = b
         self.ctx = np_init(cfg, b)
         self.stream = torch.cuda.Stream(device=dev)

@@ -246,8 +246,12 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
   if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
-  for (int i = 0; i < 2; ++i)
-    if (c->reserved[i]) return fail(ctx, NP_E_INVAL, "reserved fields must be 0");
+  if (c->dense_layers < 0 || c->dense_layers > c->n_layers)
+    return fail(ctx, NP_E_INVAL, "dense_layers must be in [0, n_layers]");
+  if (c->dense_layers > 0 && c->max_batch != 1) return fail(ctx, NP_E_INVAL, "dense_layers > 0 needs max_batch = 1");
+  if (c->dense_layers > 0 && (c->flags & (NP_F_LAYER_LAUNCHES | NP_F_DIRECT_LOADS)))
+    return fail(ctx, NP_E_INVAL, "dense_layers > 0 excludes NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS");
+  if (c->reserved[0]) return fail(ctx, NP_E_INVAL, "reserved fields must be 0");
   return NP_OK;
 }
 
@@ -309,12 +313,30 @@ int np_query_sizes(const np_config* cfg, np_sizes* out) {
   out->w1_bytes = 2ull * c.d_pred * c.d_model;
   out->w2_bytes = 2ull * c.n_layers * c.d_ffn * c.d_pred;
   out->backing_bytes = rec * c.n_layers * c.d_ffn;
-  out->row_buffer_bytes = 2ull * c.n_layers * c.capacity * c.d_model;
+  out->row_buffer_bytes = 2ull * (c.n_layers - c.dense_layers) * c.capacity * c.d_model;
+  out->dense_bytes = (uint64_t)c.dense_layers * c.d_ffn * rec;
   out->staging_bytes = rec * c.staging_rows;
   out->workspace_bytes = ws_layout(c).total;
   out->host_lists_bytes = host_lists_ints(c) * 4;
   out->logits_bytes = 4ull * c.max_batch * c.n_layers * c.d_ffn;
   out->bitmap_bytes = 4ull * c.n_layers * (c.d_ffn / 32);
+  return NP_OK;
+}
+
+int np_plan_dense_prefix(const np_config* cfg, uint64_t budget_bytes, uint64_t fixed_bytes, int32_t* d_out) {
+  if (!d_out) return fail(nullptr, NP_E_INVAL, "d_out is NULL");
+  if (!cfg) return fail(nullptr, NP_E_INVAL, "config is NULL");
+  np_config c = *cfg;
+  c.dense_layers = 0;  // the field is the answer, not an input
+  int rc = check_config(&c, nullptr);
+  if (rc) return rc;
+  const uint64_t rec = 3ull * c.d_model * 2;
+  const uint64_t dense = (uint64_t)c.d_ffn * rec, sparse = (uint64_t)c.capacity * rec;
+  *d_out = -1;
+  for (int d = 0; d <= c.n_layers; ++d) {
+    const uint64_t need = (uint64_t)d * dense + (uint64_t)(c.n_layers - d) * sparse;
+    if (need <= budget_bytes && fixed_bytes <= budget_bytes - need) *d_out = d;
+  }
   return NP_OK;
 }
 
@@ -349,12 +371,13 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   if (rc) return rc;
   if (!b) return fail(nullptr, NP_E_INVAL, "buffers is NULL");
   const bool need_staging = cfg->transfer_mode != NP_XFER_ZERO_COPY;
-  if (!b->w1 || !b->w2 || !b->backing || !b->gate_buf || !b->up_buf || !b->downT_buf || !b->workspace ||
-      !b->host_lists || (need_staging && !b->staging) ||
-      (cfg->transfer_mode == NP_XFER_HOST_GATHER && !b->host_staging))
+  const bool any_sparse = cfg->dense_layers < cfg->n_layers;
+  if (!b->w1 || !b->w2 || !b->backing || !b->workspace || !b->host_lists ||
+      (any_sparse && (!b->gate_buf || !b->up_buf || !b->downT_buf)) || (need_staging && !b->staging) ||
+      (cfg->transfer_mode == NP_XFER_HOST_GATHER && !b->host_staging) || (cfg->dense_layers > 0 && !b->dense_buf))
     return fail(nullptr, NP_E_INVAL, "a required buffer pointer is NULL");
   const void* aligned16[] = {b->w1, b->w2, b->backing, b->gate_buf, b->up_buf, b->downT_buf, b->staging,
-                             b->host_staging};
+                             b->host_staging, b->dense_buf};
   for (const void* p : aligned16)
     if ((uintptr_t)p % 16) return fail(nullptr, NP_E_INVAL, "weight, row and staging buffers must be 16-byte aligned");
   if ((uintptr_t)b->workspace % 256) return fail(nullptr, NP_E_INVAL, "workspace must be 256-byte aligned");
@@ -375,6 +398,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   d.Bmax = cfg->max_batch;
   d.ring_stages = cfg->ring_stages;
   d.rec_bytes = 3ull * d.D * 2;
+  d.dense = cfg->dense_layers;
 
 #define NP_INIT_CUDA(call)                                                                   \
   do {                                                                                       \
@@ -418,6 +442,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_did = take(LC), o_dsl = take(LC), o_eid = take(LC), o_aid = take(LC), o_asl = take(LC);
   const size_t o_ovf = take(LM), o_cnt = take((size_t)d.L * NP_N_COUNTERS), o_free = take(LC);
   const size_t o_cid = take(LC), o_ckey = take(LC), o_pred = take(LW), o_stat = take(4), o_bar = take(4);
+  const size_t o_ident = take(d.dense > 0 ? (size_t)d.M : 1);
   NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
   char* base = static_cast<char*>(ctx->slab);
   Tables& t = ctx->t;
@@ -438,6 +463,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   t.pred = reinterpret_cast<uint32_t*>(base + o_pred);
   t.status = reinterpret_cast<int32_t*>(base + o_stat);
   t.grid_bar = reinterpret_cast<unsigned int*>(base + o_bar);
+  t.identity = reinterpret_cast<int32_t*>(base + o_ident);
 
   const WsLayout wl = ws_layout(*cfg);
   char* wsb = static_cast<char*>(b->workspace);
@@ -473,6 +499,19 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
                 mlp_tc_supported(d, ctx->sm_count);
   if (cfg->max_batch > 4 && !(cfg->flags & NP_F_NO_TENSOR_CORES)) pred_tc_prepare(d, b->w2, ctx->ws.hsplit, &ctx->tc);
   memset(ctx->host_lists, 0, host_lists_ints(*cfg) * 4);
+  if (d.dense > 0) {
+    Dims dd = d;
+    dd.k = dd.C = d.M;
+    if (!chain_alu::supported(dd, ctx->sm_count) || (d.dense < d.L && !mlp_chain_supported(d, ctx->sm_count))) {
+      np_destroy(ctx);
+      return fail(nullptr, NP_E_INVAL, "dense_layers > 0: this shape is outside what the resident MLP kernels cover");
+    }
+    // the dense layers' records move to the device once; their active list is 0 .. M-1
+    NP_INIT_CUDA(cudaMemcpy(b->dense_buf, b->backing, (size_t)d.dense * d.M * d.rec_bytes, cudaMemcpyHostToDevice));
+    std::vector<int32_t> ident(d.M);
+    for (int i = 0; i < d.M; ++i) ident[i] = i;
+    NP_INIT_CUDA(cudaMemcpy(t.identity, ident.data(), (size_t)d.M * 4, cudaMemcpyHostToDevice));
+  }
   NP_INIT_CUDA(launch_tables_reset(d, t, nullptr));
   NP_INIT_CUDA(cudaDeviceSynchronize());
 #undef NP_INIT_CUDA
@@ -508,15 +547,26 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
   cudaStream_t s = as_stream(stream);
   const Dims& d = ctx->d;
   NP_LAUNCH(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
-  if (B > 4 && ctx->tc.ready) {
-    ctx->launches += 1;  // split kernel + GEMM kernel
-    NP_LAUNCH(ctx, launch_pred_l2_tc(d, ctx->tc, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
-  } else {
-    NP_LAUNCH(ctx, launch_pred_l2(d, ctx->bufs.w2, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
+  // Dense layers are not scored: the sparse layers are a contiguous suffix of W2, of the logits
+  // and of the bitmap (a dense prefix implies B = 1, so the per-sequence stride does not matter).
+  Dims ds = d;
+  ds.L = d.L - d.dense;
+  const size_t skip_rows = (size_t)d.dense * d.M;
+  float* logits = ctx->ws.logits + skip_rows;
+  if (ds.L > 0) {
+    if (B > 4 && ctx->tc.ready) {
+      ctx->launches += 1;  // split kernel + GEMM kernel
+      NP_LAUNCH(ctx, launch_pred_l2_tc(d, ctx->tc, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
+    } else {
+      NP_LAUNCH(ctx, launch_pred_l2(ds, static_cast<const char*>(ctx->bufs.w2) + skip_rows * d.H * 2, ctx->ws.hidden,
+                                  B, logits, ctx->t.status, s, ctx->sm_count));
+    }
+    NP_LAUNCH(ctx, launch_topk(ds, logits, B, ctx->t.pred + (size_t)d.dense * d.W, s));
   }
-  NP_LAUNCH(ctx, launch_topk(d, ctx->ws.logits, B, ctx->t.pred, s));
-  const size_t nlog = (size_t)B * d.L * d.M * 4, nbm = (size_t)d.L * d.W * 4;
-  if (logits_out) NP_CUDA(ctx, cudaMemcpyAsync(logits_out, ctx->ws.logits, nlog, cudaMemcpyDeviceToDevice, s));
+  if (d.dense > 0) NP_CUDA(ctx, cudaMemsetAsync(ctx->t.pred, 0, (size_t)d.dense * d.W * 4, s));
+  const size_t nlog = (size_t)B * ds.L * d.M * 4, nbm = (size_t)d.L * d.W * 4;
+  if (logits_out && nlog)
+    NP_CUDA(ctx, cudaMemcpyAsync(logits_out + skip_rows, logits, nlog, cudaMemcpyDeviceToDevice, s));
   if (bitmap_out) NP_CUDA(ctx, cudaMemcpyAsync(bitmap_out, ctx->t.pred, nbm, cudaMemcpyDeviceToDevice, s));
   ctx->have_pred = true;
   return NP_OK;
@@ -526,7 +576,12 @@ int np_topk(np_ctx* ctx, const float* logits, int32_t B, uint32_t* bitmap_out, v
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   if (!logits || !bitmap_out) return fail(ctx, NP_E_INVAL, "logits or bitmap_out is NULL");
   if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
-  NP_LAUNCH(ctx, launch_topk(ctx->d, logits, B, bitmap_out, as_stream(stream)));
+  const Dims& d = ctx->d;
+  Dims ds = d;
+  ds.L = d.L - d.dense;  // dense layers select nothing: their rows of the bitmap are zero
+  if (ds.L > 0)
+    NP_LAUNCH(ctx, launch_topk(ds, logits + (size_t)d.dense * d.M, B, bitmap_out + (size_t)d.dense * d.W, as_stream(stream)));
+  if (d.dense > 0) NP_CUDA(ctx, cudaMemsetAsync(bitmap_out, 0, (size_t)d.dense * d.W * 4, as_stream(stream)));
   return NP_OK;
 }
 
@@ -537,6 +592,8 @@ int np_centroid_select(np_ctx* ctx, const float* logits, int32_t B, int32_t K, c
   if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
   if (K < 1) return fail(ctx, NP_E_INVAL, "K=%d must be positive", K);
   NP_LAUNCH(ctx, launch_centroid_select(ctx->d, logits, B, K, bank, ids_out, bitmap_out, as_stream(stream)));
+  if (ctx->d.dense > 0)  // dense layers select nothing
+    NP_CUDA(ctx, cudaMemsetAsync(bitmap_out, 0, (size_t)ctx->d.dense * ctx->d.W * 4, as_stream(stream)));
   return NP_OK;
 }
 
@@ -547,6 +604,14 @@ int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream) {
     pred_bitmap = ctx->t.pred;
   }
   cudaStream_t s = as_stream(stream);
+  if (ctx->d.dense > 0 && pred_bitmap != ctx->t.pred) {
+    // a caller's bitmap may name rows of dense layers; those layers select nothing
+    const size_t skip = (size_t)ctx->d.dense * ctx->d.W;
+    NP_CUDA(ctx, cudaMemsetAsync(ctx->t.pred, 0, skip * 4, s));
+    NP_CUDA(ctx, cudaMemcpyAsync(ctx->t.pred + skip, pred_bitmap + skip, ((size_t)ctx->d.L * ctx->d.W - skip) * 4,
+                                 cudaMemcpyDeviceToDevice, s));
+    pred_bitmap = ctx->t.pred;
+  }
   // the previous step's installs must have landed before tables and slots are reused
   for (int l = 0; l < ctx->d.L; ++l) {
     if (ctx->install_pending[l]) {
@@ -568,6 +633,8 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
   if (layer_begin < 0 || layer_end > d.L || layer_begin > layer_end)
     return fail(ctx, NP_E_INVAL, "layer range [%d, %d) outside [0, %d)", layer_begin, layer_end, d.L);
   if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_install needs a prior np_delta");
+  layer_begin = std::max(layer_begin, d.dense);  // dense layers hold all their rows already
+  layer_end = std::max(layer_end, layer_begin);
   cudaStream_t cs = as_stream(copy_stream);
   const int check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
   const int mode = ctx->cfg.transfer_mode;
@@ -601,9 +668,9 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
       NP_LAUNCH(ctx, launch_scatter(d, store_l, true, ctx->t.delta_ids + (size_t)l * d.C,
                                   ctx->t.delta_slots + (size_t)l * d.C,
                                   ctx->t.counters + (size_t)l * NP_N_COUNTERS + NP_CNT_DELTA, 0, max_rows,
-                                  static_cast<char*>(ctx->bufs.gate_buf) + (size_t)l * d.C * row_bytes,
-                                  static_cast<char*>(ctx->bufs.up_buf) + (size_t)l * d.C * row_bytes,
-                                  static_cast<char*>(ctx->bufs.downT_buf) + (size_t)l * d.C * row_bytes,
+                                  static_cast<char*>(ctx->bufs.gate_buf) + (size_t)(l - d.dense) * d.C * row_bytes,
+                                  static_cast<char*>(ctx->bufs.up_buf) + (size_t)(l - d.dense) * d.C * row_bytes,
+                                  static_cast<char*>(ctx->bufs.downT_buf) + (size_t)(l - d.dense) * d.C * row_bytes,
                                   ctx->t.status, check, zs, ctx->sm_count));
       NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], zs));
       ctx->install_pending[l] = 1;
@@ -624,9 +691,9 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
     if (n < 0 || n > d.C) return fail(ctx, NP_E_DEVICE, "layer %d: delta count %d outside [0, %d]", l, n, d.C);
     if (cnt[NP_CNT_OVERFLOW] > 0) warn = NP_W_OVERFLOW;
     const char* store_l = store + (size_t)l * d.M * rec;
-    char* gate_l = static_cast<char*>(ctx->bufs.gate_buf) + (size_t)l * d.C * row_bytes;
-    char* up_l = static_cast<char*>(ctx->bufs.up_buf) + (size_t)l * d.C * row_bytes;
-    char* down_l = static_cast<char*>(ctx->bufs.downT_buf) + (size_t)l * d.C * row_bytes;
+    char* gate_l = static_cast<char*>(ctx->bufs.gate_buf) + (size_t)(l - d.dense) * d.C * row_bytes;
+    char* up_l = static_cast<char*>(ctx->bufs.up_buf) + (size_t)(l - d.dense) * d.C * row_bytes;
+    char* down_l = static_cast<char*>(ctx->bufs.downT_buf) + (size_t)(l - d.dense) * d.C * row_bytes;
     const int32_t* slots_dev = ctx->t.delta_slots + (size_t)l * d.C;
     const int32_t* count_dev = ctx->t.counters + (size_t)l * NP_N_COUNTERS + NP_CNT_DELTA;
 
@@ -717,9 +784,9 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   const Dims& d = ctx->d;
   const size_t row_bytes = (size_t)d.D * 2;
   MlpArgs a;
-  a.gate_l = static_cast<const char*>(ctx->bufs.gate_buf) + (size_t)layer * d.C * row_bytes;
-  a.up_l = static_cast<const char*>(ctx->bufs.up_buf) + (size_t)layer * d.C * row_bytes;
-  a.downT_l = static_cast<const char*>(ctx->bufs.downT_buf) + (size_t)layer * d.C * row_bytes;
+  a.gate_l = static_cast<const char*>(ctx->bufs.gate_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
+  a.up_l = static_cast<const char*>(ctx->bufs.up_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
+  a.downT_l = static_cast<const char*>(ctx->bufs.downT_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
   a.active_slots = ctx->t.active_slots + (size_t)layer * d.C;
   a.n_active_ptr = ctx->t.counters + (size_t)layer * NP_N_COUNTERS + NP_CNT_ACTIVE;
   a.xa = xa;
@@ -753,38 +820,61 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
 
 // residual chain: x_l = xbuf[(l+1)&1] + zbuf[(l-1)%3]; layer l accumulates MLP_l(x_l) into
 // zbuf[l%3], stores x_l to xbuf[l&1] and clears zbuf[(l+1)%3] for the next layer
-static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaStream_t s) {
+// `part`: kChainAll = the whole chain; kChainHead = its start up to the end of the dense prefix
+// (nothing there waits for an install, so np_step queues it before the host packs any rows);
+// kChainTail = the sparse layers and the result.
+enum { kChainAll = 0, kChainHead = 1, kChainTail = 2 };
+static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaStream_t s, int part = kChainAll) {
   const Dims& d = ctx->d;
   const size_t n = (size_t)B * d.D;
-  NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
   const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
                           mlp_chain_supported(d, ctx->sm_count);
-  // the accumulator of layer 0 starts at zero (later ones are cleared one layer ahead)
-  NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, (persistent ? (size_t)kZRep * d.D : n) * 4, s));
+  if (part != kChainTail) {
+    NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
+    // the accumulator of layer 0 starts at zero (later ones are cleared one layer ahead)
+    NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, (persistent ? (size_t)kZRep * d.D : n) * 4, s));
+  }
   if (persistent) {
     // runs of layers in one resident kernel each; a run starts once its layers are installed,
     // so the install of later runs still overlaps the compute of earlier ones
     const int run = std::max(1, ctx->cfg.chain_layers > 0 ? ctx->cfg.chain_layers : (d.L + 3) / 4);
-    for (int l0 = 0; l0 < d.L; l0 += run) {
+    const size_t row_bytes = (size_t)d.D * 2;
+    ChainArgs a;
+    for (int i = 0; i < 2; ++i) a.xbuf[i] = ctx->ws.xbuf[i];
+    for (int i = 0; i < 3; ++i) a.zbuf[i] = ctx->ws.zbuf[i];
+    a.grid_bar = ctx->t.grid_bar;
+    a.status = ctx->t.status;
+    a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+    a.counters = ctx->t.counters;
+    // the dense prefix first: whole records, every row active, nothing to wait for (it also
+    // widens the window in which the sparse layers' rows arrive)
+    if (d.dense > 0 && part != kChainTail) {
+      const char* dense = static_cast<const char*>(ctx->bufs.dense_buf);
+      a.gate = dense;
+      a.up = dense + row_bytes;
+      a.downT = dense + 2 * row_bytes;
+      a.active_slots = ctx->t.identity;
+      a.dense_rows = d.M;
+      a.l_begin = 0;
+      a.l_end = d.dense;
+      NP_LAUNCH(ctx, chain_alu::launch(d, a, s, ctx->sm_count));
+    }
+    // the sparse layers' buffers start at layer d; the kernels index them by absolute layer
+    const size_t shift = (size_t)d.dense * d.C * row_bytes;
+    a.gate = static_cast<const char*>(ctx->bufs.gate_buf) - shift;
+    a.up = static_cast<const char*>(ctx->bufs.up_buf) - shift;
+    a.downT = static_cast<const char*>(ctx->bufs.downT_buf) - shift;
+    a.active_slots = ctx->t.active_slots;
+    a.dense_rows = 0;
+    for (int l0 = d.dense; l0 < d.L && part != kChainHead; l0 += run) {
       const int l1 = std::min(d.L, l0 + run);
       for (int l = l0; l < l1; ++l)
         if (ctx->install_pending[l]) NP_CUDA(ctx, wait_install(ctx, l, s));
-      ChainArgs a;
-      a.gate = ctx->bufs.gate_buf;
-      a.up = ctx->bufs.up_buf;
-      a.downT = ctx->bufs.downT_buf;
-      a.active_slots = ctx->t.active_slots;
-      a.counters = ctx->t.counters;
-      for (int i = 0; i < 2; ++i) a.xbuf[i] = ctx->ws.xbuf[i];
-      for (int i = 0; i < 3; ++i) a.zbuf[i] = ctx->ws.zbuf[i];
-      a.grid_bar = ctx->t.grid_bar;
-      a.status = ctx->t.status;
       a.l_begin = l0;
       a.l_end = l1;
-      a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
       NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
     }
-  } else {
+  } else if (part != kChainHead) {
     if (ctx->mlp_tc && B >= kTcMinBatch) NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.gu[0], 0, ctx->gu_bytes, s));
     for (int l = 0; l < d.L; ++l) {
       int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
@@ -792,8 +882,9 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       if (rc < 0) return rc;
     }
   }
-  NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], persistent ? kZRep : 1, x_out,
-                                n, s));
+  if (part != kChainHead)
+    NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], persistent ? kZRep : 1,
+                                  x_out, n, s));
   return NP_OK;
 }
 
@@ -825,6 +916,7 @@ int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* 
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   const Dims& d = ctx->d;
   if (layer < 0 || layer >= d.L) return fail(ctx, NP_E_INVAL, "layer %d outside [0, %d)", layer, d.L);
+  if (layer < d.dense) return fail(ctx, NP_E_INVAL, "layer %d is dense: it runs only inside np_mlp_chain / np_step", layer);
   if (!x || !y) return fail(ctx, NP_E_INVAL, "x or y is NULL");
   if ((uintptr_t)x % 16 || (uintptr_t)y % 16) return fail(ctx, NP_E_INVAL, "x and y must be 16-byte aligned");
   if (B < 1 || B > d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, d.Bmax);
@@ -849,6 +941,12 @@ int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stre
   rc = np_delta(ctx, nullptr, stream);
   if (rc < 0) return rc;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[2], s));
+  // the dense prefix waits for no install: it is queued before the host starts on the rows
+  const bool head_first = d.dense > 0;
+  if (head_first) {
+    rc = mlp_chain(ctx, x_bf16, B, x_out, s, kChainHead);
+    if (rc < 0) return rc;
+  }
   // the copy stream is ordered after the delta step inside np_install
   NP_CUDA(ctx, cudaStreamWaitEvent(cs, ctx->ev_delta, 0));
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_c[0], cs));
@@ -856,7 +954,7 @@ int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stre
   if (warn < 0) return warn;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_c[1], cs));
 
-  rc = mlp_chain(ctx, x_bf16, B, x_out, s);
+  rc = mlp_chain(ctx, x_bf16, B, x_out, s, head_first ? kChainTail : kChainAll);
   if (rc < 0) return rc;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[3], s));
   ctx->have_step = true;

@@ -35,6 +35,7 @@ struct Tables {
   uint32_t* pred;         // [L][W]  bitmap of the last np_predict
   int32_t* status;        // [4]     device-side error word(s)
   unsigned int* grid_bar; // [1]     arrival counter of the persistent MLP kernel
+  int32_t* identity;      // [M]     0, 1, ..., M-1: the active list of a dense layer
 };
 
 // Carved out of the caller's workspace.
@@ -50,6 +51,7 @@ struct Workspace {
 
 struct Dims {
   int L, D, M, H, k, C, W, Bmax;
+  int dense;        // leading layers that are dense and fully resident (no selection, no install)
   int ring_stages;  // cap on shared-memory ring stages of the MLP kernels (0 = as many as fit)
   size_t rec_bytes;
 };
@@ -141,6 +143,8 @@ struct ChainArgs {
   unsigned int* grid_bar;
   int32_t* status;
   int l_begin, l_end, check;
+  int dense_rows;  // > 0 (ALU form only): the layers are dense_rows whole records each, `gate`/`up`/`downT` point
+                   // at the three rows of layer 0's first record, active_slots is one identity list
 };
 bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p);
 bool mlp_chain_supported(const Dims& d, int sm_count);

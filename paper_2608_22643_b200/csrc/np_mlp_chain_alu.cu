@@ -42,6 +42,9 @@ struct ChainKernelArgs {
   unsigned int* grid_bar;      // zeroed by the host before the launch
   int32_t* status;
   int l_begin, l_end, D, C, n_stages, tile_rows, rows_per_warp, check;
+  int dense_rows;              // > 0: dense layers.  Each layer is dense_rows whole records ([row][gate|up|down][D],
+                               // `gate` points at layer 0's first record), every row is active, `slots` is one
+                               // identity list shared by all layers and `counters` is not read
   int slot_cache_rows;         // capacity of the per-block slot cache (rows)
   int window_rows;             // records in flight per block (< n_stages)
 };
@@ -76,7 +79,10 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
   const int D = a.D, chunks = D >> 3;
   const uint32_t row_bytes = (uint32_t)D * 2u;
   const uint32_t rec_bytes = 3u * row_bytes;
-  const size_t layer_bytes = (size_t)a.C * row_bytes;
+  // resident slot buffers: one row per slot and projection; dense layers: whole records
+  const int cap = a.dense_rows > 0 ? a.dense_rows : a.C;               // rows a layer can hold
+  const uint32_t row_pitch = a.dense_rows > 0 ? rec_bytes : row_bytes;  // bytes from one row to the next
+  const size_t layer_bytes = (size_t)cap * row_pitch;
   // a tile is TR = RPW * (16 / SEG) rows: phase 1 gives every warp RPW (row, segment) items
   const int n_stages = a.n_stages, RPW = a.rows_per_warp, TR = a.tile_rows, SEG = kChainWarps * RPW / TR;
   const int seg_chunks = (chunks + SEG - 1) / SEG;
@@ -87,8 +93,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
 
   // ---- this block's share of every layer of the run ----
   if (tid < nl) {
-    int n = a.counters[(size_t)(a.l_begin + tid) * NP_N_COUNTERS + NP_CNT_ACTIVE];
-    if (a.check && (n < 0 || n > a.C)) {
+    int n = a.dense_rows > 0 ? a.dense_rows : a.counters[(size_t)(a.l_begin + tid) * NP_N_COUNTERS + NP_CNT_ACTIVE];
+    if (a.check && (n < 0 || n > cap)) {
       atomicOr(a.status, kStatBadCount);
       n = 0;
     }
@@ -118,8 +124,8 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
     for (int i = tid; i < nr; i += blockDim.x) {
       const int v = lay_pre[li] + i;
       if (v < total_rows) {
-        int slot = a.slots[(size_t)(a.l_begin + li) * a.C + lay_rb[li] + i];
-        if (a.check && (slot < 0 || slot >= a.C)) {
+        int slot = a.slots[(a.dense_rows > 0 ? 0 : (size_t)(a.l_begin + li) * a.C) + lay_rb[li] + i];
+        if (a.check && (slot < 0 || slot >= cap)) {
           atomicOr(a.status, kStatBadSlot);
           slot = 0;
         }
@@ -156,7 +162,7 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
           break;
         }
         while (v >= lay_pre[ll + 1]) ++ll;
-        const size_t off = (size_t)(a.l_begin + ll) * layer_bytes + (size_t)slot_cache[v] * row_bytes;
+        const size_t off = (size_t)(a.l_begin + ll) * layer_bytes + (size_t)slot_cache[v] * row_pitch;
         unsigned char* dst = csm + (size_t)s * rec_bytes;
         npp::mbar_expect_tx(&full_bar[s], rec_bytes);
         npp::bulk_g2s(dst, a.gate + off, row_bytes, &full_bar[s]);
@@ -464,7 +470,9 @@ bool supported(const Dims& d, int sm_count) {
   return alu_plan(d, sm_count, &p);
 }
 
-cudaError_t launch(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count) {
+cudaError_t launch(const Dims& d_in, const ChainArgs& a, cudaStream_t s, int sm_count) {
+  Dims d = d_in;
+  if (a.dense_rows > 0) d.k = d.C = a.dense_rows;  // plan for layers whose every row is active
   AluPlan p;
   if (!alu_plan(d, sm_count, &p)) return cudaErrorInvalidValue;
   cudaError_t e = cudaSuccess;
@@ -484,7 +492,8 @@ cudaError_t launch(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_cou
     ka.slot_cache_rows = p.slot_cache_rows;
     ka.window_rows = std::max(1, std::min(p.n_stages - 1, p.window_rows));
     ka.D = d.D;
-    ka.C = d.C;
+    ka.C = d_in.C;
+    ka.dense_rows = a.dense_rows;
     ka.n_stages = p.n_stages;
     ka.tile_rows = p.tile_rows;
     ka.rows_per_warp = p.rows_per_warp;

@@ -27,7 +27,7 @@ class Pair:
 
     def __init__(self, cfg: synth.StackConfig, policy=nb.NP_EVICT_EXACT, max_batch=1, k=None, C=None,
                  transfer_mode=nb.NP_XFER_MEMCPY_RUNS, staging_rows=None, flags=nb.NP_F_CHECK_BOUNDS,
-                 gen_device="cpu", with_oracle=True, chain_layers=0, ring_stages=0):
+                 gen_device="cpu", with_oracle=True, chain_layers=0, ring_stages=0, dense_layers=0):
         nbuild.build()
         self.cfg = cfg
         self.k = cfg.top_k if k is None else k
@@ -37,13 +37,15 @@ class Pair:
         self.backing = synth.backing_store(cfg, gen_device=gen_device)
         ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, self.k, self.C,
                               max_batch=max_batch, evict_policy=policy, staging_rows=staging_rows,
-                              transfer_mode=transfer_mode, flags=flags, chain_layers=chain_layers, ring_stages=ring_stages)
+                              transfer_mode=transfer_mode, flags=flags, chain_layers=chain_layers, ring_stages=ring_stages,
+                              dense_layers=dense_layers)
+        self.dense_layers = dense_layers
         self.eng = nb.Engine(ncfg, w1.cuda(), w2.cuda(), self.backing)
         self.store_u16 = self.backing.view(torch.int16).numpy().view(np.uint16)
         self.ora = None
         if with_oracle:
             self.ora = O.Engine(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, self.k, self.C, policy,
-                                u16(self.w1_cpu), u16(self.w2_cpu), self.store_u16)
+                                u16(self.w1_cpu), u16(self.w2_cpu), self.store_u16, dense_layers=dense_layers)
 
     def close(self):
         self.eng.close()
@@ -71,10 +73,13 @@ class Pair:
         """Every resident row of every layer holds exactly its record's bytes."""
         torch.cuda.synchronize()
         g, u, dn = (u16(t) for t in (self.eng.gate, self.eng.up, self.eng.downT))
-        for l in range(self.cfg.n_layers):
+        nd = self.dense_layers
+        for l in range(nd, self.cfg.n_layers):       # the slot buffers start at the first sparse layer
             st = self.eng.export_state(l)
             ids = np.flatnonzero(st["slot_map"] >= 0)
             slots = st["slot_map"][ids]
-            assert (g[l, slots] == self.store_u16[l, ids, 0]).all(), l
-            assert (u[l, slots] == self.store_u16[l, ids, 1]).all(), l
-            assert (dn[l, slots] == self.store_u16[l, ids, 2]).all(), l
+            assert (g[l - nd, slots] == self.store_u16[l, ids, 0]).all(), l
+            assert (u[l - nd, slots] == self.store_u16[l, ids, 1]).all(), l
+            assert (dn[l - nd, slots] == self.store_u16[l, ids, 2]).all(), l
+        if nd:
+            assert (u16(self.eng.dense) == self.store_u16[:nd]).all()

@@ -30,13 +30,13 @@ def test_every_declared_symbol_is_exported(lib):
     for n in names:
         assert hasattr(lib, n), n
     assert sorted(nb.EXPORTED) == names
-    assert nb.np_version() == 1
+    assert nb.np_version() == 2
 
 
 def test_struct_sizes_match_header():
     assert C.sizeof(nb.np_config) == 16 * 4
-    assert C.sizeof(nb.np_sizes) == 10 * 8
-    assert C.sizeof(nb.np_buffers) == 10 * C.sizeof(C.c_void_p)
+    assert C.sizeof(nb.np_sizes) == 11 * 8
+    assert C.sizeof(nb.np_buffers) == 11 * C.sizeof(C.c_void_p)
     assert C.sizeof(nb.np_delta_view) == 7 * C.sizeof(C.c_void_p)
 
 
@@ -52,12 +52,29 @@ def test_query_sizes_arithmetic(lib):
     assert s.bitmap_bytes == 32 * 344 * 4 and s.logits_bytes == 32 * 11008 * 4
     assert s.host_lists_bytes == (16 + 32 * (8 + 2 * 2752)) * 4
     assert s.workspace_bytes >= s.logits_bytes + 5 * 4096 * 4 + 512 * 4
+    assert s.dense_bytes == 0
+    # a dense prefix of 8 layers: their records in one buffer, slot buffers for the other 24
+    cfg8 = nb.make_config(32, 4096, 11008, 512, 1101, 2752, staging_rows=256, dense_layers=8)
+    s8 = nb.np_query_sizes(cfg8)
+    assert s8.dense_bytes == 8 * 11008 * 24576 and s8.row_buffer_bytes == 24 * 2752 * 4096 * 2
+
+
+def test_dense_prefix_plan_matches_the_oracle(lib):
+    from oracle import np_oracle as O
+    cfg = nb.make_config(32, 4096, 11008, 512, 1101, 2752)
+    rec = 24576
+    fixed = 5 * 2**30
+    for budget in [0, fixed, fixed + 32 * 2752 * rec, fixed + 32 * 2752 * rec + 3 * (11008 - 2752) * rec + 1,
+                   fixed + 32 * 11008 * rec - 1, fixed + 32 * 11008 * rec, 2**45]:
+        assert nb.np_plan_dense_prefix(cfg, budget, fixed) == O.dense_prefix_plan(32, 11008, 4096, 2752, budget, fixed)
+    assert nb.np_plan_dense_prefix(cfg, fixed + 32 * 2752 * rec, fixed) == 0
+    assert nb.np_plan_dense_prefix(cfg, fixed + 32 * 2752 * rec - 1, fixed) == -1
 
 
 @pytest.mark.parametrize("field,value", [
     ("n_layers", 0), ("d_model", 100), ("d_ffn", 1000), ("d_pred", 7), ("top_k", 9999), ("capacity", 0),
     ("capacity", 99999), ("max_batch", 17), ("evict_policy", 5), ("transfer_mode", 9), ("staging_rows", 0),
-    ("flags", 64),
+    ("flags", 64), ("dense_layers", -1), ("dense_layers", 3),
 ])
 def test_bad_config_is_rejected(lib, field, value):
     cfg = nb.make_config(2, 256, 1024, 64, 102, 205)
