@@ -855,9 +855,15 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       a.downT = dense + 2 * row_bytes;
       a.active_slots = ctx->t.identity;
       a.dense_rows = d.M;
-      a.l_begin = 0;
-      a.l_end = d.dense;
-      NP_LAUNCH(ctx, chain_alu::launch(d, a, s, ctx->sm_count));
+      // Short runs: while a cooperative launch is resident the install's scatter kernels do not
+      // get onto the device, so the installs of the sparse layers advance between runs
+      // (measured at the 7B shape, d = 24: 612 steps/s with runs of 3, 448 with one run).
+      constexpr int kDenseRun = 3;
+      for (int l0 = 0; l0 < d.dense; l0 += kDenseRun) {
+        a.l_begin = l0;
+        a.l_end = std::min(d.dense, l0 + kDenseRun);
+        NP_LAUNCH(ctx, chain_alu::launch(d, a, s, ctx->sm_count));
+      }
     }
     // the sparse layers' buffers start at layer d; the kernels index them by absolute layer
     const size_t shift = (size_t)d.dense * d.C * row_bytes;

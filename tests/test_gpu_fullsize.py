@@ -124,3 +124,32 @@ def test_stress_shape_batch16_few_layers():
         p.check_resident_bytes()
     finally:
         p.close()
+
+
+def test_7b_shape_with_dense_prefix():
+    """The 7B row shape on six layers, the first two dense (11008 whole records each through
+    the resident kernel), in bench.py's --dense-layers configuration."""
+    cfg = synth.CONFIGS["7b"].with_(n_layers=6)
+    L, M, D, d = cfg.n_layers, cfg.d_ffn, cfg.d_model, 2
+    p = Pair(cfg, transfer_mode=nb.NP_XFER_HOST_GATHER, staging_rows=2 * cfg.top_k, flags=0, gen_device="cuda",
+             dense_layers=d)
+    try:
+        xs = synth.hidden_states(cfg, 3)
+        logits = torch.zeros((1, L, M), dtype=torch.float32, device="cuda")
+        out = torch.empty((1, D), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, x, 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            full = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M).astype(np.float32)
+            assert rel_l2(z32[0, d:], full[0, d:]) < 1e-5 and not z32[0, :d].any()
+            full[0, d:] = z32[0, d:]
+            res = p.ora.step(u16(xs[t]), logits_f32=full)
+            cnt = p.check_delta_against(res["deltas"])
+            assert (cnt[d:, nb.NP_CNT_ACTIVE] == p.k).all() and (cnt[:d, nb.NP_CNT_ACTIVE] == 0).all()
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+        p.check_resident_bytes()
+    finally:
+        p.close()
