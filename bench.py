@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
     ap.add_argument("--dense-layers", type=int, default=0,
                     help="dense prefix: the first d layers stay whole on the GPU and take no part in selection or install")
+    ap.add_argument("--budget-gib", type=float, default=None,
+                    help="device memory for MLP weights: the dense prefix becomes the longest one that fits (memory rule)")
     ap.add_argument("--no-variants", action="store_true",
                     help="skip the extra measurement of the zero-copy transfer mode (default run only)")
     ap.add_argument("--selection", default="topk", choices=["topk", "centroid"],
@@ -290,6 +292,11 @@ def cuda_arm(args):
     mode = {"runs": nb.NP_XFER_MEMCPY_RUNS, "gather": nb.NP_XFER_HOST_GATHER,
             "zerocopy": nb.NP_XFER_ZERO_COPY}[args.transfer]
 
+    if args.budget_gib is not None:
+        plan_cfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity)
+        args.dense_layers = nb.np_plan_dense_prefix(plan_cfg, int(args.budget_gib * 2**30), 0)
+        if args.dense_layers < 0:
+            raise SystemExit("bench.py: the budget does not even hold the sparse layers' resident buffers")
     w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True)
     ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
                           max_batch=args.batch, evict_policy=policy, transfer_mode=mode,
@@ -454,7 +461,8 @@ def cuda_arm(args):
             "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
                         f"B={Bq} rho={cfg.rho} policy={args.policy} transfer={args.transfer}"
                         + (f" selection=centroid K={args.centroids}" if centroid else "")
-                        + (f" dense_layers={args.dense_layers}" if args.dense_layers else ""),
+                        + (f" dense_layers={args.dense_layers}" if args.dense_layers else "")
+                        + (f" (longest prefix within {args.budget_gib} GiB)" if args.budget_gib is not None else ""),
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
             "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
             "active_rows_per_layer": n_active, "overflow_steps": int(overflow_steps),
