@@ -100,3 +100,43 @@ def test_configurations_that_exclude_a_dense_prefix():
         with pytest.raises(nb.NpError) as e:
             nb.np_query_sizes(cfg)
         assert e.value.code == nb.NP_E_INVAL
+
+
+def test_lru_policy_reset_and_centroid_head_with_dense_prefix():
+    cfg = SMALL
+    d, K = 1, 32
+    p = Pair(cfg, policy=nb.NP_EVICT_LRU, dense_layers=d, transfer_mode=nb.NP_XFER_HOST_GATHER, C=cfg.d_ffn // 3)
+    try:
+        L, M, W, D = cfg.n_layers, cfg.d_ffn, cfg.d_ffn // 32, cfg.d_model
+        xs = synth.hidden_states(cfg, 6)
+        out = torch.empty((1, D), dtype=torch.float32, device="cuda")
+        logits = torch.zeros((1, L, M), dtype=torch.float32, device="cuda")
+
+        def run(t):
+            nb.np_predict(p.eng.ctx, xs[t].cuda(), 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, xs[t].cuda(), 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            full = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M).astype(np.float32)
+            full[0, d:] = logits.cpu().numpy()[0, d:]
+            res = p.ora.step(u16(xs[t]), logits_f32=full)
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+
+        for t in range(3):
+            run(t)
+        # reset empties the sparse layers' residency; the dense records stay where they are
+        nb.np_reset(p.eng.ctx, p.eng.stream)
+        p.ora.res.reset()
+        for t in range(3, 6):
+            run(t)
+        p.check_resident_bytes()
+        # the centroid head selects nothing in a dense layer either
+        bank = synth.centroid_bank(cfg, K).cuda()
+        z = torch.randn((1, L, 2, K), dtype=torch.float32, device="cuda")
+        words = torch.full((L, W), -1, dtype=torch.int32, device="cuda")
+        nb.np_centroid_select(p.eng.ctx, z, 1, K, bank, None, words, p.eng.stream)
+        torch.cuda.synchronize()
+        w = words.cpu().numpy()
+        assert not w[:d].any() and w[d:].any()
+    finally:
+        p.close()
