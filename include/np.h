@@ -113,8 +113,9 @@ typedef struct np_config {
                              records of each sit in dense_buf (copied from the store by
                              np_init), every row is used, and the layers take no part in
                              selection, delta or install: their rows of every bitmap read as
-                             empty and their tables stay empty.  d > 0 needs max_batch = 1 and
-                             neither NP_F_LAYER_LAUNCHES nor NP_F_DIRECT_LOADS */
+                             empty and their tables stay empty.  d > 0 excludes
+                             NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS, and with max_batch > 1
+                             also NP_F_NO_TENSOR_CORES */
   int32_t reserved[1];    /* must be 0 */
 } np_config;
 
@@ -200,8 +201,8 @@ const char* np_last_error(const np_ctx* ctx);
  *                sequence's k highest logits per layer; order = fp32 value
  *                descending (+0 above -0), ties to the lower neuron index
  * The bitmap is also kept inside the context for np_delta(ctx, NULL, ...).
- * Dense layers (dense_layers > 0) are not scored: their logits are left
- * untouched and their bitmap rows are zero.
+ * Dense layers (dense_layers > 0) select nothing: their bitmap rows are zero
+ * (with B = 1 they are not even scored and their logits are left untouched).
  * Errors: NP_E_INVAL (NULL x, B outside 1..max_batch), NP_E_CUDA. */
 int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out,
                uint32_t* bitmap_out, void* stream);

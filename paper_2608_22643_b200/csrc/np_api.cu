@@ -248,7 +248,8 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
   if (c->dense_layers < 0 || c->dense_layers > c->n_layers)
     return fail(ctx, NP_E_INVAL, "dense_layers must be in [0, n_layers]");
-  if (c->dense_layers > 0 && c->max_batch != 1) return fail(ctx, NP_E_INVAL, "dense_layers > 0 needs max_batch = 1");
+  if (c->dense_layers > 0 && c->max_batch > 1 && (c->flags & NP_F_NO_TENSOR_CORES))
+    return fail(ctx, NP_E_INVAL, "dense_layers > 0 with batches needs the tensor-core kernels");
   if (c->dense_layers > 0 && (c->flags & (NP_F_LAYER_LAUNCHES | NP_F_DIRECT_LOADS)))
     return fail(ctx, NP_E_INVAL, "dense_layers > 0 excludes NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS");
   if (c->reserved[0]) return fail(ctx, NP_E_INVAL, "reserved fields must be 0");
@@ -275,7 +276,8 @@ WsLayout ws_layout(const np_config& c) {
   off += 3 * kZRep * vec;
   // batch MLP: two dot-product accumulators, each followed by its per-sequence sums of squares
   w.gu = off;
-  w.gu_each = align_up(((size_t)c.capacity * 2 * kMaxBatch + kMaxBatch) * 4, 256);
+  const size_t gu_rows = c.dense_layers > 0 ? c.d_ffn : c.capacity;  // a dense layer has M active rows
+  w.gu_each = align_up((gu_rows * 2 * kMaxBatch + kMaxBatch) * 4, 256);
   off += 2 * w.gu_each;
   w.total = off;
   return w;
@@ -475,7 +477,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   for (int i = 0; i < 3; ++i) ctx->ws.zbuf[i] = reinterpret_cast<float*>(wsb + wl.zbuf + i * kZRep * vec);
   for (int i = 0; i < 2; ++i) {
     ctx->ws.gu[i] = reinterpret_cast<float*>(wsb + wl.gu + i * wl.gu_each);
-    ctx->ws.ssq[i] = ctx->ws.gu[i] + (size_t)cfg->capacity * 2 * kMaxBatch;
+    ctx->ws.ssq[i] = ctx->ws.gu[i] + (size_t)(cfg->dense_layers > 0 ? cfg->d_ffn : cfg->capacity) * 2 * kMaxBatch;
   }
   ctx->gu_bytes = 2 * wl.gu_each;
 
@@ -499,6 +501,10 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
                 mlp_tc_supported(d, ctx->sm_count);
   if (cfg->max_batch > 4 && !(cfg->flags & NP_F_NO_TENSOR_CORES)) pred_tc_prepare(d, b->w2, ctx->ws.hsplit, &ctx->tc);
   memset(ctx->host_lists, 0, host_lists_ints(*cfg) * 4);
+  if (d.dense > 0 && cfg->max_batch > 1 && !ctx->mlp_tc) {
+    np_destroy(ctx);
+    return fail(nullptr, NP_E_INVAL, "dense_layers > 0 with batches: this width is outside the tensor-core batch kernels");
+  }
   if (d.dense > 0) {
     Dims dd = d;
     dd.k = dd.C = d.M;
@@ -549,9 +555,12 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
   NP_LAUNCH(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
   // Dense layers are not scored: the sparse layers are a contiguous suffix of W2, of the logits
   // and of the bitmap (a dense prefix implies B = 1, so the per-sequence stride does not matter).
+  // With several sequences the per-sequence stride of the logits keeps all L layers, so every
+  // layer is scored and the dense layers' bitmap rows are cleared afterwards.
   Dims ds = d;
-  ds.L = d.L - d.dense;
-  const size_t skip_rows = (size_t)d.dense * d.M;
+  const int skip_layers = B == 1 ? d.dense : 0;
+  ds.L = d.L - skip_layers;
+  const size_t skip_rows = (size_t)skip_layers * d.M;
   float* logits = ctx->ws.logits + skip_rows;
   if (ds.L > 0) {
     if (B > 4 && ctx->tc.ready) {
@@ -561,7 +570,7 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
       NP_LAUNCH(ctx, launch_pred_l2(ds, static_cast<const char*>(ctx->bufs.w2) + skip_rows * d.H * 2, ctx->ws.hidden,
                                   B, logits, ctx->t.status, s, ctx->sm_count));
     }
-    NP_LAUNCH(ctx, launch_topk(ds, logits, B, ctx->t.pred + (size_t)d.dense * d.W, s));
+    NP_LAUNCH(ctx, launch_topk(ds, logits, B, ctx->t.pred + (size_t)skip_layers * d.W, s));
   }
   if (d.dense > 0) NP_CUDA(ctx, cudaMemsetAsync(ctx->t.pred, 0, (size_t)d.dense * d.W * 4, s));
   const size_t nlog = (size_t)B * ds.L * d.M * 4, nbm = (size_t)d.L * d.W * 4;
@@ -578,9 +587,11 @@ int np_topk(np_ctx* ctx, const float* logits, int32_t B, uint32_t* bitmap_out, v
   if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
   const Dims& d = ctx->d;
   Dims ds = d;
-  ds.L = d.L - d.dense;  // dense layers select nothing: their rows of the bitmap are zero
+  const int skip_layers = B == 1 ? d.dense : 0;  // dense layers select nothing: their rows of the bitmap are zero
+  ds.L = d.L - skip_layers;
   if (ds.L > 0)
-    NP_LAUNCH(ctx, launch_topk(ds, logits + (size_t)d.dense * d.M, B, bitmap_out + (size_t)d.dense * d.W, as_stream(stream)));
+    NP_LAUNCH(ctx, launch_topk(ds, logits + (size_t)skip_layers * d.M, B, bitmap_out + (size_t)skip_layers * d.W,
+                               as_stream(stream)));
   if (d.dense > 0) NP_CUDA(ctx, cudaMemsetAsync(bitmap_out, 0, (size_t)d.dense * d.W * 4, as_stream(stream)));
   return NP_OK;
 }
@@ -784,10 +795,21 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   const Dims& d = ctx->d;
   const size_t row_bytes = (size_t)d.D * 2;
   MlpArgs a;
-  a.gate_l = static_cast<const char*>(ctx->bufs.gate_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
-  a.up_l = static_cast<const char*>(ctx->bufs.up_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
-  a.downT_l = static_cast<const char*>(ctx->bufs.downT_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
-  a.active_slots = ctx->t.active_slots + (size_t)layer * d.C;
+  const bool dense_layer = layer < d.dense;
+  if (dense_layer) {  // whole records, every row active (tensor-core batch kernels only)
+    const char* rec0 = static_cast<const char*>(ctx->bufs.dense_buf) + (size_t)layer * d.M * d.rec_bytes;
+    a.gate_l = rec0;
+    a.up_l = rec0 + row_bytes;
+    a.downT_l = rec0 + 2 * row_bytes;
+    a.active_slots = ctx->t.identity;
+  } else {
+    a.gate_l = static_cast<const char*>(ctx->bufs.gate_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
+    a.up_l = static_cast<const char*>(ctx->bufs.up_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
+    a.downT_l = static_cast<const char*>(ctx->bufs.downT_buf) + (size_t)(layer - d.dense) * d.C * row_bytes;
+    a.active_slots = ctx->t.active_slots + (size_t)layer * d.C;
+  }
+  a.dense_rows = dense_layer ? d.M : 0;
+  a.gu_rows = d.dense > 0 ? d.M : d.C;
   a.n_active_ptr = ctx->t.counters + (size_t)layer * NP_N_COUNTERS + NP_CNT_ACTIVE;
   a.xa = xa;
   a.xb = xb;
@@ -814,6 +836,7 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
     NP_LAUNCH(ctx, launch_sparse_mlp_tc(d, a, s, ctx->sm_count));
     return NP_OK;
   }
+  if (dense_layer) return fail(ctx, NP_E_STATE, "dense layer %d reached a kernel that cannot run it", layer);
   NP_LAUNCH(ctx, launch_sparse_mlp(d, a, s, ctx->sm_count));
   return NP_OK;
 }
@@ -880,9 +903,11 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       a.l_end = l1;
       NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
     }
-  } else if (part != kChainHead) {
-    if (ctx->mlp_tc && B >= kTcMinBatch) NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.gu[0], 0, ctx->gu_bytes, s));
-    for (int l = 0; l < d.L; ++l) {
+  } else {
+    if (part != kChainTail && ctx->mlp_tc && B >= kTcMinBatch)
+      NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.gu[0], 0, ctx->gu_bytes, s));
+    const int lo = part == kChainTail ? d.dense : 0, hi = part == kChainHead ? d.dense : d.L;
+    for (int l = lo; l < hi; ++l) {
       int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
                          ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, 1, l & 1, s);
       if (rc < 0) return rc;

@@ -115,6 +115,9 @@ struct MlpArgs {
   float* gu_next;   // the next layer's, cleared by this layer (may be NULL)
   float* ssq;       // [kMaxBatch] sum of x^2 per sequence, zero on entry (needed with normalize)
   float* ssq_next;  // may be NULL
+  int gu_rows;      // rows each gu buffer holds (0 = C)
+  int dense_rows;   // > 0 (tensor-core path): a dense layer of that many whole records; gate_l / up_l / downT_l point
+                    // at the three rows of its first record, active_slots is an identity list, n_active_ptr is not read
 };
 cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count);
 // Batches on tensor cores: two launches per layer (np_mlp_tc.cu).

@@ -58,10 +58,12 @@ struct Blk {
   uint32_t row_stride;   // slice_bytes + 16: consecutive rows of a tile fall into different banks
   uint32_t slot_bytes;   // kTileRows * row_stride
   size_t slice_off;      // byte offset of this block's slice within a row
+  size_t row_pitch;      // bytes from one row to the next in the row buffers (D * 2, or a whole record for dense layers)
   int32_t* status;
 };
 
-__device__ __forceinline__ Blk make_blk(int B, int D, int C, int SW, int slice, int check, int32_t* status) {
+__device__ __forceinline__ Blk make_blk(int B, int D, int C, int SW, int slice, int check, int32_t* status,
+                                        int dense_rows) {
   Blk k;
   k.D = D, k.SW = SW, k.B = B, k.C = C, k.check = check;
   k.NJ = B > 8 ? 2 : 1;
@@ -70,6 +72,8 @@ __device__ __forceinline__ Blk make_blk(int B, int D, int C, int SW, int slice, 
   k.row_stride = k.slice_bytes + 16u;
   k.slot_bytes = (uint32_t)kTileRows * k.row_stride;
   k.slice_off = (size_t)slice * k.slice_bytes;
+  k.row_pitch = dense_rows > 0 ? (size_t)D * 6 : (size_t)D * 2;
+  if (dense_rows > 0) k.C = dense_rows;  // bound of the slot checks
   k.status = status;
   return k;
 }
@@ -156,7 +160,7 @@ __device__ __forceinline__ void issue_up_tile(const Blk& k, const unsigned char*
   if (lane == 0) mbar_expect_tx(full, (uint32_t)rows * 2u * k.slice_bytes);
   __syncwarp();
   if (lane < rows) {
-    const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r0 + lane) * k.D * 2 + k.slice_off;
+    const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r0 + lane) * k.row_pitch + k.slice_off;
     unsigned char* dst = tile + (size_t)lane * k.row_stride;
     bulk_g2s(dst, gate + src, k.slice_bytes, full);
     bulk_g2s(dst + (size_t)kUpTile * k.row_stride, up + src, k.slice_bytes, full);
@@ -172,7 +176,7 @@ __device__ __forceinline__ void issue_down_tile(const Blk& k, const unsigned cha
   __syncwarp();
   if (lane < kDownTile) {
     const int r = r0 + min(lane, rows - 1);
-    const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r) * k.D * 2 + k.slice_off;
+    const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r) * k.row_pitch + k.slice_off;
     bulk_g2s(tile + (size_t)lane * k.row_stride, downT + src, k.slice_bytes, full);
   }
 }
@@ -432,9 +436,9 @@ __device__ __forceinline__ void down_reds(const Blk& k, const float (&acc)[NJ][8
 }
 
 // every block clears its share of the next layer's accumulators
-__device__ __forceinline__ void clear_next(float* gu_next, float* ssq_next, int C, int bid, int nblk, int tid) {
+__device__ __forceinline__ void clear_next(float* gu_next, float* ssq_next, int rows, int bid, int nblk, int tid) {
   if (gu_next) {
-    const size_t total = (size_t)C * 2 * kSeq / 4;  // float4 units
+    const size_t total = (size_t)rows * 2 * kSeq / 4;  // float4 units
     const size_t lo = total * bid / nblk, hi = total * (bid + 1) / nblk;
     float4* p = reinterpret_cast<float4*>(gu_next);
     for (size_t i = lo + tid; i < hi; i += kC) p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -462,6 +466,9 @@ struct TcArgs {
   float* ssq_next;  // may be NULL
   int32_t* status;
   int B, D, C, SW, check, normalize, up_slots, down_slots;
+  int gu_rows;      // rows the GU buffers hold (all of them are cleared for the next layer)
+  int dense_rows;   // > 0: a dense layer.  gate / up / downT point at the three rows of its first record (row
+                    // pitch = one record), every one of its dense_rows rows is active, slots = an identity list
 };
 
 template <int NJ>
@@ -474,7 +481,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_up(TcArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int rb = blockIdx.x, RB = gridDim.x, ks = blockIdx.y;
   const int NS = a.up_slots;
-  const Blk k = make_blk(a.B, a.D, a.C, a.SW, ks, a.check, a.status);
+  const Blk k = make_blk(a.B, a.D, a.C, a.SW, ks, a.check, a.status, a.dense_rows);
   uint2* xf = reinterpret_cast<uint2*>(tsm);  // [n_ksteps][NJ][3 terms][32 lanes]
   unsigned char* ring = tsm + xf_bytes(k);    // [NS][kTileRows][row_stride]
 
@@ -488,7 +495,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_up(TcArgs a) {
   __syncthreads();
   pdl_launch_dependents();
 
-  const int n = checked_count(k, a.n_ptr);
+  const int n = a.dense_rows > 0 ? a.dense_rows : checked_count(k, a.n_ptr);
   const int r_begin = (int)(((long long)n * rb) / RB);
   const int r_end = (int)(((long long)n * (rb + 1)) / RB);
   const int n_tiles = (r_end - r_begin + kUpTile - 1) / kUpTile;
@@ -542,7 +549,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_down(TcArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int rb = blockIdx.x, RB = gridDim.x, cs = blockIdx.y;
   const int NS = a.down_slots;
-  const Blk k = make_blk(a.B, a.D, a.C, a.SW, cs, a.check, a.status);
+  const Blk k = make_blk(a.B, a.D, a.C, a.SW, cs, a.check, a.status, a.dense_rows);
   float* hs = reinterpret_cast<float*>(tsm);  // [kSeq][kHsStride]
   unsigned char* ring = tsm + kHsBytes;       // [NS][kTileRows][row_stride]
 
@@ -556,7 +563,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_down(TcArgs a) {
   __syncthreads();
   pdl_launch_dependents();
 
-  const int n = checked_count(k, a.n_ptr);
+  const int n = a.dense_rows > 0 ? a.dense_rows : checked_count(k, a.n_ptr);
   const int r_begin = (int)(((long long)n * rb) / RB);
   const int r_end = (int)(((long long)n * (rb + 1)) / RB);
   const int n_tiles = (r_end - r_begin + kDownTile - 1) / kDownTile;
@@ -578,7 +585,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_down(TcArgs a) {
 
   pdl_wait_prior();
   if (tid < kSeq) s_inv[tid] = a.normalize ? rsqrtf(__ldcg(a.ssq + tid) / (float)a.D + kRmsEps) : 1.f;
-  clear_next(a.gu_next, a.ssq_next, a.C, cs * RB + rb, RB * gridDim.y, tid);
+  clear_next(a.gu_next, a.ssq_next, a.gu_rows, cs * RB + rb, RB * gridDim.y, tid);
   consumer_sync();
 
   const int nt0 = wid * 8;                           // this warp's first n-tile of the slice
@@ -700,6 +707,8 @@ cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s
   ka.normalize = a.normalize;
   ka.up_slots = p.up_slots;
   ka.down_slots = p.down_slots;
+  ka.dense_rows = a.dense_rows;
+  ka.gu_rows = a.gu_rows > 0 ? a.gu_rows : a.C;
   const dim3 grid(p.RB, p.KS);
   if (a.B > 8) {
     cudaError_t e = tc_launch(k_mlp_tc_up<2>, grid, p.smem_up, ka, s);

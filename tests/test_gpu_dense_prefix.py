@@ -95,7 +95,8 @@ def test_caller_bitmaps_and_single_layer_calls_respect_the_dense_prefix():
 
 
 def test_configurations_that_exclude_a_dense_prefix():
-    for kw in (dict(max_batch=2), dict(flags=nb.NP_F_LAYER_LAUNCHES), dict(flags=nb.NP_F_DIRECT_LOADS)):
+    for kw in (dict(max_batch=2, flags=nb.NP_F_NO_TENSOR_CORES), dict(flags=nb.NP_F_LAYER_LAUNCHES),
+               dict(flags=nb.NP_F_DIRECT_LOADS)):
         cfg = nb.make_config(2, 256, 1024, 64, 102, 205, dense_layers=1, **kw)
         with pytest.raises(nb.NpError) as e:
             nb.np_query_sizes(cfg)
@@ -138,5 +139,35 @@ def test_lru_policy_reset_and_centroid_head_with_dense_prefix():
         torch.cuda.synchronize()
         w = words.cpu().numpy()
         assert not w[:d].any() and w[d:].any()
+    finally:
+        p.close()
+
+
+@pytest.mark.parametrize("cfg,d,B", [(SMALL, 1, 2), (SMALL, 2, 9), (DENSE, 2, 16), (DENSE, 4, 5)])
+def test_batches_with_dense_prefix(cfg, d, B):
+    """Several sequences: dense layers run through the tensor-core batch kernels on whole
+    records, every layer is scored (the logits keep their [B][L][M] layout) and the dense
+    layers' bitmap rows are cleared."""
+    p = Pair(cfg, max_batch=B, dense_layers=d, transfer_mode=nb.NP_XFER_ZERO_COPY, C=cfg.d_ffn // 2)
+    try:
+        L, M, W, D = cfg.n_layers, cfg.d_ffn, cfg.d_ffn // 32, cfg.d_model
+        xs = synth.hidden_states(cfg, 3, batch=B)
+        logits = torch.zeros((B, L, M), dtype=torch.float32, device="cuda")
+        bitmap = torch.full((L, W), -1, dtype=torch.int32, device="cuda")
+        out = torch.empty((B, D), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, B, logits, bitmap, p.eng.stream)
+            nb.np_step(p.eng.ctx, x, B, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            assert rel_l2(z32, O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)) < 1e-5
+            res = p.ora.step(u16(xs[t]), logits_f32=z32)
+            assert (bitmap.cpu().numpy().view(np.uint32) == res["pred"]).all() and not res["pred"][:d].any()
+            p.check_delta_against(res["deltas"])
+            got = out.cpu().numpy()
+            for b in range(B):
+                assert rel_l2(got[b], res["x_final"][b]) < 1e-5, (t, b)
+        p.check_resident_bytes()
     finally:
         p.close()
