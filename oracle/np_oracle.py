@@ -26,7 +26,9 @@ Parity unpinned against the paper (the paper is silent; these are this build's
 definitions, pinned only by invariants and determinism): the victim order of
 the LRU policy, the truncation rule when a predicted set exceeds capacity, and
 ``dense_prefix_plan`` against the paper's own operating points (found there by
-a throughput sweep on its device, not by a formula).
+a throughput sweep on its device, not by a formula), and the 8-bit record
+format of ``dequantize_records`` (the paper names quantised records only as
+future work; the rounding itself is pinned against a library conversion).
 """
 from __future__ import annotations
 
@@ -62,6 +64,30 @@ def dense_prefix_plan(L: int, M: int, D: int, C: int, budget_bytes: int, fixed_b
         if d * M * rec + (L - d) * C * rec + fixed_bytes <= budget_bytes:
             best = d
     return best
+
+
+def quantized_record_bytes(D: int) -> int:
+    """Size of an 8-bit record (a transfer-path variant the paper leaves as future work,
+    Section 6): the gate, up and transposed-down rows as int8, D values each, then their three
+    fp32 scales and four bytes of padding, so that records stay 16-byte aligned."""
+    return 3 * D + 16
+
+
+def dequantize_records(q_u8: np.ndarray, D: int) -> np.ndarray:
+    """8-bit records ``[..., 3*D + 16]`` (uint8) -> bf16 bit patterns ``[..., 3, D]`` (uint16).
+
+    Row p of a record is ``int8 q[p*D:(p+1)*D]`` with scale ``s_p`` (fp32, little endian, at byte
+    ``3*D + 4*p``); a weight is ``float32(q) * s_p`` (one fp32 multiplication) rounded to bf16,
+    ties to even.  This is this build's definition: the paper does not specify one."""
+    q_u8 = np.ascontiguousarray(q_u8, dtype=np.uint8)
+    lead = q_u8.shape[:-1]
+    assert q_u8.shape[-1] == quantized_record_bytes(D)
+    q = q_u8[..., :3 * D].view(np.int8).reshape(*lead, 3, D).astype(np.float32)
+    scales = np.ascontiguousarray(q_u8[..., 3 * D:3 * D + 12]).view(np.float32).reshape(*lead, 3)
+    w = (q * scales[..., None]).astype(np.float32)          # fp32 product, rounded once
+    bits = np.ascontiguousarray(w).view(np.uint32)
+    rounded = bits + np.uint32(0x7FFF) + ((bits >> np.uint32(16)) & np.uint32(1))
+    return (rounded >> np.uint32(16)).astype(np.uint16)
 
 
 def record_offset_bytes(layer: int, neuron: int, M: int, D: int) -> int:
