@@ -63,6 +63,8 @@ def parse_args():
                     help="dense prefix: the first d layers stay whole on the GPU and take no part in selection or install")
     ap.add_argument("--budget-gib", type=float, default=None,
                     help="device memory for MLP weights: the dense prefix becomes the longest one that fits (memory rule)")
+    ap.add_argument("--records", default="bf16", choices=["bf16", "int8"],
+                    help="int8: the store holds 8-bit rows with fp32 scales, dequantised to bf16 at install (a variant)")
     ap.add_argument("--no-variants", action="store_true",
                     help="skip the extra measurement of the zero-copy transfer mode (default run only)")
     ap.add_argument("--selection", default="topk", choices=["topk", "centroid"],
@@ -298,7 +300,14 @@ def cuda_arm(args):
         if args.dense_layers < 0:
             raise SystemExit("bench.py: the budget does not even hold the sparse layers' resident buffers")
     w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True)
+    if args.records == "int8":
+        qstore = torch.empty((cfg.n_layers, cfg.d_ffn, 3 * cfg.d_model + 16), dtype=torch.uint8)
+        nb.pin_host_tensor(qstore)
+        qstore = synth.quantize_store(store, device="cuda", out=qstore)
+        nb.unpin_host_tensor(store)                    # the bf16 store is not used any more
+        store = qstore
     ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
+                          record_format=nb.NP_REC_INT8 if args.records == "int8" else nb.NP_REC_BF16,
                           max_batch=args.batch, evict_policy=policy, transfer_mode=mode,
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
                           host_threads=args.host_threads, dense_layers=args.dense_layers,
@@ -306,7 +315,8 @@ def cuda_arm(args):
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0))
     eng = nb.Engine(ncfg, w1, w2, store, device=dev)
     L, D, M = cfg.n_layers, cfg.d_model, cfg.d_ffn
-    rec = cfg.record_bytes
+    rec = cfg.record_bytes                             # resident (bf16) bytes of a record
+    rec_store = 3 * D + 16 if args.records == "int8" else rec   # bytes of a record in the store
     T = 1 + W + K                                      # cold start + warm-up + timed
     n_detail = 16
     Bq = args.batch
@@ -461,6 +471,7 @@ def cuda_arm(args):
             "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
                         f"B={Bq} rho={cfg.rho} policy={args.policy} transfer={args.transfer}"
                         + (f" selection=centroid K={args.centroids}" if centroid else "")
+                        + (" records=int8" if args.records == "int8" else "")
                         + (f" dense_layers={args.dense_layers}" if args.dense_layers else "")
                         + (f" (longest prefix within {args.budget_gib} GiB)" if args.budget_gib is not None else ""),
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
@@ -469,7 +480,7 @@ def cuda_arm(args):
             "replicas": world,
         },
         "e2e": {"value": K * world / (e2e_ms_total / 1000.0), "unit": UNIT,
-                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * (L - nd) * rec), "d2h_bytes_per_step": int(Bq * D * 4)},
+                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * (L - nd) * rec_store), "d2h_bytes_per_step": int(Bq * D * 4)},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": mlp_kernel, "achieved": achieved, "peak": peak,
@@ -485,7 +496,8 @@ def cuda_arm(args):
 
     # ---- the same step with the other pinned-host transfer mode (reported beside, not as, the value) ----
     if (args.transfer == "gather" and not args.no_variants and not centroid and Bq == 1
-            and args.config == "7b" and not (args.layer_launches or args.direct_loads) and not args.dense_layers):
+            and args.config == "7b" and not (args.layer_launches or args.direct_loads) and not args.dense_layers
+            and args.records == "bf16"):
         eng.close()
         zcfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
                               max_batch=Bq, evict_policy=policy, transfer_mode=nb.NP_XFER_ZERO_COPY,
@@ -507,7 +519,8 @@ def cuda_arm(args):
             "value": K * world / (z_ms / 1000.0), "unit": UNIT, "ms_per_step": z_ms / K,
             "note": "scatter kernel reads the pinned store over PCIe by neuron ID; no host packing, no staging copy"}}
 
-    if rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid and not args.dense_layers:
+    if (rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid and not args.dense_layers
+            and args.records == "bf16"):
         n = args.cpu_baseline_steps
         times = run_oracle_steps(cfg, args.policy, w1.cpu(), w2.cpu(), store, xs_host, n)
         sec = float(np.mean(times))

@@ -68,6 +68,16 @@ extern "C" {
 #define NP_XFER_ZERO_COPY    2  /* the scatter kernel reads the pinned store directly by
                                    neuron ID (the paper's mapped-staging idea); no host sync */
 
+/* how the record store holds a neuron's three rows (np_config.record_format) */
+#define NP_REC_BF16  0  /* bf16 rows back to back: gate | up | downT, REC = 3 * D * 2 bytes
+                           (Section 3.5) */
+#define NP_REC_INT8  1  /* a transfer-path variant the paper leaves as future work: int8 rows
+                           gate | up | downT (D bytes each), then their three fp32 scales and 4
+                           bytes of padding, REC = 3 * D + 16.  The install path rounds
+                           float(q) * scale to bf16 (ties to even) as it places a row, so the
+                           resident buffers and the MLP kernels are unchanged and half the
+                           bytes cross PCIe.  Needs D % 16 == 0 and dense_layers == 0 */
+
 /* np_config.flags */
 #define NP_F_CHECK_BOUNDS    1  /* kernels validate every slot / neuron index and report
                                    through NP_E_DEVICE instead of touching memory */
@@ -116,14 +126,14 @@ typedef struct np_config {
                              empty and their tables stay empty.  d > 0 excludes
                              NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS, and with max_batch > 1
                              also NP_F_NO_TENSOR_CORES */
-  int32_t reserved[1];    /* must be 0 */
+  int32_t record_format;  /* NP_REC_*: how the store holds a record */
 } np_config;
 
 /* Byte counts of the caller-owned buffers for a configuration. */
 typedef struct np_sizes {
   uint64_t w1_bytes;          /* bf16 [H][D] */
   uint64_t w2_bytes;          /* bf16 [L*M][H] */
-  uint64_t backing_bytes;     /* bf16 [L][M][3][D] */
+  uint64_t backing_bytes;     /* [L][M] records of REC bytes (bf16 [L][M][3][D] with NP_REC_BF16) */
   uint64_t row_buffer_bytes;  /* bf16 [L - d][C][D], each of gate / up / downT (sparse layers only) */
   uint64_t staging_bytes;     /* staging_rows * REC (device; pinned host too for HOST_GATHER) */
   uint64_t workspace_bytes;   /* device scratch */

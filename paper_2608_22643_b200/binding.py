@@ -27,6 +27,7 @@ NP_F_CHECK_BOUNDS = 1
 NP_F_DIRECT_LOADS = 2
 NP_F_LAYER_LAUNCHES = 4
 NP_F_NO_TENSOR_CORES = 8
+NP_REC_BF16, NP_REC_INT8 = 0, 1
 (NP_CNT_PRED, NP_CNT_KEPT, NP_CNT_DELTA, NP_CNT_EVICT, NP_CNT_OVERFLOW, NP_CNT_ACTIVE,
  NP_CNT_RESIDENT, NP_CNT_STEP) = range(8)
 NP_N_COUNTERS = 8
@@ -43,7 +44,7 @@ class np_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
         "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers", "ring_stages",
-        "dense_layers")] + [("reserved", C.c_int32 * 1)]
+        "dense_layers", "record_format")]
 
 
 class np_sizes(C.Structure):
@@ -267,7 +268,7 @@ def np_predict_logits_noalloc(w1, w2, x_bf16, B: int, n_layers: int, d_model: in
 # ---- buffer owner ----------------------------------------------------------------------
 def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
                 transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0, ring_stages=0,
-                dense_layers=0) -> np_config:
+                dense_layers=0, record_format=0) -> np_config:
     cfg = np_config()
     cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
     cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
@@ -275,6 +276,7 @@ def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, st
     cfg.chain_layers = chain_layers
     cfg.ring_stages = ring_stages
     cfg.dense_layers = dense_layers
+    cfg.record_format = record_format
     cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
     return cfg
 
@@ -312,7 +314,7 @@ class Engine:
         L, D, M, Cap = cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.capacity
         assert w1.is_cuda and w2.is_cuda and not backing.is_cuda
         assert w1.numel() * 2 == self.sizes.w1_bytes and w2.numel() * 2 == self.sizes.w2_bytes
-        assert backing.numel() * 2 == self.sizes.backing_bytes and backing.is_contiguous()
+        assert backing.numel() * backing.element_size() == self.sizes.backing_bytes and backing.is_contiguous()
         self.w1, self.w2, self.backing = w1.contiguous(), w2.contiguous(), backing
         self._registered = False
         if not backing.is_pinned():

@@ -252,8 +252,15 @@ int check_config(const np_config* c, np_ctx* ctx) {
     return fail(ctx, NP_E_INVAL, "dense_layers > 0 with batches needs the tensor-core kernels");
   if (c->dense_layers > 0 && (c->flags & (NP_F_LAYER_LAUNCHES | NP_F_DIRECT_LOADS)))
     return fail(ctx, NP_E_INVAL, "dense_layers > 0 excludes NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS");
-  if (c->reserved[0]) return fail(ctx, NP_E_INVAL, "reserved fields must be 0");
+  if (c->record_format != NP_REC_BF16 && c->record_format != NP_REC_INT8)
+    return fail(ctx, NP_E_INVAL, "unknown record_format");
+  if (c->record_format == NP_REC_INT8 && (c->d_model % 16 || c->dense_layers > 0))
+    return fail(ctx, NP_E_INVAL, "8-bit records need d_model % 16 == 0 and dense_layers == 0");
   return NP_OK;
+}
+
+size_t record_bytes_of(const np_config& c) {
+  return c.record_format == NP_REC_INT8 ? 3ull * c.d_model + 16 : 3ull * c.d_model * 2;
 }
 
 struct WsLayout {
@@ -310,7 +317,7 @@ int np_query_sizes(const np_config* cfg, np_sizes* out) {
   int rc = check_config(cfg, nullptr);
   if (rc) return rc;
   const np_config& c = *cfg;
-  const uint64_t rec = 3ull * c.d_model * 2;
+  const uint64_t rec = record_bytes_of(c);
   out->record_bytes = rec;
   out->w1_bytes = 2ull * c.d_pred * c.d_model;
   out->w2_bytes = 2ull * c.n_layers * c.d_ffn * c.d_pred;
@@ -332,7 +339,7 @@ int np_plan_dense_prefix(const np_config* cfg, uint64_t budget_bytes, uint64_t f
   c.dense_layers = 0;  // the field is the answer, not an input
   int rc = check_config(&c, nullptr);
   if (rc) return rc;
-  const uint64_t rec = 3ull * c.d_model * 2;
+  const uint64_t rec = 3ull * c.d_model * 2;  // device-resident rows are bf16 whatever the store holds
   const uint64_t dense = (uint64_t)c.d_ffn * rec, sparse = (uint64_t)c.capacity * rec;
   *d_out = -1;
   for (int d = 0; d <= c.n_layers; ++d) {
@@ -399,7 +406,8 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   d.W = cfg->d_ffn / 32;
   d.Bmax = cfg->max_batch;
   d.ring_stages = cfg->ring_stages;
-  d.rec_bytes = 3ull * d.D * 2;
+  d.rec_bytes = record_bytes_of(*cfg);
+  d.rec_int8 = cfg->record_format == NP_REC_INT8;
   d.dense = cfg->dense_layers;
 
 #define NP_INIT_CUDA(call)                                                                   \

@@ -5,6 +5,8 @@
 //
 // The same kernel serves the zero-copy transfer mode, where `src` is the whole
 // layer of the pinned record store and records are addressed by neuron ID.
+#include <cuda_bf16.h>
+
 #include "np_device.cuh"
 #include "np_internal.h"
 
@@ -65,6 +67,67 @@ __global__ void __launch_bounds__(kScatterThreads) k_deinterleave_scatter(
   }
 }
 
+// 8-bit records (int8 gate | up | downT rows, three fp32 scales, padding): the rows are
+// dequantised on their way into the resident buffers, w = bf16_rn(float(q) * scale), so only
+// half the bytes of a bf16 record cross PCIe or sit in staging.  A thread turns 16 bytes of one
+// row into 32 bytes of bf16.
+__device__ __forceinline__ uint32_t dequant2(uint32_t q4, int shift, float scale) {
+  const float a = (float)(int)(signed char)((q4 >> shift) & 0xffu) * scale;
+  const float b = (float)(int)(signed char)((q4 >> (shift + 8)) & 0xffu) * scale;
+  const uint32_t lo = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(a));
+  const uint32_t hi = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(b));
+  return lo | (hi << 16);
+}
+
+template <bool kFromStore>
+__global__ void __launch_bounds__(kScatterThreads) k_dequant_scatter(
+    const unsigned char* __restrict__ src, const int32_t* __restrict__ ids, const int32_t* __restrict__ slots,
+    const int32_t* __restrict__ count_ptr, int first, int max_rows, uint4* __restrict__ gate,
+    uint4* __restrict__ up, uint4* __restrict__ downT, int D, size_t rec_bytes, int M, int C, int32_t* status,
+    int check) {
+  int n = *count_ptr - first;  // rows of this chunk
+  if (n > max_rows) n = max_rows;
+  const int q_chunks = D >> 4;  // 16-byte pieces of one int8 row
+  for (int r = blockIdx.x; r < n; r += gridDim.x) {
+    const int slot = slots[first + r];
+    size_t rec;
+    if (kFromStore) {
+      const int id = ids[first + r];
+      if (check && (id < 0 || id >= M)) {
+        if (threadIdx.x == 0) atomicOr(status, kStatBadNeuron);
+        continue;
+      }
+      rec = (size_t)id;
+    } else {
+      rec = (size_t)r;
+    }
+    if (check && (slot < 0 || slot >= C)) {
+      if (threadIdx.x == 0) atomicOr(status, kStatBadSlot);
+      continue;
+    }
+    const unsigned char* s = src + rec * rec_bytes;
+    const float* scales = reinterpret_cast<const float*>(s + (size_t)3 * D);
+    const size_t dst = (size_t)slot * (q_chunks * 2);  // uint4 units of a bf16 row
+    for (int c = threadIdx.x; c < 3 * q_chunks; c += kScatterThreads) {
+      const int p = c / q_chunks, cc = c - p * q_chunks;
+      const uint4 q = ldg_stream(s + (size_t)p * D + (size_t)cc * 16);
+      const float scale = __ldg(scales + p);
+      uint4 lo, hi;
+      lo.x = dequant2(q.x, 0, scale);
+      lo.y = dequant2(q.x, 16, scale);
+      lo.z = dequant2(q.y, 0, scale);
+      lo.w = dequant2(q.y, 16, scale);
+      hi.x = dequant2(q.z, 0, scale);
+      hi.y = dequant2(q.z, 16, scale);
+      hi.z = dequant2(q.w, 0, scale);
+      hi.w = dequant2(q.w, 16, scale);
+      uint4* row = p == 0 ? gate : (p == 1 ? up : downT);
+      row[dst + 2 * cc] = lo;
+      row[dst + 2 * cc + 1] = hi;
+    }
+  }
+}
+
 cudaError_t launch_scatter(const Dims& d, const void* src, bool src_is_store, const int32_t* ids,
                            const int32_t* slots, const int32_t* count_ptr, int first, int max_rows,
                            void* gate_l, void* up_l, void* downT_l, int32_t* status, int check,
@@ -74,6 +137,17 @@ cudaError_t launch_scatter(const Dims& d, const void* src, bool src_is_store, co
   int blocks = max_rows;
   const int cap = sm_count * 8;
   if (blocks > cap) blocks = cap;
+  if (d.rec_int8) {
+    if (src_is_store)
+      k_dequant_scatter<true><<<blocks, kScatterThreads, 0, s>>>(
+          static_cast<const unsigned char*>(src), ids, slots, count_ptr, first, max_rows, static_cast<uint4*>(gate_l),
+          static_cast<uint4*>(up_l), static_cast<uint4*>(downT_l), d.D, d.rec_bytes, d.M, d.C, status, check);
+    else
+      k_dequant_scatter<false><<<blocks, kScatterThreads, 0, s>>>(
+          static_cast<const unsigned char*>(src), ids, slots, count_ptr, first, max_rows, static_cast<uint4*>(gate_l),
+          static_cast<uint4*>(up_l), static_cast<uint4*>(downT_l), d.D, d.rec_bytes, d.M, d.C, status, check);
+    return cudaGetLastError();
+  }
   if (src_is_store) {
     k_deinterleave_scatter<true><<<blocks, kScatterThreads, 0, s>>>(
         static_cast<const uint4*>(src), ids, slots, count_ptr, first, max_rows, static_cast<uint4*>(gate_l),

@@ -232,19 +232,23 @@ def centroid_bank(cfg: StackConfig, n_centroids: int, mask_rows: Optional[int] =
     return out
 
 
-def quantize_store(store: torch.Tensor) -> torch.Tensor:
+def quantize_store(store: torch.Tensor, device: str = "cpu", out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """An 8-bit record store made from a bf16 one, uint8 ``[L, M, 3*D + 16]``: per row the int8
     values ``round(w / s)`` with ``s = max|w| / 127`` (fp32; 1 for an all-zero row), then the three
     scales as fp32 and four bytes of padding.  Input preparation only: what a weight *is* after
-    this (the product that is rounded back to bf16) is defined by whoever reads the store."""
+    this (the product that is rounded back to bf16) is defined by whoever reads the store.
+    ``device`` is where the arithmetic runs (layer by layer); the result is a host tensor."""
     L, M, three, D = store.shape
     assert three == 3 and D % 16 == 0
-    out = torch.zeros((L, M, 3 * D + 16), dtype=torch.uint8)
+    if out is None:
+        out = torch.zeros((L, M, 3 * D + 16), dtype=torch.uint8)
     for l in range(L):
-        w = store[l].to(torch.float32)                                   # [M, 3, D]
+        w = store[l].to(device).to(torch.float32)                        # [M, 3, D]
         s = w.abs().amax(dim=2) / 127.0
         s = torch.where(s > 0, s, torch.ones_like(s))
         q = torch.clamp(torch.round(w / s[..., None]), -127, 127).to(torch.int8)
-        out[l, :, :3 * D] = q.reshape(M, 3 * D).view(torch.uint8)
-        out[l, :, 3 * D:3 * D + 12] = s.contiguous().view(torch.uint8).reshape(M, 12)
+        rec = torch.zeros((M, 3 * D + 16), dtype=torch.uint8, device=w.device)
+        rec[:, :3 * D] = q.reshape(M, 3 * D).view(torch.uint8)
+        rec[:, 3 * D:3 * D + 12] = s.contiguous().view(torch.uint8).reshape(M, 12)
+        out[l].copy_(rec)
     return out
