@@ -108,22 +108,37 @@ __global__ void __launch_bounds__(kScatterThreads) k_dequant_scatter(
     const unsigned char* s = src + rec * rec_bytes;
     const float* scales = reinterpret_cast<const float*>(s + (size_t)3 * D);
     const size_t dst = (size_t)slot * (q_chunks * 2);  // uint4 units of a bf16 row
-    for (int c = threadIdx.x; c < 3 * q_chunks; c += kScatterThreads) {
-      const int p = c / q_chunks, cc = c - p * q_chunks;
-      const uint4 q = ldg_stream(s + (size_t)p * D + (size_t)cc * 16);
-      const float scale = __ldg(scales + p);
-      uint4 lo, hi;
-      lo.x = dequant2(q.x, 0, scale);
-      lo.y = dequant2(q.x, 16, scale);
-      lo.z = dequant2(q.y, 0, scale);
-      lo.w = dequant2(q.y, 16, scale);
-      hi.x = dequant2(q.z, 0, scale);
-      hi.y = dequant2(q.z, 16, scale);
-      hi.z = dequant2(q.w, 0, scale);
-      hi.w = dequant2(q.w, 16, scale);
-      uint4* row = p == 0 ? gate : (p == 1 ? up : downT);
-      row[dst + 2 * cc] = lo;
-      row[dst + 2 * cc + 1] = hi;
+    // up to four loads of a thread are issued before the first is converted
+    for (int c0 = threadIdx.x; c0 < 3 * q_chunks; c0 += kScatterThreads * 4) {
+      uint4 q[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = c0 + j * kScatterThreads;
+        if (c < 3 * q_chunks) {
+          const int p = c / q_chunks, cc = c - p * q_chunks;
+          q[j] = ldg_stream(s + (size_t)p * D + (size_t)cc * 16);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = c0 + j * kScatterThreads;
+        if (c < 3 * q_chunks) {
+          const int p = c / q_chunks, cc = c - p * q_chunks;
+          const float scale = __ldg(scales + p);
+          uint4 lo, hi;
+          lo.x = dequant2(q[j].x, 0, scale);
+          lo.y = dequant2(q[j].x, 16, scale);
+          lo.z = dequant2(q[j].y, 0, scale);
+          lo.w = dequant2(q[j].y, 16, scale);
+          hi.x = dequant2(q[j].z, 0, scale);
+          hi.y = dequant2(q[j].z, 16, scale);
+          hi.z = dequant2(q[j].w, 0, scale);
+          hi.w = dequant2(q[j].w, 16, scale);
+          uint4* row = p == 0 ? gate : (p == 1 ? up : downT);
+          row[dst + 2 * cc] = lo;
+          row[dst + 2 * cc + 1] = hi;
+        }
+      }
     }
   }
 }
