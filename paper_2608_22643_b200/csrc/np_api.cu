@@ -886,8 +886,8 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       a.downT = dense + 2 * row_bytes;
       a.active_slots = ctx->t.identity;
       a.dense_rows = d.M;
-      // Short runs: while a cooperative launch is resident the install's scatter kernels do not
-      // get onto the device, so the installs of the sparse layers advance between runs
+      // Short runs: while a resident launch is on the device the install's scatter kernels do
+      // not run beside it, so the installs of the sparse layers advance between runs
       // (measured at the 7B shape, d = 24: 612 steps/s with runs of 3, 448 with one run).
       constexpr int kDenseRun = 3;
       for (int l0 = 0; l0 < d.dense; l0 += kDenseRun) {
