@@ -64,7 +64,8 @@ extern "C" {
 #define NP_XFER_MEMCPY_RUNS  0  /* one cudaMemcpyAsync per run of adjacent neuron IDs into
                                    device staging, then the scatter kernel */
 #define NP_XFER_HOST_GATHER  1  /* host threads pack records into pinned staging, one
-                                   cudaMemcpyAsync per chunk, then the scatter kernel */
+                                   cudaMemcpyAsync per chunk, then the scatter kernel; the
+                                   staging buffers are used in up to four parts, round robin */
 #define NP_XFER_ZERO_COPY    2  /* the scatter kernel reads the pinned store directly by
                                    neuron ID (the paper's mapped-staging idea); no host sync */
 

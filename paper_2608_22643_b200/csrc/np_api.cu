@@ -159,6 +159,8 @@ class Pool {
 
 }  // namespace
 
+constexpr int kStageParts = 4;  // most parts the host-gather staging is split into
+
 struct np_ctx {
   np_config cfg;
   np_buffers bufs;
@@ -174,12 +176,12 @@ struct np_ctx {
   cudaEvent_t ev_delta = nullptr;
   std::vector<cudaEvent_t> ev_installed;
   std::vector<char> install_pending;
-  cudaEvent_t ev_half[2] = {nullptr, nullptr};  // host staging halves in flight
+  cudaEvent_t ev_half[kStageParts] = {};        // parts of the host / device staging in flight
   // library-owned side streams of the install path: [0] runs the scatter kernels behind the
   // staged copies; in zero-copy mode consecutive layers alternate between the two
   cudaStream_t aux[2] = {nullptr, nullptr};
-  cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr}, ev_copied[2] = {nullptr, nullptr};
-  bool half_pending[2] = {false, false};
+  cudaEvent_t ev_fork = nullptr, ev_join[2] = {nullptr, nullptr}, ev_copied[kStageParts] = {};
+  bool half_pending[kStageParts] = {};
   int next_half = 0;
   cudaEvent_t ev_t[4] = {nullptr, nullptr, nullptr, nullptr};  // compute-stream step timing
   cudaEvent_t ev_c[2] = {nullptr, nullptr};                    // copy-stream step timing
@@ -359,9 +361,10 @@ int np_destroy(np_ctx* ctx) {
     if (e) cudaEventDestroy(e);
   for (auto e : ctx->ev_half)
     if (e) cudaEventDestroy(e);
+  for (auto e : ctx->ev_copied)
+    if (e) cudaEventDestroy(e);
   for (int i = 0; i < 2; ++i) {
     if (ctx->ev_join[i]) cudaEventDestroy(ctx->ev_join[i]);
-    if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
     if (ctx->aux[i]) cudaStreamDestroy(ctx->aux[i]);
   }
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
@@ -495,10 +498,10 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   for (int l = 0; l < d.L; ++l)
     NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_installed[l], cudaEventDisableTiming));
   for (auto& e : ctx->ev_half) NP_INIT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  for (auto& e : ctx->ev_copied) NP_INIT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
   for (int i = 0; i < 2; ++i) {
     NP_INIT_CUDA(cudaStreamCreateWithFlags(&ctx->aux[i], cudaStreamNonBlocking));
     NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_join[i], cudaEventDisableTiming));
-    NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming));
   }
   NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
   for (auto& e : ctx->ev_t) NP_INIT_CUDA(cudaEventCreate(&e));
@@ -736,13 +739,17 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
                                     down_l, ctx->t.status, check, cs, ctx->sm_count));
       }
     } else {  // NP_XFER_HOST_GATHER: two halves of pinned staging, packed by the pool
-      const int half_rows = ctx->cfg.staging_rows / 2;
+      // the staging buffers are used in parts, round robin: a part is packed while earlier ones
+      // are copied and scattered (the scatter kernels can fall behind while a resident MLP
+      // launch holds the device; spare parts keep the host and the copy engine going)
+      const int parts = std::min(kStageParts, std::max(2, ctx->cfg.staging_rows / std::max(1, d.k / 4 + 1)));
+      const int half_rows = ctx->cfg.staging_rows / parts;
       char* hstage = static_cast<char*>(ctx->bufs.host_staging);
       if (n > half_rows && warn == NP_OK) warn = NP_W_CHUNKED;
       for (int first = 0; first < n; first += half_rows) {
         const int rows = std::min(half_rows, n - first);
-        const int h = ctx->next_half;
-        ctx->next_half ^= 1;
+        const int h = ctx->next_half % parts;
+        ctx->next_half = (h + 1) % parts;
         if (ctx->half_pending[h]) {
           NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_half[h]));
           ctx->half_pending[h] = false;
