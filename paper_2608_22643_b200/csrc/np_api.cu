@@ -243,7 +243,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
     return fail(ctx, NP_E_INVAL, "unknown transfer_mode");
   if (c->staging_rows < 1) return fail(ctx, NP_E_INVAL, "staging_rows must be >= 1");
   if (c->transfer_mode == NP_XFER_HOST_GATHER && c->staging_rows < 2)
-    return fail(ctx, NP_E_INVAL, "host gather needs staging_rows >= 2 (two halves)");
+    return fail(ctx, NP_E_INVAL, "host gather needs staging_rows >= 2 (at least two parts)");
   if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
@@ -738,7 +738,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
         NP_LAUNCH(ctx, launch_scatter(d, staging, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
                                     down_l, ctx->t.status, check, cs, ctx->sm_count));
       }
-    } else {  // NP_XFER_HOST_GATHER: two halves of pinned staging, packed by the pool
+    } else {  // NP_XFER_HOST_GATHER: parts of the pinned staging, packed by the pool
       // the staging buffers are used in parts, round robin: a part is packed while earlier ones
       // are copied and scattered (the scatter kernels can fall behind while a resident MLP
       // launch holds the device; spare parts keep the host and the copy engine going)
