@@ -536,9 +536,10 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   if (cfg->transfer_mode == NP_XFER_HOST_GATHER) {
     int n = cfg->host_threads;
     if (n == 0) {
-      // leave a few cores to the caller's thread, the driver and the copy engine's interrupts
+      // the packing is what bounds the transfer (steps/s kept rising up to 14 of 16 cores); two
+      // cores stay with the caller's thread and the driver
       const unsigned hc = std::thread::hardware_concurrency();
-      n = (int)std::max(1u, std::min(16u, hc > 8 ? hc - 4 : hc));
+      n = (int)std::max(1u, std::min(16u, hc > 8 ? hc - 2 : hc));
     }
     ctx->pool = new (std::nothrow) Pool(n - 1);  // the caller's thread works too
   }
