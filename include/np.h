@@ -77,7 +77,8 @@ extern "C" {
                            bytes of padding, REC = 3 * D + 16.  The install path rounds
                            float(q) * scale to bf16 (ties to even) as it places a row, so the
                            resident buffers and the MLP kernels are unchanged and half the
-                           bytes cross PCIe.  Needs D % 16 == 0 and dense_layers == 0 */
+                           bytes cross PCIe.  Needs D % 16 == 0.  Dense layers are rounded the
+                           same way once, in np_init */
 
 /* np_config.flags */
 #define NP_F_CHECK_BOUNDS    1  /* kernels validate every slot / neuron index and report

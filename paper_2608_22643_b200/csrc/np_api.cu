@@ -256,8 +256,8 @@ int check_config(const np_config* c, np_ctx* ctx) {
     return fail(ctx, NP_E_INVAL, "dense_layers > 0 excludes NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS");
   if (c->record_format != NP_REC_BF16 && c->record_format != NP_REC_INT8)
     return fail(ctx, NP_E_INVAL, "unknown record_format");
-  if (c->record_format == NP_REC_INT8 && (c->d_model % 16 || c->dense_layers > 0))
-    return fail(ctx, NP_E_INVAL, "8-bit records need d_model % 16 == 0 and dense_layers == 0");
+  if (c->record_format == NP_REC_INT8 && c->d_model % 16)
+    return fail(ctx, NP_E_INVAL, "8-bit records need d_model % 16 == 0");
   return NP_OK;
 }
 
@@ -325,7 +325,7 @@ int np_query_sizes(const np_config* cfg, np_sizes* out) {
   out->w2_bytes = 2ull * c.n_layers * c.d_ffn * c.d_pred;
   out->backing_bytes = rec * c.n_layers * c.d_ffn;
   out->row_buffer_bytes = 2ull * (c.n_layers - c.dense_layers) * c.capacity * c.d_model;
-  out->dense_bytes = (uint64_t)c.dense_layers * c.d_ffn * rec;
+  out->dense_bytes = (uint64_t)c.dense_layers * c.d_ffn * 3 * c.d_model * 2;  // bf16 whatever the store holds
   out->staging_bytes = rec * c.staging_rows;
   out->workspace_bytes = ws_layout(c).total;
   out->host_lists_bytes = host_lists_ints(c) * 4;
@@ -524,10 +524,19 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
       return fail(nullptr, NP_E_INVAL, "dense_layers > 0: this shape is outside what the resident MLP kernels cover");
     }
     // the dense layers' records move to the device once; their active list is 0 .. M-1
-    NP_INIT_CUDA(cudaMemcpy(b->dense_buf, b->backing, (size_t)d.dense * d.M * d.rec_bytes, cudaMemcpyHostToDevice));
     std::vector<int32_t> ident(d.M);
     for (int i = 0; i < d.M; ++i) ident[i] = i;
     NP_INIT_CUDA(cudaMemcpy(t.identity, ident.data(), (size_t)d.M * 4, cudaMemcpyHostToDevice));
+    const size_t dense_layer_bytes = (size_t)d.M * 3 * d.D * 2;
+    if (d.rec_int8) {
+      // 8-bit store: the same rounding as the install path, once, straight from the pinned store
+      for (int l = 0; l < d.dense; ++l)
+        NP_INIT_CUDA(launch_dequant_dense_layer(d, ctx->backing_dev + (size_t)l * d.M * d.rec_bytes, t.identity,
+                                                static_cast<char*>(b->dense_buf) + l * dense_layer_bytes, t.status,
+                                                nullptr, ctx->sm_count));
+    } else {
+      NP_INIT_CUDA(cudaMemcpy(b->dense_buf, b->backing, (size_t)d.dense * dense_layer_bytes, cudaMemcpyHostToDevice));
+    }
   }
   NP_INIT_CUDA(launch_tables_reset(d, t, nullptr));
   NP_INIT_CUDA(cudaDeviceSynchronize());
@@ -813,7 +822,7 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   MlpArgs a;
   const bool dense_layer = layer < d.dense;
   if (dense_layer) {  // whole records, every row active (tensor-core batch kernels only)
-    const char* rec0 = static_cast<const char*>(ctx->bufs.dense_buf) + (size_t)layer * d.M * d.rec_bytes;
+    const char* rec0 = static_cast<const char*>(ctx->bufs.dense_buf) + (size_t)layer * d.M * 3 * d.D * 2;
     a.gate_l = rec0;
     a.up_l = rec0 + row_bytes;
     a.downT_l = rec0 + 2 * row_bytes;

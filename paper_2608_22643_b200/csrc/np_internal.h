@@ -94,6 +94,9 @@ cudaError_t launch_scatter(const Dims& d, const void* src, bool src_is_store, co
                            void* gate_l, void* up_l, void* downT_l, int32_t* status, int check,
                            cudaStream_t s, int sm_count);
 
+cudaError_t launch_dequant_dense_layer(const Dims& d, const void* store_l, const int32_t* identity, void* dense_l,
+                                       int32_t* status, cudaStream_t s, int sm_count);
+
 struct MlpArgs {
   const void* gate_l;
   const void* up_l;

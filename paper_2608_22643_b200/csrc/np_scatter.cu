@@ -7,6 +7,8 @@
 // layer of the pinned record store and records are addressed by neuron ID.
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "np_device.cuh"
 #include "np_internal.h"
 
@@ -83,9 +85,10 @@ template <bool kFromStore>
 __global__ void __launch_bounds__(kScatterThreads) k_dequant_scatter(
     const unsigned char* __restrict__ src, const int32_t* __restrict__ ids, const int32_t* __restrict__ slots,
     const int32_t* __restrict__ count_ptr, int first, int max_rows, uint4* __restrict__ gate,
-    uint4* __restrict__ up, uint4* __restrict__ downT, int D, size_t rec_bytes, int M, int C, int32_t* status,
-    int check) {
-  int n = *count_ptr - first;  // rows of this chunk
+    uint4* __restrict__ up, uint4* __restrict__ downT, int D, size_t rec_bytes, int M, int C, int dst_pitch,
+    int32_t* status, int check) {
+  // count_ptr == NULL: exactly max_rows rows (the dense prefix is dequantised once, at start-up)
+  int n = count_ptr ? *count_ptr - first : max_rows;
   if (n > max_rows) n = max_rows;
   const int q_chunks = D >> 4;  // 16-byte pieces of one int8 row
   for (int r = blockIdx.x; r < n; r += gridDim.x) {
@@ -107,7 +110,7 @@ __global__ void __launch_bounds__(kScatterThreads) k_dequant_scatter(
     }
     const unsigned char* s = src + rec * rec_bytes;
     const float* scales = reinterpret_cast<const float*>(s + (size_t)3 * D);
-    const size_t dst = (size_t)slot * (q_chunks * 2);  // uint4 units of a bf16 row
+    const size_t dst = (size_t)slot * dst_pitch;  // uint4 units from one slot's row to the next
     // up to four loads of a thread are issued before the first is converted
     for (int c0 = threadIdx.x; c0 < 3 * q_chunks; c0 += kScatterThreads * 4) {
       uint4 q[4];
@@ -156,11 +159,13 @@ cudaError_t launch_scatter(const Dims& d, const void* src, bool src_is_store, co
     if (src_is_store)
       k_dequant_scatter<true><<<blocks, kScatterThreads, 0, s>>>(
           static_cast<const unsigned char*>(src), ids, slots, count_ptr, first, max_rows, static_cast<uint4*>(gate_l),
-          static_cast<uint4*>(up_l), static_cast<uint4*>(downT_l), d.D, d.rec_bytes, d.M, d.C, status, check);
+          static_cast<uint4*>(up_l), static_cast<uint4*>(downT_l), d.D, d.rec_bytes, d.M, d.C, (d.D >> 4) * 2, status,
+          check);
     else
       k_dequant_scatter<false><<<blocks, kScatterThreads, 0, s>>>(
           static_cast<const unsigned char*>(src), ids, slots, count_ptr, first, max_rows, static_cast<uint4*>(gate_l),
-          static_cast<uint4*>(up_l), static_cast<uint4*>(downT_l), d.D, d.rec_bytes, d.M, d.C, status, check);
+          static_cast<uint4*>(up_l), static_cast<uint4*>(downT_l), d.D, d.rec_bytes, d.M, d.C, (d.D >> 4) * 2, status,
+          check);
     return cudaGetLastError();
   }
   if (src_is_store) {
@@ -172,6 +177,21 @@ cudaError_t launch_scatter(const Dims& d, const void* src, bool src_is_store, co
         static_cast<const uint4*>(src), ids, slots, count_ptr, first, max_rows, static_cast<uint4*>(gate_l),
         static_cast<uint4*>(up_l), static_cast<uint4*>(downT_l), row_chunks, d.M, d.C, status, check);
   }
+  return cudaGetLastError();
+}
+
+// Start-up only: the 8-bit records of one dense layer, read from the pinned store, become whole
+// bf16 records [M][gate | up | downT][D] in the dense buffer (slot = neuron, rows three times
+// as far apart as in a slot buffer).
+cudaError_t launch_dequant_dense_layer(const Dims& d, const void* store_l, const int32_t* identity, void* dense_l,
+                                       int32_t* status, cudaStream_t s, int sm_count) {
+  const size_t row_bytes = (size_t)d.D * 2;
+  char* base = static_cast<char*>(dense_l);
+  const int blocks = std::min(d.M, sm_count * 8);
+  k_dequant_scatter<true><<<blocks, kScatterThreads, 0, s>>>(
+      static_cast<const unsigned char*>(store_l), identity, identity, nullptr, 0, d.M,
+      reinterpret_cast<uint4*>(base), reinterpret_cast<uint4*>(base + row_bytes),
+      reinterpret_cast<uint4*>(base + 2 * row_bytes), d.D, d.rec_bytes, d.M, d.M, 3 * (d.D >> 4) * 2, status, 1);
   return cudaGetLastError();
 }
 
