@@ -877,6 +877,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   const size_t n = (size_t)B * d.D;
   const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
                           mlp_chain_supported(d, ctx->sm_count);
+  const bool tc_batch = !persistent && ctx->mlp_tc && B >= kTcMinBatch && !(ctx->cfg.flags & NP_F_DIRECT_LOADS);
   if (part != kChainTail) {
     NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
     // the accumulator of layer 0 starts at zero (later ones are cleared one layer ahead)
@@ -933,14 +934,28 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.gu[0], 0, ctx->gu_bytes, s));
     const int lo = part == kChainTail ? d.dense : 0, hi = part == kChainHead ? d.dense : d.L;
     for (int l = lo; l < hi; ++l) {
-      int rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
-                         ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, 1, l & 1, s);
+      int rc;
+      if (tc_batch) {
+        // The tensor-core pair keeps x in the accumulator itself: the up kernel stores x_l into
+        // zbuf[l % 3] (its blocks of row block 0, one K slice each), the down kernel adds
+        // MLP_l(x_l) on top, and the next layer reads x_{l+1} from there: one vector to read per
+        // block instead of two, nothing to clear.
+        rc = mlp_layer(ctx, l, l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : ctx->ws.xbuf[1], nullptr, ctx->ws.zbuf[l % 3],
+                       ctx->ws.zbuf[l % 3], nullptr, B, 1, l & 1, s);
+      } else {
+        rc = mlp_layer(ctx, l, ctx->ws.xbuf[(l + 1) & 1], l > 0 ? ctx->ws.zbuf[(l - 1) % 3] : nullptr,
+                       ctx->ws.zbuf[l % 3], ctx->ws.xbuf[l & 1], ctx->ws.zbuf[(l + 1) % 3], B, 1, l & 1, s);
+      }
       if (rc < 0) return rc;
     }
   }
-  if (part != kChainHead)
-    NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], persistent ? kZRep : 1,
-                                  x_out, n, s));
+  if (part != kChainHead) {
+    if (tc_batch)  // the last accumulator holds the result
+      NP_LAUNCH(ctx, launch_add_vec(ctx->ws.zbuf[(d.L - 1) % 3], nullptr, 0, x_out, n, s));
+    else
+      NP_LAUNCH(ctx, launch_add_vec(ctx->ws.xbuf[(d.L - 1) & 1], ctx->ws.zbuf[(d.L - 1) % 3], persistent ? kZRep : 1,
+                                    x_out, n, s));
+  }
   return NP_OK;
 }
 
