@@ -20,7 +20,11 @@ bijection invariants and a set-based brute force for ``Residency.delta``;
 byte identity for ``install``; the dense SwiGLU library form when every row is
 active, linearity over disjoint sets and a scalar loop for ``sparse_mlp``; the
 paper's buffer-size arithmetic (Section 4.3) for ``record_bytes``; unit output
-RMS, scale invariance and a hand value for ``rms_normalize``.
+RMS, scale invariance and a hand value for ``rms_normalize``; a scan, boundary
+budgets and monotonicity for ``dense_prefix_plan``; the dense stack in a
+library's fp64 ops and "a dense layer is a sparse layer with every row active"
+for the dense prefix of ``Engine``; a library's fp32 -> bf16 conversion (with
+constructed ties) and hand values for ``dequantize_records``.
 
 Parity unpinned against the paper (the paper is silent; these are this build's
 definitions, pinned only by invariants and determinism): the victim order of
