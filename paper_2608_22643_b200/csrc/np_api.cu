@@ -807,7 +807,10 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
 // Orders `s` after a layer's install mark; marks that have already completed need no wait.
 static cudaError_t wait_install(np_ctx* ctx, int layer, cudaStream_t s) {
   const cudaError_t q = cudaEventQuery(ctx->ev_installed[layer]);
-  if (q == cudaSuccess) return cudaSuccess;
+  if (q == cudaSuccess) {
+    ctx->install_pending[layer] = 0;  // landed: later calls need not ask again
+    return cudaSuccess;
+  }
   if (q != cudaErrorNotReady) return q;
   (void)cudaGetLastError();
   return cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0);
