@@ -497,7 +497,7 @@ def cuda_arm(args):
     # ---- the same step with the other pinned-host transfer mode (reported beside, not as, the value) ----
     if (args.transfer == "gather" and not args.no_variants and not centroid and Bq == 1
             and args.config == "7b" and not (args.layer_launches or args.direct_loads) and not args.dense_layers
-            and args.records == "bf16"):
+            and args.records == "bf16" and world == 1):
         eng.close()
         zcfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
                               max_batch=Bq, evict_policy=policy, transfer_mode=nb.NP_XFER_ZERO_COPY,
