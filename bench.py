@@ -341,9 +341,7 @@ def cuda_arm(args):
         # bank lookup -> gate AND up -> delta -> install -> MLP chain, all through the C ABI
         nb.np_predict_logits_noalloc(eng.w1, w2c, x, Bq, L, D, 2 * Kc, cfg.d_pred, head_logits, s)
         nb.np_centroid_select(eng.ctx, head_logits, Bq, Kc, bank, None, sel_words, s)
-        nb.np_delta(eng.ctx, sel_words, s)
-        nb.np_install(eng.ctx, 0, L, cs)
-        return nb.np_mlp_chain(eng.ctx, x, Bq, out, s)
+        return nb.np_step_selected(eng.ctx, x, Bq, sel_words, out, s, cs)
 
     def barrier():
         torch.cuda.synchronize()
@@ -379,7 +377,7 @@ def cuda_arm(args):
     for i in range(n_detail):
         t = T + i                                       # the sequence simply continues
         step(xs_dev[t])
-        stage_us.append(np.full(4, np.nan, np.float32) if centroid else nb.np_last_step_times(eng.ctx))
+        stage_us.append(nb.np_last_step_times(eng.ctx))      # centroid selection: the predict stage is outside the call
         c = eng.counters()
         delta_rows.append(float(c[nd:, nb.NP_CNT_DELTA].mean()) if nd < L else 0.0)
         overflow_steps += int((c[:, nb.NP_CNT_OVERFLOW] > 0).any())

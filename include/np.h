@@ -284,6 +284,15 @@ int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* 
 int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream,
             void* copy_stream);
 
+/* The same step with the selection taken from the caller: `bitmap` (dev uint32
+ * [L][W], e.g. from np_centroid_select) replaces np_predict's top-k result;
+ * delta, install and the MLP chain run as in np_step, with the same ordering
+ * (a dense prefix is queued before the install).  np_last_step_times then
+ * reports 0 for the prediction stage.
+ * Errors: as np_step, and NP_E_INVAL for a NULL bitmap. */
+int np_step_selected(np_ctx* ctx, const void* x_bf16, int32_t B, const uint32_t* bitmap, float* x_out,
+                     void* stream, void* copy_stream);
+
 /* Stage 4 for every layer in order, nothing else: the chain of np_step,
  * x_{l+1} = x_l + MLP_l(x_l / rms(x_l)), over the rows that are active and resident now
  * (Section 3.1: the sparse suffix runs once the delta rows are in place).

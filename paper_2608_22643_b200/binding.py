@@ -34,7 +34,7 @@ NP_N_COUNTERS = 8
 
 EXPORTED = [
     "np_version", "np_query_sizes", "np_plan_dense_prefix", "np_init", "np_destroy", "np_reset", "np_last_error",
-    "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_get_delta",
+    "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_step_selected", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
     "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_last_error",
 ]
@@ -100,6 +100,7 @@ def load() -> C.CDLL:
         "np_install": [vp, i32, i32, vp],
         "np_sparse_mlp": [vp, i32, vp, i32, vp, vp],
         "np_step": [vp, vp, i32, vp, vp, vp],
+        "np_step_selected": [vp, vp, i32, vp, vp, vp, vp],
         "np_get_delta": [vp, i32, C.POINTER(np_delta_view)],
         "np_read_counters": [vp, vp, vp],
         "np_export_state": [vp, i32, vp, vp, vp, vp, vp],
@@ -212,6 +213,11 @@ def np_sparse_mlp(ctx, layer: int, x, B: int, y, stream=None) -> int:
 def np_step(ctx, x_bf16, B: int, x_out, stream, copy_stream) -> int:
     return _check(ctx, load().np_step(ctx, _ptr(x_bf16), B, _ptr(x_out), _stream(stream),
                                       _stream(copy_stream)))
+
+
+def np_step_selected(ctx, x_bf16, B: int, bitmap, x_out, stream=None, copy_stream=None) -> int:
+    return _check(ctx, load().np_step_selected(ctx, _ptr(x_bf16), B, _ptr(bitmap), _ptr(x_out), _stream(stream),
+                                               _stream(copy_stream)))
 
 
 def np_get_delta(ctx, layer: int) -> np_delta_view:

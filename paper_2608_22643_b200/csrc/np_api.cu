@@ -1001,18 +1001,23 @@ int np_sparse_mlp(np_ctx* ctx, int32_t layer, const float* x, int32_t B, float* 
   return mlp_layer(ctx, layer, x, nullptr, y, nullptr, nullptr, B, 0, -1, s);
 }
 
-int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream, void* copy_stream) {
+// One decode step; `selected` = NULL runs the library's own predictor and top-k, otherwise the
+// caller's bitmap takes their place.
+static int step_impl(np_ctx* ctx, const void* x_bf16, int32_t B, const uint32_t* selected, float* x_out,
+                     void* stream, void* copy_stream) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
-  if (!x_out) return fail(ctx, NP_E_INVAL, "x_out is NULL");
+  if (!x_bf16 || !x_out) return fail(ctx, NP_E_INVAL, "x or x_out is NULL");
   if ((uintptr_t)x_out % 16) return fail(ctx, NP_E_INVAL, "x_out must be 16-byte aligned");
-  if (stream == copy_stream) return fail(ctx, NP_E_INVAL, "np_step needs two different streams");
+  if (B < 1 || B > ctx->d.Bmax) return fail(ctx, NP_E_INVAL, "B=%d outside [1, max_batch=%d]", B, ctx->d.Bmax);
+  if (stream == copy_stream) return fail(ctx, NP_E_INVAL, "a step needs two different streams");
   const Dims& d = ctx->d;
   cudaStream_t s = as_stream(stream), cs = as_stream(copy_stream);
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[0], s));
-  int rc = np_predict(ctx, x_bf16, B, nullptr, nullptr, stream);
+  int rc = NP_OK;
+  if (!selected) rc = np_predict(ctx, x_bf16, B, nullptr, nullptr, stream);
   if (rc < 0) return rc;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[1], s));
-  rc = np_delta(ctx, nullptr, stream);
+  rc = np_delta(ctx, selected, stream);
   if (rc < 0) return rc;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[2], s));
   // the dense prefix waits for no install: it is queued before the host starts on the rows
@@ -1033,6 +1038,16 @@ int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stre
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[3], s));
   ctx->have_step = true;
   return warn;
+}
+
+int np_step(np_ctx* ctx, const void* x_bf16, int32_t B, float* x_out, void* stream, void* copy_stream) {
+  return step_impl(ctx, x_bf16, B, nullptr, x_out, stream, copy_stream);
+}
+
+int np_step_selected(np_ctx* ctx, const void* x_bf16, int32_t B, const uint32_t* bitmap, float* x_out, void* stream,
+                     void* copy_stream) {
+  if (ctx && !bitmap) return fail(ctx, NP_E_INVAL, "bitmap is NULL");
+  return step_impl(ctx, x_bf16, B, bitmap, x_out, stream, copy_stream);
 }
 
 int np_last_step_times(np_ctx* ctx, float* out_us) {

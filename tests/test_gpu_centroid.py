@@ -113,6 +113,33 @@ def test_centroid_heads_drive_the_whole_path(cfg, B, K, policy):
         p.close()
 
 
+@pytest.mark.parametrize("dense", [0, 1])
+def test_step_from_a_supplied_bitmap(dense):
+    """np_step_selected = np_step with the predictor's result replaced by the caller's bitmap:
+    same lists, tables, resident bytes and chain output as the oracle stepping on those sets."""
+    cfg, B = SMALL, 1
+    p = Pair(cfg, max_batch=B, dense_layers=dense)
+    try:
+        L, D, W = cfg.n_layers, cfg.d_model, cfg.d_ffn // 32
+        xs = synth.hidden_states(cfg, cfg.n_tokens, batch=B)
+        words = synth.random_bitmaps(L, cfg.d_ffn, p.k, 9, cfg.n_tokens, 0.8)
+        out = torch.empty((B, D), dtype=torch.float32, device="cuda")
+        for t in range(cfg.n_tokens):
+            nb.np_step_selected(p.eng.ctx, xs[t].cuda(), B, words[t].cuda(), out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            res = p.ora.step(u16(xs[t]), pred_words=words[t].numpy().view(np.uint32))
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < REL_L2_TOL, t
+            times = nb.np_last_step_times(p.eng.ctx)
+            assert times[0] < 50.0                     # no predictor pass inside the call
+        p.check_resident_bytes()
+        with pytest.raises(nb.NpError) as e:
+            nb.np_step_selected(p.eng.ctx, xs[0].cuda(), B, None, out, p.eng.stream, p.eng.copy_stream)
+        assert e.value.code == nb.NP_E_INVAL
+    finally:
+        p.close()
+
+
 def test_full_width_bank_at_7b_row_shape():
     """M = 11008, K = 512 (the paper's vocabulary) on two layers: bit-exact selection."""
     cfg = synth.StackConfig("7b2", 2, 256, 11008, 64, 10, 25, 2, 3, 0.97)
