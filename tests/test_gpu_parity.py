@@ -248,6 +248,32 @@ def test_mlp_kernel_variants_agree_with_oracle(cfg, flags, chain_layers, ring_st
         p.close()
 
 
+@pytest.mark.parametrize("flags", [nb.NP_F_CHECK_BOUNDS, nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES])
+@pytest.mark.parametrize("n_set", [0, 1, 100, 1200])
+def test_resident_chain_with_set_sizes_away_from_k(n_set, flags):
+    """Active sets the caller supplies, from empty to nearly the whole capacity: blocks without
+    rows, and shares of more rows than one tile holds (the kernels were planned for k rows)."""
+    cfg = DENSE
+    p = Pair(cfg, flags=flags)
+    try:
+        L, D = cfg.n_layers, cfg.d_model
+        assert n_set <= p.C
+        words = synth.random_bitmaps(L, cfg.d_ffn, max(n_set, 1), 77, 3, 0.6)
+        if n_set == 0:
+            words.zero_()
+        xs = synth.hidden_states(cfg, 3)
+        out = torch.empty((1, D), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            nb.np_step_selected(p.eng.ctx, xs[t].cuda(), 1, words[t].cuda(), out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            res = p.ora.step(u16(xs[t]), pred_words=words[t].numpy().view(np.uint32))
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+        p.eng.counters()
+    finally:
+        p.close()
+
+
 def test_call_order_and_argument_errors():
     p = Pair(TINY, with_oracle=False)
     try:
