@@ -43,7 +43,7 @@
 extern "C" {
 #endif
 
-#define NP_VERSION 2
+#define NP_VERSION 3
 
 /* return codes */
 #define NP_OK           0
@@ -52,6 +52,7 @@ extern "C" {
 #define NP_E_CUDA      -3   /* a CUDA runtime call failed; see np_last_error */
 #define NP_E_NOMEM     -4   /* allocation of library-owned state failed */
 #define NP_E_DEVICE    -5   /* a kernel's own bounds check tripped; state is suspect */
+#define NP_E_IO        -6   /* a read of the store file failed or came up short */
 #define NP_W_OVERFLOW   1   /* some layer's predicted set did not fit capacity */
 #define NP_W_CHUNKED    2   /* some layer's delta exceeded staging and was split */
 
@@ -68,6 +69,14 @@ extern "C" {
                                    staging buffers are used in up to four parts, round robin */
 #define NP_XFER_ZERO_COPY    2  /* the scatter kernel reads the pinned store directly by
                                    neuron ID (the paper's mapped-staging idea); no host sync */
+#define NP_XFER_FILE         3  /* the store is a file (Section 3.5): the incoming IDs of a chunk,
+                                   already ascending, are coalesced into ranges of adjacent
+                                   records and read through io_uring (np_config.io_depth reads
+                                   in flight; blocking preads from the host threads where the
+                                   kernel offers no io_uring) into parts of the pinned staging,
+                                   then one cudaMemcpyAsync per chunk and the scatter kernel as
+                                   with HOST_GATHER.  np_buffers.backing is not used;
+                                   np_buffers.backing_fd is.  Needs NP_REC_BF16 */
 
 /* how the record store holds a neuron's three rows (np_config.record_format) */
 #define NP_REC_BF16  0  /* bf16 rows back to back: gate | up | downT, REC = 3 * D * 2 bytes
@@ -129,6 +138,9 @@ typedef struct np_config {
                              NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS, and with max_batch > 1
                              also NP_F_NO_TENSOR_CORES */
   int32_t record_format;  /* NP_REC_*: how the store holds a record */
+  int32_t io_depth;       /* NP_XFER_FILE: reads in flight (0 = 256, the paper's queue depth;
+                             < 0 = no io_uring, blocking preads from the host threads) */
+  int32_t reserved;       /* 0 */
 } np_config;
 
 /* Byte counts of the caller-owned buffers for a configuration. */
@@ -149,15 +161,24 @@ typedef struct np_sizes {
 typedef struct np_buffers {
   const void* w1;          /* dev  */
   const void* w2;          /* dev  */
-  const void* backing;     /* pinned host (cudaHostAlloc or cudaHostRegister) */
+  const void* backing;     /* pinned host (cudaHostAlloc or cudaHostRegister); may be NULL with
+                              NP_XFER_FILE */
   void* gate_buf;          /* dev  */
   void* up_buf;            /* dev  */
   void* downT_buf;         /* dev  */
   void* staging;           /* dev; unused (may be NULL) with NP_XFER_ZERO_COPY */
-  void* host_staging;      /* pinned host, staging_bytes; only for NP_XFER_HOST_GATHER */
+  void* host_staging;      /* pinned host, staging_bytes; only for NP_XFER_HOST_GATHER and
+                              NP_XFER_FILE */
   void* workspace;         /* dev, 256-byte aligned */
   void* host_lists;        /* pinned host */
   void* dense_buf;         /* dev, dense_bytes; NULL when dense_layers = 0.  Filled by np_init */
+  int32_t backing_fd;      /* NP_XFER_FILE: descriptor of the store file, record (l, n) at byte
+                              (l*M + n)*REC, open for reading for the life of the context and
+                              owned by the caller.  With O_DIRECT (the paper's way; reads then
+                              bypass the page cache) REC must suit the file system's alignment
+                              rule, commonly a multiple of 512 bytes; the staging parts are
+                              4096-byte aligned when host_staging is.  Ignored otherwise */
+  int32_t reserved;        /* 0 */
 } np_buffers;
 
 /* Device views of one layer's lists from the last np_delta (valid until the next). */
@@ -249,6 +270,17 @@ int np_centroid_select(np_ctx* ctx, const float* logits, int32_t B, int32_t K, c
  * Does not synchronise.  Warnings are reported by np_install / np_read_counters. */
 int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream);
 
+/* Stage 3b of the file path on its own, no GPU involved (Section 3.5): reads records
+ * ids[0..n) (strictly ascending; record `id` = file bytes [base_offset + id*rec_bytes,
+ * +rec_bytes)) into dst + i*rec_bytes, one range per run of adjacent IDs, with io_depth reads
+ * in flight (meaning as np_config.io_depth).  Blocks until every read has completed.
+ * `dst` is host memory the caller owns (aligned as the descriptor's flags demand).
+ * *n_ranges_out (may be NULL) = coalesced ranges; *used_ring_out (may be NULL) = 1 if io_uring
+ * carried the reads, 0 if blocking preads did.
+ * Errors: NP_E_INVAL (descriptor, sizes, NULL, unsorted ids), NP_E_IO; text in np_last_error(NULL). */
+int np_read_records(int32_t fd, uint64_t base_offset, uint64_t rec_bytes, const int32_t* ids, int32_t n, void* dst,
+                    int32_t io_depth, int32_t* n_ranges_out, int32_t* used_ring_out);
+
 /* Stage 3b + 3c for layers [layer_begin, layer_end): copy each incoming record
  * (L, n) = bytes [(l*M + n)*REC, +REC) of the store to slot S[n] of the three
  * row buffers, on `copy_stream`, and mark each layer installed (np_sparse_mlp
@@ -256,12 +288,15 @@ int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream);
  * delta step.  Scatter kernels may run on streams the library owns; those are
  * ordered after the work `copy_stream` held on entry and joined back into it
  * before the call returns, so work queued on `copy_stream` afterwards sees
- * every row installed.  With NP_XFER_MEMCPY_RUNS / NP_XFER_HOST_GATHER this call blocks
- * the host until the delta lists of the last np_delta are readable; with
- * NP_XFER_ZERO_COPY it never blocks.  Deltas larger than staging_rows are split
+ * every row installed.  With NP_XFER_MEMCPY_RUNS / NP_XFER_HOST_GATHER / NP_XFER_FILE this
+ * call blocks the host until the delta lists of the last np_delta are readable (and, with
+ * NP_XFER_FILE, until the last chunk's reads have completed); with NP_XFER_ZERO_COPY it
+ * never blocks.  Deltas larger than staging_rows are split
  * into chunks in list order (result unchanged).
  * Returns NP_W_OVERFLOW / NP_W_CHUNKED (OVERFLOW wins) where it can know.
- * Errors: NP_E_STATE (no np_delta since init/reset), NP_E_INVAL, NP_E_CUDA. */
+ * Errors: NP_E_STATE (no np_delta since init/reset), NP_E_INVAL, NP_E_CUDA, NP_E_IO (a file
+ * read failed: no read is left in flight when the call returns, the layers from the failing
+ * chunk on are not marked installed). */
 int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_stream);
 
 /* Stage 4 for one layer (Section 3.4): over act = P and R of the last np_delta,

@@ -19,10 +19,10 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libnp.so")
 
-NP_OK, NP_E_INVAL, NP_E_STATE, NP_E_CUDA, NP_E_NOMEM, NP_E_DEVICE = 0, -1, -2, -3, -4, -5
+NP_OK, NP_E_INVAL, NP_E_STATE, NP_E_CUDA, NP_E_NOMEM, NP_E_DEVICE, NP_E_IO = 0, -1, -2, -3, -4, -5, -6
 NP_W_OVERFLOW, NP_W_CHUNKED = 1, 2
 NP_EVICT_EXACT, NP_EVICT_LRU = 0, 1
-NP_XFER_MEMCPY_RUNS, NP_XFER_HOST_GATHER, NP_XFER_ZERO_COPY = 0, 1, 2
+NP_XFER_MEMCPY_RUNS, NP_XFER_HOST_GATHER, NP_XFER_ZERO_COPY, NP_XFER_FILE = 0, 1, 2, 3
 NP_F_CHECK_BOUNDS = 1
 NP_F_DIRECT_LOADS = 2
 NP_F_LAYER_LAUNCHES = 4
@@ -34,7 +34,7 @@ NP_N_COUNTERS = 8
 
 EXPORTED = [
     "np_version", "np_query_sizes", "np_plan_dense_prefix", "np_init", "np_destroy", "np_reset", "np_last_error",
-    "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_install", "np_sparse_mlp", "np_step", "np_step_selected", "np_get_delta",
+    "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_read_records", "np_install", "np_sparse_mlp", "np_step", "np_step_selected", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
     "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_last_error",
 ]
@@ -44,7 +44,7 @@ class np_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
         "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers", "ring_stages",
-        "dense_layers", "record_format")]
+        "dense_layers", "record_format", "io_depth", "reserved")]
 
 
 class np_sizes(C.Structure):
@@ -56,7 +56,7 @@ class np_sizes(C.Structure):
 class np_buffers(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "w1", "w2", "backing", "gate_buf", "up_buf", "downT_buf", "staging", "host_staging", "workspace",
-        "host_lists", "dense_buf")]
+        "host_lists", "dense_buf")] + [("backing_fd", C.c_int32), ("reserved", C.c_int32)]
 
 
 class np_delta_view(C.Structure):
@@ -98,6 +98,7 @@ def load() -> C.CDLL:
         "np_centroid_select": [vp, vp, i32, i32, vp, vp, vp, vp],
         "np_delta": [vp, vp, vp],
         "np_install": [vp, i32, i32, vp],
+        "np_read_records": [i32, C.c_uint64, C.c_uint64, vp, i32, vp, i32, vp, vp],
         "np_sparse_mlp": [vp, i32, vp, i32, vp, vp],
         "np_step": [vp, vp, i32, vp, vp, vp],
         "np_step_selected": [vp, vp, i32, vp, vp, vp, vp],
@@ -202,6 +203,18 @@ def np_delta(ctx, pred_bitmap=None, stream=None) -> int:
     return _check(ctx, load().np_delta(ctx, _ptr(pred_bitmap), _stream(stream)))
 
 
+def np_read_records(fd: int, base_offset: int, rec_bytes: int, ids: np.ndarray, dst: np.ndarray, io_depth: int = 0):
+    """Reads the records ``ids`` (ascending) of a store file into ``dst``; returns
+    ``(coalesced ranges, whether io_uring carried the reads)``."""
+    ids = np.ascontiguousarray(ids, dtype=np.int32)
+    assert dst.flags["C_CONTIGUOUS"] and dst.nbytes >= ids.size * rec_bytes
+    ranges, ring = C.c_int32(0), C.c_int32(0)
+    rc = load().np_read_records(fd, base_offset, rec_bytes, ids.ctypes.data, ids.size, dst.ctypes.data, io_depth,
+                                C.addressof(ranges), C.addressof(ring))
+    _check(None, rc)
+    return ranges.value, bool(ring.value)
+
+
 def np_install(ctx, layer_begin: int, layer_end: int, copy_stream=None) -> int:
     return _check(ctx, load().np_install(ctx, layer_begin, layer_end, _stream(copy_stream)))
 
@@ -274,7 +287,7 @@ def np_predict_logits_noalloc(w1, w2, x_bf16, B: int, n_layers: int, d_model: in
 # ---- buffer owner ----------------------------------------------------------------------
 def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
                 transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0, ring_stages=0,
-                dense_layers=0, record_format=0) -> np_config:
+                dense_layers=0, record_format=0, io_depth=0) -> np_config:
     cfg = np_config()
     cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
     cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
@@ -283,6 +296,7 @@ def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, st
     cfg.ring_stages = ring_stages
     cfg.dense_layers = dense_layers
     cfg.record_format = record_format
+    cfg.io_depth = io_depth
     cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
     return cfg
 
@@ -309,23 +323,39 @@ class Engine:
     """Owns the caller-side buffers of one context and forwards to the C calls.
 
     ``w1``/``w2`` are bf16 device tensors, ``backing`` a bf16 CPU tensor
-    ``[L, M, 3, D]`` (it is page-locked here if it is not already)."""
+    ``[L, M, 3, D]`` (it is page-locked here if it is not already).  With
+    ``NP_XFER_FILE`` the store is a file instead: ``backing`` is ``None`` and
+    ``store_path`` names it; it is opened with ``O_DIRECT`` when the file
+    system allows (``direct_io`` says whether it was)."""
 
-    def __init__(self, cfg: np_config, w1: torch.Tensor, w2: torch.Tensor, backing: torch.Tensor,
-                 device: str = "cuda:0"):
+    def __init__(self, cfg: np_config, w1: torch.Tensor, w2: torch.Tensor, backing: Optional[torch.Tensor],
+                 device: str = "cuda:0", store_path: Optional[str] = None, direct: bool = True):
         self.cfg = cfg
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         self.sizes = np_query_sizes(cfg)
         L, D, M, Cap = cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.capacity
-        assert w1.is_cuda and w2.is_cuda and not backing.is_cuda
+        assert w1.is_cuda and w2.is_cuda
         assert w1.numel() * 2 == self.sizes.w1_bytes and w2.numel() * 2 == self.sizes.w2_bytes
-        assert backing.numel() * backing.element_size() == self.sizes.backing_bytes and backing.is_contiguous()
         self.w1, self.w2, self.backing = w1.contiguous(), w2.contiguous(), backing
         self._registered = False
-        if not backing.is_pinned():
-            pin_host_tensor(backing)
-            self._registered = True
+        self.store_fd, self.direct_io = -1, False
+        if cfg.transfer_mode == NP_XFER_FILE:
+            assert backing is None and store_path is not None
+            if direct:
+                try:
+                    self.store_fd = os.open(store_path, os.O_RDONLY | os.O_DIRECT)
+                    self.direct_io = True
+                except OSError:
+                    self.store_fd = -1
+            if self.store_fd < 0:
+                self.store_fd = os.open(store_path, os.O_RDONLY)
+        else:
+            assert not backing.is_cuda
+            assert backing.numel() * backing.element_size() == self.sizes.backing_bytes and backing.is_contiguous()
+            if not backing.is_pinned():
+                pin_host_tensor(backing)
+                self._registered = True
         dev = self.device
         nd = cfg.dense_layers                       # leading dense layers: no slot buffers, one record buffer
         self.gate = torch.zeros((L - nd, Cap, D), dtype=torch.bfloat16, device=dev)
@@ -334,13 +364,24 @@ class Engine:
         self.dense = torch.empty((nd, M, 3, D), dtype=torch.bfloat16, device=dev) if nd else None
         self.staging = torch.empty(int(self.sizes.staging_bytes), dtype=torch.uint8, device=dev)
         self.host_staging = None
+        self._staging_registered = False
         if cfg.transfer_mode == NP_XFER_HOST_GATHER:
             self.host_staging = torch.empty(int(self.sizes.staging_bytes), dtype=torch.uint8).pin_memory()
+        elif cfg.transfer_mode == NP_XFER_FILE:
+            # page-aligned (direct reads land here), page-locked in place
+            raw = torch.empty(int(self.sizes.staging_bytes) + 4096, dtype=torch.uint8)
+            skip = (-raw.data_ptr()) % 4096
+            self.host_staging = raw[skip:skip + int(self.sizes.staging_bytes)]
+            self._host_staging_raw = raw
+            pin_host_tensor(self.host_staging)
+            self._staging_registered = True
         self.workspace = torch.empty(int(self.sizes.workspace_bytes) + 256, dtype=torch.uint8, device=dev)
         ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
         self.host_lists = torch.zeros(int(self.sizes.host_lists_bytes) // 4, dtype=torch.int32).pin_memory()
         b = np_buffers()
-        b.w1, b.w2, b.backing = self.w1.data_ptr(), self.w2.data_ptr(), backing.data_ptr()
+        b.w1, b.w2 = self.w1.data_ptr(), self.w2.data_ptr()
+        b.backing = backing.data_ptr() if backing is not None else None
+        b.backing_fd = self.store_fd
         if L - nd > 0:
             b.gate_buf, b.up_buf, b.downT_buf = self.gate.data_ptr(), self.up.data_ptr(), self.downT.data_ptr()
         b.staging = self.staging.data_ptr()
@@ -359,6 +400,12 @@ class Engine:
         if self._registered:
             unpin_host_tensor(self.backing)
             self._registered = False
+        if getattr(self, "_staging_registered", False):
+            unpin_host_tensor(self.host_staging)
+            self._staging_registered = False
+        if getattr(self, "store_fd", -1) >= 0:
+            os.close(self.store_fd)
+            self.store_fd = -1
 
     def __del__(self):
         try:

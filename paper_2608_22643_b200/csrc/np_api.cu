@@ -11,13 +11,16 @@
 #include <functional>
 #include <mutex>
 #include <new>
+#include <deque>
 #include <thread>
 #if defined(__SSE2__)
 #include <emmintrin.h>
 #include <xmmintrin.h>
+#include <sys/stat.h>
 #endif
 
 #include "np_internal.h"
+#include "np_io.h"
 
 using namespace npi;
 
@@ -191,6 +194,7 @@ struct np_ctx {
   int step = 0;
   uint64_t launches = 0;
   Pool* pool = nullptr;
+  RecordReader reader;   // NP_XFER_FILE: reads of the store file
   PredTcState tc = {};
   size_t gu_bytes = 0;   // both dot-product accumulators of the batch MLP, contiguous
   bool mlp_tc = false;   // batches run the tensor-core MLP kernels
@@ -239,11 +243,14 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->max_batch < 1 || c->max_batch > kMaxBatch) return fail(ctx, NP_E_INVAL, "max_batch must be in [1, 16]");
   if (c->evict_policy != NP_EVICT_EXACT && c->evict_policy != NP_EVICT_LRU)
     return fail(ctx, NP_E_INVAL, "unknown evict_policy");
-  if (c->transfer_mode < NP_XFER_MEMCPY_RUNS || c->transfer_mode > NP_XFER_ZERO_COPY)
+  if (c->transfer_mode < NP_XFER_MEMCPY_RUNS || c->transfer_mode > NP_XFER_FILE)
     return fail(ctx, NP_E_INVAL, "unknown transfer_mode");
   if (c->staging_rows < 1) return fail(ctx, NP_E_INVAL, "staging_rows must be >= 1");
-  if (c->transfer_mode == NP_XFER_HOST_GATHER && c->staging_rows < 2)
-    return fail(ctx, NP_E_INVAL, "host gather needs staging_rows >= 2 (at least two parts)");
+  if ((c->transfer_mode == NP_XFER_HOST_GATHER || c->transfer_mode == NP_XFER_FILE) && c->staging_rows < 2)
+    return fail(ctx, NP_E_INVAL, "host gather and file reads need staging_rows >= 2 (at least two parts)");
+  if (c->transfer_mode == NP_XFER_FILE && c->record_format != NP_REC_BF16)
+    return fail(ctx, NP_E_INVAL, "NP_XFER_FILE needs NP_REC_BF16 records");
+  if (c->io_depth < -1 || c->io_depth > 4096) return fail(ctx, NP_E_INVAL, "io_depth must be in [-1, 4096]");
   if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
@@ -354,6 +361,7 @@ int np_plan_dense_prefix(const np_config* cfg, uint64_t budget_bytes, uint64_t f
 int np_destroy(np_ctx* ctx) {
   if (!ctx) return NP_OK;
   cudaDeviceSynchronize();
+  ctx->reader.close();  // nothing may be in flight when the pool and the buffers go
   delete ctx->pool;
   if (ctx->slab) cudaFree(ctx->slab);
   if (ctx->ev_delta) cudaEventDestroy(ctx->ev_delta);
@@ -384,10 +392,21 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   if (!b) return fail(nullptr, NP_E_INVAL, "buffers is NULL");
   const bool need_staging = cfg->transfer_mode != NP_XFER_ZERO_COPY;
   const bool any_sparse = cfg->dense_layers < cfg->n_layers;
-  if (!b->w1 || !b->w2 || !b->backing || !b->workspace || !b->host_lists ||
+  const bool from_file = cfg->transfer_mode == NP_XFER_FILE;
+  if (!b->w1 || !b->w2 || (!b->backing && !from_file) || !b->workspace || !b->host_lists ||
       (any_sparse && (!b->gate_buf || !b->up_buf || !b->downT_buf)) || (need_staging && !b->staging) ||
-      (cfg->transfer_mode == NP_XFER_HOST_GATHER && !b->host_staging) || (cfg->dense_layers > 0 && !b->dense_buf))
+      ((cfg->transfer_mode == NP_XFER_HOST_GATHER || from_file) && !b->host_staging) ||
+      (cfg->dense_layers > 0 && !b->dense_buf))
     return fail(nullptr, NP_E_INVAL, "a required buffer pointer is NULL");
+  if (from_file) {
+    struct stat st;
+    if (b->backing_fd < 0 || fstat(b->backing_fd, &st) != 0)
+      return fail(nullptr, NP_E_INVAL, "backing_fd is not an open file");
+    const uint64_t need = (uint64_t)cfg->n_layers * cfg->d_ffn * record_bytes_of(*cfg);
+    if (S_ISREG(st.st_mode) && (uint64_t)st.st_size < need)
+      return fail(nullptr, NP_E_INVAL, "the store file holds %llu bytes, the configuration needs %llu",
+                  (unsigned long long)st.st_size, (unsigned long long)need);
+  }
   const void* aligned16[] = {b->w1, b->w2, b->backing, b->gate_buf, b->up_buf, b->downT_buf, b->staging,
                              b->host_staging, b->dense_buf};
   for (const void* p : aligned16)
@@ -436,12 +455,14 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   }
   ctx->host_lists = static_cast<int32_t*>(b->host_lists);
   ctx->host_lists_dev = static_cast<int32_t*>(dev_alias);
-  if (cudaHostGetDevicePointer(&dev_alias, const_cast<void*>(b->backing), 0) != cudaSuccess) {
-    cudaGetLastError();
-    np_destroy(ctx);
-    return fail(nullptr, NP_E_INVAL, "backing store is not pinned, device-mapped host memory");
+  if (!from_file) {
+    if (cudaHostGetDevicePointer(&dev_alias, const_cast<void*>(b->backing), 0) != cudaSuccess) {
+      cudaGetLastError();
+      np_destroy(ctx);
+      return fail(nullptr, NP_E_INVAL, "backing store is not pinned, device-mapped host memory");
+    }
+    ctx->backing_dev = static_cast<const char*>(dev_alias);
   }
-  ctx->backing_dev = static_cast<const char*>(dev_alias);
 
   // library-owned slab: residency tables, lists, scratch
   const size_t LM = (size_t)d.L * d.M, LC = (size_t)d.L * d.C, LW = (size_t)d.L * d.W;
@@ -507,6 +528,28 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   for (auto& e : ctx->ev_t) NP_INIT_CUDA(cudaEventCreate(&e));
   for (auto& e : ctx->ev_c) NP_INIT_CUDA(cudaEventCreate(&e));
 
+  if (cfg->transfer_mode == NP_XFER_HOST_GATHER || from_file) {
+    int n = cfg->host_threads;
+    if (n == 0) {
+      // the packing is what bounds the transfer (steps/s kept rising up to 14 of 16 cores); two
+      // cores stay with the caller's thread and the driver
+      const unsigned hc = std::thread::hardware_concurrency();
+      n = (int)std::max(1u, std::min(16u, hc > 8 ? hc - 2 : hc));
+    }
+    ctx->pool = new (std::nothrow) Pool(n - 1);  // the caller's thread works too
+  }
+  if (from_file) {
+    Pool* pool = ctx->pool;
+    std::string note;
+    ctx->reader.open(b->backing_fd, cfg->io_depth,
+                     [pool](int count, const std::function<void(int)>& fn) {
+                       if (pool) pool->parallel_for(count, fn);
+                       else for (int i = 0; i < count; ++i) fn(i);
+                     },
+                     &note);
+    if (!note.empty()) ctx->err = note;  // readable through np_last_error: why the ring is not in use
+  }
+
   // tensor-core predictor for batches: tensor maps over W2 and the split hidden terms
   ctx->mlp_tc = cfg->max_batch >= kTcMinBatch && !(cfg->flags & (NP_F_NO_TENSOR_CORES | NP_F_DIRECT_LOADS)) &&
                 mlp_tc_supported(d, ctx->sm_count);
@@ -534,6 +577,18 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
         NP_INIT_CUDA(launch_dequant_dense_layer(d, ctx->backing_dev + (size_t)l * d.M * d.rec_bytes, t.identity,
                                                 static_cast<char*>(b->dense_buf) + l * dense_layer_bytes, t.status,
                                                 nullptr, ctx->sm_count));
+    } else if (from_file) {
+      // through the pinned staging, a staging buffer's worth at a time
+      const size_t total = (size_t)d.dense * dense_layer_bytes, step = (size_t)cfg->staging_rows * d.rec_bytes;
+      for (size_t off = 0; off < total; off += step) {
+        const size_t n = std::min(step, total - off);
+        if (!ctx->reader.submit(b->host_staging, n, off, 0) || !ctx->reader.wait_group(0)) {
+          const int e = ctx->reader.last_error();
+          np_destroy(ctx);
+          return fail(nullptr, NP_E_IO, "reading the dense layers from the store file failed: %s", strerror(e));
+        }
+        NP_INIT_CUDA(cudaMemcpy(static_cast<char*>(b->dense_buf) + off, b->host_staging, n, cudaMemcpyHostToDevice));
+      }
     } else {
       NP_INIT_CUDA(cudaMemcpy(b->dense_buf, b->backing, (size_t)d.dense * dense_layer_bytes, cudaMemcpyHostToDevice));
     }
@@ -542,16 +597,6 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   NP_INIT_CUDA(cudaDeviceSynchronize());
 #undef NP_INIT_CUDA
 
-  if (cfg->transfer_mode == NP_XFER_HOST_GATHER) {
-    int n = cfg->host_threads;
-    if (n == 0) {
-      // the packing is what bounds the transfer (steps/s kept rising up to 14 of 16 cores); two
-      // cores stay with the caller's thread and the driver
-      const unsigned hc = std::thread::hardware_concurrency();
-      n = (int)std::max(1u, std::min(16u, hc > 8 ? hc - 2 : hc));
-    }
-    ctx->pool = new (std::nothrow) Pool(n - 1);  // the caller's thread works too
-  }
   *out = ctx;
   return NP_OK;
 }
@@ -659,6 +704,113 @@ int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream) {
   return NP_OK;
 }
 
+// NP_XFER_FILE: per chunk of a layer's incoming rows, the ranges of adjacent records are read
+// from the store file into a part of the pinned staging, copied to the device and scattered.
+// The reads of the next chunk are queued before the previous chunk is waited for, so the
+// device queue does not drain at chunk boundaries.
+static int install_from_file(np_ctx* ctx, int layer_begin, int layer_end, cudaStream_t cs, int* warn) {
+  const Dims& d = ctx->d;
+  const size_t rec = d.rec_bytes, row_bytes = (size_t)d.D * 2;
+  const int check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+  char* staging = static_cast<char*>(ctx->bufs.staging);
+  char* hstage = static_cast<char*>(ctx->bufs.host_staging);
+  const size_t per_layer = NP_N_COUNTERS + 2 * (size_t)d.C;
+  const int parts = std::min(kStageParts, std::max(2, ctx->cfg.staging_rows / std::max(1, d.k / 4 + 1)));
+  const int part_rows = ctx->cfg.staging_rows / parts;
+  struct Chunk {
+    int l, first, rows, h;
+    bool last;
+  };
+  std::deque<Chunk> queued;  // reads queued, copy not yet issued
+  auto finish = [&](const Chunk& c) -> int {
+    if (!ctx->reader.wait_group(c.h)) {
+      const int e = ctx->reader.last_error();
+      ctx->reader.drain();
+      return fail(ctx, NP_E_IO, "layer %d: reading the store file failed: %s", c.l, strerror(e));
+    }
+    char* hbuf = hstage + (size_t)c.h * part_rows * rec;
+    char* dbuf = staging + (size_t)c.h * part_rows * rec;
+    NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)c.rows * rec, cudaMemcpyHostToDevice, cs));
+    NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[c.h], cs));
+    NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[c.h], 0));
+    NP_LAUNCH(ctx, launch_scatter(d, dbuf, false, nullptr, ctx->t.delta_slots + (size_t)c.l * d.C,
+                                ctx->t.counters + (size_t)c.l * NP_N_COUNTERS + NP_CNT_DELTA, c.first, c.rows,
+                                static_cast<char*>(ctx->bufs.gate_buf) + (size_t)(c.l - d.dense) * d.C * row_bytes,
+                                static_cast<char*>(ctx->bufs.up_buf) + (size_t)(c.l - d.dense) * d.C * row_bytes,
+                                static_cast<char*>(ctx->bufs.downT_buf) + (size_t)(c.l - d.dense) * d.C * row_bytes,
+                                ctx->t.status, check, ctx->aux[0], ctx->sm_count));
+    NP_CUDA(ctx, cudaEventRecord(ctx->ev_half[c.h], ctx->aux[0]));  // both copies of the part are free again
+    ctx->half_pending[c.h] = true;
+    if (c.last) {
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[c.l], ctx->aux[0]));
+      ctx->install_pending[c.l] = 1;
+    }
+    return NP_OK;
+  };
+  auto give_up = [&](int rc) {
+    ctx->reader.drain();
+    return rc;
+  };
+  for (int l = layer_begin; l < layer_end; ++l) {
+    const int32_t* cnt = ctx->host_lists + kHostHeaderInts + (size_t)l * per_layer;
+    const int32_t* ids = cnt + NP_N_COUNTERS;
+    const int n = cnt[NP_CNT_DELTA];
+    if (n < 0 || n > d.C) return give_up(fail(ctx, NP_E_DEVICE, "layer %d: delta count %d outside [0, %d]", l, n, d.C));
+    if (cnt[NP_CNT_OVERFLOW] > 0) *warn = NP_W_OVERFLOW;
+    if (n > part_rows && *warn == NP_OK) *warn = NP_W_CHUNKED;
+    if (n == 0) {  // nothing to read: the layer is installed once the earlier chunks are
+      while (!queued.empty()) {
+        const int rc = finish(queued.front());
+        queued.pop_front();
+        if (rc < 0) return give_up(rc);
+      }
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], ctx->aux[0]));
+      ctx->install_pending[l] = 1;
+      continue;
+    }
+    for (int first = 0; first < n; first += part_rows) {
+      const int rows = std::min(part_rows, n - first);
+      const int h = ctx->next_half % parts;
+      ctx->next_half = (h + 1) % parts;
+      // a part is taken again only after its earlier chunk has been copied and scattered
+      while (!queued.empty() && ((int)queued.size() >= parts - 1 || queued.front().h == h)) {
+        const int rc = finish(queued.front());
+        queued.pop_front();
+        if (rc < 0) return give_up(rc);
+      }
+      if (ctx->half_pending[h]) {
+        NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_half[h]));
+        ctx->half_pending[h] = false;
+      }
+      char* hbuf = hstage + (size_t)h * part_rows * rec;
+      // ascending IDs: adjacent IDs are adjacent records of the file -> one range per run
+      int r = 0;
+      while (r < rows) {
+        int len = 1;
+        while (r + len < rows && ids[first + r + len] == ids[first + r] + len) ++len;
+        const int id = ids[first + r];
+        if (id < 0 || id + len > d.M) return give_up(fail(ctx, NP_E_DEVICE, "layer %d: neuron id %d out of range", l, id));
+        if (!ctx->reader.submit(hbuf + (size_t)r * rec, (size_t)len * rec, ((uint64_t)l * d.M + (uint64_t)id) * rec, h))
+          return give_up(fail(ctx, NP_E_IO, "layer %d: queueing a read failed: %s", l, strerror(ctx->reader.last_error())));
+        r += len;
+      }
+      queued.push_back(Chunk{l, first, rows, h, first + rows >= n});
+      // keep one chunk's reads queued behind the one that is waited for
+      while (queued.size() > 1) {
+        const int rc = finish(queued.front());
+        queued.pop_front();
+        if (rc < 0) return give_up(rc);
+      }
+    }
+  }
+  while (!queued.empty()) {
+    const int rc = finish(queued.front());
+    queued.pop_front();
+    if (rc < 0) return give_up(rc);
+  }
+  return NP_OK;
+}
+
 int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_stream) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   const Dims& d = ctx->d;
@@ -713,6 +865,12 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
 
   // the host plans the copies: wait until the delta lists are readable
   NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_delta));
+  if (mode == NP_XFER_FILE) {
+    const int rc = install_from_file(ctx, layer_begin, layer_end, cs, &warn);
+    if (rc < 0) return rc;
+    NP_CUDA(ctx, join());
+    return warn;
+  }
   const char* store = static_cast<const char*>(ctx->bufs.backing);
   char* staging = static_cast<char*>(ctx->bufs.staging);
   const size_t per_layer = NP_N_COUNTERS + 2 * (size_t)d.C;
@@ -1125,6 +1283,34 @@ int np_import_state(np_ctx* ctx, int32_t layer, const int32_t* slot_map, const i
   NP_CUDA(ctx, cudaMemcpyAsync(ctx->t.stamp + (size_t)layer * d.M, stamp, (size_t)d.M * 4, cudaMemcpyHostToDevice, s));
   NP_CUDA(ctx, cudaStreamSynchronize(s));
   ctx->step = step;
+  return NP_OK;
+}
+
+int np_read_records(int32_t fd, uint64_t base_offset, uint64_t rec_bytes, const int32_t* ids, int32_t n, void* dst,
+                    int32_t io_depth, int32_t* n_ranges_out, int32_t* used_ring_out) {
+  if (fd < 0 || !rec_bytes || n < 0 || (n > 0 && (!ids || !dst)))
+    return fail(nullptr, NP_E_INVAL, "np_read_records: bad descriptor, record size, count or NULL pointer");
+  if (io_depth < -1 || io_depth > 4096) return fail(nullptr, NP_E_INVAL, "io_depth must be in [-1, 4096]");
+  for (int i = 0; i < n; ++i)
+    if (ids[i] < 0 || (i > 0 && ids[i] <= ids[i - 1]))
+      return fail(nullptr, NP_E_INVAL, "np_read_records: ids must be non-negative and strictly ascending");
+  RecordReader reader;
+  std::string note;
+  if (!reader.open(fd, io_depth, nullptr, &note)) return fail(nullptr, NP_E_IO, "np_read_records: cannot use the descriptor");
+  int ranges = 0, r = 0;
+  bool ok = true;
+  while (r < n && ok) {
+    int len = 1;
+    while (r + len < n && ids[r + len] == ids[r] + len) ++len;
+    ok = reader.submit(static_cast<char*>(dst) + (size_t)r * rec_bytes, (size_t)len * rec_bytes,
+                       base_offset + (uint64_t)ids[r] * rec_bytes, ranges % RecordReader::kGroups);
+    ++ranges;
+    r += len;
+  }
+  ok = reader.drain() && ok;
+  if (n_ranges_out) *n_ranges_out = ranges;
+  if (used_ring_out) *used_ring_out = reader.uses_ring() ? 1 : 0;
+  if (!ok) return fail(nullptr, NP_E_IO, "np_read_records: a read failed: %s", strerror(reader.last_error()));
   return NP_OK;
 }
 

@@ -28,7 +28,7 @@ class Pair:
     def __init__(self, cfg: synth.StackConfig, policy=nb.NP_EVICT_EXACT, max_batch=1, k=None, C=None,
                  transfer_mode=nb.NP_XFER_MEMCPY_RUNS, staging_rows=None, flags=nb.NP_F_CHECK_BOUNDS,
                  gen_device="cpu", with_oracle=True, chain_layers=0, ring_stages=0, dense_layers=0,
-                 record_format=nb.NP_REC_BF16):
+                 record_format=nb.NP_REC_BF16, store_dir=None, io_depth=0, direct=True):
         nbuild.build()
         self.cfg = cfg
         self.k = cfg.top_k if k is None else k
@@ -39,14 +39,20 @@ class Pair:
         ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, self.k, self.C,
                               max_batch=max_batch, evict_policy=policy, staging_rows=staging_rows,
                               transfer_mode=transfer_mode, flags=flags, chain_layers=chain_layers, ring_stages=ring_stages,
-                              dense_layers=dense_layers, record_format=record_format)
+                              dense_layers=dense_layers, record_format=record_format, io_depth=io_depth)
         self.dense_layers = dense_layers
         if record_format == nb.NP_REC_INT8:
             # the store the library reads is the 8-bit one; the oracle works on what those
             # records mean (its own dequantisation)
             self.backing_q = synth.quantize_store(self.backing)
             self.backing = self.backing_q
-        self.eng = nb.Engine(ncfg, w1.cuda(), w2.cuda(), self.backing)
+        if transfer_mode == nb.NP_XFER_FILE:
+            # the library sees the store only as a file; the oracle keeps the bytes in memory
+            path = str(store_dir / "store.bin")
+            self.backing.view(torch.int16).numpy().tofile(path)
+            self.eng = nb.Engine(ncfg, w1.cuda(), w2.cuda(), None, store_path=path, direct=direct)
+        else:
+            self.eng = nb.Engine(ncfg, w1.cuda(), w2.cuda(), self.backing)
         if record_format == nb.NP_REC_INT8:
             self.store_u16 = O.dequantize_records(self.backing_q.numpy(), cfg.d_model)
         else:

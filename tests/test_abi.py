@@ -30,13 +30,13 @@ def test_every_declared_symbol_is_exported(lib):
     for n in names:
         assert hasattr(lib, n), n
     assert sorted(nb.EXPORTED) == names
-    assert nb.np_version() == 2
+    assert nb.np_version() == 3
 
 
 def test_struct_sizes_match_header():
-    assert C.sizeof(nb.np_config) == 16 * 4
+    assert C.sizeof(nb.np_config) == 18 * 4
     assert C.sizeof(nb.np_sizes) == 11 * 8
-    assert C.sizeof(nb.np_buffers) == 11 * C.sizeof(C.c_void_p)
+    assert C.sizeof(nb.np_buffers) == 11 * C.sizeof(C.c_void_p) + 8
     assert C.sizeof(nb.np_delta_view) == 7 * C.sizeof(C.c_void_p)
 
 
@@ -74,7 +74,7 @@ def test_dense_prefix_plan_matches_the_oracle(lib):
 @pytest.mark.parametrize("field,value", [
     ("n_layers", 0), ("d_model", 100), ("d_ffn", 1000), ("d_pred", 7), ("top_k", 9999), ("capacity", 0),
     ("capacity", 99999), ("max_batch", 17), ("evict_policy", 5), ("transfer_mode", 9), ("staging_rows", 0),
-    ("flags", 64), ("dense_layers", -1), ("dense_layers", 3),
+    ("flags", 64), ("dense_layers", -1), ("dense_layers", 3), ("io_depth", -2), ("io_depth", 5000),
 ])
 def test_bad_config_is_rejected(lib, field, value):
     cfg = nb.make_config(2, 256, 1024, 64, 102, 205)
@@ -83,6 +83,19 @@ def test_bad_config_is_rejected(lib, field, value):
         nb.np_query_sizes(cfg)
     assert e.value.code == nb.NP_E_INVAL
     assert nb.np_last_error(None)
+
+
+def test_file_mode_config_rules(lib):
+    cfg = nb.make_config(2, 256, 1024, 64, 102, 205, transfer_mode=nb.NP_XFER_FILE, io_depth=256)
+    assert nb.np_query_sizes(cfg).record_bytes == 1536
+    cfg.record_format = nb.NP_REC_INT8               # records of 3*D + 16 bytes do not suit direct reads
+    with pytest.raises(nb.NpError) as e:
+        nb.np_query_sizes(cfg)
+    assert e.value.code == nb.NP_E_INVAL
+    cfg.record_format = nb.NP_REC_BF16
+    cfg.staging_rows = 1
+    with pytest.raises(nb.NpError):
+        nb.np_query_sizes(cfg)
 
 
 def test_null_arguments_are_rejected(lib):
