@@ -48,7 +48,11 @@ def parse_args():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--config", default="7b", choices=sorted(synth.CONFIGS))
     ap.add_argument("--policy", default="exact", choices=["exact", "lru"])
-    ap.add_argument("--transfer", default="gather", choices=["runs", "gather", "zerocopy"])
+    ap.add_argument("--transfer", default="gather", choices=["runs", "gather", "zerocopy", "file"],
+                    help="file: the record store is a file, read through io_uring with O_DIRECT (Section 3.5)")
+    ap.add_argument("--store-path", default=None, help="--transfer file: where the store file is written (default: a temp file)")
+    ap.add_argument("--io-depth", type=int, default=0, help="--transfer file: reads in flight (0 = 256; -1 = blocking preads)")
+    ap.add_argument("--buffered", action="store_true", help="--transfer file: open the store without O_DIRECT")
     ap.add_argument("--rho", type=float, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-steps", type=int, default=3)
@@ -292,7 +296,9 @@ def cuda_arm(args):
         raise SystemExit("bench.py: --warmup must be >= 3")
     policy = nb.NP_EVICT_LRU if args.policy == "lru" else nb.NP_EVICT_EXACT
     mode = {"runs": nb.NP_XFER_MEMCPY_RUNS, "gather": nb.NP_XFER_HOST_GATHER,
-            "zerocopy": nb.NP_XFER_ZERO_COPY}[args.transfer]
+            "zerocopy": nb.NP_XFER_ZERO_COPY, "file": nb.NP_XFER_FILE}[args.transfer]
+    if args.transfer == "file" and args.records != "bf16":
+        raise SystemExit("bench.py: --transfer file reads bf16 records")
 
     if args.budget_gib is not None:
         plan_cfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity)
@@ -310,10 +316,38 @@ def cuda_arm(args):
                           record_format=nb.NP_REC_INT8 if args.records == "int8" else nb.NP_REC_BF16,
                           max_batch=args.batch, evict_policy=policy, transfer_mode=mode,
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
-                          host_threads=args.host_threads, dense_layers=args.dense_layers,
+                          host_threads=args.host_threads, dense_layers=args.dense_layers, io_depth=args.io_depth,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0))
-    eng = nb.Engine(ncfg, w1, w2, store, device=dev)
+    storage = None
+    if args.transfer == "file":
+        # the store goes to a file and leaves host memory; the library sees only the descriptor
+        import tempfile
+        store_path = args.store_path or os.path.join(tempfile.gettempdir(), f"np_store_{cfg.name}_{os.getpid()}.bin")
+        t0 = time.time()
+        store.view(torch.int16).numpy().tofile(store_path)
+        fd = os.open(store_path, os.O_RDONLY)
+        os.fsync(fd)
+        os.posix_fadvise(fd, 0, 0, os.POSIX_FADV_DONTNEED)       # reads come from the device, not the page cache
+        os.close(fd)
+        write_s = time.time() - t0
+        store_bytes = store.numel() * 2
+        nb.unpin_host_tensor(store)
+        store = None
+        eng = nb.Engine(ncfg, w1, w2, None, device=dev, store_path=store_path, direct=not args.buffered)
+        # the file's own ceiling: one contiguous range of up to 2 GiB through the same reader
+        probe_recs = int(min(store_bytes, 2 << 30) // cfg.record_bytes)
+        probe = np.empty(probe_recs * cfg.record_bytes + 4096, dtype=np.uint8)
+        probe = probe[(-probe.ctypes.data) % 4096:][:probe_recs * cfg.record_bytes]
+        t0 = time.time()
+        _, used_ring = nb.np_read_records(eng.store_fd, 0, cfg.record_bytes, np.arange(probe_recs), probe, args.io_depth)
+        seq_s = time.time() - t0
+        del probe
+        storage = {"path": store_path, "file_bytes": int(store_bytes), "write_s": write_s, "direct_io": eng.direct_io,
+                   "io_uring": bool(used_ring), "io_depth": args.io_depth if args.io_depth else 256,
+                   "sequential_read_gbs": probe_recs * cfg.record_bytes / seq_s / 1e9}
+    else:
+        eng = nb.Engine(ncfg, w1, w2, store, device=dev)
     L, D, M = cfg.n_layers, cfg.d_model, cfg.d_ffn
     rec = cfg.record_bytes                             # resident (bf16) bytes of a record
     rec_store = 3 * D + 16 if args.records == "int8" else rec   # bytes of a record in the store
@@ -491,6 +525,10 @@ def cuda_arm(args):
                       "mlp_chain_alone": mlp_us * n_launch},
         "setup_s": {"generate": gen_s},
     }
+    if storage is not None:
+        # bytes the step reads from the file over the time the install takes on the copy stream
+        storage["read_gbs_during_install"] = mean_delta * (L - nd) * rec / (float(stage_us[2]) * 1e-6) / 1e9
+        result["storage"] = storage
 
     # ---- the same step with the other pinned-host transfer mode (reported beside, not as, the value) ----
     if (args.transfer == "gather" and not args.no_variants and not centroid and Bq == 1
@@ -518,7 +556,7 @@ def cuda_arm(args):
             "note": "scatter kernel reads the pinned store over PCIe by neuron ID; no host packing, no staging copy"}}
 
     if (rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid and not args.dense_layers
-            and args.records == "bf16"):
+            and args.records == "bf16" and store is not None):
         n = args.cpu_baseline_steps
         times = run_oracle_steps(cfg, args.policy, w1.cpu(), w2.cpu(), store, xs_host, n)
         sec = float(np.mean(times))
@@ -528,6 +566,8 @@ def cuda_arm(args):
     elif rank == 0:
         result["cpu_baseline"] = None
     eng.close()
+    if storage is not None and not args.store_path:
+        os.remove(storage["path"])
     if rank == 0:
         print(json.dumps(result))
     finish_replicas(dist)
