@@ -562,7 +562,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   if (d.dense > 0) {
     Dims dd = d;
     dd.k = dd.C = d.M;
-    if (!chain_alu::supported(dd, ctx->sm_count) || (d.dense < d.L && !mlp_chain_supported(d, ctx->sm_count))) {
+    if ((!dense_chain::supported(d, ctx->sm_count) && !chain_alu::supported(dd, ctx->sm_count)) || (d.dense < d.L && !mlp_chain_supported(d, ctx->sm_count))) {
       np_destroy(ctx);
       return fail(nullptr, NP_E_INVAL, "dense_layers > 0: this shape is outside what the resident MLP kernels cover");
     }
@@ -1072,7 +1072,11 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       for (int l0 = 0; l0 < d.dense; l0 += kDenseRun) {
         a.l_begin = l0;
         a.l_end = std::min(d.dense, l0 + kDenseRun);
-        NP_LAUNCH(ctx, chain_alu::launch(d, a, s, ctx->sm_count));
+        if (dense_chain::supported(d, ctx->sm_count))
+          NP_LAUNCH(ctx, dense_chain::launch(d, dense, d.M, a.xbuf, a.zbuf, a.grid_bar, a.status, a.l_begin, a.l_end, s,
+                                             ctx->sm_count));
+        else
+          NP_LAUNCH(ctx, chain_alu::launch(d, a, s, ctx->sm_count));
       }
     }
     // the sparse layers' buffers start at layer d; the kernels index them by absolute layer

@@ -156,6 +156,11 @@ struct ChainArgs {
 bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p);
 bool mlp_chain_supported(const Dims& d, int sm_count);
 cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
+namespace dense_chain {  // dense layers, direct loads (np_mlp_dense.cu); same hand-over of x as the other forms
+bool supported(const Dims& d, int sm_count);
+cudaError_t launch(const Dims& d, const void* rec0, int rows, float* const xbuf[2], float* const zbuf[3],
+                   unsigned int* grid_bar, int32_t* status, int l_begin, int l_end, cudaStream_t s, int sm_count);
+}  // namespace dense_chain
 namespace chain_alu {  // ALU form of phase 1, for shares that do not fit the ring as one tile (np_mlp_chain_alu.cu)
 bool supported(const Dims& d, int sm_count);
 cudaError_t launch(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
