@@ -1065,13 +1065,16 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       a.downT = dense + 2 * row_bytes;
       a.active_slots = ctx->t.identity;
       a.dense_rows = d.M;
-      // Short runs: while a resident launch is on the device the install's scatter kernels do
-      // not run beside it, so the installs of the sparse layers advance between runs
-      // (measured at the 7B shape, d = 24: 612 steps/s with runs of 3, 448 with one run).
-      constexpr int kDenseRun = 3;
-      for (int l0 = 0; l0 < d.dense; l0 += kDenseRun) {
+      // Runs, not one launch: while a resident launch is on the device the install's scatter
+      // kernels do not run beside it (its blocks hold the register file), so the installs of the
+      // sparse layers advance between runs.  The fewer sparse layers wait for rows, the longer a
+      // run may be (measured at the 7B shape: d = 20: 697 steps/s with runs of 3, 648 with 6;
+      // d = 24: 711 / 755 / 702 / 594 with runs of 3 / 6 / 8 / 24; d = 28: 682 / 710 / 725 with
+      // 3 / 6 / 12).
+      const int dense_run = d.dense < d.L ? std::max(3, std::min(12, 2 * d.dense / (d.L - d.dense))) : 12;
+      for (int l0 = 0; l0 < d.dense; l0 += dense_run) {
         a.l_begin = l0;
-        a.l_end = std::min(d.dense, l0 + kDenseRun);
+        a.l_end = std::min(d.dense, l0 + dense_run);
         if (dense_chain::supported(d, ctx->sm_count))
           NP_LAUNCH(ctx, dense_chain::launch(d, dense, d.M, a.xbuf, a.zbuf, a.grid_bar, a.status, a.l_begin, a.l_end, s,
                                              ctx->sm_count));
