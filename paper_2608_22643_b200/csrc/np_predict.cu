@@ -299,12 +299,118 @@ static cudaError_t l2_dispatch_nb(const uint4* w2, const float* hidden, float* l
 #undef NP_L2_LAUNCH
 }
 
+// ---------------------------------------------------------------------------
+// Layer 2 for one sequence, without the ring: LPR lanes share a row, each lane
+// keeps its CPL 16-byte chunks of `hidden` in registers for the whole kernel
+// and loads its chunks of RIF rows straight from global memory into registers
+// before it uses any (16 loads in flight per lane at H = 512); a shuffle
+// reduction per row, no shared memory, no barrier.  The hand-over per ring
+// stage (mbarrier polls, one stage at a time per warp) held the ring kernel at
+// 0.65 of the copy bandwidth; this one streams like a copy.
+// The first loads go out before the wait for layer 1: the weights do not depend
+// on it, `hidden` does.
+// ---------------------------------------------------------------------------
+constexpr int kL2dWarps = 16;
+constexpr int kL2dThreads = kL2dWarps * 32;
+
+template <int LPR, int CPL>
+__global__ void __launch_bounds__(kL2dThreads, 1) k_pred_l2_direct(const uint4* __restrict__ w2,
+                                                                   const float* hidden,  // [H]; written by the previous kernel
+                                                                   float* __restrict__ logits, long long rows, int H) {
+  constexpr int RPW = 32 / LPR;                           // rows a warp works on side by side
+  constexpr int RIF = CPL >= 16 ? 1 : (CPL >= 8 ? 2 : (CPL >= 4 ? 4 : 8));  // rows in flight per lane
+  constexpr int kGroup = RPW * RIF;                       // rows per warp and iteration
+  const int chunks = H >> 3;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int sub = lane % LPR, rsel = lane / LPR;
+  const long long r_begin = rows * blockIdx.x / gridDim.x;
+  const long long r_end = rows * (blockIdx.x + 1) / gridDim.x;
+  uint4 w[RIF][CPL];
+  // every load is issued, unconditionally: indices past the end are clamped, their results dropped
+  auto load = [&](long long base) {
+#pragma unroll
+    for (int u = 0; u < RIF; ++u) {
+      const long long r = min(base + u * RPW + rsel, r_end - 1);
+      const uint4* row = w2 + (size_t)r * chunks;
+#pragma unroll
+      for (int i = 0; i < CPL; ++i) w[u][i] = ldg_stream(row + min(sub + i * LPR, chunks - 1));
+    }
+  };
+  long long base = r_begin + (long long)wid * kGroup;
+  if (base < r_end) load(base);
+  npp::pdl_wait_prior();
+  float hreg[CPL * 8];
+#pragma unroll
+  for (int i = 0; i < CPL; ++i) {
+    const int c = sub + i * LPR;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) hreg[i * 8 + e] = c < chunks ? hidden[c * 8 + e] : 0.f;
+  }
+  while (base < r_end) {
+    float acc[RIF];
+#pragma unroll
+    for (int u = 0; u < RIF; ++u) {
+      acc[u] = 0.f;
+#pragma unroll
+      for (int i = 0; i < CPL; ++i) {
+        const float4 ha = make_float4(hreg[i * 8 + 0], hreg[i * 8 + 1], hreg[i * 8 + 2], hreg[i * 8 + 3]);
+        const float4 hb = make_float4(hreg[i * 8 + 4], hreg[i * 8 + 5], hreg[i * 8 + 6], hreg[i * 8 + 7]);
+        acc[u] = dot8(w[u][i], ha, hb, acc[u]);  // chunks past the row's end meet zeros of `hidden`
+      }
+    }
+    // the sums are complete before the registers of w are loaded again (the compiler would
+    // otherwise keep both generations of w alive, and spill)
+#pragma unroll
+    for (int u = 0; u < RIF; ++u) asm volatile("" : "+f"(acc[u]));
+    const long long cur = base;
+    base += (long long)kL2dWarps * kGroup;
+    if (base < r_end) load(base);  // the next rows are on their way while these are reduced and stored
+#pragma unroll
+    for (int u = 0; u < RIF; ++u) {
+      float v = acc[u];
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      const long long r = cur + u * RPW + rsel;
+      if (sub == 0 && r < r_end) logits[r] = v;
+    }
+  }
+}
+
+template <int LPR, int CPL>
+static cudaError_t l2_direct_launch(const uint4* w2, const float* hidden, float* logits, long long rows, int H,
+                                    int blocks, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(kL2dThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_pred_l2_direct<LPR, CPL>, w2, hidden, logits, rows, H);
+}
+
 cudaError_t launch_pred_l2(const Dims& d, const void* w2v, const float* hidden, int B, float* logits,
                            int32_t* status, cudaStream_t s, int sm_count) {
   const uint4* w2 = static_cast<const uint4*>(w2v);
   const long long rows = (long long)d.L * d.M;
   const int chunks = d.H >> 3;
   const int blocks = sm_count;
+  if (B == 1 && rows > 0) {
+#define NP_L2D(LPR, CPL) return l2_direct_launch<LPR, CPL>(w2, hidden, logits, rows, d.H, blocks, s)
+    if (chunks <= 1) NP_L2D(1, 1);
+    if (chunks <= 2) NP_L2D(2, 1);
+    if (chunks <= 4) NP_L2D(4, 1);
+    if (chunks <= 8) NP_L2D(8, 1);
+    if (chunks <= 16) NP_L2D(16, 1);
+    if (chunks <= 32) NP_L2D(16, 2);
+    if (chunks <= 64) NP_L2D(16, 4);
+    if (chunks <= 128) NP_L2D(32, 4);
+    // wider hidden vectors do not fit a lane's registers beside its loads: the ring kernel below
+#undef NP_L2D
+  }
 #define NP_L2(LPR, CPL) return l2_dispatch_nb<LPR, CPL>(w2, hidden, logits, rows, d.H, B, blocks, status, s)
   if (chunks <= 1) NP_L2(1, 1);
   if (chunks <= 2) NP_L2(2, 1);
