@@ -416,7 +416,9 @@ def cuda_arm(args):
         delta_rows.append(float(c[nd:, nb.NP_CNT_DELTA].mean()) if nd < L else 0.0)
         overflow_steps += int((c[:, nb.NP_CNT_OVERFLOW] > 0).any())
         overlap.append(float((c[nd:, nb.NP_CNT_KEPT] / np.maximum(1, c[nd:, nb.NP_CNT_PRED])).mean()) if nd < L else 1.0)
-    stage_us = np.median(np.stack(stage_us), axis=0)
+    stage_all = np.stack(stage_us)
+    step_each = stage_all[:, 0] + stage_all[:, 1] + stage_all[:, 3]   # predict + delta + chain (which waits for the installs)
+    stage_us = np.median(stage_all, axis=0)
     n_active = float(eng.counters()[nd:, nb.NP_CNT_ACTIVE].mean()) if nd < L else 0.0
 
     # ---- end-to-end timing: hidden state from pinned host, result back to the host --------
@@ -525,6 +527,13 @@ def cuda_arm(args):
                       "mlp_chain_alone": mlp_us * n_launch},
         "setup_s": {"generate": gen_s},
     }
+    if not centroid:
+        # spread over the detail steps, and the step without any transfer (context: what the GPU work alone takes)
+        result["step_us"] = {"p10": fnum(np.percentile(step_each, 10)), "median": fnum(np.median(step_each)),
+                             "p90": fnum(np.percentile(step_each, 90)), "steps": int(n_detail)}
+        compute_us = pred_us + float(stage_us[1]) + mlp_us * n_launch
+        result["compute_only"] = {"us": compute_us, "steps_per_s": 1e6 / compute_us,
+                                  "note": "predict + delta + MLP chain timed alone, rows already resident: no install"}
     if storage is not None:
         # bytes the step reads from the file over the time the install takes on the copy stream
         storage["read_gbs_during_install"] = mean_delta * (L - nd) * rec / (float(stage_us[2]) * 1e-6) / 1e9
