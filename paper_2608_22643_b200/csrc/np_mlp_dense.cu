@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_dense_chain(KArgs a) {
   // phase B: cpt threads span the row's column pieces (COLS pieces each), RG such groups share the rows
   const int cpt = min(kThreads, (chunks + COLS - 1) / COLS), RG = kThreads / cpt;
   const int rg = tid / cpt, pc = tid - rg * cpt;
+  const bool in_b = rg < RG;  // cpt need not divide the block: the threads left over sit phase B out
   if (tid == 0) s_ok = 1;
   __syncthreads();
 
@@ -193,7 +194,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_dense_chain(KArgs a) {
     for (int j = 0; j < COLS; ++j)
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[j][e] = 0.f;
-    for (int r0 = rg; r0 < nr; r0 += RG * kRowsB) {
+    for (int r0 = rg; in_b && r0 < nr; r0 += RG * kRowsB) {
       // unconditional loads again: a row past the share's end re-reads the last row with weight 0
       uint4 w[COLS][kRowsB];
 #pragma unroll
@@ -227,7 +228,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_dense_chain(KArgs a) {
       }
     }
     // the row groups meet in shared memory: group rg > 0 leaves its vector in ys[rg - 1]
-    if (rg > 0) {
+    if (rg > 0 && in_b) {
 #pragma unroll
       for (int j = 0; j < COLS; ++j) {
         const int c = pc + j * cpt;

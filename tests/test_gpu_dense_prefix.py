@@ -55,6 +55,41 @@ def test_trajectory_with_dense_prefix(cfg, d, mode):
         p.close()
 
 
+# row widths of the larger configurations (two 16-byte column pieces per thread of the dense-layer
+# kernel, uneven splits of the row over the warps), on few rows; the 8192-wide one also has a
+# predictor wider than the direct-load kernel's registers hold
+WIDE13 = synth.StackConfig("wide13", 2, 5120, 1024, 640, 10, 25, 3, 21, 0.9)
+WIDE70 = synth.StackConfig("wide70", 2, 8192, 512, 2048, 10, 25, 3, 22, 0.9)
+ODDW = synth.StackConfig("oddw", 3, 2064, 608, 72, 10, 25, 3, 23, 0.9)    # D / 8 = 258 pieces
+
+
+@pytest.mark.parametrize("cfg,d", [(WIDE13, 1), (WIDE13, 2), (WIDE70, 1), (ODDW, 2), (ODDW, 3)])
+def test_dense_layers_at_other_row_widths(cfg, d):
+    p = Pair(cfg, transfer_mode=nb.NP_XFER_HOST_GATHER, dense_layers=d)
+    try:
+        L, M = cfg.n_layers, cfg.d_ffn
+        xs = synth.hidden_states(cfg, 3)
+        logits = torch.zeros((1, L, M), dtype=torch.float32, device="cuda")
+        out = torch.empty((1, cfg.d_model), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, x, 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            z = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M).astype(np.float32)
+            z32 = logits.cpu().numpy()
+            if d < L:
+                assert rel_l2(z32[0, d:], z[0, d:]) < 1e-5
+                z[0, d:] = z32[0, d:]
+            res = p.ora.step(u16(xs[t]), logits_f32=z)
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+        p.check_resident_bytes()
+        p.eng.counters()
+    finally:
+        p.close()
+
+
 def test_all_layers_dense():
     cfg = TINY
     p = Pair(cfg, dense_layers=cfg.n_layers)
