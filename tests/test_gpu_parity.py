@@ -321,6 +321,27 @@ def test_export_import_roundtrip_resumes_trajectory():
         b.close()
 
 
+@pytest.mark.parametrize("H", [16, 24, 40, 136, 264, 520, 1024, 1032])
+@pytest.mark.parametrize("L,M", [(1, 32), (2, 96), (3, 1024)])
+def test_predictor_widths_and_row_counts(H, L, M):
+    """Hidden widths on both sides of every lane-layout boundary of the layer-2 kernels, with
+    fewer rows than blocks, a row or two per block, and many."""
+    cfg = synth.StackConfig("pw", L, 64, M, H, 25, 50, 2, 41, 0.9)
+    for B in (1, 2):
+        p = Pair(cfg, max_batch=B, with_oracle=False)
+        try:
+            xs = synth.hidden_states(cfg, 2, batch=B)
+            logits = torch.full((B, L, M), 7.0, dtype=torch.float32, device="cuda")
+            for t in range(2):
+                nb.np_predict(p.eng.ctx, xs[t].cuda(), B, logits, None, p.eng.stream)
+                p.eng.stream.synchronize()
+                z = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)
+                assert rel_l2(logits.cpu().numpy(), z) < 1e-5, (B, t)
+            p.eng.counters()
+        finally:
+            p.close()
+
+
 @pytest.mark.parametrize("shape", [
     # name, L, D, M, H, density %, capacity %
     ("max_ffn", 1, 64, 40960, 8, 10, 20),        # widest FFN the library accepts (top-k keys fill shared memory)
