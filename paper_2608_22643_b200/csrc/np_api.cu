@@ -811,6 +811,124 @@ static int install_from_file(np_ctx* ctx, int layer_begin, int layer_end, cudaSt
   return NP_OK;
 }
 
+// NP_XFER_HOST_GATHER: the pool packs the incoming records into a part of the pinned staging,
+// one cudaMemcpyAsync moves the part, scatter kernels place its rows.  The parts are used round
+// robin: one is packed while earlier ones are copied and scattered (the scatter kernels can fall
+// behind while a resident MLP launch holds the device; spare parts keep the host and the copy
+// engine going).  A part takes the rows of up to kGatherLayers consecutive layers: a copy has a
+// start-up cost, and a steady-state layer fills only a fraction of a part.
+constexpr int kGatherLayers = 2;
+
+static int install_host_gather(np_ctx* ctx, int layer_begin, int layer_end, cudaStream_t cs, int* warn) {
+  const Dims& d = ctx->d;
+  const size_t rec = d.rec_bytes, row_bytes = (size_t)d.D * 2;
+  const int check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
+  const char* store = static_cast<const char*>(ctx->bufs.backing);
+  char* staging = static_cast<char*>(ctx->bufs.staging);
+  char* hstage = static_cast<char*>(ctx->bufs.host_staging);
+  const size_t per_layer = NP_N_COUNTERS + 2 * (size_t)d.C;
+  const int parts = std::min(kStageParts, std::max(2, ctx->cfg.staging_rows / std::max(1, d.k / 4 + 1)));
+  const int part_rows = ctx->cfg.staging_rows / parts;
+  struct Piece {
+    int l, first, rows, at;  // rows [first, first + rows) of layer l's list sit at row `at` of the part
+    bool last;               // the layer is complete with this piece
+  };
+  std::vector<Piece> batch;
+  int h = -1, used = 0, layers_in = 0, last_l = -1;
+  auto open_part = [&]() -> int {
+    h = ctx->next_half % parts;
+    ctx->next_half = (h + 1) % parts;
+    if (ctx->half_pending[h]) {
+      NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_half[h]));
+      ctx->half_pending[h] = false;
+    }
+    used = 0;
+    layers_in = 0;
+    last_l = -1;
+    return NP_OK;
+  };
+  auto flush = [&]() -> int {
+    if (batch.empty()) return NP_OK;
+    char* hbuf = hstage + (size_t)h * part_rows * rec;
+    char* dbuf = staging + (size_t)h * part_rows * rec;
+    if (used > 0) {
+      bool bad = false;
+      const int nthreads = ctx->pool ? ctx->pool->size() + 1 : 1;
+      const int jobs = std::min(used, nthreads * 4);
+      auto body = [&](int job) {
+        const int lo = (int)((long long)used * job / jobs), hi = (int)((long long)used * (job + 1) / jobs);
+        size_t pi = 0;
+        for (int r = lo; r < hi; ++r) {
+          while (r >= batch[pi].at + batch[pi].rows) ++pi;  // pieces are in row order; empty ones are skipped
+          const Piece& pc = batch[pi];
+          const int32_t* ids = ctx->host_lists + kHostHeaderInts + (size_t)pc.l * per_layer + NP_N_COUNTERS;
+          const int id = ids[pc.first + (r - pc.at)];
+          if (id < 0 || id >= d.M) {
+            bad = true;
+            continue;
+          }
+          copy_record_streaming(hbuf + (size_t)r * rec, store + ((size_t)pc.l * d.M + id) * rec, rec);
+        }
+      };
+      if (ctx->pool) ctx->pool->parallel_for(jobs, body);
+      else for (int job = 0; job < jobs; ++job) body(job);
+      if (bad) return fail(ctx, NP_E_DEVICE, "layer %d: neuron id out of range", batch.front().l);
+      // the copies queue back to back on the caller's stream; the scatter kernels follow them
+      // on a side stream, so a copy never waits for the previous part's kernels
+      NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)used * rec, cudaMemcpyHostToDevice, cs));
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[h], cs));
+      NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[h], 0));
+    }
+    for (const Piece& pc : batch) {
+      if (pc.rows > 0)
+        NP_LAUNCH(ctx, launch_scatter(d, dbuf + (size_t)pc.at * rec, false, nullptr, ctx->t.delta_slots + (size_t)pc.l * d.C,
+                                    ctx->t.counters + (size_t)pc.l * NP_N_COUNTERS + NP_CNT_DELTA, pc.first, pc.rows,
+                                    static_cast<char*>(ctx->bufs.gate_buf) + (size_t)(pc.l - d.dense) * d.C * row_bytes,
+                                    static_cast<char*>(ctx->bufs.up_buf) + (size_t)(pc.l - d.dense) * d.C * row_bytes,
+                                    static_cast<char*>(ctx->bufs.downT_buf) + (size_t)(pc.l - d.dense) * d.C * row_bytes,
+                                    ctx->t.status, check, ctx->aux[0], ctx->sm_count));
+      if (pc.last) {
+        NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[pc.l], ctx->aux[0]));
+        ctx->install_pending[pc.l] = 1;
+      }
+    }
+    if (used > 0) {
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_half[h], ctx->aux[0]));  // both copies of the part are free again
+      ctx->half_pending[h] = true;
+    }
+    batch.clear();
+    h = -1;
+    return NP_OK;
+  };
+  for (int l = layer_begin; l < layer_end; ++l) {
+    const int32_t* cnt = ctx->host_lists + kHostHeaderInts + (size_t)l * per_layer;
+    const int n = cnt[NP_CNT_DELTA];
+    if (n < 0 || n > d.C) return fail(ctx, NP_E_DEVICE, "layer %d: delta count %d outside [0, %d]", l, n, d.C);
+    if (cnt[NP_CNT_OVERFLOW] > 0) *warn = NP_W_OVERFLOW;
+    if (n > part_rows && *warn == NP_OK) *warn = NP_W_CHUNKED;
+    int first = 0;
+    do {
+      const int rows = std::min(part_rows, n - first);
+      if (h >= 0 && (used + rows > part_rows || (l != last_l && layers_in >= kGatherLayers))) {
+        const int rc = flush();
+        if (rc < 0) return rc;
+      }
+      if (h < 0) {
+        const int rc = open_part();
+        if (rc < 0) return rc;
+      }
+      if (l != last_l) {
+        ++layers_in;
+        last_l = l;
+      }
+      batch.push_back(Piece{l, first, rows, used, first + rows >= n});
+      used += rows;
+      first += rows;
+    } while (first < n);
+  }
+  return flush();
+}
+
 int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_stream) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   const Dims& d = ctx->d;
@@ -865,8 +983,9 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
 
   // the host plans the copies: wait until the delta lists are readable
   NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_delta));
-  if (mode == NP_XFER_FILE) {
-    const int rc = install_from_file(ctx, layer_begin, layer_end, cs, &warn);
+  if (mode == NP_XFER_FILE || mode == NP_XFER_HOST_GATHER) {
+    const int rc = mode == NP_XFER_FILE ? install_from_file(ctx, layer_begin, layer_end, cs, &warn)
+                                        : install_host_gather(ctx, layer_begin, layer_end, cs, &warn);
     if (rc < 0) return rc;
     NP_CUDA(ctx, join());
     return warn;
@@ -906,54 +1025,6 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
         NP_LAUNCH(ctx, launch_scatter(d, staging, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
                                     down_l, ctx->t.status, check, cs, ctx->sm_count));
       }
-    } else {  // NP_XFER_HOST_GATHER: parts of the pinned staging, packed by the pool
-      // the staging buffers are used in parts, round robin: a part is packed while earlier ones
-      // are copied and scattered (the scatter kernels can fall behind while a resident MLP
-      // launch holds the device; spare parts keep the host and the copy engine going)
-      const int parts = std::min(kStageParts, std::max(2, ctx->cfg.staging_rows / std::max(1, d.k / 4 + 1)));
-      const int half_rows = ctx->cfg.staging_rows / parts;
-      char* hstage = static_cast<char*>(ctx->bufs.host_staging);
-      if (n > half_rows && warn == NP_OK) warn = NP_W_CHUNKED;
-      for (int first = 0; first < n; first += half_rows) {
-        const int rows = std::min(half_rows, n - first);
-        const int h = ctx->next_half % parts;
-        ctx->next_half = (h + 1) % parts;
-        if (ctx->half_pending[h]) {
-          NP_CUDA(ctx, cudaEventSynchronize(ctx->ev_half[h]));
-          ctx->half_pending[h] = false;
-        }
-        char* hbuf = hstage + (size_t)h * half_rows * rec;
-        char* dbuf = staging + (size_t)h * half_rows * rec;
-        bool bad = false;
-        const int nthreads = ctx->pool ? ctx->pool->size() + 1 : 1;
-        const int parts = std::min(rows, nthreads * 4);
-        auto body = [&](int part) {
-          const int lo = (int)((long long)rows * part / parts), hi = (int)((long long)rows * (part + 1) / parts);
-          for (int r = lo; r < hi; ++r) {
-            const int id = ids[first + r];
-            if (id < 0 || id >= d.M) {
-              bad = true;
-              continue;
-            }
-            copy_record_streaming(hbuf + (size_t)r * rec, store_l + (size_t)id * rec, rec);
-          }
-        };
-        if (ctx->pool) ctx->pool->parallel_for(parts, body);
-        else for (int part = 0; part < parts; ++part) body(part);
-        if (bad) return fail(ctx, NP_E_DEVICE, "layer %d: neuron id out of range", l);
-        // the copies queue back to back on the caller's stream; the scatter kernels follow them
-        // on a side stream, so a copy never waits for the previous layer's kernel
-        NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)rows * rec, cudaMemcpyHostToDevice, cs));
-        NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[h], cs));
-        NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[h], 0));
-        NP_LAUNCH(ctx, launch_scatter(d, dbuf, false, nullptr, slots_dev, count_dev, first, rows, gate_l, up_l,
-                                    down_l, ctx->t.status, check, ctx->aux[0], ctx->sm_count));
-        NP_CUDA(ctx, cudaEventRecord(ctx->ev_half[h], ctx->aux[0]));  // both copies of the half are free again
-        ctx->half_pending[h] = true;
-      }
-      NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], ctx->aux[0]));
-      ctx->install_pending[l] = 1;
-      continue;
     }
     NP_CUDA(ctx, cudaEventRecord(ctx->ev_installed[l], cs));
     ctx->install_pending[l] = 1;
