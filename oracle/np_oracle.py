@@ -24,7 +24,11 @@ RMS, scale invariance and a hand value for ``rms_normalize``; a scan, boundary
 budgets and monotonicity for ``dense_prefix_plan``; the dense stack in a
 library's fp64 ops and "a dense layer is a sparse layer with every row active"
 for the dense prefix of ``Engine``; a library's fp32 -> bf16 conversion (with
-constructed ties) and hand values for ``dequantize_records``.
+constructed ties) and hand values for ``dequantize_records``; the paper's
+parameter table for ``trunk_param_counts``, a library's LayerNorm and SiLU for
+``layer_norm`` / ``silu``, a scalar restatement on tiny sizes and structural
+properties (coordinate-copying heads, vanishing second matrices, the centroid
+half of the concatenation) for ``trunk_forward`` (Section 3.3).
 
 Parity unpinned against the paper (the paper is silent; these are this build's
 definitions, pinned only by invariants and determinism): the victim order of
@@ -33,6 +37,11 @@ the LRU policy, the truncation rule when a predicted set exceeds capacity, and
 a throughput sweep on its device, not by a formula), and the 8-bit record
 format of ``dequantize_records`` (the paper names quantised records only as
 future work; the rounding itself is pinned against a library conversion).
+In ``trunk_forward`` the paper leaves open the LayerNorm epsilon (1e-5 here),
+the width of the centroid embedding (2048 reproduces its row of the parameter
+table), the shape of the "small projection network" behind it (one block of
+the same form as the feature blocks) and whether the heads have biases (none
+here; the table's head row is met to 0.14 % either way).
 """
 from __future__ import annotations
 
@@ -210,6 +219,62 @@ def centroid_select(logits_f32: np.ndarray, bank_words: np.ndarray):
                 ids[b, l, h] = int(np.argmax(key))      # first maximum = lowest ID
             words[l] |= bank[l, 0, ids[b, l, 0]] & bank[l, 1, ids[b, l, 1]]
     return ids, words
+
+
+# --------------------------------------------------------------------------
+# the shared predictor of Section 3.3 (features -> projection blocks ->
+# residual trunk -> centroid heads), inference only (no dropout)
+# --------------------------------------------------------------------------
+LN_EPS = 1e-5   # the paper does not state the epsilon of its LayerNorms; the common default is taken
+
+
+def layer_norm(v: np.ndarray, gain: np.ndarray, bias: np.ndarray) -> np.ndarray:
+    """LayerNorm over the last axis: (v - mean) / sqrt(var + eps) * gain + bias, biased variance."""
+    v = np.asarray(v, dtype=np.float64)
+    mu = v.mean(axis=-1, keepdims=True)
+    var = ((v - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (v - mu) / np.sqrt(var + LN_EPS) * gain + bias
+
+
+def silu(v: np.ndarray) -> np.ndarray:
+    v = np.asarray(v, dtype=np.float64)
+    return v / (1.0 + np.exp(-v))
+
+
+def trunk_param_counts(T: int, feature_dims, K: int, E: int, n_blocks: int, n_heads: int) -> dict:
+    """Parameters per component of the Section 3.3 predictor (the rows of the paper's cost table),
+    with a bias on every linear layer but the heads and gain + bias on every LayerNorm."""
+    proj = sum(d * T + T + 2 * T for d in feature_dims)
+    emb = K * E + (E * 4 * T + 4 * T + 2 * 4 * T)
+    trunk = n_blocks * ((8 * T) * (4 * T) + 4 * T + 2 * 4 * T + (4 * T) * (8 * T) + 8 * T)
+    heads = 2 * n_heads * K * (8 * T)
+    return {"input_projections": proj, "centroid_embedding": emb, "residual_trunk": trunk, "output_heads": heads,
+            "total": proj + emb + trunk + heads}
+
+
+def trunk_forward(w: dict, features, centroid_id: int) -> np.ndarray:
+    """Head logits ``[n_heads, 2, K]`` of the Section 3.3 predictor for one token.
+
+    ``features``: the four continuous layer-0 features (vectors of the dims the weights were
+    made for).  Stage 1: every feature goes through its own block Linear -> LayerNorm -> SiLU to
+    T dims; the layer-0 gate centroid ID goes through an embedding and one such block to 4T dims;
+    the five results are concatenated to 8T.  Stage 2: residual blocks
+    z <- z + W2 SiLU(LayerNorm(W1 z + b1)) + b2 with W1: 8T -> 4T, W2: 4T -> 8T.  Stage 3: the
+    gate head and the up head of every sparse layer, linear, K logits each.
+    ``w`` holds fp64 arrays (bf16 values widened by the caller): ``proj[i] = (W, b, gain, bias)``,
+    ``emb`` ``[K0, E]``, ``cproj = (W, b, gain, bias)``, ``blocks[j] = (W1, b1, gain, bias, W2, b2)``,
+    ``heads`` ``[n_heads * 2 * K, 8T]`` (layer-major, gate head before up head), ``K``.
+    """
+    parts = []
+    for (W, b, g, be), f in zip(w["proj"], features):
+        parts.append(silu(layer_norm(W @ np.asarray(f, dtype=np.float64) + b, g, be)))
+    W, b, g, be = w["cproj"]
+    parts.append(silu(layer_norm(W @ w["emb"][centroid_id] + b, g, be)))
+    z = np.concatenate(parts)
+    for (W1, b1, g, be, W2, b2) in w["blocks"]:
+        z = z + W2 @ silu(layer_norm(W1 @ z + b1, g, be)) + b2
+    return (w["heads"] @ z).reshape(-1, 2, w["K"])
+
 
 
 # --------------------------------------------------------------------------

@@ -252,3 +252,57 @@ def quantize_store(store: torch.Tensor, device: str = "cpu", out: Optional[torch
         rec[:, 3 * D:3 * D + 12] = s.contiguous().view(torch.uint8).reshape(M, 12)
         out[l].copy_(rec)
     return out
+
+
+def trunk_weights(T: int, feature_dims, K0: int, E: int, n_blocks: int, n_heads: int, K: int, seed: int,
+                  device: str = "cpu") -> dict:
+    """Random weights of the Section 3.3 predictor (projection blocks, centroid embedding, residual
+    trunk, centroid heads); stands in for the trained predictor, which is not available.
+
+    Matrices are bf16, row-major ``[out][in]``; biases and LayerNorm gains / biases are fp32.  A
+    feature whose dimension is not a multiple of 8 (the scalar norm feature) gets its weight rows
+    padded with zero columns to the next multiple of 8, and is passed padded with zeros: the
+    products are unchanged.  ``feature_dims`` are the true dimensions.
+    """
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed * _SEED_MUL + 777)
+
+    def mat(rows, cols, pad_to=None, scale=None):
+        scale = (1.0 / max(cols, 1)) ** 0.5 if scale is None else scale
+        w = torch.randn(rows, cols, generator=g) * scale
+        if pad_to is not None and pad_to != cols:
+            w = torch.cat([w, torch.zeros(rows, pad_to - cols)], dim=1)
+        return w.to(torch.bfloat16).contiguous().to(device)
+
+    def vec(n, centre=0.0, scale=0.1):
+        return (centre + scale * torch.randn(n, generator=g)).to(torch.float32).contiguous().to(device)
+
+    def block(rows, cols, pad_to=None):
+        return (mat(rows, cols, pad_to), vec(rows), vec(rows, 1.0), vec(rows))
+
+    w = {"T": T, "K": K, "K0": K0, "E": E, "feature_dims": tuple(feature_dims)}
+    w["proj"] = [block(T, d, (d + 7) // 8 * 8) for d in feature_dims]
+    w["emb"] = mat(K0, E, scale=1.0)
+    w["cproj"] = block(4 * T, E)
+    w["blocks"] = []
+    for _ in range(n_blocks):
+        w1, b1, gain, bias = block(4 * T, 8 * T)
+        w["blocks"].append((w1, b1, gain, bias, mat(8 * T, 4 * T), vec(8 * T)))
+    w["heads"] = mat(n_heads * 2 * K, 8 * T)
+    return w
+
+
+def trunk_features(feature_dims, n_tokens: int, K0: int, seed: int):
+    """Synthetic layer-0 features for ``n_tokens`` tokens: one fp32 ``[n_tokens, pad8(d)]`` tensor
+    per continuous feature (zero beyond the true dimension) and int32 centroid IDs ``[n_tokens]``.
+    Stand-ins for the embedding, the pre-attention norm output, the attention sketch and the
+    post-attention norm of a real model's layer 0."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed * _SEED_MUL + 778)
+    feats = []
+    for d in feature_dims:
+        f = torch.zeros(n_tokens, (d + 7) // 8 * 8)
+        f[:, :d] = torch.randn(n_tokens, d, generator=g)
+        feats.append(f.contiguous())
+    ids = torch.randint(0, K0, (n_tokens,), generator=g, dtype=torch.int32)
+    return feats, ids
