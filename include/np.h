@@ -396,6 +396,63 @@ int np_predict_logits_noalloc(const void* w1, const void* w2, const void* x_bf16
 /* Text of the calling thread's last np_predict_logits_noalloc error.  Never NULL. */
 const char* np_noalloc_last_error(void);
 
+/* ---- The shared predictor of Section 3.3 (projection blocks -> residual trunk -> centroid
+ * heads), for one token.  Stands beside np_predict: its head logits feed np_centroid_select.
+ * No context is needed; the caller owns weights, features and workspace (all device memory).
+ *
+ * Stage 1: feature i (fp32 [feature_dim[i]]) -> Linear -> LayerNorm -> SiLU -> T values; the
+ * layer-0 gate centroid ID -> row of the embedding -> Linear -> LayerNorm -> SiLU -> 4T values;
+ * concatenated to z (8T).  Stage 2: n_blocks times z <- z + W2 SiLU(LayerNorm(W1 z + b1)) + b2,
+ * W1: 8T -> 4T, W2: 4T -> 8T.  Stage 3: head_logits[l][g][k] = heads[(l*2 + g)*K + k] . z for
+ * the n_heads sparse layers, g = 0 gate, 1 up (the layout np_centroid_select reads at B = 1).
+ * LayerNorm: biased variance, epsilon 1e-5.  Dropout is the identity (inference).
+ * Matrices are bf16, row-major [out][in], 16-byte aligned; vectors fp32.  Dimensions that are
+ * not multiples of 8 (the scalar norm feature) are passed padded with zeros, their weight rows
+ * padded with zero columns. */
+#define NP_TRUNK_MAX_BLOCKS 16
+typedef struct np_trunk_desc {
+  int32_t T;               /* width of a projection block's output, multiple of 8, <= 1024 */
+  int32_t n_features;      /* 4 */
+  int32_t feature_dim[4];  /* padded to multiples of 8 */
+  int32_t K0;              /* layer-0 gate centroid vocabulary (rows of the embedding) */
+  int32_t E;               /* embedding width, multiple of 8 */
+  int32_t n_blocks;        /* residual blocks, 0..NP_TRUNK_MAX_BLOCKS */
+  int32_t n_heads;         /* sparse layers: 2 * n_heads heads */
+  int32_t K;               /* centroid vocabulary per head */
+  int32_t reserved[5];     /* 0 */
+} np_trunk_desc;
+typedef struct np_trunk_weights {
+  const void* proj_w[4];       /* bf16 [T][feature_dim[i]] */
+  const float* proj_b[4];      /* [T] linear bias */
+  const float* proj_gain[4];   /* [T] LayerNorm gain */
+  const float* proj_bias[4];   /* [T] LayerNorm bias */
+  const void* emb;             /* bf16 [K0][E] */
+  const void* cproj_w;         /* bf16 [4T][E] */
+  const float* cproj_b;        /* [4T] */
+  const float* cproj_gain;     /* [4T] */
+  const float* cproj_bias;     /* [4T] */
+  const void* blk_w1[NP_TRUNK_MAX_BLOCKS];    /* bf16 [4T][8T] */
+  const float* blk_b1[NP_TRUNK_MAX_BLOCKS];   /* [4T] */
+  const float* blk_gain[NP_TRUNK_MAX_BLOCKS]; /* [4T] */
+  const float* blk_bias[NP_TRUNK_MAX_BLOCKS]; /* [4T] */
+  const void* blk_w2[NP_TRUNK_MAX_BLOCKS];    /* bf16 [8T][4T] */
+  const float* blk_b2[NP_TRUNK_MAX_BLOCKS];   /* [8T] */
+  const void* heads;           /* bf16 [n_heads * 2 * K][8T], no bias */
+} np_trunk_weights;
+
+/* Floats of device workspace np_trunk_forward needs for `desc` (28 * T).  NP_E_INVAL on a bad T. */
+int np_trunk_workspace_floats(const np_trunk_desc* desc, uint64_t* out);
+
+/* Queues the forward pass on `stream` (11 kernel launches at four blocks; no synchronisation,
+ * no allocation).  `features`: host array of four device pointers; `centroid_id`: device
+ * scalar in [0, K0); `workspace`: device, 16-byte aligned, np_trunk_workspace_floats floats;
+ * `head_logits`: device fp32 [n_heads][2][K].
+ * Errors: NP_E_INVAL (NULL pointer, dimension outside its range), NP_E_CUDA; text in
+ * np_trunk_last_error(). */
+int np_trunk_forward(const np_trunk_desc* desc, const np_trunk_weights* weights, const float* const* features,
+                     const int32_t* centroid_id, float* workspace, float* head_logits, void* stream);
+const char* np_trunk_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -37,6 +37,7 @@ EXPORTED = [
     "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_read_records", "np_install", "np_sparse_mlp", "np_step", "np_step_selected", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
     "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_last_error",
+    "np_trunk_workspace_floats", "np_trunk_forward", "np_trunk_last_error",
 ]
 
 
@@ -57,6 +58,23 @@ class np_buffers(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "w1", "w2", "backing", "gate_buf", "up_buf", "downT_buf", "staging", "host_staging", "workspace",
         "host_lists", "dense_buf")] + [("backing_fd", C.c_int32), ("reserved", C.c_int32)]
+
+
+NP_TRUNK_MAX_BLOCKS = 16
+
+
+class np_trunk_desc(C.Structure):
+    _fields_ = [("T", C.c_int32), ("n_features", C.c_int32), ("feature_dim", C.c_int32 * 4), ("K0", C.c_int32),
+                ("E", C.c_int32), ("n_blocks", C.c_int32), ("n_heads", C.c_int32), ("K", C.c_int32),
+                ("reserved", C.c_int32 * 5)]
+
+
+class np_trunk_weights(C.Structure):
+    _fields_ = [("proj_w", C.c_void_p * 4), ("proj_b", C.c_void_p * 4), ("proj_gain", C.c_void_p * 4),
+                ("proj_bias", C.c_void_p * 4), ("emb", C.c_void_p), ("cproj_w", C.c_void_p), ("cproj_b", C.c_void_p),
+                ("cproj_gain", C.c_void_p), ("cproj_bias", C.c_void_p)] + [
+        (n, C.c_void_p * NP_TRUNK_MAX_BLOCKS) for n in ("blk_w1", "blk_b1", "blk_gain", "blk_bias", "blk_w2", "blk_b2")
+    ] + [("heads", C.c_void_p)]
 
 
 class np_delta_view(C.Structure):
@@ -86,6 +104,8 @@ def load() -> C.CDLL:
     vp, i32 = C.c_void_p, C.c_int32
     lib.np_version.restype = C.c_int
     lib.np_last_error.restype = C.c_char_p
+    lib.np_trunk_last_error.restype = C.c_char_p
+    lib.np_trunk_last_error.argtypes = []
     lib.np_last_error.argtypes = [vp]
     sigs = {
         "np_query_sizes": [C.POINTER(np_config), C.POINTER(np_sizes)],
@@ -98,6 +118,8 @@ def load() -> C.CDLL:
         "np_centroid_select": [vp, vp, i32, i32, vp, vp, vp, vp],
         "np_delta": [vp, vp, vp],
         "np_install": [vp, i32, i32, vp],
+        "np_trunk_workspace_floats": [C.POINTER(np_trunk_desc), C.POINTER(C.c_uint64)],
+        "np_trunk_forward": [C.POINTER(np_trunk_desc), C.POINTER(np_trunk_weights), C.POINTER(vp), vp, vp, vp, vp],
         "np_read_records": [i32, C.c_uint64, C.c_uint64, vp, i32, vp, i32, vp, vp],
         "np_sparse_mlp": [vp, i32, vp, i32, vp, vp],
         "np_step": [vp, vp, i32, vp, vp, vp],
@@ -213,6 +235,45 @@ def np_read_records(fd: int, base_offset: int, rec_bytes: int, ids: np.ndarray, 
                                 C.addressof(ranges), C.addressof(ring))
     _check(None, rc)
     return ranges.value, bool(ring.value)
+
+
+def trunk_pack(w: dict, n_heads: int):
+    """The C descriptor and pointer table for a weight dict of ``synth.trunk_weights`` whose tensors
+    live on the device (the dict must stay alive while the table is in use)."""
+    d = np_trunk_desc()
+    d.T, d.n_features, d.K0, d.E, d.K = w["T"], 4, w["K0"], w["E"], w["K"]
+    d.n_blocks, d.n_heads = len(w["blocks"]), n_heads
+    for i, dim in enumerate(w["feature_dims"]):
+        d.feature_dim[i] = (dim + 7) // 8 * 8
+    t = np_trunk_weights()
+    for i, (W, b, g, be) in enumerate(w["proj"]):
+        t.proj_w[i], t.proj_b[i], t.proj_gain[i], t.proj_bias[i] = W.data_ptr(), b.data_ptr(), g.data_ptr(), be.data_ptr()
+    t.emb = w["emb"].data_ptr()
+    W, b, g, be = w["cproj"]
+    t.cproj_w, t.cproj_b, t.cproj_gain, t.cproj_bias = W.data_ptr(), b.data_ptr(), g.data_ptr(), be.data_ptr()
+    for j, (W1, b1, g, be, W2, b2) in enumerate(w["blocks"]):
+        t.blk_w1[j], t.blk_b1[j], t.blk_gain[j], t.blk_bias[j] = W1.data_ptr(), b1.data_ptr(), g.data_ptr(), be.data_ptr()
+        t.blk_w2[j], t.blk_b2[j] = W2.data_ptr(), b2.data_ptr()
+    t.heads = w["heads"].data_ptr()
+    return d, t
+
+
+def np_trunk_workspace_floats(desc: np_trunk_desc) -> int:
+    out = C.c_uint64(0)
+    rc = load().np_trunk_workspace_floats(C.byref(desc), C.byref(out))
+    if rc < 0:
+        raise NpError(rc, load().np_trunk_last_error().decode())
+    return int(out.value)
+
+
+def np_trunk_forward(desc, table, features, centroid_id, workspace, head_logits, stream=None) -> int:
+    """``features``: four device fp32 vectors; ``centroid_id``: device int32 scalar."""
+    ptrs = (C.c_void_p * 4)(*[_ptr(f) for f in features])
+    rc = load().np_trunk_forward(C.byref(desc), C.byref(table), ptrs, _ptr(centroid_id), _ptr(workspace),
+                                 _ptr(head_logits), _stream(stream))
+    if rc < 0:
+        raise NpError(rc, load().np_trunk_last_error().decode())
+    return rc
 
 
 def np_install(ctx, layer_begin: int, layer_end: int, copy_stream=None) -> int:
