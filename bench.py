@@ -74,6 +74,9 @@ def parse_args():
     ap.add_argument("--selection", default="topk", choices=["topk", "centroid"],
                     help="topk: the metric's selection; centroid: centroid heads + bank lookup + gate AND up")
     ap.add_argument("--centroids", type=int, default=512, help="centroid vocabulary per head (centroid selection)")
+    ap.add_argument("--predictor", default="mlp", choices=["mlp", "trunk"],
+                    help="centroid selection: head logits from the two-layer predictor (mlp) or from the paper's own "
+                         "predictor, projection blocks -> residual trunk -> heads (trunk; one sequence)")
     return ap.parse_args()
 
 
@@ -367,13 +370,41 @@ def cuda_arm(args):
         bank = synth.centroid_bank(cfg, Kc).to(dev)
         head_logits = torch.empty((Bq, L, 2, Kc), dtype=torch.float32, device=dev)
         sel_words = torch.empty((L, M // 32), dtype=torch.int32, device=dev)
+    trunk = centroid and args.predictor == "trunk"
+    if trunk:
+        if Bq != 1:
+            raise SystemExit("bench.py: --predictor trunk runs one sequence")
+        # The paper's predictor at its sizes (T = 512, four blocks), one gate and one up head per layer
+        # of this stack.  Its five layer-0 features are stand-ins made from the step's hidden state
+        # (no model is available): the state itself, its LayerNorm, its first 128 values, its RMS, and
+        # the arg-max of a fixed random projection as the layer-0 gate centroid ID.
+        tT, tK0, tE = 512, 512, 2048
+        tdims = (D, D, 128, 1)
+        tw = synth.trunk_weights(tT, tdims, tK0, tE, 4, L, Kc, cfg.seed, device="cuda")
+        tdesc, ttable = nb.trunk_pack(tw, L)
+        tws = torch.empty(nb.np_trunk_workspace_floats(tdesc), dtype=torch.float32, device=dev)
+        xf = xs_host[:, 0].to(torch.float32)                                  # [T + n_detail, D]
+        gproj = torch.randn(D, tK0, generator=torch.Generator().manual_seed(cfg.seed + 5)) / D ** 0.5
+        rms = xf.pow(2).mean(dim=1, keepdim=True).sqrt()
+        feats_host = [xf.contiguous(), torch.nn.functional.layer_norm(xf, (D,)).contiguous(), xf[:, :128].contiguous(),
+                      torch.cat([rms, torch.zeros(xf.shape[0], 7)], dim=1).contiguous()]
+        feats_host = [f.pin_memory() for f in feats_host]
+        ids_host = (xf @ gproj).argmax(dim=1).to(torch.int32).pin_memory()
+        feats_dev = [f.to(dev) for f in feats_host]
+        ids_dev = ids_host.to(dev)
+        feat_stage = [torch.empty_like(f[0], device=dev) for f in feats_host]
+        id_stage = torch.empty(1, dtype=torch.int32, device=dev)
+        trunk_in_bytes = sum(f[0].numel() * 4 for f in feats_host) + 4
 
-    def step(x):
+    def step(x, feats=None, cid=None):
         if not centroid:
             return nb.np_step(eng.ctx, x, Bq, out, s, cs)
         # the same path with the selection stage swapped: head logits -> arg-max centroids ->
         # bank lookup -> gate AND up -> delta -> install -> MLP chain, all through the C ABI
-        nb.np_predict_logits_noalloc(eng.w1, w2c, x, Bq, L, D, 2 * Kc, cfg.d_pred, head_logits, s)
+        if trunk:
+            nb.np_trunk_forward(tdesc, ttable, feats, cid, tws, head_logits, s)
+        else:
+            nb.np_predict_logits_noalloc(eng.w1, w2c, x, Bq, L, D, 2 * Kc, cfg.d_pred, head_logits, s)
         nb.np_centroid_select(eng.ctx, head_logits, Bq, Kc, bank, None, sel_words, s)
         return nb.np_step_selected(eng.ctx, x, Bq, sel_words, out, s, cs)
 
@@ -385,7 +416,10 @@ def cuda_arm(args):
 
     def run_resident(t_lo, t_hi, stats=None):
         for t in range(t_lo, t_hi):
-            step(xs_dev[t])
+            if trunk:
+                step(xs_dev[t], [f[t] for f in feats_dev], ids_dev[t:t + 1])
+            else:
+                step(xs_dev[t])
             if stats is not None:
                 stats.append(eng.counters().copy())
 
@@ -410,7 +444,10 @@ def cuda_arm(args):
     stage_us, delta_rows, overlap, overflow_steps = [], [], [], 0
     for i in range(n_detail):
         t = T + i                                       # the sequence simply continues
-        step(xs_dev[t])
+        if trunk:
+            step(xs_dev[t], [f[t] for f in feats_dev], ids_dev[t:t + 1])
+        else:
+            step(xs_dev[t])
         stage_us.append(nb.np_last_step_times(eng.ctx))      # centroid selection: the predict stage is outside the call
         c = eng.counters()
         delta_rows.append(float(c[nd:, nb.NP_CNT_DELTA].mean()) if nd < L else 0.0)
@@ -427,7 +464,14 @@ def cuda_arm(args):
         for t in range(t_lo, t_hi):
             with torch.cuda.stream(s):
                 x_stage.copy_(xs_host[t], non_blocking=True)
-            step(x_stage)
+                if trunk:
+                    for dst, src in zip(feat_stage, feats_host):
+                        dst.copy_(src[t], non_blocking=True)
+                    id_stage.copy_(ids_host[t:t + 1], non_blocking=True)
+            if trunk:
+                step(x_stage, feat_stage, id_stage)
+            else:
+                step(x_stage)
             with torch.cuda.stream(s):
                 out_host.copy_(out, non_blocking=True)
             s.synchronize()                              # the caller consumes the result every step
@@ -469,7 +513,9 @@ def cuda_arm(args):
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record(s)
     for _ in range(reps):
-        if centroid:
+        if trunk:
+            nb.np_trunk_forward(tdesc, ttable, [f[T - 1] for f in feats_dev], ids_dev[T - 1:T], tws, head_logits, s)
+        elif centroid:
             nb.np_predict_logits_noalloc(eng.w1, w2c, xs_dev[T - 1], Bq, L, D, 2 * Kc, cfg.d_pred, head_logits, s)
             nb.np_centroid_select(eng.ctx, head_logits, Bq, Kc, bank, None, sel_words, s)
         else:
@@ -496,6 +542,9 @@ def cuda_arm(args):
     traffic = 27.52e6 * L / n_launch if cfg.name == "7b" and not nd else None
     pred_rows = L * 2 * args.centroids if centroid else L * M
     pred_bytes = 2 * cfg.d_pred * D + 2 * pred_rows * cfg.d_pred + 4 * pred_rows
+    if trunk:   # every matrix of the predictor once, plus the logits
+        pred_bytes = 2 * (sum(blk[0].numel() for blk in tw["proj"]) + tw["cproj"][0].numel() + tw["heads"].numel()
+                          + sum(b[0].numel() + b[4].numel() for b in tw["blocks"])) + 4 * pred_rows
     mean_delta = float(np.mean(delta_rows))
     result = {
         "metric": METRIC, "value": K * world / (ms_total / 1000.0), "unit": UNIT, "n_gpus": world,
@@ -505,6 +554,7 @@ def cuda_arm(args):
             "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
                         f"B={Bq} rho={cfg.rho} policy={args.policy} transfer={args.transfer}"
                         + (f" selection=centroid K={args.centroids}" if centroid else "")
+                        + (" predictor=trunk(T=512, 4 blocks)" if trunk else "")
                         + (" records=int8" if args.records == "int8" else "")
                         + (f" dense_layers={args.dense_layers}" if args.dense_layers else "")
                         + (f" (longest prefix within {args.budget_gib} GiB)" if args.budget_gib is not None else ""),
@@ -514,7 +564,8 @@ def cuda_arm(args):
             "replicas": world,
         },
         "e2e": {"value": K * world / (e2e_ms_total / 1000.0), "unit": UNIT,
-                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * (L - nd) * rec_store), "d2h_bytes_per_step": int(Bq * D * 4)},
+                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * (L - nd) * rec_store + (trunk_in_bytes if trunk else 0)),
+                "d2h_bytes_per_step": int(Bq * D * 4)},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": mlp_kernel, "achieved": achieved, "peak": peak,
