@@ -212,7 +212,9 @@ static cudaError_t gemv(const GemvArgs& a, int n_seg, cudaStream_t s, int sm_cou
     max_rows = std::max(max_rows, a.seg[i].rows);
   }
   const size_t smem = (size_t)max_in * 4;
-  const bool wide = max_rows >= 2 * kWarps * sm_count;  // two rows for every warp of the device
+  // two rows per warp where every warp of the device gets two, and where a row is so short that
+  // one row's pieces would leave half of a lane's loads unused
+  const bool wide = max_rows >= 2 * kWarps * sm_count || max_in <= 2048;
   auto kfn = wide ? k_gemv<2, 8> : k_gemv<1, 16>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
