@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--policy", default="exact", choices=["exact", "lru"])
     ap.add_argument("--transfer", default="gather", choices=["runs", "gather", "zerocopy", "file"],
                     help="file: the record store is a file, read through io_uring with O_DIRECT (Section 3.5)")
+    ap.add_argument("--mapped-staging", action="store_true",
+                    help="gather / file transfer: the scatter kernel reads the pinned staging itself, no staging copy")
     ap.add_argument("--store-path", default=None, help="--transfer file: where the store file is written (default: a temp file)")
     ap.add_argument("--io-depth", type=int, default=0, help="--transfer file: reads in flight (0 = 256; -1 = blocking preads)")
     ap.add_argument("--buffered", action="store_true", help="--transfer file: open the store without O_DIRECT")
@@ -321,7 +323,8 @@ def cuda_arm(args):
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
                           host_threads=args.host_threads, dense_layers=args.dense_layers, io_depth=args.io_depth,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
-                          | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0))
+                          | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0)
+                          | (nb.NP_F_MAPPED_STAGING if args.mapped_staging else 0))
     storage = None
     if args.transfer == "file":
         # the store goes to a file and leaves host memory; the library sees only the descriptor
@@ -556,6 +559,7 @@ def cuda_arm(args):
                         + (f" selection=centroid K={args.centroids}" if centroid else "")
                         + (" predictor=trunk(T=512, 4 blocks)" if trunk else "")
                         + (" records=int8" if args.records == "int8" else "")
+                        + (" mapped_staging" if args.mapped_staging else "")
                         + (f" dense_layers={args.dense_layers}" if args.dense_layers else "")
                         + (f" (longest prefix within {args.budget_gib} GiB)" if args.budget_gib is not None else ""),
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",

@@ -98,6 +98,11 @@ extern "C" {
                                    (for comparison runs) */
 #define NP_F_LAYER_LAUNCHES  4  /* np_step / np_mlp_chain: one kernel launch per layer instead
                                    of resident kernels spanning runs of layers */
+#define NP_F_MAPPED_STAGING 16  /* NP_XFER_HOST_GATHER / NP_XFER_FILE: no staging copy; the scatter kernel
+                                   reads the records in the pinned staging buffer through its device
+                                   mapping (Section 3.5: page-aligned host staging registered as mapped,
+                                   read by the kernels "without an explicit cudaMemcpy").  host_staging
+                                   must be device-mapped pinned memory; np_buffers.staging is not used */
 
 /* per-layer counters written by np_delta (np_read_counters) */
 #define NP_CNT_PRED      0  /* |P|                      */

@@ -176,6 +176,7 @@ struct np_ctx {
   int32_t* host_lists = nullptr;      // host address
   int32_t* host_lists_dev = nullptr;  // device alias
   const char* backing_dev = nullptr;  // device alias of the record store
+  char* hstage_dev = nullptr;         // device alias of the pinned staging (NP_F_MAPPED_STAGING)
   cudaEvent_t ev_delta = nullptr;
   std::vector<cudaEvent_t> ev_installed;
   std::vector<char> install_pending;
@@ -251,7 +252,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->transfer_mode == NP_XFER_FILE && c->record_format != NP_REC_BF16)
     return fail(ctx, NP_E_INVAL, "NP_XFER_FILE needs NP_REC_BF16 records");
   if (c->io_depth < -1 || c->io_depth > 4096) return fail(ctx, NP_E_INVAL, "io_depth must be in [-1, 4096]");
-  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
+  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES | NP_F_MAPPED_STAGING)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
   if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
@@ -390,7 +391,9 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   int rc = check_config(cfg, nullptr);
   if (rc) return rc;
   if (!b) return fail(nullptr, NP_E_INVAL, "buffers is NULL");
-  const bool need_staging = cfg->transfer_mode != NP_XFER_ZERO_COPY;
+  const bool mapped_staging = (cfg->flags & NP_F_MAPPED_STAGING) &&
+                              (cfg->transfer_mode == NP_XFER_HOST_GATHER || cfg->transfer_mode == NP_XFER_FILE);
+  const bool need_staging = cfg->transfer_mode != NP_XFER_ZERO_COPY && !mapped_staging;
   const bool any_sparse = cfg->dense_layers < cfg->n_layers;
   const bool from_file = cfg->transfer_mode == NP_XFER_FILE;
   if (!b->w1 || !b->w2 || (!b->backing && !from_file) || !b->workspace || !b->host_lists ||
@@ -455,6 +458,14 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   }
   ctx->host_lists = static_cast<int32_t*>(b->host_lists);
   ctx->host_lists_dev = static_cast<int32_t*>(dev_alias);
+  if (mapped_staging) {
+    if (cudaHostGetDevicePointer(&dev_alias, b->host_staging, 0) != cudaSuccess) {
+      cudaGetLastError();
+      np_destroy(ctx);
+      return fail(nullptr, NP_E_INVAL, "host_staging is not pinned, device-mapped host memory (NP_F_MAPPED_STAGING)");
+    }
+    ctx->hstage_dev = static_cast<char*>(dev_alias);
+  }
   if (!from_file) {
     if (cudaHostGetDevicePointer(&dev_alias, const_cast<void*>(b->backing), 0) != cudaSuccess) {
       cudaGetLastError();
@@ -730,9 +741,14 @@ static int install_from_file(np_ctx* ctx, int layer_begin, int layer_end, cudaSt
     }
     char* hbuf = hstage + (size_t)c.h * part_rows * rec;
     char* dbuf = staging + (size_t)c.h * part_rows * rec;
-    NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)c.rows * rec, cudaMemcpyHostToDevice, cs));
-    NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[c.h], cs));
-    NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[c.h], 0));
+    if (ctx->hstage_dev) {
+      // mapped staging (the paper's way): the scatter kernel reads the staged records over the bus itself
+      dbuf = ctx->hstage_dev + (size_t)c.h * part_rows * rec;
+    } else {
+      NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)c.rows * rec, cudaMemcpyHostToDevice, cs));
+      NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[c.h], cs));
+      NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[c.h], 0));
+    }
     NP_LAUNCH(ctx, launch_scatter(d, dbuf, false, nullptr, ctx->t.delta_slots + (size_t)c.l * d.C,
                                 ctx->t.counters + (size_t)c.l * NP_N_COUNTERS + NP_CNT_DELTA, c.first, c.rows,
                                 static_cast<char*>(ctx->bufs.gate_buf) + (size_t)(c.l - d.dense) * d.C * row_bytes,
@@ -875,9 +891,13 @@ static int install_host_gather(np_ctx* ctx, int layer_begin, int layer_end, cuda
       if (bad) return fail(ctx, NP_E_DEVICE, "layer %d: neuron id out of range", batch.front().l);
       // the copies queue back to back on the caller's stream; the scatter kernels follow them
       // on a side stream, so a copy never waits for the previous part's kernels
-      NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)used * rec, cudaMemcpyHostToDevice, cs));
-      NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[h], cs));
-      NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[h], 0));
+      if (ctx->hstage_dev) {
+        dbuf = ctx->hstage_dev + (size_t)h * part_rows * rec;  // mapped staging: no staging copy
+      } else {
+        NP_CUDA(ctx, cudaMemcpyAsync(dbuf, hbuf, (size_t)used * rec, cudaMemcpyHostToDevice, cs));
+        NP_CUDA(ctx, cudaEventRecord(ctx->ev_copied[h], cs));
+        NP_CUDA(ctx, cudaStreamWaitEvent(ctx->aux[0], ctx->ev_copied[h], 0));
+      }
     }
     for (const Piece& pc : batch) {
       if (pc.rows > 0)

@@ -57,6 +57,21 @@ def test_small_staging_splits_a_layer_into_chunks(tmp_path, direct):
         p.close()
 
 
+@pytest.mark.parametrize("mode", [nb.NP_XFER_FILE, nb.NP_XFER_HOST_GATHER])
+@pytest.mark.parametrize("policy", [nb.NP_EVICT_EXACT, nb.NP_EVICT_LRU])
+def test_mapped_staging_needs_no_staging_copy(tmp_path, mode, policy):
+    """NP_F_MAPPED_STAGING: the scatter kernel reads the pinned staging through its device
+    mapping (the paper's coherent mapped path); same result, chunked or not."""
+    cfg = SMALL
+    for staging_rows in (None, 16):
+        p = Pair(cfg, policy=policy, transfer_mode=mode, store_dir=tmp_path, staging_rows=staging_rows,
+                 flags=nb.NP_F_CHECK_BOUNDS | nb.NP_F_MAPPED_STAGING)
+        try:
+            _run_steps(p, cfg, n=4)
+        finally:
+            p.close()
+
+
 def test_dense_prefix_is_filled_from_the_file(tmp_path):
     cfg = SMALL
     p = Pair(cfg, transfer_mode=nb.NP_XFER_FILE, store_dir=tmp_path, dense_layers=2, staging_rows=64)
