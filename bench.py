@@ -427,8 +427,13 @@ def cuda_arm(args):
                 stats.append(eng.counters().copy())
 
     # ---- device-resident timing ("value") ----------------------------------------------
-    run_resident(0, 1 + W)                              # cold start + warm-up
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record(s)
+    run_resident(0, 1)                                  # cold start: every predicted row of every layer is installed
+    c1.record(s)
+    run_resident(1, 1 + W)                              # warm-up
     barrier()
+    cold_ms = c0.elapsed_time(c1)
     eng.counters()                                      # raises if a kernel reported a fault or a timed-out wait
     sampler = ClockSampler(local)
     sampler.start()
@@ -581,6 +586,8 @@ def cuda_arm(args):
                       "predict_alone": pred_us, "predict_gbs": pred_bytes / (pred_us * 1e-6) / 1e9,
                       "mlp_chain_alone": mlp_us * n_launch},
         "setup_s": {"generate": gen_s},
+        "cold_start": {"ms": cold_ms, "note": "step 0, reported apart from the steady state: empty buffers, every "
+                                               "predicted row of every sparse layer crosses to the device"},
     }
     if not centroid:
         # spread over the detail steps, and the step without any transfer (context: what the GPU work alone takes)
