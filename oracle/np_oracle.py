@@ -16,7 +16,9 @@ Pins (see tests/test_oracle_*.py): exact rational brute force and structured
 closed forms for ``predict``; full-sort brute force, constructed ties and
 degenerate k for ``topk_bitmap``; a per-bit scalar loop, constructed ties and
 the one-hot/identity-bank special cases for ``centroid_select``; the set identities of Eq. 2-3, slot-map
-bijection invariants and a set-based brute force for ``Residency.delta``;
+bijection invariants and a set-based brute force for ``Residency.delta``
+(``validity_errors`` is the order-free form of those invariants, itself checked
+on hand-made valid and invalid states);
 byte identity for ``install``; the dense SwiGLU library form when every row is
 active, linearity over disjoint sets and a scalar loop for ``sparse_mlp``; the
 paper's buffer-size arithmetic (Section 4.3) for ``record_bytes``; unit output
@@ -367,6 +369,42 @@ class Residency:
 
     def resident_words(self) -> np.ndarray:
         return bool_to_bitmap(self.R)
+
+
+def validity_errors(slot_map: np.ndarray, owner: np.ndarray, resident: np.ndarray, C: int,
+                    pred: np.ndarray = None, active_ids: np.ndarray = None) -> list:
+    """Order-free validity of one layer's residency state (Section 3.4: "correctness depends on
+    row presence and slot address", not on which free slot a row took).  Returns the violated
+    conditions as text, an empty list for any correct assignment: the slot map restricted to the
+    resident rows is injective into [0, C), absent rows map to -1, ``owner`` is its inverse and -1
+    elsewhere, and (when given) the active rows are exactly the predicted rows that are resident.
+    Used to tell "wrong" from "differently ordered" when a list differs from the canonical one."""
+    errs = []
+    S = np.asarray(slot_map)
+    R = np.asarray(resident, dtype=bool)
+    ow = np.asarray(owner)
+    if not ((S >= 0) == R).all():
+        errs.append("slot map is >= 0 on a row that is not resident, or -1 on one that is")
+    slots = S[R]
+    if slots.size and (slots.min() < 0 or slots.max() >= C):
+        errs.append("a resident row's slot lies outside [0, C)")
+    elif np.unique(slots).size != slots.size:
+        errs.append("two resident rows share a slot")
+    else:
+        if slots.size and not (ow[slots] == np.flatnonzero(R)).all():
+            errs.append("owner is not the inverse of the slot map")
+        free = np.ones(C, dtype=bool)
+        free[slots] = False
+        if not (ow[free] == -1).all():
+            errs.append("a free slot has an owner")
+    if int(R.sum()) > C:
+        errs.append("more resident rows than capacity")
+    if pred is not None and active_ids is not None:
+        want = np.flatnonzero(np.asarray(pred, dtype=bool) & R)
+        if not np.array_equal(np.sort(np.asarray(active_ids)), want):
+            errs.append("the active rows are not the predicted rows that are resident")
+    return errs
+
 
 
 # --------------------------------------------------------------------------

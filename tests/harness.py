@@ -78,6 +78,10 @@ class Pair:
             assert cnt[l][nb.NP_CNT_RESIDENT] == int(self.ora.res.R[l].sum())
             assert cnt[l][nb.NP_CNT_STEP] == self.ora.res.t - 1
             st = self.eng.export_state(l)
+            # order-free validity first: a failure here is a wrong state, one below only a different order
+            resident = O.bitmap_to_bool(st["resident"], self.cfg.d_ffn)
+            assert O.validity_errors(st["slot_map"], st["owner"], resident, self.C) == [], l
+            assert set(got["active_ids"].tolist()) <= set(np.flatnonzero(resident).tolist()), l   # act is a subset of R
             assert (st["slot_map"] == self.ora.res.S[l]).all(), l
             assert (st["owner"] == self.ora.res.owner[l]).all(), l
             assert (st["resident"] == O.bool_to_bitmap(self.ora.res.R[l])).all(), l

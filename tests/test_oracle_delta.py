@@ -11,8 +11,43 @@ def _words(T, L, M, n_set, seed, persistence=0.8):
     return synth.random_bitmaps(L, M, n_set, seed, T, persistence).numpy().view(np.uint32)
 
 
+def test_validity_checker_accepts_any_correct_assignment_and_names_what_is_wrong():
+    M, C = 64, 8
+    R = np.zeros(M, bool)
+    rows = np.array([3, 17, 40, 63])
+    R[rows] = True
+    P = np.zeros(M, bool)
+    P[[3, 40, 50]] = True
+    for slots in ([0, 1, 2, 3], [7, 2, 5, 0]):                # canonical order or not: both valid
+        S = np.full(M, -1)
+        S[rows] = slots
+        owner = np.full(C, -1)
+        owner[slots] = rows
+        assert O.validity_errors(S, owner, R, C, P, np.array([40, 3])) == []
+    S = np.full(M, -1)
+    S[rows] = [0, 1, 1, 3]                                     # two rows in one slot
+    owner = np.full(C, -1)
+    owner[[0, 1, 3]] = [3, 40, 63]
+    assert any("share a slot" in e for e in O.validity_errors(S, owner, R, C))
+    S[rows] = [0, 1, 2, 9]                                     # slot outside the buffer
+    assert any("outside" in e for e in O.validity_errors(S, owner, R, C))
+    S[rows] = [0, 1, 2, 3]
+    owner = np.full(C, -1)
+    owner[[0, 1, 2, 3]] = [3, 17, 40, 62]                      # owner names the wrong row
+    assert any("inverse" in e for e in O.validity_errors(S, owner, R, C))
+    owner[[0, 1, 2, 3, 6]] = [3, 17, 40, 63, 5]                # a free slot with an owner
+    assert any("free slot" in e for e in O.validity_errors(S, owner, R, C))
+    owner[6] = -1
+    S[5] = 4                                                   # mapped but not resident
+    assert any("not resident" in e for e in O.validity_errors(S, owner, R, C))
+    S[5] = -1
+    assert any("active rows" in e for e in O.validity_errors(S, owner, R, C, P, np.array([3])))
+
+
 def _check_tables(res: O.Residency):
     """S and owner are mutually inverse; S[n] >= 0 exactly on resident rows."""
+    for l in range(res.L):
+        assert O.validity_errors(res.S[l], res.owner[l], res.R[l], res.C) == []
     for l in range(res.L):
         R, S, owner = res.R[l], res.S[l], res.owner[l]
         assert ((S >= 0) == R).all()
