@@ -449,7 +449,7 @@ def cuda_arm(args):
 
     nd = args.dense_layers
     # ---- per-stage detail on a few more steady-state steps (untimed region) ----------------
-    stage_us, delta_rows, overlap, overflow_steps = [], [], [], 0
+    stage_us, delta_rows, overlap, overflow_steps, active_max = [], [], [], 0, 0
     for i in range(n_detail):
         t = T + i                                       # the sequence simply continues
         if trunk:
@@ -460,6 +460,7 @@ def cuda_arm(args):
         c = eng.counters()
         delta_rows.append(float(c[nd:, nb.NP_CNT_DELTA].mean()) if nd < L else 0.0)
         overflow_steps += int((c[:, nb.NP_CNT_OVERFLOW] > 0).any())
+        active_max = max(active_max, int(c[nd:, nb.NP_CNT_ACTIVE].max()) if nd < L else 0)
         overlap.append(float((c[nd:, nb.NP_CNT_KEPT] / np.maximum(1, c[nd:, nb.NP_CNT_PRED])).mean()) if nd < L else 1.0)
     stage_all = np.stack(stage_us)
     step_each = stage_all[:, 0] + stage_all[:, 1] + stage_all[:, 3]   # predict + delta + chain (which waits for the installs)
@@ -569,7 +570,7 @@ def cuda_arm(args):
                         + (f" (longest prefix within {args.budget_gib} GiB)" if args.budget_gib is not None else ""),
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
             "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
-            "active_rows_per_layer": n_active, "overflow_steps": int(overflow_steps),
+            "active_rows_per_layer": n_active, "active_rows_max": active_max, "overflow_steps": int(overflow_steps),
             "replicas": world,
         },
         "e2e": {"value": K * world / (e2e_ms_total / 1000.0), "unit": UNIT,
