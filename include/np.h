@@ -100,8 +100,8 @@ extern "C" {
                                    of resident kernels spanning runs of layers */
 #define NP_F_MAPPED_STAGING 16  /* NP_XFER_HOST_GATHER / NP_XFER_FILE: no staging copy; the scatter kernel
                                    reads the records in the pinned staging buffer through its device
-                                   mapping (Section 3.5: page-aligned host staging registered as mapped,
-                                   read by the kernels "without an explicit cudaMemcpy").  host_staging
+                                   mapping (Section 3.5: the staging is page-aligned host memory registered
+                                   as mapped, so kernels reach it with no copy call in between).  host_staging
                                    must be device-mapped pinned memory; np_buffers.staging is not used */
 
 /* per-layer counters written by np_delta (np_read_counters) */
@@ -204,8 +204,8 @@ int np_version(void);
  * size: Section 3.5; buffer size: Section 4.3).  NP_E_INVAL on a bad config. */
 int np_query_sizes(const np_config* cfg, np_sizes* out);
 
-/* The dense/sparse split's memory rule (Section 3.1: "the largest dense prefix
- * that fits within the memory budget"): the largest d in [0, L] with
+/* The dense/sparse split's memory rule (Section 3.1: as many leading layers stay
+ * dense as the memory budget has room for): the largest d in [0, L] with
  *   d * M * REC + (L - d) * C * REC + fixed_bytes <= budget_bytes,
  * i.e. d dense layers, resident buffers of C records for the rest, next to
  * fixed_bytes of other resident state.  cfg->dense_layers is ignored.
@@ -387,8 +387,12 @@ int np_last_step_times(np_ctx* ctx, float* out_us);
  * context; here the scratch between the two predictor layers is a fixed array inside the library.
  *   w1 dev bf16 [d_pred][d_model], w2 dev bf16 [n_layers*d_ffn][d_pred], x_bf16 dev bf16 [B][d_model]
  *   logits_out dev fp32 [B][n_layers][d_ffn]   (all caller-owned, 16-byte aligned)
- * Same kernels and results as np_predict's logits.  Calls no cudaMalloc / cudaFree or allocating
- * library routine.  The first call on a device looks up the scratch array's device address
+ * Bit-identical to np_predict's logits in a context created with NP_F_NO_TENSOR_CORES (the same
+ * plain-core kernels); a default context takes the tensor-core kernel for B > 4, whose rounding
+ * differs (both are within rel-L2 1e-5 of the exact product).  Calls no cudaMalloc / cudaFree or
+ * allocating library routine.  Every call first clears the status words in the scratch; a kernel
+ * whose bounded wait runs out records a bit there, leaves part of logits_out unwritten and the
+ * call still returns NP_OK (it does not synchronise): np_noalloc_check reports it.  The first call on a device looks up the scratch array's device address
  * (cudaGetSymbolAddress, with that device current); make that first call before any stream
  * capture.  All calls on a device share the one scratch array: calls that may overlap on the GPU
  * (different streams) race on it and must be serialised by the caller.
@@ -398,7 +402,14 @@ int np_predict_logits_noalloc(const void* w1, const void* w2, const void* x_bf16
                               int32_t n_layers, int32_t d_model, int32_t d_ffn, int32_t d_pred,
                               float* logits_out, void* stream);
 
-/* Text of the calling thread's last np_predict_logits_noalloc error.  Never NULL. */
+/* Waits for `stream` and returns NP_E_DEVICE if the kernels of the last
+ * np_predict_logits_noalloc on the current device recorded a status bit (a bounded wait ran
+ * out: logits incomplete), NP_OK if not, NP_E_STATE if that entry point never ran on this
+ * device.  Allocates nothing (the word is copied to the caller's stack).  The paper has no
+ * counterpart. */
+int np_noalloc_check(void* stream);
+
+/* Text of the calling thread's last np_predict_logits_noalloc / np_noalloc_check error.  Never NULL. */
 const char* np_noalloc_last_error(void);
 
 /* ---- The shared predictor of Section 3.3 (projection blocks -> residual trunk -> centroid

@@ -37,7 +37,7 @@ EXPORTED = [
     "np_version", "np_query_sizes", "np_plan_dense_prefix", "np_init", "np_destroy", "np_reset", "np_last_error",
     "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_read_records", "np_install", "np_sparse_mlp", "np_step", "np_step_selected", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
-    "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_last_error",
+    "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_check", "np_noalloc_last_error",
     "np_trunk_workspace_floats", "np_trunk_forward", "np_trunk_last_error",
 ]
 
@@ -137,6 +137,7 @@ def load() -> C.CDLL:
     lib.np_noalloc_last_error.restype = C.c_char_p
     lib.np_noalloc_last_error.argtypes = []
     sigs["np_predict_logits_noalloc"] = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+    sigs["np_noalloc_check"] = [vp]
     for name, args in sigs.items():
         fn = getattr(lib, name)
         fn.argtypes = args
@@ -341,6 +342,14 @@ def np_predict_logits_noalloc(w1, w2, x_bf16, B: int, n_layers: int, d_model: in
     """Predictor logits without a context and without allocating (see include/np.h)."""
     rc = load().np_predict_logits_noalloc(_ptr(w1), _ptr(w2), _ptr(x_bf16), B, n_layers, d_model, d_ffn,
                                           d_pred, _ptr(logits_out), _stream(stream))
+    if rc < 0:
+        raise NpError(rc, load().np_noalloc_last_error().decode())
+    return rc
+
+
+def np_noalloc_check(stream=None) -> int:
+    """Waits for `stream`; raises if the last allocation-free predictor call recorded a status bit."""
+    rc = load().np_noalloc_check(_stream(stream))
     if rc < 0:
         raise NpError(rc, load().np_noalloc_last_error().decode())
     return rc

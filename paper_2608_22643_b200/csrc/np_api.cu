@@ -266,6 +266,18 @@ int check_config(const np_config* c, np_ctx* ctx) {
     return fail(ctx, NP_E_INVAL, "unknown record_format");
   if (c->record_format == NP_REC_INT8 && c->d_model % 16)
     return fail(ctx, NP_E_INVAL, "8-bit records need d_model % 16 == 0");
+  {
+    // batches the tensor-core predictor does not take (B <= 4, no tensor cores, or a width
+    // outside its K blocks) run the ring kernel, whose shared memory holds the batch's hidden
+    // vectors beside at least two stages of W2 rows
+    Dims pd = {};
+    pd.H = c->d_pred;
+    const bool tc = c->max_batch > 4 && !(c->flags & NP_F_NO_TENSOR_CORES) && pred_tc_supported(pd);
+    const int b_ring = tc ? 4 : c->max_batch;
+    if (b_ring >= 2 && !pred_l2_ring_fits(c->d_pred, b_ring))
+      return fail(ctx, NP_E_INVAL, "max_batch=%d with d_pred=%d: the hidden vectors of %d sequences do not fit the "
+                  "predictor kernel's shared memory", c->max_batch, c->d_pred, b_ring);
+  }
   return NP_OK;
 }
 
@@ -565,6 +577,18 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   ctx->mlp_tc = cfg->max_batch >= kTcMinBatch && !(cfg->flags & (NP_F_NO_TENSOR_CORES | NP_F_DIRECT_LOADS)) &&
                 mlp_tc_supported(d, ctx->sm_count);
   if (cfg->max_batch > 4 && !(cfg->flags & NP_F_NO_TENSOR_CORES)) pred_tc_prepare(d, b->w2, ctx->ws.hsplit, &ctx->tc);
+  {
+    // batches the tensor-core predictor does not take go through the ring kernel, whose shared
+    // memory holds the batch's hidden vectors beside at least two stages of W2 rows
+    const int b_ring = ctx->tc.ready ? std::min(cfg->max_batch, 4) : cfg->max_batch;
+    if (b_ring >= 2 && !pred_l2_ring_fits(d.H, b_ring)) {
+      np_destroy(ctx);
+      return fail(nullptr, NP_E_INVAL,
+                  "max_batch=%d with d_pred=%d: the hidden vectors of %d sequences do not fit the predictor kernel's "
+                  "shared memory%s", cfg->max_batch, d.H, b_ring,
+                  (cfg->flags & NP_F_NO_TENSOR_CORES) ? " (NP_F_NO_TENSOR_CORES is set)" : "");
+    }
+  }
   memset(ctx->host_lists, 0, host_lists_ints(*cfg) * 4);
   if (d.dense > 0 && cfg->max_batch > 1 && !ctx->mlp_tc) {
     np_destroy(ctx);

@@ -64,6 +64,8 @@ cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, in
                            cudaStream_t s);
 cudaError_t launch_pred_l2(const Dims& d, const void* w2, const float* hidden, int B, float* logits,
                            int32_t* status, cudaStream_t s, int sm_count);
+// whether the ring form of layer 2 (batches without the tensor-core kernel) has room for B hidden vectors of H values
+bool pred_l2_ring_fits(int H, int B);
 // Tensor-core form of predictor layer 2 for batches (np_predict_tc.cu).
 struct PredTcState {
   alignas(64) unsigned char map_w2[128];  // CUtensorMap of W2 [L*M][H]

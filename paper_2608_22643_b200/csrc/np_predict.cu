@@ -262,18 +262,36 @@ __global__ void __launch_bounds__(kL2Threads, 1) k_pred_l2(const uint4* __restri
   }
 }
 
+// Ring geometry of k_pred_l2 for rows of H values, B sequences and LPR lanes per row: a stage is
+// about 32 KB of whole rows (a multiple of the rows one pass of all consumer warps covers); the
+// hidden vectors of a batch sit beside the ring.  False when they and two stages do not fit.
+static bool l2_ring_plan(int H, int B, int lpr, int* stage_rows_out, int* n_stages_out) {
+  const long long row_bytes = (long long)H * 2;
+  const int pass_rows = kL2ConsumerWarps * (32 / lpr);
+  int stage_rows = (int)std::max<long long>(1, 32768 / row_bytes);
+  stage_rows = std::max(pass_rows, stage_rows / pass_rows * pass_rows);
+  const long long stage_bytes = stage_rows * row_bytes;
+  const long long hs_bytes = B > 1 ? (long long)B * H * 4 : 0;
+  const long long n = std::min<long long>(kL2MaxStages, (200 * 1024 - hs_bytes) / stage_bytes);  // signed: may be <= 0
+  if (n < 2) return false;
+  *stage_rows_out = stage_rows;
+  *n_stages_out = (int)n;
+  return true;
+}
+static int l2_ring_lpr(int chunks) { return chunks <= 1 ? 1 : chunks <= 2 ? 2 : chunks <= 4 ? 4 : chunks <= 96 ? 8 : chunks <= 128 ? 16 : 32; }
+
+bool pred_l2_ring_fits(int H, int B) {
+  int a, b;
+  return l2_ring_plan(H, B, l2_ring_lpr(H >> 3), &a, &b);
+}
+
 template <int LPR, int CPL>
 static cudaError_t l2_dispatch_nb(const uint4* w2, const float* hidden, float* logits, long long rows,
                                   int H, int B, int blocks, int32_t* status, cudaStream_t s) {
-  // stage: about 32 KB of whole rows, a multiple of the rows one pass of all consumer warps covers
-  const int row_bytes = H * 2;
-  const int pass_rows = kL2ConsumerWarps * (32 / LPR);
-  int stage_rows = std::max(1, 32768 / row_bytes);
-  stage_rows = std::max(pass_rows, stage_rows / pass_rows * pass_rows);
-  const size_t stage_bytes = (size_t)stage_rows * row_bytes;
+  int stage_rows = 0, n_stages = 0;
+  if (!l2_ring_plan(H, B, LPR, &stage_rows, &n_stages)) return cudaErrorInvalidValue;
+  const size_t stage_bytes = (size_t)stage_rows * H * 2;
   const size_t hs_bytes = B > 1 ? (size_t)B * H * 4 : 0;
-  int n_stages = (int)std::min<size_t>(kL2MaxStages, (200 * 1024 - hs_bytes) / stage_bytes);
-  if (n_stages < 2) return cudaErrorInvalidValue;
   const size_t sm = (size_t)n_stages * stage_bytes + hs_bytes;
 
   cudaLaunchConfig_t cfg = {};

@@ -93,11 +93,42 @@ int np_predict_logits_noalloc(const void* w1, const void* w2, const void* x_bf16
   d.H = d_pred;
   d.W = d_ffn / 32;
   d.Bmax = B;
-  cudaError_t e = npi::launch_pred_l1(d, w1, x_bf16, B, hidden, s);
+  // the status words start every call at zero (the array keeps the last call's contents), so
+  // that np_noalloc_check reports only what this call's kernels recorded
+  cudaError_t e = cudaMemsetAsync(status, 0, kStatusInts * sizeof(int32_t), s);
+  if (e == cudaSuccess) e = npi::launch_pred_l1(d, w1, x_bf16, B, hidden, s);
   if (e == cudaSuccess) e = npi::launch_pred_l2(d, w2, hidden, B, logits_out, status, s, sm_count);
   if (e != cudaSuccess) {
     snprintf(g_err, sizeof g_err, "kernel launch failed: %s", cudaGetErrorString(e));
     return NP_E_CUDA;
+  }
+  return NP_OK;
+}
+
+int np_noalloc_check(void* stream) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return fail(NP_E_CUDA, "cudaGetDevice failed");
+  if (dev < 0 || dev >= kMaxDevices) return fail(NP_E_INVAL, "device ordinal above 63");
+  float* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    scratch = g_scratch_addr[dev];
+  }
+  if (!scratch) return fail(NP_E_STATE, "np_predict_logits_noalloc has not run on this device");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t word = 0;  // on the caller's stack: nothing is allocated
+  cudaError_t e = cudaMemcpyAsync(&word, scratch, sizeof word, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) {
+    snprintf(g_err, sizeof g_err, "reading the status word failed: %s", cudaGetErrorString(e));
+    return NP_E_CUDA;
+  }
+  if (word != 0) {
+    snprintf(g_err, sizeof g_err,
+             "the last np_predict_logits_noalloc on this device recorded status 0x%x (a bounded wait ran out): "
+             "its logits are incomplete",
+             (unsigned)word);
+    return NP_E_DEVICE;
   }
   return NP_OK;
 }

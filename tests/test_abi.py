@@ -85,6 +85,22 @@ def test_bad_config_is_rejected(lib, field, value):
     assert nb.np_last_error(None)
 
 
+def test_batches_whose_hidden_vectors_do_not_fit_are_rejected(lib):
+    """Sixteen sequences of 4096 hidden values need 256 KB beside the ring of the plain-core
+    predictor kernel: refused at configuration time, not at the first np_predict."""
+    cfg = nb.make_config(2, 256, 1024, 4096, 102, 205, max_batch=16, flags=nb.NP_F_NO_TENSOR_CORES)
+    with pytest.raises(nb.NpError) as e:
+        nb.np_query_sizes(cfg)
+    assert e.value.code == nb.NP_E_INVAL and "do not fit" in str(e.value)
+    cfg.flags = 0                                    # the tensor-core kernel takes B > 4; the ring sees at most 4
+    nb.np_query_sizes(cfg)
+    cfg.flags = nb.NP_F_NO_TENSOR_CORES
+    cfg.max_batch = 4
+    nb.np_query_sizes(cfg)
+    cfg.max_batch, cfg.d_pred = 16, 2048             # 128 KB of hidden vectors + two 32 KB stages
+    nb.np_query_sizes(cfg)
+
+
 def test_file_mode_config_rules(lib):
     cfg = nb.make_config(2, 256, 1024, 64, 102, 205, transfer_mode=nb.NP_XFER_FILE, io_depth=256)
     assert nb.np_query_sizes(cfg).record_bytes == 1536

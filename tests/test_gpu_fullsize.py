@@ -65,15 +65,19 @@ def test_7b_shape_steps_match_oracle(policy):
         p.close()
 
 
-@pytest.mark.parametrize("name,n_layers,mode", [
-    ("13b", 3, nb.NP_XFER_HOST_GATHER), ("70b", 2, nb.NP_XFER_ZERO_COPY), ("70b", 2, nb.NP_XFER_MEMCPY_RUNS),
+@pytest.mark.parametrize("name,n_layers,mode,chain_layers", [
+    ("13b", 3, nb.NP_XFER_HOST_GATHER, 0), ("70b", 2, nb.NP_XFER_ZERO_COPY, 0), ("70b", 2, nb.NP_XFER_MEMCPY_RUNS, 0),
+    # several layers per resident launch (the cross-layer hand-over of x at these row widths)
+    ("13b", 4, nb.NP_XFER_HOST_GATHER, 4), ("13b", 4, nb.NP_XFER_ZERO_COPY, 2),
+    ("70b", 4, nb.NP_XFER_ZERO_COPY, 4), ("70b", 4, nb.NP_XFER_HOST_GATHER, 2),
 ])
-def test_larger_shapes_few_layers(name, n_layers, mode):
+def test_larger_shapes_few_layers(name, n_layers, mode, chain_layers):
     """The 13B- and 70B-shaped rows (D = 5120 / 8192, M = 13824 / 28672) on a few layers:
-    other ring depths, column rounds and segment splits than the 7B shape."""
+    other ring depths, column rounds and segment splits than the 7B shape, with one and with
+    several layers per resident launch."""
     cfg = synth.CONFIGS[name].with_(n_layers=n_layers)
     L, M, D, W = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_ffn // 32
-    p = Pair(cfg, transfer_mode=mode, flags=nb.NP_F_CHECK_BOUNDS, gen_device="cuda")
+    p = Pair(cfg, transfer_mode=mode, flags=nb.NP_F_CHECK_BOUNDS, gen_device="cuda", chain_layers=chain_layers)
     try:
         xs = synth.hidden_states(cfg, 3)
         logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")

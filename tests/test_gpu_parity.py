@@ -350,11 +350,11 @@ def test_predictor_widths_and_row_counts(H, L, M):
     ("min_all", 1, 8, 32, 8, 10, 20),            # smallest legal sizes
 ])
 @pytest.mark.parametrize("B", [1, 3])
-def test_limit_shapes(shape, B):
+def test_limit_shapes(shape, B, chain_layers=0):
     """The extreme sizes np_init accepts run the whole path and match the oracle."""
     name, L, D, M, H, dens, cap = shape
     cfg = synth.StackConfig(name, L, D, M, H, dens, cap, 3, 31, 0.9)
-    p = Pair(cfg, max_batch=B, k=max(1, cfg.top_k), C=max(2, cfg.capacity))
+    p = Pair(cfg, max_batch=B, k=max(1, cfg.top_k), C=max(2, cfg.capacity), chain_layers=chain_layers)
     try:
         xs = synth.hidden_states(cfg, 3, batch=B)
         out = torch.empty((B, D), dtype=torch.float32, device="cuda")
@@ -371,6 +371,13 @@ def test_limit_shapes(shape, B):
         p.check_resident_bytes()
     finally:
         p.close()
+
+
+@pytest.mark.parametrize("chain_layers", [2, 4])
+def test_widest_model_with_several_layers_per_launch(chain_layers):
+    """D = 16384 on four layers, two and four of them per resident launch: x is handed from
+    layer to layer inside the kernel at the widest row the library accepts."""
+    test_limit_shapes(("max_model_chain", 4, 16384, 64, 64, 25, 50), 1, chain_layers=chain_layers)
 
 
 def test_bounded_wait_times_out_and_context_survives():

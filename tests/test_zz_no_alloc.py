@@ -1,4 +1,4 @@
-"""The allocation-free predictor entry point gives np_predict's logits.
+"""The allocation-free predictor entry point gives the oracle's (and np_predict's) logits.
 
 Collected last on purpose (file name): a failure here cannot hide the result of
 any other test in a run that stops at the first failure.
@@ -10,18 +10,23 @@ import torch
 from paper_2608_22643_b200 import binding as nb
 from paper_2608_22643_b200 import build as nbuild
 from paper_2608_22643_b200 import synth
-from tests.harness import Pair, rel_l2
+from oracle import np_oracle as O
+from tests.harness import Pair, rel_l2, u16
 
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,B", [("small", 1), ("small", 3)])
-def test_noalloc_predictor_matches_context_path_twice(name, B):
+_WIDE = synth.StackConfig("noalloc_wide", 2, 256, 1024 + 32, 2048, 10, 20, 4, 13, 0.9)   # B = 1 takes the ring kernel
+_FULL = synth.StackConfig("noalloc_full", 2, 512, 2048 + 32, 1024, 10, 20, 4, 17, 0.9)   # 16 x 1024 = the whole scratch
+
+
+@pytest.mark.parametrize("cfg,B", [(synth.CONFIGS["small"], 1), (synth.CONFIGS["small"], 3), (_WIDE, 1), (_FULL, 16)])
+def test_noalloc_predictor_matches_context_path_twice(cfg, B):
     """Callers that cannot allocate device memory (pool-owned memory, allocation-free decode
     loops) use np_predict_logits_noalloc; two calls in a row on the library's fixed scratch
-    must both reproduce what np_predict computes with its workspace."""
-    cfg = synth.CONFIGS[name]
-    p = Pair(cfg, max_batch=B, with_oracle=False)
+    must both reproduce the oracle's predictor within tolerance and, bit for bit, what
+    np_predict computes with its workspace on the same plain-core kernels."""
+    p = Pair(cfg, max_batch=B, with_oracle=False, flags=nb.NP_F_CHECK_BOUNDS | nb.NP_F_NO_TENSOR_CORES)
     try:
         L, M, D, H = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_pred
         xs = synth.hidden_states(cfg, 2, batch=B)
@@ -32,9 +37,12 @@ def test_noalloc_predictor_matches_context_path_twice(name, B):
             nb.np_predict(p.eng.ctx, x, B, want, None, p.eng.stream)
             p.eng.stream.synchronize()
             nb.np_predict_logits_noalloc(p.eng.w1, p.eng.w2, x, B, L, D, M, H, got, p.eng.stream)
-            p.eng.stream.synchronize()
-            assert rel_l2(got.cpu().numpy(), want.cpu().numpy()) < 1e-5
+            assert nb.np_noalloc_check(p.eng.stream) == nb.NP_OK      # no bounded wait ran out
+            z = O.predict(u16(p.w1_cpu), u16(p.w2_cpu), u16(xs[t]), L, M)
+            assert rel_l2(got.cpu().numpy(), z) < 1e-5
             assert np.isfinite(got.cpu().numpy()).all()
+            assert torch.equal(got, want)
+            got.fill_(float("nan"))
     finally:
         p.close()
 
