@@ -197,6 +197,8 @@ struct np_ctx {
   Pool* pool = nullptr;
   RecordReader reader;   // NP_XFER_FILE: reads of the store file
   PredTcState tc = {};
+  chain_slices::State slices = {};  // column-sliced resident MLP kernel: its counters, exchange words and their values
+  bool use_slices = false;
   size_t gu_bytes = 0;   // both dot-product accumulators of the batch MLP, contiguous
   bool mlp_tc = false;   // batches run the tensor-core MLP kernels
   std::string err;
@@ -252,7 +254,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->transfer_mode == NP_XFER_FILE && c->record_format != NP_REC_BF16)
     return fail(ctx, NP_E_INVAL, "NP_XFER_FILE needs NP_REC_BF16 records");
   if (c->io_depth < -1 || c->io_depth > 4096) return fail(ctx, NP_E_INVAL, "io_depth must be in [-1, 4096]");
-  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES | NP_F_MAPPED_STAGING)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
+  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES | NP_F_MAPPED_STAGING | NP_F_ROW_CHAIN)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
   if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
@@ -500,6 +502,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_ovf = take(LM), o_cnt = take((size_t)d.L * NP_N_COUNTERS), o_free = take(LC);
   const size_t o_cid = take(LC), o_ckey = take(LC), o_pred = take(LW), o_stat = take(4), o_bar = take(4);
   const size_t o_ident = take(d.dense > 0 ? (size_t)d.M : 1);
+  const size_t o_sbar = take(chain_slices::bar_words()), o_sxch = take(2 * chain_slices::xch_words(d, ctx->sm_count));
   NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
   char* base = static_cast<char*>(ctx->slab);
   Tables& t = ctx->t;
@@ -521,6 +524,12 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   t.status = reinterpret_cast<int32_t*>(base + o_stat);
   t.grid_bar = reinterpret_cast<unsigned int*>(base + o_bar);
   t.identity = reinterpret_cast<int32_t*>(base + o_ident);
+  ctx->slices.bars = reinterpret_cast<unsigned int*>(base + o_sbar);
+  ctx->slices.xch = reinterpret_cast<unsigned long long*>(base + o_sxch);
+  ctx->slices.bar_base = ctx->slices.seq_base = 0;
+  NP_INIT_CUDA(cudaMemset(ctx->slices.bars, 0, chain_slices::bar_words() * 4));
+  NP_INIT_CUDA(cudaMemset(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8));
+  ctx->use_slices = !(cfg->flags & NP_F_ROW_CHAIN) && chain_slices::supported(d, ctx->sm_count);
 
   const WsLayout wl = ws_layout(*cfg);
   char* wsb = static_cast<char*>(b->workspace);
@@ -639,6 +648,10 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
 int np_reset(np_ctx* ctx, void* stream) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   NP_LAUNCH(ctx, launch_tables_reset(ctx->d, ctx->t, as_stream(stream)));
+  // a launch that gave up may have left the sliced kernel's counters and stamps anywhere
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.bars, 0, chain_slices::bar_words() * 4, as_stream(stream)));
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8, as_stream(stream)));
+  ctx->slices.bar_base = ctx->slices.seq_base = 0;
   ctx->have_delta = ctx->have_pred = ctx->have_step = false;
   std::fill(ctx->install_pending.begin(), ctx->install_pending.end(), 0);
   ctx->step = 0;
@@ -1152,7 +1165,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   const Dims& d = ctx->d;
   const size_t n = (size_t)B * d.D;
   const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
-                          mlp_chain_supported(d, ctx->sm_count);
+                          (ctx->use_slices || mlp_chain_supported(d, ctx->sm_count));
   const bool tc_batch = !persistent && ctx->mlp_tc && B >= kTcMinBatch && !(ctx->cfg.flags & NP_F_DIRECT_LOADS);
   if (part != kChainTail) {
     NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
@@ -1210,7 +1223,10 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
         if (ctx->install_pending[l]) NP_CUDA(ctx, wait_install(ctx, l, s));
       a.l_begin = l0;
       a.l_end = l1;
-      NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
+      if (ctx->use_slices)
+        NP_LAUNCH(ctx, chain_slices::launch(d, a, &ctx->slices, s, ctx->sm_count));
+      else
+        NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
     }
   } else {
     if (part != kChainTail && ctx->mlp_tc && B >= kTcMinBatch)

@@ -168,6 +168,25 @@ bool supported(const Dims& d, int sm_count);
 cudaError_t launch(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
 }  // namespace chain_alu
 
+namespace chain_slices {  // column-sliced resident form for one sequence (np_mlp_slices.cu); same hand-over of x
+struct Plan {
+  int R, ks, vg_shift, gw_shift, ng, window, run_layers, slot_cache_rows, max_rows, xch_stride;
+  size_t group_bytes, smem;
+};
+// Library-owned device words and the host's running record of them: the arrival counters and
+// the exchange stamps only ever grow, so nothing has to be cleared between launches.
+struct State {
+  unsigned int* bars;       // [bar_words()] zero at init / reset
+  unsigned long long* xch;  // [xch_words(d, sm_count)] zero at init / reset
+  unsigned int bar_base, seq_base;
+};
+bool plan(const Dims& d, int sm_count, Plan* p);
+bool supported(const Dims& d, int sm_count);
+size_t xch_words(const Dims& d, int sm_count);
+size_t bar_words();
+cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s, int sm_count);
+}  // namespace chain_slices
+
 cudaError_t launch_selftest_wait(int32_t* status, cudaStream_t s);
 cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s);
 // out = a + sum of `reps` consecutive copies of b (each n floats)
