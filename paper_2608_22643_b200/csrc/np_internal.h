@@ -14,7 +14,10 @@ namespace npi {
 constexpr int kMaxBatch = 16;
 constexpr int kHostHeaderInts = 16;
 constexpr float kRmsEps = 1e-6f;  // x / sqrt(mean(x^2) + eps) in front of every MLP of the chain
-constexpr int kZRep = 4;  // copies of each MLP accumulator vector (spreads same-address adds)  // global header of the host list mirror
+#ifndef NP_ZREP
+#define NP_ZREP 4
+#endif
+constexpr int kZRep = NP_ZREP;  // copies of each MLP accumulator vector (spreads same-address adds)  // global header of the host list mirror
 
 // Device-resident tables and lists of all layers (one slab, library-owned).
 struct Tables {

@@ -89,6 +89,8 @@ struct KArgs {
 
 #ifdef NP_TRACE  // development builds only: time stamps of four blocks, read back by np_debug_trace
 __device__ unsigned long long np_trace_buf[4][64][32];
+__device__ unsigned long long np_trace_all[160][8][8];
+extern "C" int np_debug_trace_all(void* out) { return (int)cudaMemcpyFromSymbol(out, np_trace_all, sizeof(np_trace_all)); }
 __device__ __forceinline__ unsigned long long gtime() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -101,6 +103,7 @@ extern "C" int np_debug_clk(void* out) { return (int)cudaMemcpyFromSymbol(out, n
   do {                                                                                                    \
     const int tb__ = blockIdx.x < 4 ? (int)blockIdx.x : -1;                                               \
     if (threadIdx.x == 0 && tb__ >= 0 && li < 64 && (slot) < 32) np_trace_buf[tb__][li][slot] = gtime();  \
+    if (threadIdx.x == 0 && blockIdx.x < 160 && li < 8 && (slot) < 8) np_trace_all[blockIdx.x][li][slot] = gtime(); \
   } while (0)
 extern "C" int np_debug_trace(void* out) { return (int)cudaMemcpyFromSymbol(out, np_trace_buf, sizeof(np_trace_buf)); }
 #else
@@ -759,7 +762,7 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   if (fixed + 3 * group_bytes > budget) return false;
   int ng = (int)std::min<size_t>(kMaxGroups, (budget - fixed) / group_bytes);
   if (d.ring_stages >= 2) ng = std::max(3, std::min(ng, d.ring_stages));
-  int window = std::max(1, std::min(ng - 1, (int)((72 * 1024 + group_bytes / 2) / group_bytes)));
+  int window = std::max(1, std::min(ng - 1, (int)(40 * 1024 / group_bytes)));
 #ifdef NP_TUNE  // development builds only: geometry from the environment
   if (const char* e = getenv("NP_SL_NG")) ng = std::max(2, std::min(ng, atoi(e)));
   if (const char* e = getenv("NP_SL_WIN")) window = std::min(atoi(e), std::min(kHist - 1, ng - 1));
