@@ -38,6 +38,11 @@ from paper_2608_22643_b200 import synth  # noqa: E402
 METRIC = "decode steps/s (predict+delta+install+sparse MLP, 7B shape)"
 UNIT = "steps/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per layer (dram__bytes_read.sum + dram__bytes_write.sum of one launch / its layers) of the
+# sparse-MLP kernels, from the ncu captures summarised under profiles/: (kernel, config) -> (bytes, file)
+NCU_TRAFFIC = {
+    ("k_mlp_chain", "7b"): (27.52e6, "profiles/k_mlp_chain_7b.md"),
+}
 
 
 def parse_args():
@@ -62,6 +67,12 @@ def parse_args():
     ap.add_argument("--direct-loads", action="store_true", help="MLP rows by plain global loads")
     ap.add_argument("--chain-layers", type=int, default=0, help="layers per resident MLP kernel")
     ap.add_argument("--capacity-pct", type=int, default=None, help="resident capacity in percent of FFN rows")
+    ap.add_argument("--store-layers", default="auto",
+                    help="layers of records the host store holds (layer l reads layer l mod this); 'auto' = all of them "
+                         "unless the host cannot hold and pin the whole store, 0 = all")
+    ap.add_argument("--min-timed-steps", type=int, default=240,
+                    help="the timed region repeats the K steps (the sequence simply continues) until it spans at "
+                         "least this many; ms_per_step is the mean over all of them")
     ap.add_argument("--batch", type=int, default=1, help="sequences per step (the metric's workload is 1)")
     ap.add_argument("--gamma", type=float, default=0.9, help="shared-driver weight of batched hidden states")
     ap.add_argument("--host-threads", type=int, default=0, help="threads packing records (gather transfer)")
@@ -164,10 +175,43 @@ def oracle_threads() -> int:
         return 1
 
 
-def make_workload(cfg, gen_device: str, pin: bool):
+def host_mem_available() -> int:
+    try:
+        with open("/proc/meminfo") as f:
+            for line in f:
+                if line.startswith("MemAvailable:"):
+                    return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
+
+
+def plan_store_layers(cfg, requested: str, world: int):
+    """Layers of records the host store holds.  'auto': the whole stack when a host of this size can hold
+    and pin it beside everything else (at most half of what is available, per replica), else as many
+    layers as that allows; the stack then reads layer l mod Lp (shapes and traffic unchanged)."""
+    L = cfg.n_layers
+    if requested != "auto":
+        n = int(requested)
+        return (L if n <= 0 else min(L, n)), "requested"
+    layer_bytes = cfg.d_ffn * cfg.record_bytes
+    avail = host_mem_available()
+    if avail <= 0 or L * layer_bytes <= avail // (2 * max(1, world)):
+        return L, "whole store"
+    return max(1, min(L, int(avail // (2 * max(1, world)) // layer_bytes))), f"host has {avail / 2**30:.0f} GiB available"
+
+
+def make_workload(cfg, gen_device: str, pin: bool, store_layers=None):
     """Weights (CPU + generator device), the record store on the host, hidden states."""
     t0 = time.time()
     w1, w2 = synth.predictor_weights(cfg, gen_device)
+    if store_layers is not None and store_layers < cfg.n_layers:
+        store = torch.empty((store_layers, cfg.d_ffn, 3, cfg.d_model), dtype=torch.bfloat16)
+        if pin:
+            from paper_2608_22643_b200 import binding as nb
+            nb.pin_host_tensor(store)
+        synth.fill_backing_store(cfg.with_(n_layers=store_layers), store, gen_device)
+        return w1, w2, store, time.time() - t0
     store = torch.empty((cfg.n_layers, cfg.d_ffn, 3, cfg.d_model), dtype=torch.bfloat16)
     if pin:
         from paper_2608_22643_b200 import binding as nb
@@ -310,9 +354,15 @@ def cuda_arm(args):
         args.dense_layers = nb.np_plan_dense_prefix(plan_cfg, int(args.budget_gib * 2**30), 0)
         if args.dense_layers < 0:
             raise SystemExit("bench.py: the budget does not even hold the sparse layers' resident buffers")
-    w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True)
+    Lp, lp_why = plan_store_layers(cfg, args.store_layers, int(os.environ.get("LOCAL_WORLD_SIZE", world)))
+    if Lp < cfg.n_layers and (args.transfer == "file" or args.dense_layers > Lp):
+        raise SystemExit("bench.py: an aliased store is not combined with --transfer file or a longer dense prefix here")
+    w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True, store_layers=Lp)
+    # replicas share one host: the packing threads of the gather transfer are divided among them
+    if args.host_threads == 0 and world > 1:
+        args.host_threads = nb.replica_host_threads(int(os.environ.get("LOCAL_WORLD_SIZE", world)))
     if args.records == "int8":
-        qstore = torch.empty((cfg.n_layers, cfg.d_ffn, 3 * cfg.d_model + 16), dtype=torch.uint8)
+        qstore = torch.empty((Lp, cfg.d_ffn, 3 * cfg.d_model + 16), dtype=torch.uint8)
         nb.pin_host_tensor(qstore)
         qstore = synth.quantize_store(store, device="cuda", out=qstore)
         nb.unpin_host_tensor(store)                    # the bf16 store is not used any more
@@ -322,6 +372,7 @@ def cuda_arm(args):
                           max_batch=args.batch, evict_policy=policy, transfer_mode=mode,
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
                           host_threads=args.host_threads, dense_layers=args.dense_layers, io_depth=args.io_depth,
+                          store_layers=Lp if Lp < cfg.n_layers else 0,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0)
                           | (nb.NP_F_MAPPED_STAGING if args.mapped_staging else 0))
@@ -357,7 +408,9 @@ def cuda_arm(args):
     L, D, M = cfg.n_layers, cfg.d_model, cfg.d_ffn
     rec = cfg.record_bytes                             # resident (bf16) bytes of a record
     rec_store = 3 * D + 16 if args.records == "int8" else rec   # bytes of a record in the store
-    T = 1 + W + K                                      # cold start + warm-up + timed
+    reps_timed = max(1, -(-args.min_timed_steps // K))   # the K steps are repeated until the timed region is long enough
+    KT = K * reps_timed
+    T = 1 + W + KT                                     # cold start + warm-up + timed
     n_detail = 16
     Bq = args.batch
     xs_host = synth.hidden_states(cfg, T + n_detail, batch=Bq, gamma=args.gamma).pin_memory()  # [T + n_detail, B, D] bf16
@@ -510,14 +563,9 @@ def cuda_arm(args):
     if args.layer_launches or args.direct_loads or Bq > 1:
         chain_layers = 1
     n_launch = -(-L // chain_layers)                                # MLP kernel launches per chain
-    if chain_layers > 1:
-        mlp_kernel = "k_mlp_chain"
-    elif args.direct_loads:
-        mlp_kernel = "k_sparse_mlp"
-    elif Bq > 1:
-        mlp_kernel = "k_mlp_tc_up + k_mlp_tc_down (the two launches of one layer)"
-    else:
-        mlp_kernel = "k_sparse_mlp_pipe"
+    mlp_kernel = nb.np_mlp_kernel_name(eng.ctx, Bq)       # the kernel the library chose for this shape and batch
+    if Bq > 1:
+        mlp_kernel += " (the two launches of one layer)"
     mlp_us = k0.elapsed_time(k1) * 1000.0 / (reps * n_launch)      # per launch, gaps included
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record(s)
@@ -546,9 +594,10 @@ def cuda_arm(args):
         mlp_bytes = nd * (M * rec + 8 * D) + (L - nd) * layer_bytes
         mlp_kernel = "whole MLP chain (dense prefix + sparse layers)"
     achieved = mlp_bytes / (mlp_us * 1e-6) / 1e9
-    # DRAM bytes of one layer from the ncu capture in profiles/k_mlp_chain_7b.md (7B shape):
-    # (216.63 MB read + 3.51 MB written) / 8 layers; scaled by the layers a launch spans
-    traffic = 27.52e6 * L / n_launch if cfg.name == "7b" and not nd else None
+    # DRAM bytes per layer of the dominant kernel from its ncu capture, by kernel and shape; a kernel or
+    # shape without a capture reports null rather than another kernel's figure
+    per_layer, traffic_src = NCU_TRAFFIC.get((mlp_kernel, cfg.name), (None, None))
+    traffic = per_layer * L / n_launch if per_layer is not None and not nd else None
     pred_rows = L * 2 * args.centroids if centroid else L * M
     pred_bytes = 2 * cfg.d_pred * D + 2 * pred_rows * cfg.d_pred + 4 * pred_rows
     if trunk:   # every matrix of the predictor once, plus the logits
@@ -556,8 +605,8 @@ def cuda_arm(args):
                           + sum(b[0].numel() + b[4].numel() for b in tw["blocks"])) + 4 * pred_rows
     mean_delta = float(np.mean(delta_rows))
     result = {
-        "metric": METRIC, "value": K * world / (ms_total / 1000.0), "unit": UNIT, "n_gpus": world,
-        "steps": K, "warmup": W, "ms_per_step": ms_total / K, "higher_is_better": True,
+        "metric": METRIC, "value": KT * world / (ms_total / 1000.0), "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": W, "ms_per_step": ms_total / KT, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": f"{cfg.name}: L={L} D={D} M={M} H={cfg.d_pred} k={cfg.top_k} C={cfg.capacity} "
@@ -572,15 +621,21 @@ def cuda_arm(args):
             "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
             "active_rows_per_layer": n_active, "active_rows_max": active_max, "overflow_steps": int(overflow_steps),
             "replicas": world,
+            "timed_steps": KT,   # --steps repeated (the sequence continues) so that the timed region is not a few ms
+            "store": (f"host store holds all {L} layers" if Lp == L else
+                      f"host store aliased over {Lp} of {L} layers (layer l reads layer l mod {Lp}; {lp_why}); shapes, "
+                      f"rows and bytes per step are those of the {L}-layer stack"),
+            "host_threads": int(args.host_threads),
         },
-        "e2e": {"value": K * world / (e2e_ms_total / 1000.0), "unit": UNIT,
+        "e2e": {"value": KT * world / (e2e_ms_total / 1000.0), "unit": UNIT,
                 "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * (L - nd) * rec_store + (trunk_in_bytes if trunk else 0)),
                 "d2h_bytes_per_step": int(Bq * D * 4)},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": mlp_kernel, "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind + " copy bandwidth (burst)",
-                     "traffic": traffic, "us_per_launch": mlp_us, "bytes_per_launch": mlp_bytes,
+                     "traffic": traffic, "traffic_source": traffic_src if traffic is not None else None,
+                     "us_per_launch": mlp_us, "bytes_per_launch": mlp_bytes,
                      "layers_per_launch": L / n_launch},
         "stages_us": {"predict_topk": fnum(stage_us[0]), "delta": fnum(stage_us[1]),
                       "install_copy_stream": fnum(stage_us[2]), "mlp_chain_incl_waits": fnum(stage_us[3]),
@@ -602,33 +657,83 @@ def cuda_arm(args):
         storage["read_gbs_during_install"] = mean_delta * (L - nd) * rec / (float(stage_us[2]) * 1e-6) / 1e9
         result["storage"] = storage
 
-    # ---- the same step with the other pinned-host transfer mode (reported beside, not as, the value) ----
+    # ---- pinned host -> device copy rate of this machine, measured in the run: the ceiling of the install stage ----
+    h2d_gbs = None
+    if store is not None:
+        probe_bytes = int(min(256 << 20, store.numel() * store.element_size()))
+        probe_src = store.view(torch.uint8).view(-1)[:probe_bytes]        # the head of the pinned store, contiguous
+        probe_dst = torch.empty(probe_bytes, dtype=torch.uint8, device=dev)
+        best = float("inf")
+        for _ in range(4):
+            h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            h0.record(s)
+            with torch.cuda.stream(s):
+                probe_dst.copy_(probe_src, non_blocking=True)
+            h1.record(s)
+            s.synchronize()
+            best = min(best, h0.elapsed_time(h1))
+        h2d_gbs = probe_bytes / (best * 1e-3) / 1e9
+        del probe_dst
+        install_bytes = mean_delta * (L - nd) * rec_store
+        inst_us = float(stage_us[2])
+        if inst_us > 0:
+            result["roofline_install"] = {
+                "bound": "pcie", "achieved": install_bytes / (inst_us * 1e-6) / 1e9, "peak": h2d_gbs, "unit": "GB/s",
+                "frac": install_bytes / (inst_us * 1e-6) / 1e9 / h2d_gbs,
+                "peak_kind": f"one contiguous {probe_bytes >> 20} MiB copy from the pinned store, best of 4, in this run",
+                "bytes_per_step": install_bytes, "us_per_step": inst_us,
+                "note": "the step's bound: scattered records of REC bytes cross to the device while the GPU work "
+                        "(compute_only) takes a fraction of the step"}
+
+    # ---- the same step in other settings (reported beside, not as, the value) ----
     if (args.transfer == "gather" and not args.no_variants and not centroid and Bq == 1
             and args.config == "7b" and not (args.layer_launches or args.direct_loads) and not args.dense_layers
-            and args.records == "bf16" and world == 1):
+            and args.records == "bf16" and world == 1 and args.policy == "exact"):
         eng.close()
-        zcfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity,
-                              max_batch=Bq, evict_policy=policy, transfer_mode=nb.NP_XFER_ZERO_COPY,
-                              chain_layers=args.chain_layers)
-        eng = nb.Engine(zcfg, w1, w2, store, device=dev)
-        s, cs = eng.stream, eng.copy_stream
-        for t in range(0, 1 + W):
-            nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
-        barrier()
-        z0, z1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        z0.record(s)
-        for t in range(1 + W, T):
-            nb.np_step(eng.ctx, xs_dev[t], Bq, out, s, cs)
-        z1.record(s)
-        barrier()
-        eng.counters()
-        (z_ms,) = max_over_ranks(dist, [z0.elapsed_time(z1)], dev)
-        result["variants"] = {"transfer=zerocopy": {
-            "value": K * world / (z_ms / 1000.0), "unit": UNIT, "ms_per_step": z_ms / K,
-            "note": "scatter kernel reads the pinned store over PCIe by neuron ID; no host packing, no staging copy"}}
+
+        def variant(note, vstore=None, **kw):
+            vkw = dict(max_batch=Bq, evict_policy=policy, transfer_mode=mode, staging_rows=2 * cfg.top_k,
+                       chain_layers=args.chain_layers, host_threads=args.host_threads,
+                       store_layers=Lp if Lp < cfg.n_layers else 0)
+            vkw.update(kw)
+            vcfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, cfg.top_k, cfg.capacity, **vkw)
+            veng = nb.Engine(vcfg, w1, w2, store if vstore is None else vstore, device=dev)
+            vs, vcs = veng.stream, veng.copy_stream
+            for t in range(0, 1 + W):
+                nb.np_step(veng.ctx, xs_dev[t], Bq, out, vs, vcs)
+            barrier()
+            z0, z1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            z0.record(vs)
+            for t in range(1 + W, T):
+                nb.np_step(veng.ctx, xs_dev[t], Bq, out, vs, vcs)
+            z1.record(vs)
+            barrier()
+            cnt = veng.counters()
+            veng.close()
+            (z_ms,) = max_over_ranks(dist, [z0.elapsed_time(z1)], dev)
+            return {"value": KT * world / (z_ms / 1000.0), "unit": UNIT, "ms_per_step": z_ms / KT,
+                    "delta_rows_per_layer": float(cnt[:, nb.NP_CNT_DELTA].mean()), "note": note}
+
+        result["variants"] = {
+            "transfer=zerocopy": variant("scatter kernel reads the pinned store over PCIe by neuron ID; no host packing, "
+                                         "no staging copy", transfer_mode=nb.NP_XFER_ZERO_COPY),
+            "policy=lru": variant("rows stay resident while capacity allows (least recently predicted leave first): "
+                                  "fewer incoming rows per step than under Eq. 3's exact replacement",
+                                  evict_policy=nb.NP_EVICT_LRU),
+        }
+        qstore = torch.empty((store.shape[0], cfg.d_ffn, 3 * cfg.d_model + 16), dtype=torch.uint8)
+        nb.pin_host_tensor(qstore)
+        qstore = synth.quantize_store(store, device="cuda", out=qstore)
+        result["variants"]["records=int8"] = variant(
+            "8-bit row records (int8 rows + fp32 scales), dequantised to bf16 at install: half the bytes cross to the "
+            "device; a different workload (the weights are the dequantised ones)", vstore=qstore,
+            record_format=nb.NP_REC_INT8)
+        nb.unpin_host_tensor(qstore)
+        del qstore
+        eng = None
 
     if (rank == 0 and not args.no_cpu_baseline and world == 1 and Bq == 1 and not centroid and not args.dense_layers
-            and args.records == "bf16" and store is not None):
+            and args.records == "bf16" and store is not None and Lp == cfg.n_layers):
         n = args.cpu_baseline_steps
         times = run_oracle_steps(cfg, args.policy, w1.cpu(), w2.cpu(), store, xs_host, n)
         sec = float(np.mean(times))
@@ -637,7 +742,8 @@ def cuda_arm(args):
             "sample": f"{n} steady-state decode steps of the same stack (all {L} layers), after an untimed cold start"}
     elif rank == 0:
         result["cpu_baseline"] = None
-    eng.close()
+    if eng is not None:
+        eng.close()
     if storage is not None and not args.store_path:
         os.remove(storage["path"])
     if rank == 0:

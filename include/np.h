@@ -147,14 +147,17 @@ typedef struct np_config {
   int32_t record_format;  /* NP_REC_*: how the store holds a record */
   int32_t io_depth;       /* NP_XFER_FILE: reads in flight (0 = 256, the paper's queue depth;
                              < 0 = no io_uring, blocking preads from the host threads) */
-  int32_t reserved;       /* 0 */
+  int32_t store_layers;   /* Lp, 0 or 1 <= Lp <= L: the store holds Lp layers of records and layer l reads
+                             layer l mod Lp of it (0 = L, every layer its own).  For stacks whose whole
+                             store the host cannot hold or pin: shapes, row counts and traffic per step
+                             stay those of the L-layer stack */
 } np_config;
 
 /* Byte counts of the caller-owned buffers for a configuration. */
 typedef struct np_sizes {
   uint64_t w1_bytes;          /* bf16 [H][D] */
   uint64_t w2_bytes;          /* bf16 [L*M][H] */
-  uint64_t backing_bytes;     /* [L][M] records of REC bytes (bf16 [L][M][3][D] with NP_REC_BF16) */
+  uint64_t backing_bytes;     /* [Lp][M] records of REC bytes (bf16 [L][M][3][D] with NP_REC_BF16 and store_layers = 0) */
   uint64_t row_buffer_bytes;  /* bf16 [L - d][C][D], each of gate / up / downT (sparse layers only) */
   uint64_t staging_bytes;     /* staging_rows * REC (device; pinned host too for HOST_GATHER) */
   uint64_t workspace_bytes;   /* device scratch */
@@ -370,6 +373,11 @@ int np_export_state(np_ctx* ctx, int32_t layer, int32_t* slot_map, int32_t* owne
  * step counter; the caller vouches for their consistency.  Synchronises. */
 int np_import_state(np_ctx* ctx, int32_t layer, const int32_t* slot_map, const int32_t* owner,
                     const uint32_t* resident, const int32_t* stamp, int32_t step, void* stream);
+
+/* Name of the kernel np_mlp_chain / np_step run the sparse layers' MLP with for B sequences in this
+ * context (a static string: "k_mlp_slices", "k_mlp_chain", "k_mlp_chain_alu", "k_mlp_tc_up + k_mlp_tc_down",
+ * "k_sparse_mlp_pipe" or "k_sparse_mlp").  For reports; NULL if ctx is NULL or B is out of range. */
+const char* np_mlp_kernel_name(np_ctx* ctx, int32_t B);
 
 /* Timing of the last np_step in microseconds, host float [4]: predict+top-k,
  * delta, install (copy stream, first enqueue to last mark), MLP chain.

@@ -38,7 +38,7 @@ EXPORTED = [
     "np_version", "np_query_sizes", "np_plan_dense_prefix", "np_init", "np_destroy", "np_reset", "np_last_error",
     "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_read_records", "np_install", "np_sparse_mlp", "np_step", "np_step_selected", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
-    "np_launch_count", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_check", "np_noalloc_last_error",
+    "np_launch_count", "np_mlp_kernel_name", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_check", "np_noalloc_last_error",
     "np_trunk_workspace_floats", "np_trunk_forward", "np_trunk_last_error",
 ]
 
@@ -47,7 +47,7 @@ class np_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
         "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers", "ring_stages",
-        "dense_layers", "record_format", "io_depth", "reserved")]
+        "dense_layers", "record_format", "io_depth", "store_layers")]
 
 
 class np_sizes(C.Structure):
@@ -135,6 +135,8 @@ def load() -> C.CDLL:
         "np_selftest_bounded_wait": [vp, vp],
         "np_launch_count": [vp, C.POINTER(C.c_uint64)],
     }
+    lib.np_mlp_kernel_name.restype = C.c_char_p
+    lib.np_mlp_kernel_name.argtypes = [vp, i32]
     lib.np_noalloc_last_error.restype = C.c_char_p
     lib.np_noalloc_last_error.argtypes = []
     sigs["np_predict_logits_noalloc"] = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
@@ -348,6 +350,11 @@ def np_predict_logits_noalloc(w1, w2, x_bf16, B: int, n_layers: int, d_model: in
     return rc
 
 
+def np_mlp_kernel_name(ctx, B: int = 1) -> str:
+    name = load().np_mlp_kernel_name(ctx, B)
+    return name.decode() if name else ""
+
+
 def np_noalloc_check(stream=None) -> int:
     """Waits for `stream`; raises if the last allocation-free predictor call recorded a status bit."""
     rc = load().np_noalloc_check(_stream(stream))
@@ -359,7 +366,7 @@ def np_noalloc_check(stream=None) -> int:
 # ---- buffer owner ----------------------------------------------------------------------
 def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
                 transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0, ring_stages=0,
-                dense_layers=0, record_format=0, io_depth=0) -> np_config:
+                dense_layers=0, record_format=0, io_depth=0, store_layers=0) -> np_config:
     cfg = np_config()
     cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
     cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
@@ -369,8 +376,19 @@ def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, st
     cfg.dense_layers = dense_layers
     cfg.record_format = record_format
     cfg.io_depth = io_depth
+    cfg.store_layers = store_layers
     cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
     return cfg
+
+
+def replica_host_threads(local_world_size: int) -> int:
+    """Packing threads for one of ``local_world_size`` contexts that share a host (NP_XFER_HOST_GATHER).
+
+    A context on its own takes all cores but two (``host_threads = 0``); replicas on one host get an equal
+    share of that, at least one each, so that N contexts do not start N times the host's cores in threads.
+    """
+    cores = os.cpu_count() or 1
+    return max(1, (cores - 2) // max(1, local_world_size))
 
 
 def pin_host_tensor(t: torch.Tensor) -> None:

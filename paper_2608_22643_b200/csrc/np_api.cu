@@ -266,6 +266,8 @@ int check_config(const np_config* c, np_ctx* ctx) {
     return fail(ctx, NP_E_INVAL, "dense_layers > 0 excludes NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS");
   if (c->record_format != NP_REC_BF16 && c->record_format != NP_REC_INT8)
     return fail(ctx, NP_E_INVAL, "unknown record_format");
+  if (c->store_layers < 0 || c->store_layers > c->n_layers)
+    return fail(ctx, NP_E_INVAL, "store_layers must be 0 or in [1, n_layers]");
   if (c->record_format == NP_REC_INT8 && c->d_model % 16)
     return fail(ctx, NP_E_INVAL, "8-bit records need d_model % 16 == 0");
   {
@@ -345,7 +347,7 @@ int np_query_sizes(const np_config* cfg, np_sizes* out) {
   out->record_bytes = rec;
   out->w1_bytes = 2ull * c.d_pred * c.d_model;
   out->w2_bytes = 2ull * c.n_layers * c.d_ffn * c.d_pred;
-  out->backing_bytes = rec * c.n_layers * c.d_ffn;
+  out->backing_bytes = rec * (c.store_layers > 0 ? c.store_layers : c.n_layers) * c.d_ffn;
   out->row_buffer_bytes = 2ull * (c.n_layers - c.dense_layers) * c.capacity * c.d_model;
   out->dense_bytes = (uint64_t)c.dense_layers * c.d_ffn * 3 * c.d_model * 2;  // bf16 whatever the store holds
   out->staging_bytes = rec * c.staging_rows;
@@ -419,7 +421,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
     struct stat st;
     if (b->backing_fd < 0 || fstat(b->backing_fd, &st) != 0)
       return fail(nullptr, NP_E_INVAL, "backing_fd is not an open file");
-    const uint64_t need = (uint64_t)cfg->n_layers * cfg->d_ffn * record_bytes_of(*cfg);
+    const uint64_t need = (uint64_t)(cfg->store_layers > 0 ? cfg->store_layers : cfg->n_layers) * cfg->d_ffn * record_bytes_of(*cfg);
     if (S_ISREG(st.st_mode) && (uint64_t)st.st_size < need)
       return fail(nullptr, NP_E_INVAL, "the store file holds %llu bytes, the configuration needs %llu",
                   (unsigned long long)st.st_size, (unsigned long long)need);
@@ -445,6 +447,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   d.W = cfg->d_ffn / 32;
   d.Bmax = cfg->max_batch;
   d.ring_stages = cfg->ring_stages;
+  d.Lp = cfg->store_layers > 0 ? cfg->store_layers : cfg->n_layers;
   d.rec_bytes = record_bytes_of(*cfg);
   d.rec_int8 = cfg->record_format == NP_REC_INT8;
   d.dense = cfg->dense_layers;
@@ -618,23 +621,30 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
     if (d.rec_int8) {
       // 8-bit store: the same rounding as the install path, once, straight from the pinned store
       for (int l = 0; l < d.dense; ++l)
-        NP_INIT_CUDA(launch_dequant_dense_layer(d, ctx->backing_dev + (size_t)l * d.M * d.rec_bytes, t.identity,
+        NP_INIT_CUDA(launch_dequant_dense_layer(d, ctx->backing_dev + (size_t)(l % d.Lp) * d.M * d.rec_bytes, t.identity,
                                                 static_cast<char*>(b->dense_buf) + l * dense_layer_bytes, t.status,
                                                 nullptr, ctx->sm_count));
     } else if (from_file) {
       // through the pinned staging, a staging buffer's worth at a time
       const size_t total = (size_t)d.dense * dense_layer_bytes, step = (size_t)cfg->staging_rows * d.rec_bytes;
-      for (size_t off = 0; off < total; off += step) {
-        const size_t n = std::min(step, total - off);
-        if (!ctx->reader.submit(b->host_staging, n, off, 0) || !ctx->reader.wait_group(0)) {
+      const size_t file_bytes = (size_t)d.Lp * dense_layer_bytes;  // the file holds Lp layers; later layers wrap around
+      size_t off = 0;
+      while (off < total) {
+        const size_t foff = off % file_bytes;
+        const size_t n = std::min(std::min(step, total - off), file_bytes - foff);
+        if (!ctx->reader.submit(b->host_staging, n, foff, 0) || !ctx->reader.wait_group(0)) {
           const int e = ctx->reader.last_error();
           np_destroy(ctx);
           return fail(nullptr, NP_E_IO, "reading the dense layers from the store file failed: %s", strerror(e));
         }
         NP_INIT_CUDA(cudaMemcpy(static_cast<char*>(b->dense_buf) + off, b->host_staging, n, cudaMemcpyHostToDevice));
+        off += n;
       }
     } else {
-      NP_INIT_CUDA(cudaMemcpy(b->dense_buf, b->backing, (size_t)d.dense * dense_layer_bytes, cudaMemcpyHostToDevice));
+      for (int l = 0; l < d.dense; ++l)
+        NP_INIT_CUDA(cudaMemcpy(static_cast<char*>(b->dense_buf) + l * dense_layer_bytes,
+                                static_cast<const char*>(b->backing) + (size_t)(l % d.Lp) * dense_layer_bytes,
+                                dense_layer_bytes, cudaMemcpyHostToDevice));
     }
   }
   NP_INIT_CUDA(launch_tables_reset(d, t, nullptr));
@@ -843,7 +853,7 @@ static int install_from_file(np_ctx* ctx, int layer_begin, int layer_end, cudaSt
         while (r + len < rows && ids[first + r + len] == ids[first + r] + len) ++len;
         const int id = ids[first + r];
         if (id < 0 || id + len > d.M) return give_up(fail(ctx, NP_E_DEVICE, "layer %d: neuron id %d out of range", l, id));
-        if (!ctx->reader.submit(hbuf + (size_t)r * rec, (size_t)len * rec, ((uint64_t)l * d.M + (uint64_t)id) * rec, h))
+        if (!ctx->reader.submit(hbuf + (size_t)r * rec, (size_t)len * rec, ((uint64_t)(l % d.Lp) * d.M + (uint64_t)id) * rec, h))
           return give_up(fail(ctx, NP_E_IO, "layer %d: queueing a read failed: %s", l, strerror(ctx->reader.last_error())));
         r += len;
       }
@@ -920,7 +930,7 @@ static int install_host_gather(np_ctx* ctx, int layer_begin, int layer_end, cuda
             bad = true;
             continue;
           }
-          copy_record_streaming(hbuf + (size_t)r * rec, store + ((size_t)pc.l * d.M + id) * rec, rec);
+          copy_record_streaming(hbuf + (size_t)r * rec, store + ((size_t)(pc.l % d.Lp) * d.M + id) * rec, rec);
         }
       };
       if (ctx->pool) ctx->pool->parallel_for(jobs, body);
@@ -1023,7 +1033,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
     const int max_rows = d.C;
     for (int l = layer_begin; l < layer_end; ++l) {
       cudaStream_t zs = ctx->aux[l & 1];
-      const char* store_l = ctx->backing_dev + (size_t)l * d.M * rec;
+      const char* store_l = ctx->backing_dev + (size_t)(l % d.Lp) * d.M * rec;
       NP_LAUNCH(ctx, launch_scatter(d, store_l, true, ctx->t.delta_ids + (size_t)l * d.C,
                                   ctx->t.delta_slots + (size_t)l * d.C,
                                   ctx->t.counters + (size_t)l * NP_N_COUNTERS + NP_CNT_DELTA, 0, max_rows,
@@ -1056,7 +1066,7 @@ int np_install(np_ctx* ctx, int32_t layer_begin, int32_t layer_end, void* copy_s
     const int n = cnt[NP_CNT_DELTA];
     if (n < 0 || n > d.C) return fail(ctx, NP_E_DEVICE, "layer %d: delta count %d outside [0, %d]", l, n, d.C);
     if (cnt[NP_CNT_OVERFLOW] > 0) warn = NP_W_OVERFLOW;
-    const char* store_l = store + (size_t)l * d.M * rec;
+    const char* store_l = store + (size_t)(l % d.Lp) * d.M * rec;
     char* gate_l = static_cast<char*>(ctx->bufs.gate_buf) + (size_t)(l - d.dense) * d.C * row_bytes;
     char* up_l = static_cast<char*>(ctx->bufs.up_buf) + (size_t)(l - d.dense) * d.C * row_bytes;
     char* down_l = static_cast<char*>(ctx->bufs.downT_buf) + (size_t)(l - d.dense) * d.C * row_bytes;
@@ -1273,6 +1283,20 @@ int np_selftest_bounded_wait(np_ctx* ctx, void* stream) {
   NP_LAUNCH(ctx, launch_selftest_wait(ctx->t.status, s));
   const int rc = check_device_status(ctx, s);
   return rc == NP_E_DEVICE ? NP_E_DEVICE : (rc < 0 ? rc : fail(ctx, NP_E_STATE, "the wait did not time out"));
+}
+
+const char* np_mlp_kernel_name(np_ctx* ctx, int32_t B) {
+  if (!ctx || B < 1 || B > ctx->d.Bmax) return nullptr;
+  const Dims& d = ctx->d;
+  const int flags = ctx->cfg.flags;
+  if (B == 1 && !(flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES))) {
+    if (ctx->use_slices) return "k_mlp_slices";
+    ChainPlan p;
+    if (mlp_chain_plan(d, ctx->sm_count, &p) && (p.single_tile || !chain_alu::supported(d, ctx->sm_count))) return "k_mlp_chain";
+    if (chain_alu::supported(d, ctx->sm_count)) return "k_mlp_chain_alu";
+  }
+  if (ctx->mlp_tc && B >= kTcMinBatch && !(flags & NP_F_DIRECT_LOADS)) return "k_mlp_tc_up + k_mlp_tc_down";
+  return (flags & NP_F_DIRECT_LOADS) ? "k_sparse_mlp" : "k_sparse_mlp_pipe";
 }
 
 int np_launch_count(np_ctx* ctx, uint64_t* out) {

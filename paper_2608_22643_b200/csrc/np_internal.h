@@ -57,6 +57,7 @@ struct Dims {
   int dense;        // leading layers that are dense and fully resident (no selection, no install)
   int rec_int8;     // the store holds 8-bit records (int8 rows + fp32 scales); rec_bytes says how long they are
   int ring_stages;  // cap on shared-memory ring stages of the MLP kernels (0 = as many as fit)
+  int Lp;           // layers the record store holds: layer l reads layer l % Lp of it
   size_t rec_bytes;
 };
 

@@ -28,18 +28,21 @@ class Pair:
     def __init__(self, cfg: synth.StackConfig, policy=nb.NP_EVICT_EXACT, max_batch=1, k=None, C=None,
                  transfer_mode=nb.NP_XFER_MEMCPY_RUNS, staging_rows=None, flags=nb.NP_F_CHECK_BOUNDS,
                  gen_device="cpu", with_oracle=True, chain_layers=0, ring_stages=0, dense_layers=0,
-                 record_format=nb.NP_REC_BF16, store_dir=None, io_depth=0, direct=True):
+                 record_format=nb.NP_REC_BF16, store_dir=None, io_depth=0, direct=True, store_layers=0):
         nbuild.build()
         self.cfg = cfg
         self.k = cfg.top_k if k is None else k
         self.C = cfg.capacity if C is None else C
         w1, w2 = synth.predictor_weights(cfg, gen_device)
         self.w1_cpu, self.w2_cpu = w1.cpu(), w2.cpu()
-        self.backing = synth.backing_store(cfg, gen_device=gen_device)
+        # store_layers = Lp > 0: the store holds the first Lp layers and layer l reads layer l % Lp of it
+        Lp = store_layers if store_layers > 0 else cfg.n_layers
+        self.backing = synth.backing_store(cfg.with_(n_layers=Lp), gen_device=gen_device)
         ncfg = nb.make_config(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, self.k, self.C,
                               max_batch=max_batch, evict_policy=policy, staging_rows=staging_rows,
                               transfer_mode=transfer_mode, flags=flags, chain_layers=chain_layers, ring_stages=ring_stages,
-                              dense_layers=dense_layers, record_format=record_format, io_depth=io_depth)
+                              dense_layers=dense_layers, record_format=record_format, io_depth=io_depth,
+                              store_layers=store_layers)
         self.dense_layers = dense_layers
         if record_format == nb.NP_REC_INT8:
             # the store the library reads is the 8-bit one; the oracle works on what those
@@ -57,6 +60,8 @@ class Pair:
             self.store_u16 = O.dequantize_records(self.backing_q.numpy(), cfg.d_model)
         else:
             self.store_u16 = self.backing.view(torch.int16).numpy().view(np.uint16)
+        if Lp != cfg.n_layers:      # what the oracle sees: every layer's records written out
+            self.store_u16 = self.store_u16[np.arange(cfg.n_layers) % Lp]
         self.ora = None
         if with_oracle:
             self.ora = O.Engine(cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred, self.k, self.C, policy,

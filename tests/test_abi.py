@@ -74,7 +74,7 @@ def test_dense_prefix_plan_matches_the_oracle(lib):
 @pytest.mark.parametrize("field,value", [
     ("n_layers", 0), ("d_model", 100), ("d_ffn", 1000), ("d_pred", 7), ("top_k", 9999), ("capacity", 0),
     ("capacity", 99999), ("max_batch", 17), ("evict_policy", 5), ("transfer_mode", 9), ("staging_rows", 0),
-    ("flags", 32), ("dense_layers", -1), ("dense_layers", 3), ("io_depth", -2), ("io_depth", 5000),
+    ("flags", 64), ("store_layers", -1), ("store_layers", 3), ("dense_layers", -1), ("dense_layers", 3), ("io_depth", -2), ("io_depth", 5000),
 ])
 def test_bad_config_is_rejected(lib, field, value):
     cfg = nb.make_config(2, 256, 1024, 64, 102, 205)
@@ -83,6 +83,13 @@ def test_bad_config_is_rejected(lib, field, value):
         nb.np_query_sizes(cfg)
     assert e.value.code == nb.NP_E_INVAL
     assert nb.np_last_error(None)
+
+
+def test_aliased_store_is_sized_by_its_own_layers(lib):
+    cfg = nb.make_config(8, 256, 1024, 64, 102, 205, store_layers=3)
+    full = nb.np_query_sizes(nb.make_config(8, 256, 1024, 64, 102, 205))
+    sz = nb.np_query_sizes(cfg)
+    assert sz.backing_bytes * 8 == full.backing_bytes * 3 and sz.row_buffer_bytes == full.row_buffer_bytes
 
 
 def test_batches_whose_hidden_vectors_do_not_fit_are_rejected(lib):

@@ -380,6 +380,32 @@ def test_widest_model_with_several_layers_per_launch(chain_layers):
     test_limit_shapes(("max_model_chain", 4, 16384, 64, 64, 25, 50), 1, chain_layers=chain_layers)
 
 
+@pytest.mark.parametrize("mode,dense", [(nb.NP_XFER_MEMCPY_RUNS, 0), (nb.NP_XFER_HOST_GATHER, 0), (nb.NP_XFER_ZERO_COPY, 0),
+                                        (nb.NP_XFER_HOST_GATHER, 3), (nb.NP_XFER_FILE, 0), (nb.NP_XFER_FILE, 3)])
+def test_store_aliased_over_fewer_layers(mode, dense, tmp_path):
+    """store_layers = 2 on a five-layer stack: layer l reads the records of layer l mod 2 (a stack whose
+    whole store the host cannot hold), through every transfer mode and through a dense prefix that
+    wraps around the store; the oracle is handed the five layers written out."""
+    cfg = SMALL.with_(n_layers=5)
+    p = Pair(cfg, transfer_mode=mode, store_layers=2, dense_layers=dense, store_dir=tmp_path)
+    try:
+        assert p.backing.shape[0] == 2
+        xs = synth.hidden_states(cfg, 4)
+        L, M = cfg.n_layers, cfg.d_ffn
+        out = torch.empty((1, cfg.d_model), dtype=torch.float32, device="cuda")
+        logits = torch.zeros((1, L, M), dtype=torch.float32, device="cuda")
+        for t in range(4):
+            nb.np_predict(p.eng.ctx, xs[t].cuda(), 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, xs[t].cuda(), 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            res = p.ora.step(u16(xs[t]), logits_f32=logits.cpu().numpy())
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+        p.check_resident_bytes()
+    finally:
+        p.close()
+
+
 def test_bounded_wait_times_out_and_context_survives():
     """A wait that nothing satisfies gives up, is reported as NP_E_DEVICE, and after np_reset
     the context computes correctly again (no hang, no trap)."""

@@ -20,7 +20,9 @@ def test_two_replicas_reduce_to_the_slowest_rank(tmp_path):
         "cfg = bench.replica_config(synth.CONFIGS['tiny'], rank)\n"
         "ms = bench.max_over_ranks(dist, [10.0 + 5.0 * rank, 3.0 - rank], 'cpu')\n"
         "x = synth.hidden_states(cfg, 2)\n"
-        "print(json.dumps({'rank': rank, 'seed': cfg.seed, 'ms': ms, 'x0': float(x.float().sum())}))\n"
+        "from paper_2608_22643_b200 import binding as nb\n"
+        "threads = nb.replica_host_threads(int(os.environ['WORLD_SIZE']))\n"
+        "print(json.dumps({'rank': rank, 'seed': cfg.seed, 'ms': ms, 'x0': float(x.float().sum()), 'threads': threads}))\n"
         "bench.finish_replicas(dist)\n")
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29611", WORLD_SIZE="2")
     procs = [subprocess.Popen([sys.executable, str(script)], env=dict(env, RANK=str(r), LOCAL_RANK=str(r)),
@@ -33,6 +35,20 @@ def test_two_replicas_reduce_to_the_slowest_rank(tmp_path):
     outs.sort(key=lambda d: d["rank"])
     assert outs[0]["ms"] == outs[1]["ms"] == [15.0, 3.0]          # every rank sees the slowest rank's time
     assert outs[0]["seed"] != outs[1]["seed"] and outs[0]["x0"] != outs[1]["x0"]   # own sequence per replica
+    # the replicas of one host share its cores: together their packing threads stay within them
+    cores = os.cpu_count() or 1
+    assert all(o["threads"] >= 1 for o in outs)
+    assert sum(o["threads"] for o in outs) <= max(2, cores - 2)
+
+
+def test_packing_threads_are_divided_among_replicas():
+    sys.path.insert(0, ROOT)
+    from paper_2608_22643_b200 import binding as nb
+    cores = os.cpu_count() or 1
+    assert nb.replica_host_threads(1) == max(1, cores - 2)
+    for n in (2, 4, 8):
+        assert 1 <= nb.replica_host_threads(n) <= max(1, (cores - 2) // n)
+        assert n * nb.replica_host_threads(n) <= max(n, cores - 2)
 
 
 def test_reference_arm_runs_on_rank_zero_only():
