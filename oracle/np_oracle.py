@@ -32,8 +32,13 @@ parameter table for ``trunk_param_counts``, a library's LayerNorm and SiLU for
 properties (coordinate-copying heads, vanishing second matrices, the centroid
 half of the concatenation) for ``trunk_forward`` (Section 3.3).
 
+``Residency.speculate`` (the deeper prefetch the paper names as future work): it never evicts, keeps
+every table valid, leaves the chain's output bit-identical, and under exact replacement the next
+step's incoming set shrinks by exactly the speculative rows that are predicted (set brute force).
+
 Parity unpinned against the paper (the paper is silent; these are this build's
-definitions, pinned only by invariants and determinism): the victim order of
+definitions, pinned only by invariants and determinism): the candidate and slot rule of
+``Residency.speculate``, the victim order of
 the LRU policy, the truncation rule when a predicted set exceeds capacity, and
 ``dense_prefix_plan`` against the paper's own operating points (found there by
 a throughput sweep on its device, not by a formula), and the 8-bit record
@@ -370,6 +375,35 @@ class Residency:
     def resident_words(self) -> np.ndarray:
         return bool_to_bitmap(self.R)
 
+    def speculate(self, cand_words: np.ndarray, budget: int) -> list:
+        """Speculative residency, after this step's ``delta`` and before the next one.
+
+        The paper names a deeper prefetch pipeline as future work (Section 6): rows are fetched
+        before a token asks for them.  Residency is a cache (a resident row that is not
+        predicted is simply not used), so rows may be made resident ahead of time without
+        changing any result; what changes is the next token's incoming set, ``P \\ R``.
+        Rule (this build's; the paper gives none): per layer, of the candidate rows that are not
+        resident, the ``min(budget, free slots)`` lowest-indexed ones become resident; the i-th
+        of them (ascending neuron) takes the i-th free slot (ascending slot), exactly as
+        incoming rows do.  Nothing is evicted and no stamp changes, so under the LRU policy a
+        speculative row that is never predicted is among the first to leave, and under Eq. 3's
+        exact replacement it leaves at the next step.  Returns one ``(ids, slots)`` pair of
+        int32 arrays per layer."""
+        cand_all = bitmap_to_bool(cand_words, self.M)
+        out = []
+        for l in range(self.L):
+            R, S, owner = self.R[l], self.S[l], self.owner[l]
+            want = np.flatnonzero(cand_all[l] & ~R)
+            avail = np.flatnonzero(owner == -1)
+            n = max(0, min(int(budget), int(want.size), int(avail.size)))
+            ids, slots = want[:n].astype(np.int32), avail[:n].astype(np.int32)
+            for i in range(n):
+                S[ids[i]] = slots[i]
+                owner[slots[i]] = ids[i]
+                R[ids[i]] = True
+            out.append((ids, slots))
+        return out
+
 
 def validity_errors(slot_map: np.ndarray, owner: np.ndarray, resident: np.ndarray, C: int,
                     pred: np.ndarray = None, active_ids: np.ndarray = None) -> list:
@@ -504,11 +538,17 @@ class Engine:
         self.up = np.zeros((L, C, D), dtype=np.uint16)
         self.downT = np.zeros((L, C, D), dtype=np.uint16)
 
-    def step(self, x_u16: np.ndarray, pred_words: np.ndarray = None, logits_f32: np.ndarray = None):
+    def step(self, x_u16: np.ndarray, pred_words: np.ndarray = None, logits_f32: np.ndarray = None,
+             spec_extra: int = 0, spec_words: np.ndarray = None):
         """Run predict -> top-k -> delta -> install -> MLP chain for one token.
 
         ``pred_words`` (or ``logits_f32``) may be supplied to take the selection
-        (or the logits) from elsewhere; returns a dict of everything produced."""
+        (or the logits) from elsewhere; returns a dict of everything produced.
+        ``spec_extra`` > 0 adds the speculative prefetch of ``Residency.speculate`` behind the
+        step: the candidates are the rows ranked k+1 .. k+spec_extra by the same order as the
+        selection (or ``spec_words``, a candidate bitmap from elsewhere), the budget per layer is
+        ``spec_extra``; their records are installed like incoming rows.  The step's own output
+        does not depend on it."""
         out = {}
         if pred_words is None:
             if logits_f32 is None:
@@ -541,4 +581,16 @@ class Engine:
         out["y_layers"] = ys
         out["x_layers"] = xs
         out["x_final"] = x
+        if spec_extra > 0:
+            if spec_words is None:
+                assert logits_f32 is not None, "the candidate rule ranks this step's logits"
+                spec_words = topk_bitmap(logits_f32, min(self.M, self.k + spec_extra))
+            if self.dense_layers:
+                spec_words = np.array(spec_words, copy=True)
+                spec_words[:self.dense_layers] = 0
+            specs = self.res.speculate(spec_words, spec_extra)
+            for l, (ids, slots) in enumerate(specs):
+                nbytes += install(self.backing, self.gate, self.up, self.downT, l, ids, slots)
+            out["specs"] = specs
+            out["installed_bytes"] = nbytes
         return out
