@@ -70,6 +70,8 @@ def parse_args():
     ap.add_argument("--store-layers", default="auto",
                     help="layers of records the host store holds (layer l reads layer l mod this); 'auto' = all of them "
                          "unless the host cannot hold and pin the whole store, 0 = all")
+    ap.add_argument("--spec-rows", type=int, default=0,
+                    help="speculative prefetch behind every step: rows ranked k+1 .. k+N of the step's logits per layer")
     ap.add_argument("--min-timed-steps", type=int, default=240,
                     help="the timed region repeats the K steps (the sequence simply continues) until it spans at "
                          "least this many; ms_per_step is the mean over all of them")
@@ -372,7 +374,7 @@ def cuda_arm(args):
                           max_batch=args.batch, evict_policy=policy, transfer_mode=mode,
                           staging_rows=2 * cfg.top_k, chain_layers=args.chain_layers,
                           host_threads=args.host_threads, dense_layers=args.dense_layers, io_depth=args.io_depth,
-                          store_layers=Lp if Lp < cfg.n_layers else 0,
+                          store_layers=Lp if Lp < cfg.n_layers else 0, spec_rows=args.spec_rows,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0)
                           | (nb.NP_F_MAPPED_STAGING if args.mapped_staging else 0))
@@ -502,7 +504,7 @@ def cuda_arm(args):
 
     nd = args.dense_layers
     # ---- per-stage detail on a few more steady-state steps (untimed region) ----------------
-    stage_us, delta_rows, overlap, overflow_steps, active_max = [], [], [], 0, 0
+    stage_us, delta_rows, overlap, overflow_steps, active_max, spec_rows_seen = [], [], [], 0, 0, []
     for i in range(n_detail):
         t = T + i                                       # the sequence simply continues
         if trunk:
@@ -511,6 +513,8 @@ def cuda_arm(args):
             step(xs_dev[t])
         stage_us.append(nb.np_last_step_times(eng.ctx))      # centroid selection: the predict stage is outside the call
         c = eng.counters()
+        if args.spec_rows and not centroid:
+            spec_rows_seen.append(float(np.mean([eng.speculative_lists(l)[0].size for l in range(nd, L)])))
         delta_rows.append(float(c[nd:, nb.NP_CNT_DELTA].mean()) if nd < L else 0.0)
         overflow_steps += int((c[:, nb.NP_CNT_OVERFLOW] > 0).any())
         active_max = max(active_max, int(c[nd:, nb.NP_CNT_ACTIVE].max()) if nd < L else 0)
@@ -559,10 +563,9 @@ def cuda_arm(args):
         nb.np_mlp_chain(eng.ctx, xs_dev[T - 1], Bq, out, s)
     k1.record(s)
     s.synchronize()
-    chain_layers = args.chain_layers if args.chain_layers > 0 else (L + 3) // 4
-    if args.layer_launches or args.direct_loads or Bq > 1:
-        chain_layers = 1
-    n_launch = -(-L // chain_layers)                                # MLP kernel launches per chain
+    n_launch = nb.np_chain_launches(eng.ctx)                        # resident launches the chain was cut into
+    if n_launch <= 0:
+        n_launch = L - nd                                           # per-layer (or batch) kernels
     mlp_kernel = nb.np_mlp_kernel_name(eng.ctx, Bq)       # the kernel the library chose for this shape and batch
     if Bq > 1:
         mlp_kernel += " (the two launches of one layer)"
@@ -604,6 +607,7 @@ def cuda_arm(args):
         pred_bytes = 2 * (sum(blk[0].numel() for blk in tw["proj"]) + tw["cproj"][0].numel() + tw["heads"].numel()
                           + sum(b[0].numel() + b[4].numel() for b in tw["blocks"])) + 4 * pred_rows
     mean_delta = float(np.mean(delta_rows))
+    mean_spec = float(np.mean(spec_rows_seen)) if spec_rows_seen else 0.0
     result = {
         "metric": METRIC, "value": KT * world / (ms_total / 1000.0), "unit": UNIT, "n_gpus": world,
         "steps": K, "warmup": W, "ms_per_step": ms_total / KT, "higher_is_better": True,
@@ -616,10 +620,11 @@ def cuda_arm(args):
                         + (" records=int8" if args.records == "int8" else "")
                         + (" mapped_staging" if args.mapped_staging else "")
                         + (f" dense_layers={args.dense_layers}" if args.dense_layers else "")
+                        + (f" spec_rows={args.spec_rows}" if args.spec_rows else "")
                         + (f" (longest prefix within {args.budget_gib} GiB)" if args.budget_gib is not None else ""),
             "l2": "inputs exceed L2 (per step 866 MB of rows + 365 MB of predictor weights stream through a 126 MB L2)",
             "overlap_measured": float(np.mean(overlap)), "delta_rows_per_layer": mean_delta,
-            "active_rows_per_layer": n_active, "active_rows_max": active_max, "overflow_steps": int(overflow_steps),
+            "speculative_rows_per_layer": mean_spec, "active_rows_per_layer": n_active, "active_rows_max": active_max, "overflow_steps": int(overflow_steps),
             "replicas": world,
             "timed_steps": KT,   # --steps repeated (the sequence continues) so that the timed region is not a few ms
             "store": (f"host store holds all {L} layers" if Lp == L else
@@ -628,7 +633,7 @@ def cuda_arm(args):
             "host_threads": int(args.host_threads),
         },
         "e2e": {"value": KT * world / (e2e_ms_total / 1000.0), "unit": UNIT,
-                "h2d_bytes_per_step": int(Bq * D * 2 + mean_delta * (L - nd) * rec_store + (trunk_in_bytes if trunk else 0)),
+                "h2d_bytes_per_step": int(Bq * D * 2 + (mean_delta + mean_spec) * (L - nd) * rec_store + (trunk_in_bytes if trunk else 0)),
                 "d2h_bytes_per_step": int(Bq * D * 4)},
         "gpu_launches": int(launches),
         "clocks": clocks,
@@ -688,7 +693,7 @@ def cuda_arm(args):
     # ---- the same step in other settings (reported beside, not as, the value) ----
     if (args.transfer == "gather" and not args.no_variants and not centroid and Bq == 1
             and args.config == "7b" and not (args.layer_launches or args.direct_loads) and not args.dense_layers
-            and args.records == "bf16" and world == 1 and args.policy == "exact"):
+            and args.records == "bf16" and world == 1 and args.policy == "exact" and not args.spec_rows):
         eng.close()
 
         def variant(note, vstore=None, **kw):

@@ -133,8 +133,9 @@ typedef struct np_config {
   int32_t transfer_mode;  /* NP_XFER_* */
   int32_t flags;          /* NP_F_* */
   int32_t host_threads;   /* worker threads for NP_XFER_HOST_GATHER (0 = pick) */
-  int32_t chain_layers;   /* layers per resident MLP kernel in np_step / np_mlp_chain
-                             (0 = a quarter of the stack) */
+  int32_t chain_layers;   /* layers per resident MLP kernel in np_step / np_mlp_chain (0 = runs that
+                             shrink towards the end: the last run is an eighth of the stack, the one
+                             before it a quarter, the first takes the rest) */
   int32_t ring_stages;    /* cap on the records the MLP kernels stage in shared memory
                              (0 = as many as fit; >= 2 otherwise) */
   int32_t dense_layers;   /* d, 0 <= d <= L: the first d layers are dense (Section 3.1): all M
@@ -151,6 +152,11 @@ typedef struct np_config {
                              layer l mod Lp of it (0 = L, every layer its own).  For stacks whose whole
                              store the host cannot hold or pin: shapes, row counts and traffic per step
                              stay those of the L-layer stack */
+  int32_t spec_rows;      /* s >= 0: np_step / np_step_selected add a speculative prefetch behind every step (see
+                             np_speculate): per layer up to s rows ranked k+1 .. k+s by the step's own logits
+                             (np_step) become resident in free slots and are transferred after the step's
+                             incoming rows.  0 = none */
+  int32_t reserved;       /* 0 */
 } np_config;
 
 /* Byte counts of the caller-owned buffers for a configuration. */
@@ -373,6 +379,28 @@ int np_export_state(np_ctx* ctx, int32_t layer, int32_t* slot_map, int32_t* owne
  * step counter; the caller vouches for their consistency.  Synchronises. */
 int np_import_state(np_ctx* ctx, int32_t layer, const int32_t* slot_map, const int32_t* owner,
                     const uint32_t* resident, const int32_t* stamp, int32_t step, void* stream);
+
+/* Speculative residency behind a step: the "deeper prefetch pipeline" the paper names as future work
+ * (Section 6).  Residency is a cache: a row may be made resident before any token asks for it without
+ * changing a result; what changes is the next token's incoming set P \ R (Eq. 2).  After np_delta and
+ * before the next one, per layer: of the rows of cand_bitmap (dev uint32 [L][W]) that are not resident,
+ * the min(budget, free slots) lowest-indexed become resident; the i-th of them (ascending neuron) takes
+ * the i-th free slot (ascending slot), as incoming rows do.  Nothing is evicted, no stamp changes (under
+ * NP_EVICT_LRU a speculative row that is never predicted is among the first to leave; under
+ * NP_EVICT_EXACT it leaves at the next step).  The rule is this library's: the paper gives none.
+ * The lists (np_get_speculative) are mirrored to the host; np_install_speculative transfers the rows
+ * exactly as np_install transfers incoming rows (same transfer mode, chunking and per-layer marks), and
+ * is meant to be queued after the step's own np_install and MLP launches.  Dense layers take none.
+ * Errors: NP_E_STATE (no np_delta yet / np_install_speculative without np_speculate), NP_E_INVAL, NP_E_CUDA. */
+int np_speculate(np_ctx* ctx, const uint32_t* cand_bitmap, int32_t budget, void* stream);
+int np_install_speculative(np_ctx* ctx, void* copy_stream);
+/* Device views of one layer's speculative rows of the last np_speculate: ids and slots (ascending neuron),
+ * and their count.  Valid until the next np_speculate. */
+int np_get_speculative(np_ctx* ctx, int32_t layer, const int32_t** ids, const int32_t** slots, const int32_t** count);
+
+/* Launches of the resident MLP kernel (sparse layers, one sequence) made by the last np_mlp_chain / np_step:
+ * the runs the chain was cut into.  0 when that call ran per-layer or batch kernels.  For reports. */
+int np_chain_launches(np_ctx* ctx, int32_t* out);
 
 /* Name of the kernel np_mlp_chain / np_step run the sparse layers' MLP with for B sequences in this
  * context (a static string: "k_mlp_slices", "k_mlp_chain", "k_mlp_chain_alu", "k_mlp_tc_up + k_mlp_tc_down",

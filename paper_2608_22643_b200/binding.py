@@ -38,7 +38,7 @@ EXPORTED = [
     "np_version", "np_query_sizes", "np_plan_dense_prefix", "np_init", "np_destroy", "np_reset", "np_last_error",
     "np_predict", "np_topk", "np_centroid_select", "np_delta", "np_read_records", "np_install", "np_sparse_mlp", "np_step", "np_step_selected", "np_get_delta",
     "np_read_counters", "np_export_state", "np_import_state", "np_last_step_times", "np_mlp_chain",
-    "np_launch_count", "np_mlp_kernel_name", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_check", "np_noalloc_last_error",
+    "np_launch_count", "np_chain_launches", "np_speculate", "np_install_speculative", "np_get_speculative", "np_mlp_kernel_name", "np_selftest_bounded_wait", "np_predict_logits_noalloc", "np_noalloc_check", "np_noalloc_last_error",
     "np_trunk_workspace_floats", "np_trunk_forward", "np_trunk_last_error",
 ]
 
@@ -47,7 +47,7 @@ class np_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "d_model", "d_ffn", "d_pred", "top_k", "capacity", "max_batch", "evict_policy",
         "staging_rows", "transfer_mode", "flags", "host_threads", "chain_layers", "ring_stages",
-        "dense_layers", "record_format", "io_depth", "store_layers")]
+        "dense_layers", "record_format", "io_depth", "store_layers", "spec_rows", "reserved")]
 
 
 class np_sizes(C.Structure):
@@ -141,6 +141,10 @@ def load() -> C.CDLL:
     lib.np_noalloc_last_error.argtypes = []
     sigs["np_predict_logits_noalloc"] = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
     sigs["np_noalloc_check"] = [vp]
+    sigs["np_speculate"] = [vp, vp, i32, vp]
+    sigs["np_chain_launches"] = [vp, C.POINTER(C.c_int32)]
+    sigs["np_install_speculative"] = [vp, vp]
+    sigs["np_get_speculative"] = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
     for name, args in sigs.items():
         fn = getattr(lib, name)
         fn.argtypes = args
@@ -350,6 +354,20 @@ def np_predict_logits_noalloc(w1, w2, x_bf16, B: int, n_layers: int, d_model: in
     return rc
 
 
+def np_speculate(ctx, cand_bitmap, budget: int, stream=None) -> int:
+    return _check(ctx, load().np_speculate(ctx, _ptr(cand_bitmap), budget, _stream(stream)))
+
+
+def np_install_speculative(ctx, copy_stream=None) -> int:
+    return _check(ctx, load().np_install_speculative(ctx, _stream(copy_stream)))
+
+
+def np_chain_launches(ctx) -> int:
+    out = C.c_int32(0)
+    _check(ctx, load().np_chain_launches(ctx, C.byref(out)))
+    return int(out.value)
+
+
 def np_mlp_kernel_name(ctx, B: int = 1) -> str:
     name = load().np_mlp_kernel_name(ctx, B)
     return name.decode() if name else ""
@@ -366,7 +384,7 @@ def np_noalloc_check(stream=None) -> int:
 # ---- buffer owner ----------------------------------------------------------------------
 def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, staging_rows=None,
                 transfer_mode=NP_XFER_MEMCPY_RUNS, flags=0, host_threads=0, chain_layers=0, ring_stages=0,
-                dense_layers=0, record_format=0, io_depth=0, store_layers=0) -> np_config:
+                dense_layers=0, record_format=0, io_depth=0, store_layers=0, spec_rows=0) -> np_config:
     cfg = np_config()
     cfg.n_layers, cfg.d_model, cfg.d_ffn, cfg.d_pred = L, D, M, H
     cfg.top_k, cfg.capacity, cfg.max_batch = k, Cap, max_batch
@@ -377,6 +395,7 @@ def make_config(L, D, M, H, k, Cap, max_batch=1, evict_policy=NP_EVICT_EXACT, st
     cfg.record_format = record_format
     cfg.io_depth = io_depth
     cfg.store_layers = store_layers
+    cfg.spec_rows = spec_rows
     cfg.staging_rows = staging_rows if staging_rows is not None else max(2, min(Cap, 2 * max(1, k)))
     return cfg
 
@@ -526,6 +545,14 @@ class Engine:
             "active_ids": self._read_i32(v.active_ids, int(c[NP_CNT_ACTIVE])),
             "active_slots": self._read_i32(v.active_slots, int(c[NP_CNT_ACTIVE])),
         }
+
+    def speculative_lists(self, layer: int):
+        """(ids, slots) of the layer's rows made resident by the last np_speculate."""
+        torch.cuda.synchronize(self.device)
+        ids, slots, cnt = C.c_void_p(), C.c_void_p(), C.c_void_p()
+        _check(self.ctx, load().np_get_speculative(self.ctx, layer, C.byref(ids), C.byref(slots), C.byref(cnt)))
+        n = int(self._read_i32(cnt.value, 1)[0])
+        return self._read_i32(ids.value, n), self._read_i32(slots.value, n)
 
     def export_state(self, layer: int) -> dict:
         M, Cap, W = self.cfg.d_ffn, self.cfg.capacity, self.cfg.d_ffn // 32

@@ -178,6 +178,7 @@ struct np_ctx {
   const char* backing_dev = nullptr;  // device alias of the record store
   char* hstage_dev = nullptr;         // device alias of the pinned staging (NP_F_MAPPED_STAGING)
   cudaEvent_t ev_delta = nullptr;
+  cudaEvent_t ev_spec = nullptr;      // the lists of the last np_speculate are written
   std::vector<cudaEvent_t> ev_installed;
   std::vector<char> install_pending;
   cudaEvent_t ev_half[kStageParts] = {};        // parts of the host / device staging in flight
@@ -190,6 +191,7 @@ struct np_ctx {
   cudaEvent_t ev_t[4] = {nullptr, nullptr, nullptr, nullptr};  // compute-stream step timing
   cudaEvent_t ev_c[2] = {nullptr, nullptr};                    // copy-stream step timing
   bool have_delta = false;
+  bool have_spec = false;   // np_speculate has run since the last np_delta
   bool have_pred = false;
   bool have_step = false;
   int step = 0;
@@ -199,6 +201,7 @@ struct np_ctx {
   PredTcState tc = {};
   chain_slices::State slices = {};  // column-sliced resident MLP kernel: its counters, exchange words and their values
   bool use_slices = false;
+  int chain_kernel_launches = 0;    // MLP kernel launches of the last np_mlp_chain / np_step
   size_t gu_bytes = 0;   // both dot-product accumulators of the batch MLP, contiguous
   bool mlp_tc = false;   // batches run the tensor-core MLP kernels
   std::string err;
@@ -266,6 +269,8 @@ int check_config(const np_config* c, np_ctx* ctx) {
     return fail(ctx, NP_E_INVAL, "dense_layers > 0 excludes NP_F_LAYER_LAUNCHES and NP_F_DIRECT_LOADS");
   if (c->record_format != NP_REC_BF16 && c->record_format != NP_REC_INT8)
     return fail(ctx, NP_E_INVAL, "unknown record_format");
+  if (c->spec_rows < 0 || c->spec_rows > c->capacity) return fail(ctx, NP_E_INVAL, "spec_rows must be in [0, capacity]");
+  if (c->reserved != 0) return fail(ctx, NP_E_INVAL, "reserved must be 0");
   if (c->store_layers < 0 || c->store_layers > c->n_layers)
     return fail(ctx, NP_E_INVAL, "store_layers must be 0 or in [1, n_layers]");
   if (c->record_format == NP_REC_INT8 && c->d_model % 16)
@@ -316,9 +321,12 @@ WsLayout ws_layout(const np_config& c) {
   return w;
 }
 
-size_t host_lists_ints(const np_config& c) {
+// one list area of the host mirror: [header][layer: counters, ids[C], slots[C]]
+size_t host_area_ints(const np_config& c) {
   return kHostHeaderInts + (size_t)c.n_layers * (NP_N_COUNTERS + 2 * (size_t)c.capacity);
 }
+// two areas: the incoming rows of np_delta, then the speculative rows of np_speculate
+size_t host_lists_ints(const np_config& c) { return 2 * host_area_ints(c); }
 
 cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
 
@@ -382,6 +390,7 @@ int np_destroy(np_ctx* ctx) {
   delete ctx->pool;
   if (ctx->slab) cudaFree(ctx->slab);
   if (ctx->ev_delta) cudaEventDestroy(ctx->ev_delta);
+  if (ctx->ev_spec) cudaEventDestroy(ctx->ev_spec);
   for (auto e : ctx->ev_installed)
     if (e) cudaEventDestroy(e);
   for (auto e : ctx->ev_half)
@@ -505,6 +514,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_ovf = take(LM), o_cnt = take((size_t)d.L * NP_N_COUNTERS), o_free = take(LC);
   const size_t o_cid = take(LC), o_ckey = take(LC), o_pred = take(LW), o_stat = take(4), o_bar = take(4);
   const size_t o_ident = take(d.dense > 0 ? (size_t)d.M : 1);
+  const size_t o_spid = take(LC), o_spsl = take(LC), o_spcnt = take((size_t)d.L * NP_N_COUNTERS), o_spcand = take(LW);
   const size_t o_sbar = take(chain_slices::bar_words()), o_sxch = take(2 * chain_slices::xch_words(d, ctx->sm_count));
   NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
   char* base = static_cast<char*>(ctx->slab);
@@ -527,6 +537,10 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   t.status = reinterpret_cast<int32_t*>(base + o_stat);
   t.grid_bar = reinterpret_cast<unsigned int*>(base + o_bar);
   t.identity = reinterpret_cast<int32_t*>(base + o_ident);
+  t.spec_ids = reinterpret_cast<int32_t*>(base + o_spid);
+  t.spec_slots = reinterpret_cast<int32_t*>(base + o_spsl);
+  t.spec_counters = reinterpret_cast<int32_t*>(base + o_spcnt);
+  t.spec_cand = reinterpret_cast<uint32_t*>(base + o_spcand);
   ctx->slices.bars = reinterpret_cast<unsigned int*>(base + o_sbar);
   ctx->slices.xch = reinterpret_cast<unsigned long long*>(base + o_sxch);
   ctx->slices.bar_base = ctx->slices.seq_base = 0;
@@ -549,6 +563,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   ctx->gu_bytes = 2 * wl.gu_each;
 
   NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_delta, cudaEventDisableTiming));
+  NP_INIT_CUDA(cudaEventCreateWithFlags(&ctx->ev_spec, cudaEventDisableTiming));
   ctx->ev_installed.assign(d.L, nullptr);
   ctx->install_pending.assign(d.L, 0);
   for (int l = 0; l < d.L; ++l)
@@ -662,7 +677,7 @@ int np_reset(np_ctx* ctx, void* stream) {
   NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.bars, 0, chain_slices::bar_words() * 4, as_stream(stream)));
   NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8, as_stream(stream)));
   ctx->slices.bar_base = ctx->slices.seq_base = 0;
-  ctx->have_delta = ctx->have_pred = ctx->have_step = false;
+  ctx->have_delta = ctx->have_pred = ctx->have_step = ctx->have_spec = false;
   std::fill(ctx->install_pending.begin(), ctx->install_pending.end(), 0);
   ctx->step = 0;
   return NP_OK;
@@ -759,6 +774,7 @@ int np_delta(np_ctx* ctx, const uint32_t* pred_bitmap, void* stream) {
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_delta, s));
   ctx->step += 1;
   ctx->have_delta = true;
+  ctx->have_spec = false;
   return NP_OK;
 }
 
@@ -1177,8 +1193,11 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
                           (ctx->use_slices || mlp_chain_supported(d, ctx->sm_count));
   const bool tc_batch = !persistent && ctx->mlp_tc && B >= kTcMinBatch && !(ctx->cfg.flags & NP_F_DIRECT_LOADS);
+  if (part != kChainTail) ctx->chain_kernel_launches = 0;
+  // the sliced kernel widens the stack's bf16 input itself when it runs layer 0
+  const bool fold_widen = persistent && ctx->use_slices && d.dense == 0;
   if (part != kChainTail) {
-    NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
+    if (!fold_widen) NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
     // the accumulator of layer 0 starts at zero (later ones are cleared one layer ahead)
     NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, (persistent ? (size_t)kZRep * d.D : n) * 4, s));
   }
@@ -1194,6 +1213,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
     a.status = ctx->t.status;
     a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
     a.counters = ctx->t.counters;
+    a.x_bf16 = fold_widen ? x_bf16 : nullptr;
     // the dense prefix first: whole records, every row active, nothing to wait for (it also
     // widens the window in which the sparse layers' rows arrive)
     if (d.dense > 0 && part != kChainTail) {
@@ -1227,16 +1247,39 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
     a.downT = static_cast<const char*>(ctx->bufs.downT_buf) - shift;
     a.active_slots = ctx->t.active_slots;
     a.dense_rows = 0;
-    for (int l0 = d.dense; l0 < d.L && part != kChainHead; l0 += run) {
-      const int l1 = std::min(d.L, l0 + run);
+    // Runs of the sparse layers.  A run starts once its layers are installed, so what the step waits for
+    // after its last row has landed is the last run: with chain_layers = 0 the runs shrink towards the end
+    // (the tail is an eighth of the stack, the run before it a quarter, the first run takes the rest), which
+    // also makes fewer launches than equal runs of a quarter each.
+    std::vector<int> runs;
+    {
+      const int ns = d.L - d.dense;
+      if (ctx->cfg.chain_layers > 0) {
+        for (int l0 = 0; l0 < ns; l0 += run) runs.push_back(std::min(run, ns - l0));
+      } else if (ns > 0) {
+        const int tail = std::max(1, ns / 8), mid = std::min(ns - tail, 2 * tail), first = ns - tail - mid;
+        if (first > 0) runs.push_back(first);
+        if (mid > 0) runs.push_back(mid);
+        runs.push_back(tail);
+      }
+    }
+    int l0 = d.dense;
+    for (size_t ri = 0; ri < runs.size() && part != kChainHead; ++ri) {
+      const int l1 = l0 + runs[ri];
       for (int l = l0; l < l1; ++l)
         if (ctx->install_pending[l]) NP_CUDA(ctx, wait_install(ctx, l, s));
       a.l_begin = l0;
       a.l_end = l1;
-      if (ctx->use_slices)
+      if (ctx->use_slices) {
+        chain_slices::Plan sp;
+        chain_slices::plan(d, ctx->sm_count, &sp);
+        ctx->chain_kernel_launches += (l1 - l0 + sp.run_layers - 1) / sp.run_layers;
         NP_LAUNCH(ctx, chain_slices::launch(d, a, &ctx->slices, s, ctx->sm_count));
-      else
+      } else {
+        ctx->chain_kernel_launches += 1;
         NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
+      }
+      l0 = l1;
     }
   } else {
     if (part != kChainTail && ctx->mlp_tc && B >= kTcMinBatch)
@@ -1283,6 +1326,62 @@ int np_selftest_bounded_wait(np_ctx* ctx, void* stream) {
   NP_LAUNCH(ctx, launch_selftest_wait(ctx->t.status, s));
   const int rc = check_device_status(ctx, s);
   return rc == NP_E_DEVICE ? NP_E_DEVICE : (rc < 0 ? rc : fail(ctx, NP_E_STATE, "the wait did not time out"));
+}
+
+int np_speculate(np_ctx* ctx, const uint32_t* cand_bitmap, int32_t budget, void* stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!cand_bitmap) return fail(ctx, NP_E_INVAL, "cand_bitmap is NULL");
+  if (budget < 0) return fail(ctx, NP_E_INVAL, "budget must be >= 0");
+  if (!ctx->have_delta) return fail(ctx, NP_E_STATE, "np_speculate needs a prior np_delta");
+  cudaStream_t s = as_stream(stream);
+  // rows brought in ahead of time by an earlier call must have landed before their tables move again
+  for (int l = 0; l < ctx->d.L; ++l)
+    if (ctx->have_spec && ctx->install_pending[l]) NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[l], 0));
+  NP_LAUNCH(ctx, launch_speculate(ctx->d, ctx->t, cand_bitmap, std::min(budget, ctx->d.C),
+                                  ctx->host_lists_dev + host_area_ints(ctx->cfg), s));
+  NP_CUDA(ctx, cudaEventRecord(ctx->ev_spec, s));
+  ctx->have_spec = true;
+  return NP_OK;
+}
+
+int np_install_speculative(np_ctx* ctx, void* copy_stream) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!ctx->have_spec) return fail(ctx, NP_E_STATE, "np_install_speculative needs a prior np_speculate");
+  // The speculative rows take the very path of the incoming rows: for the length of this call the
+  // install code is pointed at the second list area (host mirror, device lists, counts, event).
+  struct Saved {
+    int32_t *host, *ids, *slots, *counters;
+    cudaEvent_t ev;
+  } keep = {ctx->host_lists, ctx->t.delta_ids, ctx->t.delta_slots, ctx->t.counters, ctx->ev_delta};
+  ctx->host_lists += host_area_ints(ctx->cfg);
+  ctx->t.delta_ids = ctx->t.spec_ids;
+  ctx->t.delta_slots = ctx->t.spec_slots;
+  ctx->t.counters = ctx->t.spec_counters;
+  ctx->ev_delta = ctx->ev_spec;
+  const int rc = np_install(ctx, 0, ctx->d.L, copy_stream);
+  ctx->host_lists = keep.host;
+  ctx->t.delta_ids = keep.ids;
+  ctx->t.delta_slots = keep.slots;
+  ctx->t.counters = keep.counters;
+  ctx->ev_delta = keep.ev;
+  return rc;
+}
+
+int np_get_speculative(np_ctx* ctx, int32_t layer, const int32_t** ids, const int32_t** slots, const int32_t** count) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (layer < 0 || layer >= ctx->d.L) return fail(ctx, NP_E_INVAL, "layer %d outside [0, %d)", layer, ctx->d.L);
+  if (!ctx->have_spec) return fail(ctx, NP_E_STATE, "np_get_speculative needs a prior np_speculate");
+  if (ids) *ids = ctx->t.spec_ids + (size_t)layer * ctx->d.C;
+  if (slots) *slots = ctx->t.spec_slots + (size_t)layer * ctx->d.C;
+  if (count) *count = ctx->t.spec_counters + (size_t)layer * NP_N_COUNTERS + NP_CNT_DELTA;
+  return NP_OK;
+}
+
+int np_chain_launches(np_ctx* ctx, int32_t* out) {
+  if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
+  if (!out) return fail(ctx, NP_E_INVAL, "out is NULL");
+  *out = ctx->chain_kernel_launches;
+  return NP_OK;
 }
 
 const char* np_mlp_kernel_name(np_ctx* ctx, int32_t B) {
@@ -1340,6 +1439,24 @@ static int step_impl(np_ctx* ctx, const void* x_bf16, int32_t B, const uint32_t*
   rc = np_delta(ctx, selected, stream);
   if (rc < 0) return rc;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[2], s));
+  // Speculative prefetch behind the step (Section 6's future work).  Its candidates are the rows ranked
+  // k+1 .. k+s by this step's own logits (a caller's selection has no ranking to extend: the caller then
+  // calls np_speculate itself).  The second selection and the table update run right behind the delta
+  // step (the MLP launches read only the step's active lists and their slots, which a speculative row
+  // never takes); the transfer is queued last, behind the incoming rows and the MLP launches.
+  const bool spec = ctx->cfg.spec_rows > 0 && !selected;
+  if (spec) {
+    Dims ds = d;
+    const int skip_layers = B == 1 ? d.dense : 0;
+    ds.L = d.L - skip_layers;
+    ds.k = std::min(d.M, d.k + ctx->cfg.spec_rows);
+    if (ds.L > 0)
+      NP_LAUNCH(ctx, launch_topk(ds, ctx->ws.logits + (size_t)skip_layers * d.M, B,
+                                 ctx->t.spec_cand + (size_t)skip_layers * d.W, s));
+    if (d.dense > 0) NP_CUDA(ctx, cudaMemsetAsync(ctx->t.spec_cand, 0, (size_t)d.dense * d.W * 4, s));
+    rc = np_speculate(ctx, ctx->t.spec_cand, ctx->cfg.spec_rows, stream);
+    if (rc < 0) return rc;
+  }
   // the dense prefix waits for no install: it is queued before the host starts on the rows
   const bool head_first = d.dense > 0;
   if (head_first) {
@@ -1357,6 +1474,11 @@ static int step_impl(np_ctx* ctx, const void* x_bf16, int32_t B, const uint32_t*
   if (rc < 0) return rc;
   NP_CUDA(ctx, cudaEventRecord(ctx->ev_t[3], s));
   ctx->have_step = true;
+  if (spec) {
+    // the guessed rows cross behind the step's own rows, while its MLP launches run
+    rc = np_install_speculative(ctx, copy_stream);
+    if (rc < 0) return rc;
+  }
   return warn;
 }
 

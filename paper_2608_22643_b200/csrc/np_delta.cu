@@ -310,6 +310,83 @@ __global__ void __launch_bounds__(kDeltaThreads) k_delta(DeltaParams p) {
   }
 }
 
+// Speculative residency behind a step (the deeper prefetch of the paper's future work, Section 6):
+// per layer, the candidates that are not resident, lowest index first, take the free slots in
+// ascending order, as many as the budget and the free slots allow.  Nothing leaves, no stamp changes.
+__global__ void __launch_bounds__(kDeltaThreads) k_speculate(Tables t, const uint32_t* __restrict__ cand, int32_t* host_lists,
+                                                             int M, int C, int W, int budget, int first_layer) {
+  extern __shared__ __align__(16) int ssm[];
+  uint32_t* w_sp = reinterpret_cast<uint32_t*>(ssm);  // [W] candidate and not resident
+  int* scan = reinterpret_cast<int*>(w_sp + W);       // [W]
+  int* red = scan + W;                                // [48]
+  const int layer = first_layer + blockIdx.x, tid = threadIdx.x;
+  uint32_t* R = t.resident + (size_t)layer * W;
+  int32_t* S = t.slot_map + (size_t)layer * M;
+  int32_t* owner = t.owner + (size_t)layer * C;
+  int32_t* free_slots = t.free_slots + (size_t)layer * C;
+  int32_t* ids = t.spec_ids + (size_t)layer * C;
+  int32_t* slots = t.spec_slots + (size_t)layer * C;
+  int32_t* cnt = t.spec_counters + (size_t)layer * NP_N_COUNTERS;
+  int32_t* h_cnt = nullptr;
+  int32_t* h_ids = nullptr;
+  int32_t* h_slots = nullptr;
+  if (host_lists) {  // the second list area of the host mirror, laid out like the first
+    h_cnt = host_lists + kHostHeaderInts + (size_t)layer * (NP_N_COUNTERS + 2 * (size_t)C);
+    h_ids = h_cnt + NP_N_COUNTERS;
+    h_slots = h_ids + C;
+  }
+  const uint32_t* cw = cand + (size_t)layer * W;
+  for (int w = tid; w < W; w += blockDim.x) {
+    const uint32_t m = cw[w] & ~R[w];
+    w_sp[w] = m;
+    scan[w] = __popc(m);
+  }
+  const int n_want = block_exclusive_scan(scan, W, red);
+  const int n_avail = compact_indices(
+      C, red, [&](int s) { return owner[s] < 0; }, [&](int pos, int s) { free_slots[pos] = s; });
+  const int n = max(0, min(budget, min(n_want, n_avail)));
+  for (int w = tid; w < W; w += blockDim.x) {
+    uint32_t m = w_sp[w];
+    int pos = scan[w];
+    uint32_t placed = 0u;
+    while (m && pos < n) {
+      const int bit = __ffs(m) - 1;
+      const int nid = w * 32 + bit;
+      m &= m - 1;
+      const int s = free_slots[pos];
+      S[nid] = s;
+      owner[s] = nid;
+      ids[pos] = nid;
+      slots[pos] = s;
+      if (h_ids) {
+        h_ids[pos] = nid;
+        h_slots[pos] = s;
+      }
+      placed |= 1u << bit;
+      ++pos;
+    }
+    if (placed) R[w] |= placed;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    for (int i = 0; i < NP_N_COUNTERS; ++i) cnt[i] = 0;
+    cnt[NP_CNT_DELTA] = n;
+    t.counters[(size_t)layer * NP_N_COUNTERS + NP_CNT_RESIDENT] += n;
+    if (h_cnt) {
+      __threadfence_system();  // the list entries of the other threads precede the count the host reads
+      for (int i = 0; i < NP_N_COUNTERS; ++i) h_cnt[i] = i == NP_CNT_DELTA ? n : 0;
+    }
+  }
+}
+
+cudaError_t launch_speculate(const Dims& d, const Tables& t, const uint32_t* cand, int budget, int32_t* host_lists_dev,
+                             cudaStream_t s) {
+  if (d.L <= d.dense) return cudaSuccess;
+  const size_t sm = (size_t)d.W * 8 + 48 * 4;
+  k_speculate<<<d.L - d.dense, kDeltaThreads, sm, s>>>(t, cand, host_lists_dev, d.M, d.C, d.W, budget, d.dense);
+  return cudaGetLastError();
+}
+
 __global__ void k_tables_reset(Tables t, int L, int M, int C, int W) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t nLM = (size_t)L * M, nLC = (size_t)L * C, nLW = (size_t)L * W;
@@ -322,7 +399,10 @@ __global__ void k_tables_reset(Tables t, int L, int M, int C, int W) {
     t.resident[i] = 0u;
     t.pred[i] = 0u;
   }
-  if (i < (size_t)L * NP_N_COUNTERS) t.counters[i] = 0;
+  if (i < (size_t)L * NP_N_COUNTERS) {
+    t.counters[i] = 0;
+    t.spec_counters[i] = 0;
+  }
   if (i < 4) t.status[i] = 0;
 }
 

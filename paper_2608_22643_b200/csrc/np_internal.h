@@ -39,6 +39,10 @@ struct Tables {
   int32_t* status;        // [4]     device-side error word(s)
   unsigned int* grid_bar; // [1]     arrival counter of the persistent MLP kernel
   int32_t* identity;      // [M]     0, 1, ..., M-1: the active list of a dense layer
+  int32_t* spec_ids;      // [L][C]  rows made resident ahead of time by the last np_speculate
+  int32_t* spec_slots;    // [L][C]
+  int32_t* spec_counters; // [L][NP_N_COUNTERS] their count sits at NP_CNT_DELTA (the install path reads it there)
+  uint32_t* spec_cand;    // [L][W]  candidate bitmap of np_step's own speculation
 };
 
 // Carved out of the caller's workspace.
@@ -92,6 +96,9 @@ cudaError_t launch_centroid_select(const Dims& d, const float* logits, int B, in
 
 cudaError_t launch_delta(const Dims& d, const Tables& t, const uint32_t* pred, int policy, int step,
                          int32_t* host_lists_dev, int check, cudaStream_t s);
+// speculative residency: candidates that are not resident take free slots (np_delta.cu)
+cudaError_t launch_speculate(const Dims& d, const Tables& t, const uint32_t* cand, int budget, int32_t* host_lists_dev,
+                             cudaStream_t s);
 
 // src_is_store: records are read from the whole-layer store by neuron ID
 // (zero-copy); otherwise record r of `src` is the r-th entry of the lists.
@@ -151,6 +158,7 @@ struct ChainArgs {
   const void* downT;
   const int32_t* active_slots;  // [L][C]
   const int32_t* counters;      // [L][NP_N_COUNTERS]
+  const void* x_bf16;  // sliced kernel only, may be NULL: the stack's input, read by the run that starts at layer 0
   float* xbuf[2];
   float* zbuf[3];
   unsigned int* grid_bar;

@@ -71,6 +71,7 @@ struct KArgs {
   const unsigned char* downT;
   const int32_t* slots;        // active_slots [L][C]
   const int32_t* counters;     // [L][NP_N_COUNTERS]
+  const uint16_t* x_bf16;      // not NULL: the run starts the stack (layer 0) and reads its input from here (bf16 [D])
   float* xbuf[2];              // x_l of the run's last layer is stored to xbuf[l & 1]
   float* zbuf[3];              // MLP_l(x_l) accumulates into zbuf[l % 3]: kZRep copies of [D]
   unsigned int* bars;          // [kQ][kBarStride] arrival counters, never reset: the host tracks their value
@@ -498,7 +499,14 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       for (int j = 0; j < J4; ++j) {  // every load of the pass is issued before any is used
         const int c = tid + j * kThreads;
         if (c < nf4) {
-          if (li == 0) xown[j] = __ldcg(reinterpret_cast<const float4*>(xa) + c);
+          if (li == 0) {
+            if (a.x_bf16) {  // the stack's input: bf16 values widened here (no kernel in front for that)
+              const uint2 h = __ldg(reinterpret_cast<const uint2*>(a.x_bf16 + qoff) + c);
+              xown[j] = make_float4(bf16_lo(h.x), bf16_hi(h.x), bf16_lo(h.y), bf16_hi(h.y));
+            } else {
+              xown[j] = __ldcg(reinterpret_cast<const float4*>(xa) + c);
+            }
+          }
           if (zb) {
 #pragma unroll
             for (int rep = 0; rep < kZRep; ++rep) w[j][rep] = __ldcg(reinterpret_cast<const float4*>(zb + (size_t)rep * D) + c);
@@ -826,6 +834,7 @@ cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s,
     ka.downT = static_cast<const unsigned char*>(a.downT);
     ka.slots = a.active_slots;
     ka.counters = a.counters;
+    ka.x_bf16 = l0 == 0 ? static_cast<const uint16_t*>(a.x_bf16) : nullptr;
     for (int i = 0; i < 2; ++i) ka.xbuf[i] = a.xbuf[i];
     for (int i = 0; i < 3; ++i) ka.zbuf[i] = a.zbuf[i];
     ka.bars = st->bars;

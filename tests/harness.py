@@ -28,7 +28,7 @@ class Pair:
     def __init__(self, cfg: synth.StackConfig, policy=nb.NP_EVICT_EXACT, max_batch=1, k=None, C=None,
                  transfer_mode=nb.NP_XFER_MEMCPY_RUNS, staging_rows=None, flags=nb.NP_F_CHECK_BOUNDS,
                  gen_device="cpu", with_oracle=True, chain_layers=0, ring_stages=0, dense_layers=0,
-                 record_format=nb.NP_REC_BF16, store_dir=None, io_depth=0, direct=True, store_layers=0):
+                 record_format=nb.NP_REC_BF16, store_dir=None, io_depth=0, direct=True, store_layers=0, spec_rows=0):
         nbuild.build()
         self.cfg = cfg
         self.k = cfg.top_k if k is None else k
@@ -42,7 +42,7 @@ class Pair:
                               max_batch=max_batch, evict_policy=policy, staging_rows=staging_rows,
                               transfer_mode=transfer_mode, flags=flags, chain_layers=chain_layers, ring_stages=ring_stages,
                               dense_layers=dense_layers, record_format=record_format, io_depth=io_depth,
-                              store_layers=store_layers)
+                              store_layers=store_layers, spec_rows=spec_rows)
         self.dense_layers = dense_layers
         if record_format == nb.NP_REC_INT8:
             # the store the library reads is the 8-bit one; the oracle works on what those

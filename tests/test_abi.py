@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_struct_sizes_match_header():
-    assert C.sizeof(nb.np_config) == 18 * 4
+    assert C.sizeof(nb.np_config) == 20 * 4
     assert C.sizeof(nb.np_sizes) == 11 * 8
     assert C.sizeof(nb.np_buffers) == 11 * C.sizeof(C.c_void_p) + 8
     assert C.sizeof(nb.np_delta_view) == 7 * C.sizeof(C.c_void_p)
@@ -50,7 +50,7 @@ def test_query_sizes_arithmetic(lib):
     assert s.row_buffer_bytes == 32 * 2752 * 4096 * 2
     assert s.staging_bytes == 256 * 24576
     assert s.bitmap_bytes == 32 * 344 * 4 and s.logits_bytes == 32 * 11008 * 4
-    assert s.host_lists_bytes == (16 + 32 * (8 + 2 * 2752)) * 4
+    assert s.host_lists_bytes == 2 * (16 + 32 * (8 + 2 * 2752)) * 4     # incoming rows, then speculative rows
     assert s.workspace_bytes >= s.logits_bytes + 5 * 4096 * 4 + 512 * 4
     assert s.dense_bytes == 0
     # a dense prefix of 8 layers: their records in one buffer, slot buffers for the other 24
@@ -74,7 +74,7 @@ def test_dense_prefix_plan_matches_the_oracle(lib):
 @pytest.mark.parametrize("field,value", [
     ("n_layers", 0), ("d_model", 100), ("d_ffn", 1000), ("d_pred", 7), ("top_k", 9999), ("capacity", 0),
     ("capacity", 99999), ("max_batch", 17), ("evict_policy", 5), ("transfer_mode", 9), ("staging_rows", 0),
-    ("flags", 64), ("store_layers", -1), ("store_layers", 3), ("dense_layers", -1), ("dense_layers", 3), ("io_depth", -2), ("io_depth", 5000),
+    ("flags", 64), ("store_layers", -1), ("store_layers", 3), ("spec_rows", -1), ("spec_rows", 206), ("reserved", 1), ("dense_layers", -1), ("dense_layers", 3), ("io_depth", -2), ("io_depth", 5000),
 ])
 def test_bad_config_is_rejected(lib, field, value):
     cfg = nb.make_config(2, 256, 1024, 64, 102, 205)
