@@ -403,7 +403,7 @@ int np_get_speculative(np_ctx* ctx, int32_t layer, const int32_t** ids, const in
 int np_chain_launches(np_ctx* ctx, int32_t* out);
 
 /* Name of the kernel np_mlp_chain / np_step run the sparse layers' MLP with for B sequences in this
- * context (a static string: "k_mlp_slices", "k_mlp_chain", "k_mlp_chain_alu", "k_mlp_tc_up + k_mlp_tc_down",
+ * context (a static string: "k_mlp_slices", "k_mlp_chain_alu", "k_mlp_tc_up + k_mlp_tc_down",
  * "k_sparse_mlp_pipe" or "k_sparse_mlp").  For reports; NULL if ctx is NULL or B is out of range. */
 const char* np_mlp_kernel_name(np_ctx* ctx, int32_t B);
 

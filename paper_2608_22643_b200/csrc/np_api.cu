@@ -624,7 +624,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   if (d.dense > 0) {
     Dims dd = d;
     dd.k = dd.C = d.M;
-    if ((!dense_chain::supported(d, ctx->sm_count) && !chain_alu::supported(dd, ctx->sm_count)) || (d.dense < d.L && !mlp_chain_supported(d, ctx->sm_count))) {
+    if ((!dense_chain::supported(d, ctx->sm_count) && !chain_alu::supported(dd, ctx->sm_count)) || (d.dense < d.L && !chain_slices::supported(d, ctx->sm_count) && !chain_alu::supported(d, ctx->sm_count))) {
       np_destroy(ctx);
       return fail(nullptr, NP_E_INVAL, "dense_layers > 0: this shape is outside what the resident MLP kernels cover");
     }
@@ -1191,7 +1191,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   const Dims& d = ctx->d;
   const size_t n = (size_t)B * d.D;
   const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
-                          (ctx->use_slices || mlp_chain_supported(d, ctx->sm_count));
+                          (ctx->use_slices || chain_alu::supported(d, ctx->sm_count));
   const bool tc_batch = !persistent && ctx->mlp_tc && B >= kTcMinBatch && !(ctx->cfg.flags & NP_F_DIRECT_LOADS);
   if (part != kChainTail) ctx->chain_kernel_launches = 0;
   // the sliced kernel widens the stack's bf16 input itself when it runs layer 0
@@ -1277,7 +1277,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
         NP_LAUNCH(ctx, chain_slices::launch(d, a, &ctx->slices, s, ctx->sm_count));
       } else {
         ctx->chain_kernel_launches += 1;
-        NP_LAUNCH(ctx, launch_mlp_chain(d, a, s, ctx->sm_count));
+        NP_LAUNCH(ctx, chain_alu::launch(d, a, s, ctx->sm_count));
       }
       l0 = l1;
     }
@@ -1390,8 +1390,6 @@ const char* np_mlp_kernel_name(np_ctx* ctx, int32_t B) {
   const int flags = ctx->cfg.flags;
   if (B == 1 && !(flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES))) {
     if (ctx->use_slices) return "k_mlp_slices";
-    ChainPlan p;
-    if (mlp_chain_plan(d, ctx->sm_count, &p) && (p.single_tile || !chain_alu::supported(d, ctx->sm_count))) return "k_mlp_chain";
     if (chain_alu::supported(d, ctx->sm_count)) return "k_mlp_chain_alu";
   }
   if (ctx->mlp_tc && B >= kTcMinBatch && !(flags & NP_F_DIRECT_LOADS)) return "k_mlp_tc_up + k_mlp_tc_down";

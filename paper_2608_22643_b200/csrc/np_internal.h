@@ -143,15 +143,7 @@ bool mlp_tc_supported(const Dims& d, int sm_count);
 size_t mlp_tc_gu_floats(const Dims& d);
 cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count);
 
-// Persistent multi-layer form of the sparse MLP for one sequence (np_mlp_chain.cu).
-struct ChainPlan {
-  int n_stages, tile_rows, cols;
-  int single_tile;      // the block's expected share of a layer fits the ring as one tile
-  int run_layers;       // layers one launch can span (bounded by the slot cache)
-  int slot_cache_rows;
-  int window_rows;      // records in flight per block (producer pacing)
-  size_t smem;
-};
+// Arguments of the resident multi-layer kernels for one sequence.
 struct ChainArgs {
   const void* gate;  // layer 0 of each row buffer
   const void* up;
@@ -167,15 +159,12 @@ struct ChainArgs {
   int dense_rows;  // > 0 (ALU form only): the layers are dense_rows whole records each, `gate`/`up`/`downT` point
                    // at the three rows of layer 0's first record, active_slots is one identity list
 };
-bool mlp_chain_plan(const Dims& d, int sm_count, ChainPlan* p);
-bool mlp_chain_supported(const Dims& d, int sm_count);
-cudaError_t launch_mlp_chain(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
 namespace dense_chain {  // dense layers, direct loads (np_mlp_dense.cu); same hand-over of x as the other forms
 bool supported(const Dims& d, int sm_count);
 cudaError_t launch(const Dims& d, const void* rec0, int rows, float* const xbuf[2], float* const zbuf[3],
                    unsigned int* grid_bar, int32_t* status, int l_begin, int l_end, cudaStream_t s, int sm_count);
 }  // namespace dense_chain
-namespace chain_alu {  // ALU form of phase 1, for shares that do not fit the ring as one tile (np_mlp_chain_alu.cu)
+namespace chain_alu {  // row-partitioned resident kernel (np_mlp_chain_alu.cu): any row width; the sliced kernel's fallback
 bool supported(const Dims& d, int sm_count);
 cudaError_t launch(const Dims& d, const ChainArgs& a, cudaStream_t s, int sm_count);
 }  // namespace chain_alu

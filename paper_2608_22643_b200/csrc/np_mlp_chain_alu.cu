@@ -1,12 +1,17 @@
-// Stage 4 over a run of layers in one resident kernel, ALU form of phase 1.
+// Stage 4 over a run of layers in one resident kernel, rows dealt whole to the blocks (B = 1).
 //
-// Same structure as np_mlp_chain.cu (one block per SM, ring of shared-memory stages filled by
-// bulk copies, replicated accumulators, grid barrier per layer), but the gate/up dot products
-// run on the ALUs with a (row, segment) item per warp and x_l in shared memory as fp32.  It
-// serves the shapes whose per-block share of a layer does not fit the ring as one tile
-// (D = 5120 and 8192 at the 13B / 70B shapes): there a tile has few rows, and the
-// tensor-core form, which walks the whole K range for 16 MMA rows per tile whatever the
-// tile holds, loses more to its per-tile cost than it gains.
+//   x_{l+1} = x_l + sum_{i in act_l} silu(gate_l[s_i].n_l) * (up_l[s_i].n_l) * downT_l[s_i],
+//   n_l = x_l / sqrt(mean(x_l^2) + 1e-6)
+//
+// (Section 3.4: the sparse MLP reads each active row through the slot map.)  One block per SM
+// stays resident over the run (cooperative launch); every block owns a share of a layer's
+// active rows and a ring of shared-memory stages of one record each, filled by 1-D bulk copies
+// from a producer lane; the gate/up dot products run on the ALUs with a (row, segment) item per
+// warp and x_l in shared memory as fp32; every block adds its partial vector of all D outputs to
+// one of kZRep accumulator copies and a grid-wide counter barrier publishes x_{l+1}.
+// It takes any row width, and is what runs where the column-sliced kernel (np_mlp_slices.cu)
+// does not apply: row widths that are not a multiple of 64, dense layers without the
+// direct-load kernel, and NP_F_ROW_CHAIN.  Every wait is bounded (kStatTimeout on expiry).
 #include <algorithm>
 
 #include "np_device.cuh"

@@ -65,11 +65,49 @@ def test_7b_shape_steps_match_oracle(policy):
         p.close()
 
 
+def test_7b_long_trajectory_every_logit_and_resident_row():
+    """Cold start and fifteen steady-state steps of the whole 32-layer 7B-shaped stack in the benchmark's
+    launch configuration: every logit against the oracle's predictor, the whole selection, every list
+    and table, every resident row of every layer byte for byte, and the chain's output, each step."""
+    cfg = synth.CONFIGS["7b"]
+    L, M, D, W = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_ffn // 32
+    free, _ = torch.cuda.mem_get_info()
+    if free < 8 * 2**30:
+        pytest.skip("needs 8 GB of device memory")
+    p = Pair(cfg, transfer_mode=nb.NP_XFER_HOST_GATHER, staging_rows=2 * cfg.top_k, flags=0, gen_device="cuda")
+    try:
+        n_steps = 16
+        xs = synth.hidden_states(cfg, n_steps)
+        logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")
+        bitmap = torch.empty((L, W), dtype=torch.int32, device="cuda")
+        out = torch.empty((1, D), dtype=torch.float32, device="cuda")
+        w1_u16, w2_u16 = u16(p.w1_cpu), u16(p.w2_cpu)
+        for t in range(n_steps):
+            x = xs[t].cuda()
+            nb.np_predict(p.eng.ctx, x, 1, logits, bitmap, p.eng.stream)
+            rc = nb.np_step(p.eng.ctx, x, 1, out, p.eng.stream, p.eng.copy_stream)
+            assert rc in (nb.NP_OK, nb.NP_W_CHUNKED)
+            torch.cuda.synchronize()
+            z32 = logits.cpu().numpy()
+            z = O.predict(w1_u16, w2_u16, u16(xs[t]), L, M)
+            assert rel_l2(z32, z) < 1e-5 and np.max(np.abs(z32 - z)) < 1e-4 * np.max(np.abs(z)), t
+            assert (bitmap.cpu().numpy().view(np.uint32) == O.topk_bitmap(z32, p.k)).all(), t
+            res = p.ora.step(u16(xs[t]), logits_f32=z32)
+            cnt = p.check_delta_against(res["deltas"])
+            assert (cnt[:, nb.NP_CNT_ACTIVE] == p.k).all() and (cnt[:, nb.NP_CNT_OVERFLOW] == 0).all()
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+            p.check_resident_bytes()
+    finally:
+        p.close()
+
+
 @pytest.mark.parametrize("name,n_layers,mode,chain_layers", [
     ("13b", 3, nb.NP_XFER_HOST_GATHER, 0), ("70b", 2, nb.NP_XFER_ZERO_COPY, 0), ("70b", 2, nb.NP_XFER_MEMCPY_RUNS, 0),
     # several layers per resident launch (the cross-layer hand-over of x at these row widths)
     ("13b", 4, nb.NP_XFER_HOST_GATHER, 4), ("13b", 4, nb.NP_XFER_ZERO_COPY, 2),
     ("70b", 4, nb.NP_XFER_ZERO_COPY, 4), ("70b", 4, nb.NP_XFER_HOST_GATHER, 2),
+    # the row-partitioned resident kernel (the fallback of the column-sliced one) at the same widths
+    ("13b", 4, nb.NP_XFER_HOST_GATHER, -4), ("70b", 4, nb.NP_XFER_ZERO_COPY, -2),
 ])
 def test_larger_shapes_few_layers(name, n_layers, mode, chain_layers):
     """The 13B- and 70B-shaped rows (D = 5120 / 8192, M = 13824 / 28672) on a few layers:
@@ -77,7 +115,8 @@ def test_larger_shapes_few_layers(name, n_layers, mode, chain_layers):
     several layers per resident launch."""
     cfg = synth.CONFIGS[name].with_(n_layers=n_layers)
     L, M, D, W = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_ffn // 32
-    p = Pair(cfg, transfer_mode=mode, flags=nb.NP_F_CHECK_BOUNDS, gen_device="cuda", chain_layers=chain_layers)
+    flags = nb.NP_F_CHECK_BOUNDS | (nb.NP_F_ROW_CHAIN if chain_layers < 0 else 0)     # negative: the row kernel
+    p = Pair(cfg, transfer_mode=mode, flags=flags, gen_device="cuda", chain_layers=abs(chain_layers))
     try:
         xs = synth.hidden_states(cfg, 3)
         logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")

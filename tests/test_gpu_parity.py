@@ -217,6 +217,7 @@ DENSE = synth.StackConfig("dense", 4, 512, 2048, 64, 44, 60, 5, 13, 0.9)
 @pytest.mark.parametrize("flags,chain_layers,ring_stages", [
     (nb.NP_F_CHECK_BOUNDS, 1, 0), (nb.NP_F_CHECK_BOUNDS, 2, 0), (nb.NP_F_CHECK_BOUNDS, 0, 0), (0, 0, 0),
     (nb.NP_F_CHECK_BOUNDS, 0, 2), (nb.NP_F_CHECK_BOUNDS, 3, 3), (nb.NP_F_CHECK_BOUNDS, 0, 4),
+    (nb.NP_F_CHECK_BOUNDS | nb.NP_F_ROW_CHAIN, 0, 0), (nb.NP_F_CHECK_BOUNDS | nb.NP_F_ROW_CHAIN, 2, 3),
     (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0, 0),
     (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0, 2),
     (nb.NP_F_CHECK_BOUNDS | nb.NP_F_LAYER_LAUNCHES, 0, 5),
