@@ -1252,15 +1252,34 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
     // (the tail is an eighth of the stack, the run before it a quarter, the first run takes the rest), which
     // also makes fewer launches than equal runs of a quarter each.
     std::vector<int> runs;
-    {
-      const int ns = d.L - d.dense;
+    if (part != kChainHead) {
+      // layers whose rows have all landed already need no run of their own to wait in: they go into one
+      // first run (the whole stack when nothing is pending, as in np_mlp_chain on resident rows)
+      int landed = d.dense;
+      while (landed < d.L) {
+        if (ctx->install_pending[landed]) {
+          const cudaError_t q = cudaEventQuery(ctx->ev_installed[landed]);
+          if (q == cudaErrorNotReady) {
+            (void)cudaGetLastError();
+            break;
+          }
+          if (q != cudaSuccess) return fail(ctx, NP_E_CUDA, "cudaEventQuery failed: %s", cudaGetErrorString(q));
+          ctx->install_pending[landed] = 0;
+        }
+        ++landed;
+      }
+      const int ns = d.L - landed;  // layers that still wait for rows
       if (ctx->cfg.chain_layers > 0) {
-        for (int l0 = 0; l0 < ns; l0 += run) runs.push_back(std::min(run, ns - l0));
-      } else if (ns > 0) {
-        const int tail = std::max(1, ns / 8), mid = std::min(ns - tail, 2 * tail), first = ns - tail - mid;
-        if (first > 0) runs.push_back(first);
-        if (mid > 0) runs.push_back(mid);
-        runs.push_back(tail);
+        for (int l0 = d.dense; l0 < d.L; l0 += run) runs.push_back(std::min(run, d.L - l0));
+      } else {
+        if (landed > d.dense) runs.push_back(landed - d.dense);
+        if (ns > 0) {
+          const int unit = std::max(1, (d.L - d.dense) / 8);
+          const int tail = std::min(ns, unit), mid = std::min(ns - tail, 2 * unit), first = ns - tail - mid;
+          if (first > 0) runs.push_back(first);
+          if (mid > 0) runs.push_back(mid);
+          runs.push_back(tail);
+        }
       }
     }
     int l0 = d.dense;

@@ -755,8 +755,6 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   const int VG = 1 << vg_shift;
   const size_t group_bytes = (size_t)VG * pstride;
   const size_t budget = 227 * 1024 - 2048;  // static shared memory of the kernel
-  p->run_layers = std::max(1, std::min(kMaxLayers, 8192 / (4 * max_rows)));
-  p->slot_cache_rows = p->run_layers * max_rows;
   const int apad = ((max_rows + 15) & ~15) + 16;
   const int n_gu_max = (2 * max_rows + VG - 1) / VG;
   // phase 1 deals a layer's gate|up groups to sets of GW warps: as many sets as the expected share has groups
@@ -765,11 +763,17 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   int gw_shift = 3;
   while (gw_shift > 0 && (kWarps >> gw_shift) < n_gu_typ) --gw_shift;
   const int GW = 1 << gw_shift;
-  const size_t fixed = 3 * pstride + (size_t)Ds * 4 + (size_t)n_gu_max * GW * VG * 4 + (size_t)(3 * apad + (apad & 1)) * 2 +
-                       (size_t)p->slot_cache_rows * 4 + 64;
-  if (fixed + 3 * group_bytes > budget) return false;
-  int ng = (int)std::min<size_t>(kMaxGroups, (budget - fixed) / group_bytes);
+  // everything but the ring and the slot cache; the cache (the slots of a launch's rows) takes a minimum first
+  // and, once the ring's slots are counted, whatever is left, so that a launch can span more layers
+  const size_t fixed0 = 3 * pstride + (size_t)Ds * 4 + (size_t)n_gu_max * GW * VG * 4 + (size_t)(3 * apad + (apad & 1)) * 2 + 64;
+  const size_t cache_min = std::max<size_t>(4 * (size_t)max_rows, std::min<size_t>(8192, 4 * (size_t)max_rows * 8));
+  if (fixed0 + cache_min + 3 * group_bytes > budget) return false;
+  int ng = (int)std::min<size_t>(kMaxGroups, (budget - fixed0 - cache_min) / group_bytes);
   if (d.ring_stages >= 2) ng = std::max(3, std::min(ng, d.ring_stages));
+  const size_t cache_bytes = std::min<size_t>(budget - fixed0 - (size_t)ng * group_bytes, 4 * (size_t)max_rows * kMaxLayers);
+  p->run_layers = (int)std::max<size_t>(1, std::min<size_t>(kMaxLayers, cache_bytes / (4 * (size_t)max_rows)));
+  p->slot_cache_rows = p->run_layers * max_rows;
+  const size_t fixed = fixed0 + (size_t)p->slot_cache_rows * 4;
   int window = std::max(1, std::min(ng - 1, (int)(40 * 1024 / group_bytes)));
 #ifdef NP_TUNE  // development builds only: geometry from the environment
   if (const char* e = getenv("NP_SL_NG")) ng = std::max(2, std::min(ng, atoi(e)));
