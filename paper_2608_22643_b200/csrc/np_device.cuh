@@ -113,6 +113,33 @@ __device__ __forceinline__ int block_exclusive_scan(int* a, int n, int* red) {
   return total;
 }
 
+// Inclusive scan of one int per thread over a block of 1024 threads, in thread order; returns
+// this thread's inclusive value and leaves the block's total in wsum[32].  wsum: 33 ints of
+// shared scratch.  Two block-wide barriers; a caller that scans again puts one between the calls.
+__device__ __forceinline__ int block_inclusive_scan_1024(int v, int* wsum, int lane, int wid) {
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) wsum[wid] = inc;
+  __syncthreads();
+  if (wid == 0) {
+    const int ws = wsum[lane];
+    int winc = ws;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    wsum[lane] = winc - ws;
+    if (lane == 31) wsum[32] = winc;
+  }
+  __syncthreads();
+  return wsum[wid] + inc;
+}
+
 // The n lowest set bits of m (all of m if it has fewer).
 __device__ __forceinline__ uint32_t lowest_bits(uint32_t m, int n) {
   if (n <= 0) return 0u;

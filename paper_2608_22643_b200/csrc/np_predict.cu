@@ -61,6 +61,38 @@ __global__ void __launch_bounds__(128) k_pred_l1(const uint4* __restrict__ w1,
   }
 }
 
+// One sequence: a row per block, a quarter of the row per warp, so that (for rows of up to
+// 4096 values) every weight load of the kernel is issued at once and the kernel lasts one
+// trip to memory, not four; the layer behind it waits for exactly this kernel.
+__global__ void __launch_bounds__(128) k_pred_l1_row(const uint4* __restrict__ w1, const uint4* __restrict__ x,
+                                                      float* __restrict__ hidden, int H, int D) {
+  __shared__ float part[4];
+  npp::pdl_launch_dependents();  // layer 2 may start prefetching its weights now
+  const int row = blockIdx.x, lane = threadIdx.x & 31, wq = threadIdx.x >> 5;
+  const int chunks = D >> 3;  // 16-byte chunks per row
+  const uint4* wr = w1 + (size_t)row * chunks;
+  float acc = 0.f;
+  for (int c0 = wq * 128; c0 < chunks; c0 += 512) {
+    uint4 w[4], xv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = c0 + u * 32 + lane;
+      w[u] = c < chunks ? ldg_stream(wr + c) : make_uint4(0, 0, 0, 0);
+      xv[u] = c < chunks ? __ldg(x + c) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float4 xa = make_float4(bf16_lo(xv[u].x), bf16_hi(xv[u].x), bf16_lo(xv[u].y), bf16_hi(xv[u].y));
+      const float4 xb = make_float4(bf16_lo(xv[u].z), bf16_hi(xv[u].z), bf16_lo(xv[u].w), bf16_hi(xv[u].w));
+      acc = dot8(w[u], xa, xb, acc);
+    }
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) part[wq] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) hidden[row] = fmaxf((part[0] + part[1]) + (part[2] + part[3]), 0.f);
+}
+
 // Batched form (B > 4): the B input vectors are staged once per block in shared memory (as
 // bf16), so that a weight chunk is multiplied with all sequences without going back to L1/L2
 // for x; one warp per output row.
@@ -108,7 +140,7 @@ cudaError_t launch_pred_l1(const Dims& d, const void* w1, const void* x_bf16, in
   const uint4* w = static_cast<const uint4*>(w1);
   const uint4* x = static_cast<const uint4*>(x_bf16);
   if (B == 1)
-    k_pred_l1<1><<<blocks, threads, 0, s>>>(w, x, hidden, d.H, d.D, B);
+    k_pred_l1_row<<<d.H, threads, 0, s>>>(w, x, hidden, d.H, d.D);
   else if (B <= 4)
     k_pred_l1<4><<<blocks, threads, 0, s>>>(w, x, hidden, d.H, d.D, B);
   else {
@@ -357,6 +389,7 @@ __global__ void __launch_bounds__(kL2dThreads, 1) k_pred_l2_direct(const uint4* 
   long long base = r_begin + (long long)wid * kGroup;
   if (base < r_end) load(base);
   npp::pdl_wait_prior();
+  npp::pdl_launch_dependents();  // the selection's blocks take the SMs as this grid's blocks leave them
   float hreg[CPL * 8];
 #pragma unroll
   for (int i = 0; i < CPL; ++i) {

@@ -85,10 +85,12 @@ def test_topk_edge_cases():
 @pytest.mark.parametrize("cfg,n_set,C,persist", [
     (TINY, 102, 205, 0.8), (TINY, 102, 102, 0.6), (SMALL, 208, 520, 0.83), (SMALL, 700, 520, 0.7),
     (TINY, 1, 1, 0.0), (TINY, 0, 4, 0.5),
+    (TINY.with_(d_ffn=12288), 5000, 6000, 0.3), (TINY.with_(d_ffn=12288), 7000, 6000, 0.3),
 ])
 def test_delta_lists_and_tables_bit_exact(policy, cfg, n_set, C, persist):
     """Injected bitmap sequences (fixed-size sets, full replacement, oversize sets that
-    overflow capacity, the empty set) against the oracle, every step."""
+    overflow capacity, the empty set, lists of several thousand rows: longer than what the
+    kernel keeps in shared memory) against the oracle, every step."""
     T = 10
     p = Pair(cfg, policy=policy, k=min(n_set, C), C=C)
     try:
