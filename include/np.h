@@ -99,7 +99,11 @@ extern "C" {
 #define NP_F_LAYER_LAUNCHES  4  /* np_step / np_mlp_chain: one kernel launch per layer instead
                                    of resident kernels spanning runs of layers */
 #define NP_F_ROW_CHAIN      32  /* np_step / np_mlp_chain, one sequence: the resident MLP kernel that deals whole rows
-                                   to the blocks instead of the column-sliced one (for comparison runs) */
+                                   to single blocks and reduces through global memory only, instead of the cluster or the
+                                   column-sliced one (for comparison runs) */
+#define NP_F_CLUSTER_ROWS   64  /* np_step / np_mlp_chain, one sequence: the resident MLP kernel that deals whole rows to
+                                   blocks in clusters of four and reduces inside the cluster first (where it applies:
+                                   row widths of 1024 to 4096 in steps of 1024), instead of the column-sliced one */
 #define NP_F_MAPPED_STAGING 16  /* NP_XFER_HOST_GATHER / NP_XFER_FILE: no staging copy; the scatter kernel
                                    reads the records in the pinned staging buffer through its device
                                    mapping (Section 3.5: the staging is page-aligned host memory registered

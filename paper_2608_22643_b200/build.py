@@ -14,7 +14,7 @@ INCLUDE = os.path.join(ROOT, "include")
 OBJ_DIR = os.path.join(HERE, "build")
 LIB_PATH = os.path.join(HERE, "libnp.so")
 
-SOURCES = ["np_api.cu", "np_predict.cu", "np_topk.cu", "np_centroid.cu", "np_delta.cu", "np_scatter.cu", "np_mlp.cu", "np_mlp_tc.cu", "np_mlp_chain_alu.cu", "np_mlp_slices.cu", "np_mlp_dense.cu", "np_static.cu", "np_io.cu", "np_trunk.cu", "np_predict_tc.cu"]
+SOURCES = ["np_api.cu", "np_predict.cu", "np_topk.cu", "np_centroid.cu", "np_delta.cu", "np_scatter.cu", "np_mlp.cu", "np_mlp_tc.cu", "np_mlp_chain_alu.cu", "np_mlp_slices.cu", "np_mlp_rows.cu", "np_mlp_dense.cu", "np_static.cu", "np_io.cu", "np_trunk.cu", "np_predict_tc.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

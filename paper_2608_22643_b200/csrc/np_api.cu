@@ -201,6 +201,8 @@ struct np_ctx {
   PredTcState tc = {};
   chain_slices::State slices = {};  // column-sliced resident MLP kernel: its counters, exchange words and their values
   bool use_slices = false;
+  chain_rows::State rows = {};  // cluster form of the resident MLP kernel (whole rows per block): its accumulators and counters
+  bool use_rows = false;
   int chain_kernel_launches = 0;    // MLP kernel launches of the last np_mlp_chain / np_step
   size_t gu_bytes = 0;   // both dot-product accumulators of the batch MLP, contiguous
   bool mlp_tc = false;   // batches run the tensor-core MLP kernels
@@ -257,7 +259,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->transfer_mode == NP_XFER_FILE && c->record_format != NP_REC_BF16)
     return fail(ctx, NP_E_INVAL, "NP_XFER_FILE needs NP_REC_BF16 records");
   if (c->io_depth < -1 || c->io_depth > 4096) return fail(ctx, NP_E_INVAL, "io_depth must be in [-1, 4096]");
-  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES | NP_F_MAPPED_STAGING | NP_F_ROW_CHAIN)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
+  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES | NP_F_MAPPED_STAGING | NP_F_ROW_CHAIN | NP_F_CLUSTER_ROWS)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
   if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
@@ -516,6 +518,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_ident = take(d.dense > 0 ? (size_t)d.M : 1);
   const size_t o_spid = take(LC), o_spsl = take(LC), o_spcnt = take((size_t)d.L * NP_N_COUNTERS), o_spcand = take(LW);
   const size_t o_sbar = take(chain_slices::bar_words()), o_sxch = take(2 * chain_slices::xch_words(d, ctx->sm_count));
+  const size_t o_rz = take(chain_rows::z_floats(d)), o_rcnt = take(4);
   NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
   char* base = static_cast<char*>(ctx->slab);
   Tables& t = ctx->t;
@@ -547,6 +550,12 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   NP_INIT_CUDA(cudaMemset(ctx->slices.bars, 0, chain_slices::bar_words() * 4));
   NP_INIT_CUDA(cudaMemset(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8));
   ctx->use_slices = !(cfg->flags & NP_F_ROW_CHAIN) && chain_slices::supported(d, ctx->sm_count);
+  ctx->rows.z4 = reinterpret_cast<float*>(base + o_rz);
+  ctx->rows.cnt = reinterpret_cast<unsigned int*>(base + o_rcnt);
+  ctx->rows.cnt_base = ctx->rows.seq = 0;
+  NP_INIT_CUDA(cudaMemset(ctx->rows.z4, 0, chain_rows::z_floats(d) * 4));
+  NP_INIT_CUDA(cudaMemset(ctx->rows.cnt, 0, 4 * 4));
+  ctx->use_rows = (cfg->flags & NP_F_CLUSTER_ROWS) && !(cfg->flags & NP_F_ROW_CHAIN) && d.dense < d.L && chain_rows::prepare(d, ctx->sm_count, &ctx->rows);
 
   const WsLayout wl = ws_layout(*cfg);
   char* wsb = static_cast<char*>(b->workspace);
@@ -677,6 +686,9 @@ int np_reset(np_ctx* ctx, void* stream) {
   NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.bars, 0, chain_slices::bar_words() * 4, as_stream(stream)));
   NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8, as_stream(stream)));
   ctx->slices.bar_base = ctx->slices.seq_base = 0;
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->rows.z4, 0, chain_rows::z_floats(ctx->d) * 4, as_stream(stream)));
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->rows.cnt, 0, 4 * 4, as_stream(stream)));
+  ctx->rows.cnt_base = ctx->rows.seq = 0;
   ctx->have_delta = ctx->have_pred = ctx->have_step = ctx->have_spec = false;
   std::fill(ctx->install_pending.begin(), ctx->install_pending.end(), 0);
   ctx->step = 0;
@@ -914,6 +926,8 @@ static int install_host_gather(np_ctx* ctx, int layer_begin, int layer_end, cuda
   };
   std::vector<Piece> batch;
   int h = -1, used = 0, layers_in = 0, last_l = -1;
+  int flushed = 0;  // parts handed to the copy engine by this call
+  const int first_small = 1;  // the first part takes one layer: the copy engine starts sooner
   auto open_part = [&]() -> int {
     h = ctx->next_half % parts;
     ctx->next_half = (h + 1) % parts;
@@ -981,6 +995,7 @@ static int install_host_gather(np_ctx* ctx, int layer_begin, int layer_end, cuda
     }
     batch.clear();
     h = -1;
+    ++flushed;
     return NP_OK;
   };
   for (int l = layer_begin; l < layer_end; ++l) {
@@ -992,7 +1007,7 @@ static int install_host_gather(np_ctx* ctx, int layer_begin, int layer_end, cuda
     int first = 0;
     do {
       const int rows = std::min(part_rows, n - first);
-      if (h >= 0 && (used + rows > part_rows || (l != last_l && layers_in >= kGatherLayers))) {
+      if (h >= 0 && (used + rows > part_rows || (l != last_l && layers_in >= (flushed < first_small ? 1 : kGatherLayers)))) {
         const int rc = flush();
         if (rc < 0) return rc;
       }
@@ -1191,11 +1206,11 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   const Dims& d = ctx->d;
   const size_t n = (size_t)B * d.D;
   const bool persistent = B == 1 && !(ctx->cfg.flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES)) &&
-                          (ctx->use_slices || chain_alu::supported(d, ctx->sm_count));
+                          (ctx->use_rows || ctx->use_slices || chain_alu::supported(d, ctx->sm_count));
   const bool tc_batch = !persistent && ctx->mlp_tc && B >= kTcMinBatch && !(ctx->cfg.flags & NP_F_DIRECT_LOADS);
   if (part != kChainTail) ctx->chain_kernel_launches = 0;
   // the sliced kernel widens the stack's bf16 input itself when it runs layer 0
-  const bool fold_widen = persistent && ctx->use_slices && d.dense == 0;
+  const bool fold_widen = persistent && (ctx->use_rows || ctx->use_slices) && d.dense == 0;
   if (part != kChainTail) {
     if (!fold_widen) NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
     // the accumulator of layer 0 starts at zero (later ones are cleared one layer ahead)
@@ -1289,7 +1304,11 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
         if (ctx->install_pending[l]) NP_CUDA(ctx, wait_install(ctx, l, s));
       a.l_begin = l0;
       a.l_end = l1;
-      if (ctx->use_slices) {
+      if (ctx->use_rows) {
+        const int rl = chain_rows::run_layers(d, ctx->rows);
+        ctx->chain_kernel_launches += (l1 - l0 + rl - 1) / rl;
+        NP_LAUNCH(ctx, chain_rows::launch(d, a, &ctx->rows, s));
+      } else if (ctx->use_slices) {
         chain_slices::Plan sp;
         chain_slices::plan(d, ctx->sm_count, &sp);
         ctx->chain_kernel_launches += (l1 - l0 + sp.run_layers - 1) / sp.run_layers;
@@ -1408,6 +1427,7 @@ const char* np_mlp_kernel_name(np_ctx* ctx, int32_t B) {
   const Dims& d = ctx->d;
   const int flags = ctx->cfg.flags;
   if (B == 1 && !(flags & (NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES))) {
+    if (ctx->use_rows) return "k_mlp_rows";
     if (ctx->use_slices) return "k_mlp_slices";
     if (chain_alu::supported(d, ctx->sm_count)) return "k_mlp_chain_alu";
   }

@@ -188,6 +188,22 @@ size_t bar_words();
 cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s, int sm_count);
 }  // namespace chain_slices
 
+namespace chain_rows {  // whole rows per block, blocks in clusters (np_mlp_rows.cu); same hand-over of x
+// Library-owned device words and the host's running record of them: the counters only ever grow
+// and the accumulators are used in rotation, so nothing has to be cleared between launches.
+struct State {
+  float* z4;          // [z_floats(d)] zero at init / reset
+  unsigned int* cnt;  // [4] zero at init / reset
+  unsigned int cnt_base, seq;
+  int grid;           // blocks of a launch (0: the kernel does not apply)
+};
+size_t z_floats(const Dims& d);
+bool prepare(const Dims& d, int sm_count, State* st);
+bool supported(const Dims& d, const State& st);
+int run_layers(const Dims& d, const State& st);
+cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s);
+}  // namespace chain_rows
+
 cudaError_t launch_selftest_wait(int32_t* status, cudaStream_t s);
 cudaError_t launch_widen_bf16(const void* x_bf16, float* out, size_t n, cudaStream_t s);
 // out = a + sum of `reps` consecutive copies of b (each n floats)
