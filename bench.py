@@ -66,6 +66,9 @@ def parse_args():
     ap.add_argument("--layer-launches", action="store_true", help="one MLP kernel launch per layer")
     ap.add_argument("--direct-loads", action="store_true", help="MLP rows by plain global loads")
     ap.add_argument("--chain-layers", type=int, default=0, help="layers per resident MLP kernel")
+    ap.add_argument("--mlp-kernel", default="auto", choices=["auto", "cluster-rows", "row-chain"],
+                    help="resident sparse-MLP kernel for one sequence: the library's choice, whole rows per block with "
+                         "blocks in clusters (NP_F_CLUSTER_ROWS), or whole rows with a global reduction only (NP_F_ROW_CHAIN)")
     ap.add_argument("--capacity-pct", type=int, default=None, help="resident capacity in percent of FFN rows")
     ap.add_argument("--store-layers", default="auto",
                     help="layers of records the host store holds (layer l reads layer l mod this); 'auto' = all of them "
@@ -376,6 +379,7 @@ def cuda_arm(args):
                           host_threads=args.host_threads, dense_layers=args.dense_layers, io_depth=args.io_depth,
                           store_layers=Lp if Lp < cfg.n_layers else 0, spec_rows=args.spec_rows,
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
+                          | {"auto": 0, "cluster-rows": nb.NP_F_CLUSTER_ROWS, "row-chain": nb.NP_F_ROW_CHAIN}[args.mlp_kernel]
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0)
                           | (nb.NP_F_MAPPED_STAGING if args.mapped_staging else 0))
     storage = None

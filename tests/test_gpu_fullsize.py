@@ -12,16 +12,17 @@ from tests.harness import REL_L2_TOL, Pair, rel_l2, u16
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("policy", [nb.NP_EVICT_EXACT, nb.NP_EVICT_LRU])
-def test_7b_shape_steps_match_oracle(policy):
+@pytest.mark.parametrize("policy,mlp_flags", [(nb.NP_EVICT_EXACT, 0), (nb.NP_EVICT_LRU, 0), (nb.NP_EVICT_EXACT, nb.NP_F_CLUSTER_ROWS)])
+def test_7b_shape_steps_match_oracle(policy, mlp_flags):
     cfg = synth.CONFIGS["7b"]
     L, M, D, W = cfg.n_layers, cfg.d_ffn, cfg.d_model, cfg.d_ffn // 32
     free, _ = torch.cuda.mem_get_info()
     if free < 8 * 2**30:
         pytest.skip("needs 8 GB of device memory")
     p = Pair(cfg, policy=policy, transfer_mode=nb.NP_XFER_HOST_GATHER, staging_rows=2 * cfg.top_k,
-             flags=0, gen_device="cuda")
+             flags=mlp_flags, gen_device="cuda")
     try:
+        assert nb.np_mlp_kernel_name(p.eng.ctx, 1) == ("k_mlp_rows" if mlp_flags else "k_mlp_slices")
         n_steps = 3
         xs = synth.hidden_states(cfg, n_steps)
         logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")

@@ -383,6 +383,40 @@ def test_widest_model_with_several_layers_per_launch(chain_layers):
     test_limit_shapes(("max_model_chain", 4, 16384, 64, 64, 25, 50), 1, chain_layers=chain_layers)
 
 
+@pytest.mark.parametrize("D,M,L,chain_layers,dense,policy", [
+    (1024, 4096, 5, 0, 0, nb.NP_EVICT_EXACT),     # three rows a block, all layers in one launch
+    (2048, 2048, 4, 2, 0, nb.NP_EVICT_LRU),       # x handed from launch to launch
+    (4096, 4096, 3, 1, 0, nb.NP_EVICT_EXACT),     # the 7B row width, a launch per layer
+    (1024, 16384, 3, 0, 0, nb.NP_EVICT_EXACT),    # eleven rows a block: two MMA row blocks, two batches of tensor-memory reads
+    (1024, 4096, 5, 0, 2, nb.NP_EVICT_EXACT),     # behind a dense prefix: the run starts from another kernel's hand-over
+])
+def test_cluster_rows_kernel(D, M, L, chain_layers, dense, policy):
+    """NP_F_CLUSTER_ROWS: whole rows per block, blocks in clusters that reduce among themselves through distributed
+    shared memory, down rows parked in tensor memory.  The whole step against the oracle, every step."""
+    cfg = synth.StackConfig("cluster_rows", L, D, M, 64, 10, 25, 4, 77, 0.9)
+    p = Pair(cfg, policy=policy, flags=nb.NP_F_CHECK_BOUNDS | nb.NP_F_CLUSTER_ROWS, chain_layers=chain_layers, dense_layers=dense)
+    try:
+        assert nb.np_mlp_kernel_name(p.eng.ctx, 1) == "k_mlp_rows"
+        xs = synth.hidden_states(cfg, 4)
+        out = torch.empty((1, D), dtype=torch.float32, device="cuda")
+        logits = torch.empty((1, L, M), dtype=torch.float32, device="cuda")
+        for t in range(4):
+            nb.np_predict(p.eng.ctx, xs[t].cuda(), 1, logits, None, p.eng.stream)
+            nb.np_step(p.eng.ctx, xs[t].cuda(), 1, out, p.eng.stream, p.eng.copy_stream)
+            torch.cuda.synchronize()
+            res = p.ora.step(u16(xs[t]), logits_f32=logits.cpu().numpy())
+            p.check_delta_against(res["deltas"])
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5, t
+        # the chain alone, twice: the kernel's counters and accumulators carry over from launch to launch
+        for _ in range(2):
+            nb.np_mlp_chain(p.eng.ctx, xs[3].cuda(), 1, out, p.eng.stream)
+            torch.cuda.synchronize()
+            assert rel_l2(out.cpu().numpy(), res["x_final"]) < 1e-5
+        p.eng.counters()    # reading the counters also checks the status word
+    finally:
+        p.close()
+
+
 @pytest.mark.parametrize("mode,dense", [(nb.NP_XFER_MEMCPY_RUNS, 0), (nb.NP_XFER_HOST_GATHER, 0), (nb.NP_XFER_ZERO_COPY, 0),
                                         (nb.NP_XFER_HOST_GATHER, 3), (nb.NP_XFER_FILE, 0), (nb.NP_XFER_FILE, 3)])
 def test_store_aliased_over_fewer_layers(mode, dense, tmp_path):
