@@ -632,9 +632,16 @@ cudaError_t launch_delta(const Dims& d, const Tables& t, const uint32_t* pred, i
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (sm > 48 * 1024) {  // only the widest layers with every row resident
-    cudaError_t e = cudaFuncSetAttribute(k_delta, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+  if (sm > 48 * 1024) {
+    static size_t allowed[64] = {};  // per device: the attribute sticks to the function, set it when a launch needs more than before
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || sm > allowed[dev]) {
+      e = cudaFuncSetAttribute(k_delta, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+      if (e != cudaSuccess) return e;
+      if (dev >= 0 && dev < 64) allowed[dev] = sm;
+    }
   }
   return cudaLaunchKernelEx(&cfg, k_delta, p);
 }
