@@ -62,7 +62,7 @@ constexpr int kMaxGroups = 16;         // ring slots
 constexpr int kMaxLayers = 64;         // layers per launch (longer runs are split by the host)
 constexpr int kBarStride = 32;         // one 128-byte line per barrier counter
 constexpr int kHist = 8;               // pacing history of the producer (> window)
-constexpr int kGroupTarget = 36 * 1024;
+constexpr int kGroupTarget = 42 * 1024;
 constexpr int kPad = 16;               // bytes between pieces in shared memory
 
 struct KArgs {
