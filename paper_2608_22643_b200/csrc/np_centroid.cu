@@ -16,8 +16,7 @@ using namespace npd;
 
 constexpr int kCentroidThreads = 256;
 
-__device__ __forceinline__ uint32_t centroid_order_key(float z) {
-  const uint32_t b = __float_as_uint(z);
+__device__ __forceinline__ uint32_t centroid_order_key(uint32_t b) {  // the fp32 value's bit pattern (a float move may flush a denormal)
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
@@ -37,7 +36,7 @@ __global__ void __launch_bounds__(kCentroidThreads)
     unsigned long long best = 0ull;  // below every real entry: keys are never 0 with index bits set
     for (int c = tid; c < K; c += kCentroidThreads) {
       const unsigned long long v =
-          ((unsigned long long)centroid_order_key(__ldg(z + (size_t)h * K + c)) << 32) | (uint32_t)(~(uint32_t)c);
+          ((unsigned long long)centroid_order_key(__ldg(reinterpret_cast<const uint32_t*>(z) + (size_t)h * K + c)) << 32) | (uint32_t)(~(uint32_t)c);
       best = v > best ? v : best;
     }
 #pragma unroll

@@ -39,10 +39,8 @@ extern "C" int np_debug_tk(void* out) { return (int)cudaMemcpyFromSymbol(out, np
 #define TK(ev) do { } while (0)
 #endif
 
-__device__ __forceinline__ uint32_t order_key(float z) {
-  const uint32_t b = __float_as_uint(z);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
+// bit pattern of an fp32 value -> order-preserving uint32 (larger float, larger key; +0 above -0)
+__device__ __forceinline__ uint32_t order_key(uint32_t b) { return (b & 0x80000000u) ? ~b : (b | 0x80000000u); }
 
 // KPT: keys per thread, ceil(M / 1024)
 template <int KPT>
@@ -80,20 +78,23 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
     return;
   }
 
-  float zv[KPT];
+  // The logits are kept as bit patterns: the keys must be exact, and floating-point moves under flush-to-zero
+  // arithmetic need not preserve a denormal.  Only the fast path's bin arithmetic looks at them as numbers.
+  uint32_t zb[KPT];
   float lo = __int_as_float(0x7f800000), hi = __int_as_float(0xff800000);
   int bad = 0;
+  const uint32_t* zbits = reinterpret_cast<const uint32_t*>(z);
 #pragma unroll
   for (int j = 0; j < KPT; ++j) {
     const int i = tid + kTopkThreads * j;
-    zv[j] = i < M ? z[i] : 0.f;  // entries past the layer's end are never counted (every use tests the index)
+    zb[j] = i < M ? zbits[i] : 0u;  // entries past the layer's end are never counted (every use tests the index)
   }
 #pragma unroll
   for (int j = 0; j < KPT; ++j) {
     if (tid + kTopkThreads * j < M) {
-      bad |= (__float_as_uint(zv[j]) & 0x7f800000u) == 0x7f800000u;  // infinity or NaN
-      lo = fminf(lo, zv[j]);
-      hi = fmaxf(hi, zv[j]);
+      bad |= (zb[j] & 0x7f800000u) == 0x7f800000u;  // infinity or NaN
+      lo = fminf(lo, __uint_as_float(zb[j]));
+      hi = fmaxf(hi, __uint_as_float(zb[j]));
     }
   }
   hist[tid] = 0;
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
     auto bin_of = [&](float v) { return min(kLinBins - 1, (int)((v - lo) * scale)); };
 #pragma unroll
     for (int j = 0; j < KPT; ++j)
-      if (tid + kTopkThreads * j < M) atomicAdd(&hist[bin_of(zv[j])], 1);
+      if (tid + kTopkThreads * j < M) atomicAdd(&hist[bin_of(__uint_as_float(zb[j]))], 1);
     __syncthreads();
     TK(4);
     // the bin of the k-th largest key: thread t takes the two highest bins not taken by the threads below it
@@ -153,7 +154,7 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
       for (int j = 0; j < KPT; ++j) {
         const int i = tid + kTopkThreads * j;
         const int w = wid + 32 * j;  // the word of neurons 32 w .. 32 w + 31: this warp's logits of round j
-        const int bn = i < M ? bin_of(zv[j]) : -1;
+        const int bn = i < M ? bin_of(__uint_as_float(zb[j])) : -1;
         const uint32_t gt = __ballot_sync(0xffffffffu, bn > bstar);
         if (lane == 0 && w < W) {
           if (use_atomic) {
@@ -164,7 +165,7 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
         }
         if (bn == bstar) {
           const int q = atomicAdd(&s_ncand, 1);
-          ckey[q] = order_key(zv[j]);
+          ckey[q] = order_key(zb[j]);
           cidx[q] = i;
         }
       }
@@ -208,7 +209,7 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
     int* my_hist = pass == 0 ? hist + wid * 256 : hist;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
-      const uint32_t key = order_key(zv[j]);
+      const uint32_t key = order_key(zb[j]);
       const bool in = tid + kTopkThreads * j < M && (key & mask) == prefix;
       // lanes with the same digit add once
       const uint32_t d = in ? (key >> shift) & dmask : 0xffffffffu;
@@ -261,7 +262,7 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
       const int w = wid + 32 * j;
-      const uint32_t eq = __ballot_sync(0xffffffffu, tid + kTopkThreads * j < M && order_key(zv[j]) == thr);
+      const uint32_t eq = __ballot_sync(0xffffffffu, tid + kTopkThreads * j < M && order_key(zb[j]) == thr);
       if (lane == 0 && w < W) wsm[w] = __popc(eq);
     }
     block_exclusive_scan(wsm, W, hist);
@@ -270,7 +271,7 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk(const float* __restrict__
   for (int j = 0; j < KPT; ++j) {
     const int w = wid + 32 * j;
     const bool valid = tid + kTopkThreads * j < M;
-    const uint32_t key = order_key(zv[j]);
+    const uint32_t key = order_key(zb[j]);
     const uint32_t gt = __ballot_sync(0xffffffffu, valid && key > thr);
     const uint32_t eq = __ballot_sync(0xffffffffu, valid && key == thr);
     if (lane == 0 && w < W) {

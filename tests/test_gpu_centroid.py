@@ -39,6 +39,7 @@ def test_select_matches_oracle_bit_for_bit(cfg, B, K):
             z[-1, -1, 1, K // 2] = 0.0
             z[0, -1, 0, K - 1] = np.inf
             z[0, -1, 0, 0] = -np.inf
+            z[0, 0, 1, :] = (rng.standard_normal(K) * 1e-42).astype(np.float32)    # a head whose logits are all denormal
         ids, words = _select(p, torch.from_numpy(z).cuda(), B, K, bank.cuda())
         want_ids, want_words = O.centroid_select(z, bank.numpy().view(np.uint32))
         assert (ids == want_ids).all()

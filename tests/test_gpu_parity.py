@@ -81,6 +81,40 @@ def test_topk_edge_cases():
             p.close()
 
 
+def test_topk_paths_of_the_selection_kernel():
+    """The selection kernel bins the logits linearly and ranks the deciding bin directly; ranges, ties and
+    clusters that it has to hand to its general (radix) path, and the boundary between the two."""
+    cfg = TINY.with_(d_ffn=4096)
+    L, M = cfg.n_layers, cfg.d_ffn
+    rng = np.random.default_rng(5)
+    p = Pair(cfg, with_oracle=False)
+    try:
+        k = p.k
+        assert 300 < k < 1000
+        z = rng.standard_normal((1, L, M)).astype(np.float32)
+        z[:, :, 7] = 3e38; z[:, :, 9] = -3e38                               # max - min overflows
+        _topk_case(p, z)
+        for n_tie in (1024, 1025, 2000):                                    # n_tie equal keys around the k-th place
+            z = rng.standard_normal((1, L, M)).astype(np.float32)
+            order = np.argsort(-z[0], axis=1)
+            for l in range(L):
+                v = z[0, l, order[l, k]]
+                idx = rng.permutation(order[l, k - 200:k - 200 + n_tie])    # 200 of them above the cut, the rest below
+                z[0, l, idx] = v
+            _topk_case(p, z)
+        z = (1.0 + rng.permutation(M)[None, None, :].repeat(L, 1) * 2.0**-23).astype(np.float32)   # consecutive floats
+        _topk_case(p, z)
+        z = rng.standard_normal((1, L, M)).astype(np.float32) * 1e-3        # two far clusters, the cut inside the lower one
+        z[:, :, :200] += 1e6
+        _topk_case(p, z)
+        z = rng.standard_normal((1, L, M)).astype(np.float32) * 1e-42       # denormals only
+        _topk_case(p, z)
+        z = np.where(rng.random((1, L, M)) < 0.5, -0.0, 0.0).astype(np.float32)   # signed zeros only
+        _topk_case(p, z)
+    finally:
+        p.close()
+
+
 @pytest.mark.parametrize("policy", [nb.NP_EVICT_EXACT, nb.NP_EVICT_LRU])
 @pytest.mark.parametrize("cfg,n_set,C,persist", [
     (TINY, 102, 205, 0.8), (TINY, 102, 102, 0.6), (SMALL, 208, 520, 0.83), (SMALL, 700, 520, 0.7),
