@@ -519,6 +519,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_spid = take(LC), o_spsl = take(LC), o_spcnt = take((size_t)d.L * NP_N_COUNTERS), o_spcand = take(LW);
   const size_t o_sbar = take(chain_slices::bar_words()), o_sxch = take(2 * chain_slices::xch_words(d, ctx->sm_count));
   const size_t o_rz = take(chain_rows::z_floats(d)), o_rcnt = take(4);
+  const size_t o_l1p = take(cfg->max_batch > 4 ? (size_t)kPredL1Parts * 16 * d.H : 1);
   NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
   char* base = static_cast<char*>(ctx->slab);
   Tables& t = ctx->t;
@@ -612,7 +613,8 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   // tensor-core predictor for batches: tensor maps over W2 and the split hidden terms
   ctx->mlp_tc = cfg->max_batch >= kTcMinBatch && !(cfg->flags & (NP_F_NO_TENSOR_CORES | NP_F_DIRECT_LOADS)) &&
                 mlp_tc_supported(d, ctx->sm_count);
-  if (cfg->max_batch > 4 && !(cfg->flags & NP_F_NO_TENSOR_CORES)) pred_tc_prepare(d, b->w2, ctx->ws.hsplit, &ctx->tc);
+  if (cfg->max_batch > 4 && !(cfg->flags & NP_F_NO_TENSOR_CORES))
+    pred_tc_prepare(d, b->w1, b->w2, ctx->ws.hsplit, reinterpret_cast<float*>(static_cast<char*>(ctx->slab) + o_l1p), ctx->sm_count, &ctx->tc);
   {
     // batches the tensor-core predictor does not take go through the ring kernel, whose shared
     // memory holds the batch's hidden vectors beside at least two stages of W2 rows
@@ -703,7 +705,13 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
   if ((uintptr_t)x_bf16 % 16) return fail(ctx, NP_E_INVAL, "x must be 16-byte aligned");
   cudaStream_t s = as_stream(stream);
   const Dims& d = ctx->d;
-  NP_LAUNCH(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
+  // batches: both layers on the tensor cores where the shapes allow (layer 1 leaves partial sums that layer 2's
+  // split kernel adds up)
+  const bool l1_tc = B > 4 && ctx->tc.ready && ctx->tc.l1_ready && d.dense == 0;
+  if (l1_tc)
+    NP_LAUNCH(ctx, launch_pred_l1_tc(d, ctx->tc, x_bf16, B, ctx->t.status, s));
+  else
+    NP_LAUNCH(ctx, launch_pred_l1(d, ctx->bufs.w1, x_bf16, B, ctx->ws.hidden, s));
   // Dense layers are not scored: the sparse layers are a contiguous suffix of W2, of the logits
   // and of the bitmap (a dense prefix implies B = 1, so the per-sequence stride does not matter).
   // With several sequences the per-sequence stride of the logits keeps all L layers, so every
@@ -716,7 +724,8 @@ int np_predict(np_ctx* ctx, const void* x_bf16, int32_t B, float* logits_out, ui
   if (ds.L > 0) {
     if (B > 4 && ctx->tc.ready) {
       ctx->launches += 1;  // split kernel + GEMM kernel
-      NP_LAUNCH(ctx, launch_pred_l2_tc(d, ctx->tc, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count));
+      NP_LAUNCH(ctx, launch_pred_l2_tc(d, ctx->tc, ctx->ws.hidden, B, ctx->ws.logits, ctx->t.status, s, ctx->sm_count,
+                                       l1_tc ? ctx->tc.l1_parts : 0));
     } else {
       NP_LAUNCH(ctx, launch_pred_l2(ds, static_cast<const char*>(ctx->bufs.w2) + skip_rows * d.H * 2, ctx->ws.hidden,
                                   B, logits, ctx->t.status, s, ctx->sm_count));

@@ -75,18 +75,23 @@ cudaError_t launch_pred_l2(const Dims& d, const void* w2, const float* hidden, i
 // whether the ring form of layer 2 (batches without the tensor-core kernel) has room for B hidden vectors of H values
 bool pred_l2_ring_fits(int H, int B);
 // Tensor-core form of predictor layer 2 for batches (np_predict_tc.cu).
+constexpr int kPredL1Parts = 16;  // K ranges (partial sums) of the tensor-core layer 1, at most
 struct PredTcState {
   alignas(64) unsigned char map_w2[128];  // CUtensorMap of W2 [L*M][H]
   alignas(64) unsigned char map_h[128];   // CUtensorMap of the split hidden terms [48][H]
+  alignas(64) unsigned char map_w1[128];  // CUtensorMap of W1 [H][D]
   void* hsplit;                           // device bf16 [48][H] (workspace)
+  float* l1_part;                         // device fp32 [kPredL1Parts][16][H]: layer 1's partial sums per K range
   int n_stages;
   size_t smem;
   int ready;
+  int l1_ready, l1_parts, l1_kb_per_block;
 };
 bool pred_tc_supported(const Dims& d);
-bool pred_tc_prepare(const Dims& d, const void* w2, void* hsplit, PredTcState* st);
-cudaError_t launch_pred_l2_tc(const Dims& d, const PredTcState& st, const float* hidden, int B, float* logits,
-                              int32_t* status, cudaStream_t s, int sm_count);
+bool pred_tc_prepare(const Dims& d, const void* w1, const void* w2, void* hsplit, float* l1_part, int sm_count, PredTcState* st);
+cudaError_t launch_pred_l1_tc(const Dims& d, const PredTcState& st, const void* x_bf16, int B, int32_t* status, cudaStream_t s);
+cudaError_t launch_pred_l2_tc(const Dims& d, const PredTcState& st, float* hidden, int B, float* logits,
+                              int32_t* status, cudaStream_t s, int sm_count, int l1_parts);
 
 cudaError_t launch_topk(const Dims& d, const float* logits, int B, uint32_t* bitmap, cudaStream_t s);
 

@@ -87,13 +87,26 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
       : "r"(taddr));
 }
 
-// hidden fp32 [B][H] -> three bf16 terms, rows [term * 16 + b] of a [48][H] array (zero for b >= B)
-__global__ void k_split_hidden(const float* __restrict__ hidden, __nv_bfloat16* __restrict__ out, int H, int B) {
+// hidden fp32 [B][H] -> three bf16 terms, rows [term * 16 + b] of a [48][H] array (zero for b >= B).
+// n_part > 0: `hidden` holds n_part partial sums [n_part][16][H] of layer 1 (one per K range of the tensor-core
+// kernel below); they are added in a fixed order, the ReLU is applied, and the result is also stored to `sum_out`.
+__global__ void k_split_hidden(const float* __restrict__ hidden, __nv_bfloat16* __restrict__ out, int H, int B, int n_part,
+                               float* __restrict__ sum_out) {
   npp::pdl_launch_dependents();
+  npp::pdl_wait_prior();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= 16 * H) return;
   const int b = i / H, m = i - b * H;
-  float v = b < B ? hidden[(size_t)b * H + m] : 0.f;
+  float v = 0.f;
+  if (b < B) {
+    if (n_part > 0) {
+      for (int p = 0; p < n_part; ++p) v += hidden[((size_t)p * 16 + b) * H + m];
+      v = fmaxf(v, 0.f);
+      sum_out[(size_t)b * H + m] = v;
+    } else {
+      v = hidden[(size_t)b * H + m];
+    }
+  }
   const __nv_bfloat16 t0 = __float2bfloat16_rn(v);
   v -= __bfloat162float(t0);
   const __nv_bfloat16 t1 = __float2bfloat16_rn(v);
@@ -259,6 +272,96 @@ k_pred_l2_tc(const __grid_constant__ CUtensorMap map_w2, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------------
+// Layer 1 for batches on the same tensor cores: raw[b][r] = sum_d W1[r][d] * x[b][d], r < H.  W1 is 4 MB and x is
+// bf16 already (one term, N = 16), so the kernel is all latency: the grid is (row tiles of 128) x (K ranges), every
+// block loads its few K blocks (a 16 KB tile of W1 and a 2 KB tile of x each) at once, multiplies, and stores its
+// partial sums [K range][sequence][row]; k_split_hidden adds the ranges in a fixed order (no atomics: the result
+// does not depend on the order in which blocks finish) and applies the ReLU.
+constexpr int kL1N = 16;
+constexpr int kL1MaxKb = 8;  // K blocks per block, all in flight at once
+constexpr uint32_t kL1XBytes = kL1N * kTcKBlock * 2;
+constexpr uint32_t kL1StageBytes = kTcStageBytes + kL1XBytes;  // a multiple of 1024: both tiles stay swizzle-aligned
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+k_pred_l1_tc(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_x, float* __restrict__ part,
+             int H, int n_kb, int kb_per_block, int32_t* status) {
+  extern __shared__ __align__(1024) unsigned char tsm[];
+  __shared__ __align__(8) uint64_t full_bar[kL1MaxKb];
+  __shared__ __align__(8) uint64_t acc_full;
+  __shared__ uint32_t s_tmem_base;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tsm) + 1023) & ~(uintptr_t)1023);
+  const int mt = blockIdx.x, kr = blockIdx.y;
+  const int kb0 = kr * kb_per_block, nkb = min(kb_per_block, n_kb - kb0);
+  if (tid == 0) {
+    for (int i = 0; i < kL1MaxKb; ++i) npp::mbar_init(&full_bar[i], 1);
+    npp::mbar_init(&acc_full, 1);
+    npp::fence_barrier_init();
+  }
+  if (wid == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(npp::smem_addr(&s_tmem_base)), "r"(32) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  npp::pdl_launch_dependents();
+  const uint32_t tmem_base = s_tmem_base;
+  if (wid == 0) {
+    if (lane == 0) {
+      // W1 does not depend on anything before this kernel; x may be the previous operation's
+      for (int i = 0; i < nkb; ++i) {
+        npp::mbar_expect_tx(&full_bar[i], kL1StageBytes);
+        tma_load_2d(base + (size_t)i * kL1StageBytes, &map_w1, (kb0 + i) * kTcKBlock, mt * kTcTileRows, &full_bar[i]);
+      }
+      npp::pdl_wait_prior();
+      for (int i = 0; i < nkb; ++i)
+        tma_load_2d(base + (size_t)i * kL1StageBytes + kTcStageBytes, &map_x, (kb0 + i) * kTcKBlock, 0, &full_bar[i]);
+    }
+  } else if (wid == 1) {
+    if (lane == 0) {
+      // instruction descriptor: D fp32, A and B bf16, both K-major, N = 16, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kL1N >> 3) << 17) | ((uint32_t)(kTcTileRows >> 4) << 24);
+      bool ok = true;
+      for (int i = 0; i < nkb && ok; ++i) {
+        if (!npp::mbar_wait(&full_bar[i], 0)) {
+          atomicOr(status, npp::kStatTimeout);
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint64_t a0 = tc_smem_desc(base + (size_t)i * kL1StageBytes);
+        const uint64_t b0 = tc_smem_desc(base + (size_t)i * kL1StageBytes + kTcStageBytes);
+#pragma unroll
+        for (int k = 0; k < kTcKBlock / 16; ++k) tc_mma(tmem_base, a0 + (uint64_t)(2 * k), b0 + (uint64_t)(2 * k), idesc, (i | k) != 0 ? 1u : 0u);
+      }
+      tc_commit(&acc_full);  // also on a timeout: the epilogue must not wait in vain
+    }
+  } else {
+    const int q = wid & 3;  // the TMEM lane quarter this warp may read
+    if (npp::mbar_wait(&acc_full, 0)) {
+      tc_fence_after();
+      uint32_t t0[16];
+      tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16), t0);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      const int r = mt * kTcTileRows + q * 32 + lane;
+      if (r < H && nkb > 0) {
+#pragma unroll
+        for (int b = 0; b < kL1N; ++b) part[((size_t)kr * kL1N + b) * H + r] = __uint_as_float(t0[b]);
+      }
+    } else if (lane == 0) {
+      atomicOr(status, npp::kStatTimeout);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (wid == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(32) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------
 namespace {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -294,10 +397,28 @@ bool make_map(CUtensorMap* map, const void* gptr, uint64_t inner, uint64_t outer
 
 bool pred_tc_supported(const Dims& d) { return d.H % kTcKBlock == 0 && d.H >= kTcKBlock; }
 
-bool pred_tc_prepare(const Dims& d, const void* w2, void* hsplit, PredTcState* st) {
+bool pred_tc_prepare(const Dims& d, const void* w1, const void* w2, void* hsplit, float* l1_part, int sm_count, PredTcState* st) {
   static_assert(sizeof(CUtensorMap) <= sizeof(st->map_w2), "tensor map blob too small");
   st->ready = 0;
+  st->l1_ready = 0;
   if (!pred_tc_supported(d)) return false;
+  // layer 1 on the tensor cores: whole row tiles of W1 and whole K blocks, and room for the partial sums
+  if (l1_part && d.H % kTcTileRows == 0 && d.D % kTcKBlock == 0) {
+    CUtensorMap w;
+    if (make_map(&w, w1, (uint64_t)d.D, (uint64_t)d.H, kTcKBlock, kTcTileRows)) {
+      memcpy(st->map_w1, &w, sizeof w);
+      const int n_kb = d.D / kTcKBlock, n_mt = d.H / kTcTileRows;
+      // K ranges: enough blocks to fill the machine, at most kPredL1Parts partial sums, at most kL1MaxKb K blocks each
+      int parts = std::min(std::min(n_kb, kPredL1Parts), std::max(1, sm_count / n_mt));
+      int per = (n_kb + parts - 1) / parts;
+      if (per <= kL1MaxKb) {
+        st->l1_kb_per_block = per;
+        st->l1_parts = (n_kb + per - 1) / per;
+        st->l1_part = l1_part;
+        st->l1_ready = 1;
+      }
+    }
+  }
   CUtensorMap a, b;
   const uint64_t rows = (uint64_t)d.L * d.M;
   if (!make_map(&a, w2, (uint64_t)d.H, rows, kTcKBlock, kTcTileRows)) return false;
@@ -314,14 +435,31 @@ bool pred_tc_prepare(const Dims& d, const void* w2, void* hsplit, PredTcState* s
   return true;
 }
 
-cudaError_t launch_pred_l2_tc(const Dims& d, const PredTcState& st, const float* hidden, int B, float* logits,
-                              int32_t* status, cudaStream_t s, int sm_count) {
+cudaError_t launch_pred_l1_tc(const Dims& d, const PredTcState& st, const void* x_bf16, int B, int32_t* status, cudaStream_t s) {
+  if (!st.ready || !st.l1_ready) return cudaErrorInvalidValue;
+  CUtensorMap w, x;
+  memcpy(&w, st.map_w1, sizeof w);
+  // x is the caller's buffer: its map is made per call.  The box has 16 rows, the tensor B: rows past the end read zero.
+  if (!make_map(&x, x_bf16, (uint64_t)d.D, (uint64_t)B, kTcKBlock, kL1N)) return cudaErrorInvalidValue;
+  const size_t smem = (size_t)st.l1_kb_per_block * kL1StageBytes + 1024;
+  cudaError_t e = cudaFuncSetAttribute(k_pred_l1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  k_pred_l1_tc<<<dim3(d.H / kTcTileRows, st.l1_parts), kTcThreads, smem, s>>>(w, x, st.l1_part, d.H, d.D / kTcKBlock, st.l1_kb_per_block,
+                                                                              status);
+  return cudaGetLastError();
+}
+
+// l1_parts > 0: layer 1 ran on the tensor cores and left that many partial sums; the split kernel adds them up,
+// applies the ReLU and stores the hidden vectors to `hidden` as the other layer-1 kernels do.
+cudaError_t launch_pred_l2_tc(const Dims& d, const PredTcState& st, float* hidden, int B, float* logits,
+                              int32_t* status, cudaStream_t s, int sm_count, int l1_parts) {
   if (!st.ready) return cudaErrorInvalidValue;
   CUtensorMap a, b;
   memcpy(&a, st.map_w2, sizeof a);
   memcpy(&b, st.map_h, sizeof b);
   const int n = 16 * d.H;
-  k_split_hidden<<<(n + 255) / 256, 256, 0, s>>>(hidden, static_cast<__nv_bfloat16*>(st.hsplit), d.H, B);
+  k_split_hidden<<<(n + 255) / 256, 256, 0, s>>>(l1_parts > 0 ? st.l1_part : hidden, static_cast<__nv_bfloat16*>(st.hsplit), d.H, B,
+                                                 l1_parts, hidden);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(k_pred_l2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)st.smem);

@@ -17,11 +17,17 @@ SMALL = synth.CONFIGS["small"]     # ragged: M = 2080 (65 words), H = 96, 3 laye
 # predictor width a multiple of 64 (three k-blocks) and a row count that is not a multiple of
 # the 128-row MMA tile: the batch path runs on the tensor cores with a ragged last tile
 TCW = synth.StackConfig("tcw", 3, 512, 2080, 192, 10, 25, 4, 21, 0.9)
+# predictor width a multiple of the 128-row MMA tile: layer 1 of a batch runs on the tensor cores too (one K range
+# per block at D = 512, sixteen ranges of four K blocks at D = 4096, a ragged last range at D = 4160)
+TC1 = synth.StackConfig("tc1", 2, 512, 1024, 128, 10, 25, 4, 22, 0.9)
+TC1W = synth.StackConfig("tc1w", 2, 4096, 1024, 256, 10, 25, 4, 23, 0.9)
+TC1R = synth.StackConfig("tc1r", 2, 4160, 1024, 384, 10, 25, 4, 24, 0.9)
 
 
 @pytest.mark.parametrize("cfg,B,flags", [
     (TINY, 1, 0), (SMALL, 1, 0), (SMALL, 3, 0), (TINY, 16, 0), (TCW, 16, 0), (TCW, 7, 0), (TCW, 5, 0),
     (TCW, 16, nb.NP_F_NO_TENSOR_CORES), (SMALL, 9, 0),
+    (TC1, 5, 0), (TC1, 16, 0), (TC1W, 16, 0), (TC1W, 9, 0), (TC1R, 16, 0), (TC1R, 6, 0),
 ])
 def test_predict_logits_and_bitmap(cfg, B, flags):
     p = Pair(cfg, max_batch=B, flags=flags | nb.NP_F_CHECK_BOUNDS)
