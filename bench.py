@@ -69,6 +69,9 @@ def parse_args():
     ap.add_argument("--mlp-kernel", default="auto", choices=["auto", "cluster-rows", "row-chain"],
                     help="resident sparse-MLP kernel for one sequence: the library's choice, whole rows per block with "
                          "blocks in clusters (NP_F_CLUSTER_ROWS), or whole rows with a global reduction only (NP_F_ROW_CHAIN)")
+    ap.add_argument("--batch-up-kernel", default="mma-sync", choices=["mma-sync", "tcgen05"],
+                    help="--batch > 1: the up phase of the batched sparse MLP on the mma.sync kernel or the tcgen05 one "
+                         "(NP_F_TCGEN05_BATCH)")
     ap.add_argument("--capacity-pct", type=int, default=None, help="resident capacity in percent of FFN rows")
     ap.add_argument("--store-layers", default="auto",
                     help="layers of records the host store holds (layer l reads layer l mod this); 'auto' = all of them "
@@ -381,6 +384,7 @@ def cuda_arm(args):
                           flags=(nb.NP_F_LAYER_LAUNCHES if args.layer_launches or args.direct_loads else 0)
                           | {"auto": 0, "cluster-rows": nb.NP_F_CLUSTER_ROWS, "row-chain": nb.NP_F_ROW_CHAIN}[args.mlp_kernel]
                           | (nb.NP_F_DIRECT_LOADS if args.direct_loads else 0)
+                          | (nb.NP_F_TCGEN05_BATCH if args.batch_up_kernel == "tcgen05" else 0)
                           | (nb.NP_F_MAPPED_STAGING if args.mapped_staging else 0))
     storage = None
     if args.transfer == "file":
@@ -572,7 +576,7 @@ def cuda_arm(args):
         n_launch = L - nd                                           # per-layer (or batch) kernels
     mlp_kernel = nb.np_mlp_kernel_name(eng.ctx, Bq)       # the kernel the library chose for this shape and batch
     if Bq > 1:
-        mlp_kernel += " (the two launches of one layer)"
+        mlp_kernel += " (the launches of one layer)"
     mlp_us = k0.elapsed_time(k1) * 1000.0 / (reps * n_launch)      # per launch, gaps included
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record(s)

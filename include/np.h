@@ -104,6 +104,12 @@ extern "C" {
 #define NP_F_CLUSTER_ROWS   64  /* np_step / np_mlp_chain, one sequence: the resident MLP kernel that deals whole rows to
                                    blocks in clusters of four and reduces inside the cluster first (where it applies:
                                    row widths of 1024 to 4096 in steps of 1024), instead of the column-sliced one */
+#define NP_F_TCGEN05_BATCH 128  /* batches: the up phase of the sparse MLP as a tcgen05 kernel (rows gathered into
+                                   unswizzled K-major tiles, accumulators in tensor memory, x split into bf16 terms
+                                   once per layer by a kernel of its own) instead of the mma.sync kernel; applies to
+                                   sparse layers whose row width is a multiple of 256, other shapes keep the default.
+                                   Results agree with the default to rounding order; measured slower at sixteen
+                                   sequences, so off by default */
 #define NP_F_MAPPED_STAGING 16  /* NP_XFER_HOST_GATHER / NP_XFER_FILE: no staging copy; the scatter kernel
                                    reads the records in the pinned staging buffer through its device
                                    mapping (Section 3.5: the staging is page-aligned host memory registered

@@ -30,6 +30,7 @@ NP_F_MAPPED_STAGING = 16
 NP_F_NO_TENSOR_CORES = 8
 NP_F_ROW_CHAIN = 32
 NP_F_CLUSTER_ROWS = 64
+NP_F_TCGEN05_BATCH = 128
 NP_REC_BF16, NP_REC_INT8 = 0, 1
 (NP_CNT_PRED, NP_CNT_KEPT, NP_CNT_DELTA, NP_CNT_EVICT, NP_CNT_OVERFLOW, NP_CNT_ACTIVE,
  NP_CNT_RESIDENT, NP_CNT_STEP) = range(8)

@@ -201,6 +201,7 @@ struct np_ctx {
   PredTcState tc = {};
   chain_slices::State slices = {};  // column-sliced resident MLP kernel: its counters, exchange words and their values
   bool use_slices = false;
+  void* xterms = nullptr;  // scratch of the tcgen05 up kernel of the batch MLP
   chain_rows::State rows = {};  // cluster form of the resident MLP kernel (whole rows per block): its accumulators and counters
   bool use_rows = false;
   int chain_kernel_launches = 0;    // MLP kernel launches of the last np_mlp_chain / np_step
@@ -259,7 +260,7 @@ int check_config(const np_config* c, np_ctx* ctx) {
   if (c->transfer_mode == NP_XFER_FILE && c->record_format != NP_REC_BF16)
     return fail(ctx, NP_E_INVAL, "NP_XFER_FILE needs NP_REC_BF16 records");
   if (c->io_depth < -1 || c->io_depth > 4096) return fail(ctx, NP_E_INVAL, "io_depth must be in [-1, 4096]");
-  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES | NP_F_MAPPED_STAGING | NP_F_ROW_CHAIN | NP_F_CLUSTER_ROWS)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
+  if (c->flags & ~(NP_F_CHECK_BOUNDS | NP_F_DIRECT_LOADS | NP_F_LAYER_LAUNCHES | NP_F_NO_TENSOR_CORES | NP_F_MAPPED_STAGING | NP_F_ROW_CHAIN | NP_F_CLUSTER_ROWS | NP_F_TCGEN05_BATCH)) return fail(ctx, NP_E_INVAL, "unknown flag bits");
   if (c->host_threads < 0 || c->host_threads > 256) return fail(ctx, NP_E_INVAL, "host_threads out of range");
   if (c->chain_layers < 0) return fail(ctx, NP_E_INVAL, "chain_layers must be >= 0");
   if (c->ring_stages < 0 || c->ring_stages == 1) return fail(ctx, NP_E_INVAL, "ring_stages must be 0 or >= 2");
@@ -520,6 +521,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_sbar = take(chain_slices::bar_words()), o_sxch = take(2 * chain_slices::xch_words(d, ctx->sm_count));
   const size_t o_rz = take(chain_rows::z_floats(d)), o_rcnt = take(4);
   const size_t o_l1p = take(cfg->max_batch > 4 ? (size_t)kPredL1Parts * 16 * d.H : 1);
+  const size_t o_xt = take(cfg->max_batch >= kTcMinBatch ? mlp_tc_xterms_bytes(d) / 4 : 1);
   NP_INIT_CUDA(cudaMalloc(&ctx->slab, off));
   char* base = static_cast<char*>(ctx->slab);
   Tables& t = ctx->t;
@@ -551,6 +553,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   NP_INIT_CUDA(cudaMemset(ctx->slices.bars, 0, chain_slices::bar_words() * 4));
   NP_INIT_CUDA(cudaMemset(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8));
   ctx->use_slices = !(cfg->flags & NP_F_ROW_CHAIN) && chain_slices::supported(d, ctx->sm_count);
+  ctx->xterms = base + o_xt;
   ctx->rows.z4 = reinterpret_cast<float*>(base + o_rz);
   ctx->rows.cnt = reinterpret_cast<unsigned int*>(base + o_rcnt);
   ctx->rows.cnt_base = ctx->rows.seq = 0;
@@ -1187,6 +1190,7 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
   a.force_direct = (ctx->cfg.flags & NP_F_DIRECT_LOADS) ? 1 : 0;
   a.status = ctx->t.status;
   a.gu = a.gu_next = a.ssq = a.ssq_next = nullptr;
+  a.xterms = (ctx->cfg.flags & NP_F_TCGEN05_BATCH) ? ctx->xterms : nullptr;
   if (ctx->install_pending[layer]) NP_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_installed[layer], 0));
   if (ctx->mlp_tc && B >= kTcMinBatch && !a.force_direct) {
     const int cur = gu_sel < 0 ? 0 : gu_sel;
@@ -1196,7 +1200,8 @@ static int mlp_layer(np_ctx* ctx, int layer, const float* xa, const float* xb, f
       a.gu_next = ctx->ws.gu[cur ^ 1];
       a.ssq_next = ctx->ws.ssq[cur ^ 1];
     }
-    ctx->launches += 1;  // two kernels per layer
+    // two kernels per layer; three where the tcgen05 up kernel runs (x is split by a kernel of its own)
+    ctx->launches += (a.xterms && !dense_layer && mlp_tc_up_on_tcgen05(d, ctx->sm_count)) ? 2 : 1;
     NP_LAUNCH(ctx, launch_sparse_mlp_tc(d, a, s, ctx->sm_count));
     return NP_OK;
   }
@@ -1440,7 +1445,8 @@ const char* np_mlp_kernel_name(np_ctx* ctx, int32_t B) {
     if (ctx->use_slices) return "k_mlp_slices";
     if (chain_alu::supported(d, ctx->sm_count)) return "k_mlp_chain_alu";
   }
-  if (ctx->mlp_tc && B >= kTcMinBatch && !(flags & NP_F_DIRECT_LOADS)) return "k_mlp_tc_up + k_mlp_tc_down";
+  if (ctx->mlp_tc && B >= kTcMinBatch && !(flags & NP_F_DIRECT_LOADS))
+    return ((flags & NP_F_TCGEN05_BATCH) && mlp_tc_up_on_tcgen05(d, ctx->sm_count)) ? "k_mlp_up5 + k_mlp_tc_down" : "k_mlp_tc_up + k_mlp_tc_down";
   return (flags & NP_F_DIRECT_LOADS) ? "k_sparse_mlp" : "k_sparse_mlp_pipe";
 }
 

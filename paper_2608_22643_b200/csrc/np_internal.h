@@ -138,6 +138,7 @@ struct MlpArgs {
   float* ssq;       // [kMaxBatch] sum of x^2 per sequence, zero on entry (needed with normalize)
   float* ssq_next;  // may be NULL
   int gu_rows;      // rows each gu buffer holds (0 = C)
+  void* xterms;     // scratch of mlp_tc_xterms_bytes(): x as three bf16 terms for the tcgen05 up kernel (NULL: mma.sync up kernel)
   int dense_rows;   // > 0 (tensor-core path): a dense layer of that many whole records; gate_l / up_l / downT_l point
                     // at the three rows of its first record, active_slots is an identity list, n_active_ptr is not read
 };
@@ -146,6 +147,8 @@ cudaError_t launch_sparse_mlp(const Dims& d, const MlpArgs& a, cudaStream_t s, i
 constexpr int kTcMinBatch = 2;
 bool mlp_tc_supported(const Dims& d, int sm_count);
 size_t mlp_tc_gu_floats(const Dims& d);
+size_t mlp_tc_xterms_bytes(const Dims& d);
+bool mlp_tc_up_on_tcgen05(const Dims& d, int sm_count);  // sparse layers of this shape take the tcgen05 up kernel
 cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count);
 
 // Arguments of the resident multi-layer kernels for one sequence.

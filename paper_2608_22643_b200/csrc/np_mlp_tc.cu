@@ -467,6 +467,8 @@ struct TcArgs {
   int32_t* status;
   int B, D, C, SW, check, normalize, up_slots, down_slots;
   int gu_rows;      // rows the GU buffers hold (all of them are cleared for the next layer)
+  void* xterms;     // tcgen05 up phase: x as three bf16 terms, [D / 8][48][8] (may be NULL: legacy up kernel)
+  int up_rp;        // tcgen05 up phase: rows of a chunk plane (the most rows a block can have, rounded up to 8)
   int dense_rows;   // > 0: a dense layer.  gate / up / downT point at the three rows of its first record (row
                     // pitch = one record), every one of its dense_rows rows is active, slots = an identity list
 };
@@ -623,6 +625,288 @@ __global__ void __launch_bounds__(kThreads, 1) k_mlp_tc_down(TcArgs a) {
   if (r_end > r_begin && ok) down_reds<NJ>(k, acc, a.yacc + (size_t)cs * a.SW, nt0, my_nt, lane);
 }
 
+// ---------------------------------------------------------------------------
+// Up phase on the 5th-generation tensor cores (B >= 2, sparse layers): GU[row][gate|up][b] += W[row][K slice] . x_b.
+//
+// M = 128 rows of a row block, N = 48 = 16 sequences x 3 bf16 terms of x, K = 16 per MMA, fp32 accumulators in
+// tensor memory (gate in columns 0-47, up in 64-111).  The rows are scattered over the slot buffers, so no tiled
+// TMA copy can fetch a tile; four warps gather them with 16-byte cp.async into the layout the MMA reads without
+// swizzling: 8 x 16-byte core matrices, here simply [16-byte chunk of K][row] (row r of chunk j at 2048 j + 16 r:
+// groups of 8 rows 128 bytes apart, K-adjacent core matrices 2048 bytes apart).  Eight consecutive threads copy
+// the 128 bytes a row has in a K block, so every 32-byte sector that is read is used.  x comes as one bulk copy:
+// k_x_terms has split it once per layer, already in this layout ([chunk][48][8]), where the legacy kernel's blocks
+// each rebuilt their slice (5 us of the 17).  One lane issues the MMAs; a commit per stage hands the stage back to
+// the gathering warps, which at the end read the accumulators (tcgen05.ld), add the three terms and reduce into GU.
+// ---------------------------------------------------------------------------
+constexpr int kUpRows = 128;                         // MMA M
+constexpr int kUpN = 48;                             // MMA N
+constexpr int kUpKb = 64;                            // K per stage
+constexpr int kUpStages = 6;                         // five stages in flight: a gather is bound by what it has in flight
+constexpr int kUpLoaders = 256;                      // gathering threads (eight warps: one warp alone issues a copy every 13
+                                                     // clocks or so); the first four warps also read the accumulators back
+constexpr int kUpThreads = kUpLoaders + 32;          // plus the MMA warp
+// A stage holds, per matrix (gate, up), 8 chunk planes of `rp` rows x 16 bytes, rp = the most rows a block can have,
+// rounded up to 8: a plane is as long as the block's rows need, not 128 rows (the MMA still reads 128 rows per plane:
+// those past rp are the next planes' bytes, and their results are not used).
+__host__ __device__ constexpr uint32_t up_stage_bytes(int rp) { return 2u * 8u * (uint32_t)rp * 16u; }
+constexpr uint32_t kUpChunkN = kUpN * 16;                // bytes of x per 16-byte K chunk: 48 x 16
+
+__device__ __forceinline__ void tc5_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc5_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc5_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+// K-major operand without swizzle: core matrices of 8 rows x 16 bytes; lbo = bytes between K-adjacent core
+// matrices, sbo = bytes between groups of 8 rows
+__device__ __forceinline__ uint64_t tc5_desc(const void* p, uint32_t lbo, uint32_t sbo) {
+  const uint64_t addr = (uint64_t)(smem_addr(p) & 0x3ffffu) >> 4;
+  return addr | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
+}
+__device__ __forceinline__ void tc5_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void tc5_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+
+// x = xa (+ xb) of a layer, once: three bf16 terms per value in the up kernel's operand layout [D / 8][48][8]
+// (row 16 t + b of chunk j = term t of x_b[8 j .. 8 j + 7]; rows of sequences past B are zero), and the chain's side
+// effects: x is stored, the accumulator one layer ahead is cleared, sum(x^2) per sequence is added to ssq.
+__global__ void __launch_bounds__(256) k_x_terms(const float* __restrict__ xa, const float* __restrict__ xb, float* __restrict__ x_store,
+                                                 float* __restrict__ zero_out, float* __restrict__ ssq, uint4* __restrict__ xt, int B, int D) {
+  pdl_launch_dependents();
+  pdl_wait_prior();
+  const int chunks = D >> 3;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= kSeq * chunks) return;
+  const int b = i / chunks, j = i - b * chunks;  // a warp's threads share b (chunks is a multiple of 32)
+  float v[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) v[e] = 0.f;
+  if (b < B) {
+    const size_t gi = (size_t)b * D + (size_t)j * 8;
+    const float4 a0 = __ldcg(reinterpret_cast<const float4*>(xa + gi)), a1 = __ldcg(reinterpret_cast<const float4*>(xa + gi + 4));
+    v[0] = a0.x, v[1] = a0.y, v[2] = a0.z, v[3] = a0.w, v[4] = a1.x, v[5] = a1.y, v[6] = a1.z, v[7] = a1.w;
+    if (xb) {
+      const float4 b0 = __ldcg(reinterpret_cast<const float4*>(xb + gi)), b1 = __ldcg(reinterpret_cast<const float4*>(xb + gi + 4));
+      v[0] += b0.x, v[1] += b0.y, v[2] += b0.z, v[3] += b0.w, v[4] += b1.x, v[5] += b1.y, v[6] += b1.z, v[7] += b1.w;
+    }
+    if (x_store) {
+      *reinterpret_cast<float4*>(x_store + gi) = make_float4(v[0], v[1], v[2], v[3]);
+      *reinterpret_cast<float4*>(x_store + gi + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    }
+    if (zero_out) {
+      *reinterpret_cast<float4*>(zero_out + gi) = make_float4(0.f, 0.f, 0.f, 0.f);
+      *reinterpret_cast<float4*>(zero_out + gi + 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  uint32_t t[8][3];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) split3(v[e], t[e][0], t[e][1], t[e][2]);
+#pragma unroll
+  for (int k = 0; k < 3; ++k)
+    xt[(size_t)j * kUpN + k * kSeq + b] = make_uint4(pack2(t[0][k], t[1][k]), pack2(t[2][k], t[3][k]), pack2(t[4][k], t[5][k]), pack2(t[6][k], t[7][k]));
+  if (ssq) {
+    float ss = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) ss += v[e] * v[e];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0 && b < B) atomicAdd(ssq + b, ss);
+  }
+}
+
+#ifdef NP_TRACE  // development builds only
+__device__ long long np_up5_clk[64];
+#define UK(ev) do { if (blockIdx.x == 3 && blockIdx.y == 1 && (threadIdx.x & 31) == 0) np_up5_clk[ev] = clock64(); } while (0)
+#else
+#define UK(ev) do { } while (0)
+#endif
+
+__global__ void __launch_bounds__(kUpThreads, 1) k_mlp_up5(TcArgs a) {
+  extern __shared__ __align__(128) unsigned char tsm[];
+  __shared__ __align__(8) uint64_t full_bar[kUpStages];   // a stage's rows have landed (every gathering thread arrives)
+  __shared__ __align__(8) uint64_t empty_bar[kUpStages];  // the MMAs that read the stage are done
+  __shared__ __align__(8) uint64_t x_bar, acc_bar;
+  __shared__ uint32_t s_tmem_base;
+  __shared__ uint32_t rowoff[kUpRows];                    // byte offset of a row's K slice in the slot buffers, in 16-byte units
+
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int rb = blockIdx.x, RB = gridDim.x, ks = blockIdx.y;
+  const int SW = a.SW, nkb = SW / kUpKb;
+  const size_t row_pitch = (size_t)a.D * 2;
+  unsigned char* xsm = tsm;                                        // [SW / 8][48][16 bytes]
+  unsigned char* stages = tsm + (size_t)(SW / 8) * kUpChunkN;      // [kUpStages][gate | up][8 chunks][rp rows][16 bytes]
+  const uint32_t plane = (uint32_t)a.up_rp * 16u, tile_bytes = 8u * plane, stage_bytes = 2u * tile_bytes;
+
+  if (tid == 0) UK(0);
+  if (tid == 0) {
+    for (int i = 0; i < kUpStages; ++i) {
+      mbar_init(&full_bar[i], kUpLoaders);
+      mbar_init(&empty_bar[i], 1);
+    }
+    mbar_init(&x_bar, 1);
+    mbar_init(&acc_bar, 1);
+    fence_barrier_init();
+  }
+  if (wid == kUpLoaders / 32) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&s_tmem_base)), "r"(128) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  int n = *a.n_ptr;
+  if (a.check && (n < 0 || n > a.C)) {
+    if (tid == 0) atomicOr(a.status, kStatBadCount);
+    n = 0;
+  }
+  const int r_begin = (int)(((long long)n * rb) / RB);
+  int nrows = (int)(((long long)n * (rb + 1)) / RB) - r_begin;
+  if (nrows > kUpRows) {  // more rows than a tile: the launch code does not choose this kernel for such shapes
+    if (tid == 0) atomicOr(a.status, kStatBadCount);
+    nrows = kUpRows;
+  }
+  if (tid < nrows) {
+    int slot = a.slots[r_begin + tid];
+    if (a.check && (slot < 0 || slot >= a.C)) {
+      atomicOr(a.status, kStatBadSlot);
+      slot = 0;
+    }
+    rowoff[tid] = (uint32_t)(((size_t)slot * row_pitch + (size_t)ks * SW * 2) >> 4);
+  }
+  tc5_fence_before();
+  __syncthreads();
+  tc5_fence_after();
+  pdl_launch_dependents();
+  const uint32_t tmem_base = s_tmem_base;
+  if (tid == 0) UK(1);
+
+  if (wid < kUpLoaders / 32) {
+    // ---------------- gathering warps: the weight rows do not depend on the previous kernel ----------------
+    const int chunk = tid & 7, row0 = tid >> 3;  // 8 threads per row, 32 rows per round
+    constexpr int kRounds = kUpRows / (kUpLoaders / 8);
+    size_t src_off[kRounds];   // this thread's rows: byte offset of its chunk of K block 0 (the same in gate and up)
+    uint32_t dst_off[kRounds]; // ... and where it goes inside a stage
+#pragma unroll
+    for (int i = 0; i < kRounds; ++i) {
+      const int row = row0 + (kUpLoaders / 8) * i;
+      src_off[i] = row < nrows ? ((size_t)rowoff[row] << 4) + (size_t)chunk * 16 : 0;
+      dst_off[i] = (uint32_t)chunk * plane + (uint32_t)row * 16u;
+    }
+    bool ok = true;
+    for (int kb = 0; kb < nkb; ++kb) {
+      const int s = kb % kUpStages;
+      if (kb >= kUpStages && ok && !mbar_wait(&empty_bar[s], (uint32_t)((kb / kUpStages - 1) & 1))) {
+        atomicOr(a.status, kStatTimeout);
+        ok = false;
+      }
+      const uint32_t dst0 = smem_addr(stages + (size_t)s * stage_bytes);
+      const size_t koff = (size_t)kb * (kUpKb * 2);
+#pragma unroll
+      for (int i = 0; i < kRounds; ++i) {
+        if (row0 + (kUpLoaders / 8) * i < nrows) {
+          cp_async16(dst0 + dst_off[i], a.gate + src_off[i] + koff);
+          cp_async16(dst0 + tile_bytes + dst_off[i], a.up + src_off[i] + koff);
+        }
+      }
+      // the thread's arrival on the stage's barrier happens when its copies above have landed: nothing here waits,
+      // so a stage is announced as soon as it is complete, whatever the thread is doing by then
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_addr(&full_bar[s])) : "memory");
+      if (tid == 0 && kb < 16) UK(8 + kb);
+    }
+    if (wid >= 4) goto done;  // the other four warps read the accumulators
+    // ---------------- epilogue: the same warps read the accumulators of their 32 rows ----------------
+    const int q = wid & 3;
+    if (mbar_wait(&acc_bar, 0)) {
+      tc5_fence_after();
+      if (tid == 0) UK(2);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+      uint32_t g0[16], g1[16], g2[16];
+      tc5_ld16(taddr, g0);
+      tc5_ld16(taddr + 16, g1);
+      tc5_ld16(taddr + 32, g2);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      const int row = q * 32 + lane;
+      float* dst = a.gu + (size_t)(r_begin + row) * 2 * kSeq;
+      if (row < nrows) {
+#pragma unroll
+        for (int b4 = 0; b4 < kSeq; b4 += 4)
+          if (b4 < a.B)
+            red_add_v4(dst + b4, (__uint_as_float(g2[b4]) + __uint_as_float(g1[b4])) + __uint_as_float(g0[b4]),
+                       (__uint_as_float(g2[b4 + 1]) + __uint_as_float(g1[b4 + 1])) + __uint_as_float(g0[b4 + 1]),
+                       (__uint_as_float(g2[b4 + 2]) + __uint_as_float(g1[b4 + 2])) + __uint_as_float(g0[b4 + 2]),
+                       (__uint_as_float(g2[b4 + 3]) + __uint_as_float(g1[b4 + 3])) + __uint_as_float(g0[b4 + 3]));
+      }
+      tc5_ld16(taddr + 64, g0);
+      tc5_ld16(taddr + 80, g1);
+      tc5_ld16(taddr + 96, g2);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      if (row < nrows) {
+#pragma unroll
+        for (int b4 = 0; b4 < kSeq; b4 += 4)
+          if (b4 < a.B)
+            red_add_v4(dst + kSeq + b4, (__uint_as_float(g2[b4]) + __uint_as_float(g1[b4])) + __uint_as_float(g0[b4]),
+                       (__uint_as_float(g2[b4 + 1]) + __uint_as_float(g1[b4 + 1])) + __uint_as_float(g0[b4 + 1]),
+                       (__uint_as_float(g2[b4 + 2]) + __uint_as_float(g1[b4 + 2])) + __uint_as_float(g0[b4 + 2]),
+                       (__uint_as_float(g2[b4 + 3]) + __uint_as_float(g1[b4 + 3])) + __uint_as_float(g0[b4 + 3]));
+      }
+    } else if (lane == 0) {
+      atomicOr(a.status, kStatTimeout);
+    }
+    if (tid == 0) UK(3);
+  } else if (lane == 0) {
+    // ---------------- MMA lane ----------------
+    pdl_wait_prior();  // the terms of x are the previous kernel's
+    UK(4);
+    const uint32_t x_bytes = (uint32_t)(SW / 8) * kUpChunkN;
+    mbar_expect_tx(&x_bar, x_bytes);
+    bulk_g2s(xsm, static_cast<const unsigned char*>(a.xterms) + (size_t)ks * x_bytes, x_bytes, &x_bar);
+    // instruction descriptor: D fp32, A and B bf16, both K-major, N = 48, M = 128
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUpN >> 3) << 17) | ((uint32_t)(kUpRows >> 4) << 24);
+    bool ok = mbar_wait(&x_bar, 0);
+    if (!ok) atomicOr(a.status, kStatTimeout);
+    UK(5);
+    for (int kb = 0; kb < nkb && ok; ++kb) {
+      const int s = kb % kUpStages;
+      if (!mbar_wait(&full_bar[s], (uint32_t)(kb / kUpStages) & 1u)) {
+        atomicOr(a.status, kStatTimeout);
+        ok = false;
+        break;
+      }
+      fence_proxy_async();  // the rows were written by cp.async; the MMA reads shared memory through the async proxy
+      tc5_fence_after();
+      const unsigned char* st = stages + (size_t)s * stage_bytes;
+#pragma unroll
+      for (int k = 0; k < kUpKb / 16; ++k) {  // 16 K values = two 16-byte chunks
+        const uint64_t bd = tc5_desc(xsm + (size_t)(kb * 8 + k * 2) * kUpChunkN, kUpChunkN, 128);
+        tc5_mma(tmem_base, tc5_desc(st + (size_t)k * 2 * plane, plane, 128), bd, idesc, (kb | k) != 0 ? 1u : 0u);
+        tc5_mma(tmem_base + 64, tc5_desc(st + tile_bytes + (size_t)k * 2 * plane, plane, 128), bd, idesc, (kb | k) != 0 ? 1u : 0u);
+      }
+      tc5_commit(&empty_bar[s]);
+      if (kb < 16) UK(32 + kb);
+    }
+    tc5_commit(&acc_bar);
+    UK(6);  // also after a timeout: the epilogue must not wait in vain
+  }
+done:
+  tc5_fence_before();
+  __syncthreads();
+  if (wid == kUpLoaders / 32) {
+    tc5_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(128) : "memory");
+  }
+}
+
 struct TcPlan {
   int KS, SW, RB;
   int up_slots, down_slots;
@@ -680,6 +964,25 @@ bool mlp_tc_supported(const Dims& d, int sm_count) {
 
 size_t mlp_tc_gu_floats(const Dims& d) { return (size_t)d.C * 2 * kSeq; }
 
+size_t mlp_tc_xterms_bytes(const Dims& d) { return (size_t)d.D / 8 * kUpChunkN; }
+
+// The tcgen05 up kernel applies to sparse layers whose K slices are whole stages and whose row blocks fit one tile.
+static int up5_rp(const Dims& d, const TcPlan& p) { return ((d.C + p.RB - 1) / p.RB + 7) & ~7; }
+// x terms | stages | slack for the rows the MMA reads past the last plane
+static size_t up5_smem(const Dims& d, const TcPlan& p) {
+  return (size_t)(p.SW / 8) * kUpChunkN + (size_t)kUpStages * up_stage_bytes(up5_rp(d, p)) + kUpRows * 16;
+}
+static bool up5_shape_ok(const Dims& d, const TcPlan& p) {
+  return p.SW % kUpKb == 0 && d.D % 256 == 0 && up5_rp(d, p) <= kUpRows && up5_smem(d, p) <= 224 * 1024;
+}
+static bool up5_applies(const Dims& d, const TcPlan& p, const MlpArgs& a) {
+  return a.xterms && a.dense_rows == 0 && a.C == d.C && up5_shape_ok(d, p);
+}
+bool mlp_tc_up_on_tcgen05(const Dims& d, int sm_count) {
+  TcPlan p;
+  return tc_plan(d, sm_count, kMaxBatch, &p) && up5_shape_ok(d, p);
+}
+
 cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s, int sm_count) {
   TcPlan p;
   if (!tc_plan(d, sm_count, a.B, &p) || !a.gu || (a.normalize && !a.ssq)) return cudaErrorInvalidValue;
@@ -709,7 +1012,33 @@ cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s
   ka.down_slots = p.down_slots;
   ka.dense_rows = a.dense_rows;
   ka.gu_rows = a.gu_rows > 0 ? a.gu_rows : a.C;
+  ka.xterms = a.xterms;
   const dim3 grid(p.RB, p.KS);
+  if (up5_applies(d, p, a)) {
+    // x once per layer (split, side effects), the up phase on tcgen05, the down phase as before
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((kSeq * (d.D / 8) + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_x_terms, a.xa, a.xb, a.x_store, a.zero_out, a.normalize ? a.ssq : (float*)nullptr,
+                                       static_cast<uint4*>(a.xterms), a.B, d.D);
+    if (e != cudaSuccess) return e;
+    const size_t smem_up5 = up5_smem(d, p);
+    ka.up_rp = up5_rp(d, p);
+    e = cudaFuncSetAttribute(k_mlp_up5, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_up5);
+    if (e != cudaSuccess) return e;
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kUpThreads);
+    cfg.dynamicSmemBytes = smem_up5;
+    e = cudaLaunchKernelEx(&cfg, k_mlp_up5, ka);
+    if (e != cudaSuccess) return e;
+    return a.B > 8 ? tc_launch(k_mlp_tc_down<2>, grid, p.smem_down, ka, s) : tc_launch(k_mlp_tc_down<1>, grid, p.smem_down, ka, s);
+  }
   if (a.B > 8) {
     cudaError_t e = tc_launch(k_mlp_tc_up<2>, grid, p.smem_up, ka, s);
     return e != cudaSuccess ? e : tc_launch(k_mlp_tc_down<2>, grid, p.smem_down, ka, s);
@@ -719,3 +1048,7 @@ cudaError_t launch_sparse_mlp_tc(const Dims& d, const MlpArgs& a, cudaStream_t s
 }
 
 }  // namespace npi
+
+#ifdef NP_TRACE
+extern "C" int np_debug_up5(void* out) { return (int)cudaMemcpyFromSymbol(out, npi::np_up5_clk, sizeof(npi::np_up5_clk)); }
+#endif

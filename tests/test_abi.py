@@ -74,7 +74,7 @@ def test_dense_prefix_plan_matches_the_oracle(lib):
 @pytest.mark.parametrize("field,value", [
     ("n_layers", 0), ("d_model", 100), ("d_ffn", 1000), ("d_pred", 7), ("top_k", 9999), ("capacity", 0),
     ("capacity", 99999), ("max_batch", 17), ("evict_policy", 5), ("transfer_mode", 9), ("staging_rows", 0),
-    ("flags", 128), ("store_layers", -1), ("store_layers", 3), ("spec_rows", -1), ("spec_rows", 206), ("reserved", 1), ("dense_layers", -1), ("dense_layers", 3), ("io_depth", -2), ("io_depth", 5000),
+    ("flags", 256), ("store_layers", -1), ("store_layers", 3), ("spec_rows", -1), ("spec_rows", 206), ("reserved", 1), ("dense_layers", -1), ("dense_layers", 3), ("io_depth", -2), ("io_depth", 5000),
 ])
 def test_bad_config_is_rejected(lib, field, value):
     cfg = nb.make_config(2, 256, 1024, 64, 102, 205)

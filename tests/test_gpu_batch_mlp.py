@@ -20,6 +20,7 @@ ODD = synth.StackConfig("odd", 2, 320, 1024, 32, 25, 50, 4, 17, 0.9)
 WIDE = synth.StackConfig("wide", 1, 128, 20480, 16, 100, 100, 2, 19, 0.9)
 
 TC, ALU = 0, nb.NP_F_NO_TENSOR_CORES
+TC5 = nb.NP_F_TCGEN05_BATCH   # up phase on tcgen05 where the shape allows it (row widths that are multiples of 256)
 
 
 def _install_random_sets(p, words):
@@ -32,7 +33,7 @@ def _install_random_sets(p, words):
     return deltas
 
 
-@pytest.mark.parametrize("flags", [TC, ALU])
+@pytest.mark.parametrize("flags", [TC, ALU, TC5])
 @pytest.mark.parametrize("cfg,B,ring", [(SMALL, 2, 0), (SMALL, 3, 0), (SMALL, 8, 0), (SMALL, 9, 0), (SMALL, 16, 0),
                                         (DENSE, 4, 0), (DENSE, 16, 0), (DENSE, 16, 3), (DENSE, 7, 2), (ODD, 5, 0),
                                         (ODD, 12, 0)])
@@ -59,7 +60,7 @@ def test_single_layer_matches_oracle(cfg, B, ring, flags):
         p.close()
 
 
-@pytest.mark.parametrize("flags", [TC, ALU])
+@pytest.mark.parametrize("flags", [TC, ALU, TC5])
 @pytest.mark.parametrize("cfg,B", [(SMALL, 2), (SMALL, 11), (DENSE, 16), (ODD, 6)])
 def test_chain_matches_oracle(cfg, B, flags):
     """The residual chain with the pre-MLP normalisation, several tokens in a row (the
@@ -85,6 +86,18 @@ def test_chain_matches_oracle(cfg, B, flags):
             assert rel_l2(out2.cpu().numpy(), res["x_final"]) < 1e-5
     finally:
         p.close()
+
+
+def test_kernel_choice_follows_the_flag():
+    """The library names the kernels it launches for a batch: the tcgen05 up kernel only with its flag and only for
+    row widths it covers."""
+    for cfg, flags, want in [(DENSE, TC, "k_mlp_tc_up + k_mlp_tc_down"), (DENSE, TC5, "k_mlp_up5 + k_mlp_tc_down"),
+                             (ODD, TC5, "k_mlp_tc_up + k_mlp_tc_down")]:
+        p = Pair(cfg, max_batch=16, flags=flags)
+        try:
+            assert nb.np_mlp_kernel_name(p.eng.ctx, 16) == want, (cfg.name, flags)
+        finally:
+            p.close()
 
 
 @pytest.mark.parametrize("B", [3, 16])

@@ -138,15 +138,19 @@ def test_larger_shapes_few_layers(name, n_layers, mode, chain_layers):
         p.close()
 
 
-def test_stress_shape_batch16_few_layers():
+@pytest.mark.parametrize("flags,kernel", [(0, "k_mlp_tc_up + k_mlp_tc_down"),
+                                          (nb.NP_F_TCGEN05_BATCH, "k_mlp_up5 + k_mlp_tc_down")])
+def test_stress_shape_batch16_few_layers(flags, kernel):
     """Sixteen sequences at the 7B row shape (the delta-stress workload) on four layers: the
     tensor-core predictor and the tensor-core batch MLP in the configuration bench.py --batch 16
-    times; unions of the per-sequence sets, tables bit-exact, chain within tolerance."""
+    times (and with the up phase on tcgen05); unions of the per-sequence sets, tables bit-exact,
+    chain within tolerance."""
     cfg = synth.CONFIGS["stress"].with_(n_layers=4)
     L, M, D, B = cfg.n_layers, cfg.d_ffn, cfg.d_model, 16
-    p = Pair(cfg, max_batch=B, transfer_mode=nb.NP_XFER_HOST_GATHER, staging_rows=2 * cfg.top_k, flags=0,
+    p = Pair(cfg, max_batch=B, transfer_mode=nb.NP_XFER_HOST_GATHER, staging_rows=2 * cfg.top_k, flags=flags,
              gen_device="cuda")
     try:
+        assert nb.np_mlp_kernel_name(p.eng.ctx, B) == kernel
         xs = synth.hidden_states(cfg, 3, batch=B, gamma=0.9)
         logits = torch.empty((B, L, M), dtype=torch.float32, device="cuda")
         out = torch.empty((B, D), dtype=torch.float32, device="cuda")
