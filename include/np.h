@@ -51,7 +51,10 @@ extern "C" {
 #define NP_E_STATE     -2   /* call out of order (e.g. install before delta) */
 #define NP_E_CUDA      -3   /* a CUDA runtime call failed; see np_last_error */
 #define NP_E_NOMEM     -4   /* allocation of library-owned state failed */
-#define NP_E_DEVICE    -5   /* a kernel's own bounds check tripped; state is suspect */
+#define NP_E_DEVICE    -5   /* a kernel recorded a status bit (np_last_error prints them): 1 slot, 2 neuron id or
+                               4 count out of range; 8 a bounded wait ran out; 16 a block's partial MLP sum was
+                               not finite or reached 2^19 in magnitude (the resident one-sequence kernel hands
+                               sums between layers in fixed point, resolution 2^-30); state is suspect */
 #define NP_E_IO        -6   /* a read of the store file failed or came up short */
 #define NP_W_OVERFLOW   1   /* some layer's predicted set did not fit capacity */
 #define NP_W_CHUNKED    2   /* some layer's delta exceeded staging and was split */

@@ -518,7 +518,7 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   const size_t o_cid = take(LC), o_ckey = take(LC), o_pred = take(LW), o_stat = take(4), o_bar = take(4);
   const size_t o_ident = take(d.dense > 0 ? (size_t)d.M : 1);
   const size_t o_spid = take(LC), o_spsl = take(LC), o_spcnt = take((size_t)d.L * NP_N_COUNTERS), o_spcand = take(LW);
-  const size_t o_sbar = take(chain_slices::bar_words()), o_sxch = take(2 * chain_slices::xch_words(d, ctx->sm_count));
+  const size_t o_sfix = take(2 * chain_slices::zfix_words(d)), o_sbar = take(chain_slices::bar_words()), o_sxch = take(2 * chain_slices::xch_words(d, ctx->sm_count));
   const size_t o_rz = take(chain_rows::z_floats(d)), o_rcnt = take(4);
   const size_t o_l1p = take(cfg->max_batch > 4 ? (size_t)kPredL1Parts * 16 * d.H : 1);
   const size_t o_xt = take(cfg->max_batch >= kTcMinBatch ? mlp_tc_xterms_bytes(d) / 4 : 1);
@@ -547,9 +547,11 @@ int np_init(np_ctx** out, const np_config* cfg, const np_buffers* b) {
   t.spec_slots = reinterpret_cast<int32_t*>(base + o_spsl);
   t.spec_counters = reinterpret_cast<int32_t*>(base + o_spcnt);
   t.spec_cand = reinterpret_cast<uint32_t*>(base + o_spcand);
+  ctx->slices.zfix = reinterpret_cast<unsigned long long*>(base + o_sfix);
   ctx->slices.bars = reinterpret_cast<unsigned int*>(base + o_sbar);
   ctx->slices.xch = reinterpret_cast<unsigned long long*>(base + o_sxch);
-  ctx->slices.bar_base = ctx->slices.seq_base = 0;
+  ctx->slices.seq_base = ctx->slices.bar_base = 0;
+  NP_INIT_CUDA(cudaMemset(ctx->slices.zfix, 0, chain_slices::zfix_words(ctx->d) * 8));
   NP_INIT_CUDA(cudaMemset(ctx->slices.bars, 0, chain_slices::bar_words() * 4));
   NP_INIT_CUDA(cudaMemset(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8));
   ctx->use_slices = !(cfg->flags & NP_F_ROW_CHAIN) && chain_slices::supported(d, ctx->sm_count);
@@ -688,9 +690,10 @@ int np_reset(np_ctx* ctx, void* stream) {
   if (!ctx) return fail(nullptr, NP_E_INVAL, "ctx is NULL");
   NP_LAUNCH(ctx, launch_tables_reset(ctx->d, ctx->t, as_stream(stream)));
   // a launch that gave up may have left the sliced kernel's counters and stamps anywhere
+  NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.zfix, 0, chain_slices::zfix_words(ctx->d) * 8, as_stream(stream)));
   NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.bars, 0, chain_slices::bar_words() * 4, as_stream(stream)));
   NP_CUDA(ctx, cudaMemsetAsync(ctx->slices.xch, 0, chain_slices::xch_words(ctx->d, ctx->sm_count) * 8, as_stream(stream)));
-  ctx->slices.bar_base = ctx->slices.seq_base = 0;
+  ctx->slices.seq_base = ctx->slices.bar_base = 0;
   NP_CUDA(ctx, cudaMemsetAsync(ctx->rows.z4, 0, chain_rows::z_floats(ctx->d) * 4, as_stream(stream)));
   NP_CUDA(ctx, cudaMemsetAsync(ctx->rows.cnt, 0, 4 * 4, as_stream(stream)));
   ctx->rows.cnt_base = ctx->rows.seq = 0;

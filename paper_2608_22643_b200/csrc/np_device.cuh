@@ -10,6 +10,7 @@ namespace npd {
 constexpr int kStatBadSlot = 1;     // slot index outside [0, C)
 constexpr int kStatBadNeuron = 2;   // neuron index outside [0, M)
 constexpr int kStatBadCount = 4;    // a list count larger than its capacity
+constexpr int kStatRange = 16;      // a partial MLP sum outside the range of the counted fixed-point words (or not a number)
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }

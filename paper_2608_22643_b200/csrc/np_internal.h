@@ -182,16 +182,18 @@ struct Plan {
   int R, ks, vg_shift, gw_shift, ng, window, run_layers, slot_cache_rows, max_rows, xch_stride;
   size_t group_bytes, smem;
 };
-// Library-owned device words and the host's running record of them: the arrival counters and
-// the exchange stamps only ever grow, so nothing has to be cleared between launches.
+// Library-owned device words and the host's running record of them: the counted sums and the
+// exchange stamps only ever grow, so nothing has to be cleared between launches.
 struct State {
-  unsigned int* bars;       // [bar_words()] zero at init / reset
-  unsigned long long* xch;  // [xch_words(d, sm_count)] zero at init / reset
+  unsigned long long* zfix;  // [zfix_words(d)] zero at init / reset
+  unsigned int* bars;        // [bar_words()] zero at init / reset
+  unsigned long long* xch;   // [xch_words(d, sm_count)] zero at init / reset
   unsigned int bar_base, seq_base;
 };
 bool plan(const Dims& d, int sm_count, Plan* p);
 bool supported(const Dims& d, int sm_count);
 size_t xch_words(const Dims& d, int sm_count);
+size_t zfix_words(const Dims& d);
 size_t bar_words();
 cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s, int sm_count);
 }  // namespace chain_slices

@@ -19,10 +19,34 @@
 //    (value, stamp) words that are written with one store and polled by the readers: no fence,
 //    no counter.  Phase 2 gives a partial sum of its quarter of the outputs only: a quarter of
 //    the reduction volume and of the accumulator re-read of a kernel that deals whole rows to
-//    the blocks (np_mlp_chain.cu), and the barrier that publishes x_{l+1} spans only the R
-//    blocks of the same quarter (x's quarter q is all block (r, q) ever needs: its K range in
-//    phase 1 is its column range in phase 2).  The sum of squares of x for the normalisation
-//    travels with the exchange.
+//    the blocks (np_mlp_chain.cu), and the hand-over of x_{l+1} spans only the R blocks of the
+//    same quarter (x's quarter q is all block (r, q) ever needs: its K range in phase 1 is its
+//    column range in phase 2).  The sum of squares of x for the normalisation travels with the
+//    exchange.
+//
+//    Between two layers of a launch the R partial sums of a column meet in 64-bit words that
+//    carry their own arrival count: a block adds, with one 64-bit reduction per column,
+//    2^56 + round(y * 2^30), so the word's top byte counts the blocks that have added and the
+//    rest is their sum in fixed point (resolution 2^-30, |y| < 2^19 per block, checked).  A
+//    reader polls the words of its own columns until the count is R: no fence, no arrival
+//    counter and no second trip to read the sums, the adds commute exactly (the result does not
+//    depend on their order), and nothing is cleared while it is in use: the words only grow, two
+//    sets of them alternate by layer, and a reader subtracts what it saw at the set's previous
+//    completion (all arithmetic modulo 2^64).  What the sets held when the launch began is read at
+//    its start (which also brings the words into the L2: a launch that found them zeroed by its
+//    predecessor instead measured 340-400 us per 32 layers against 261); a block's first adds wait
+//    until every block of its slice has done that reading (one arrival counter per slice, counted
+//    once per launch and long complete by the time the first layer ends).  The launch's last layer
+//    leaves its sums as fp32 in the stack's rotating accumulators, the form every other kernel of
+//    the chain reads.
+//
+//    This form is used where a thread owns one 4-column granule of the slice (row widths up to
+//    4096).  Wider slices keep the fp32 form between all layers: 16-byte fp32 reductions into the
+//    rotating accumulators (kZRep copies), a fence, one arrival counter per slice that the next
+//    layer's first thread polls, then every thread reads the copies of its columns.  There the
+//    counted words measured slower (13B shape 0.49 against 0.52-0.56 of the HBM peak, 70B shape
+//    0.45 against 0.53): twice the bytes per column, in 8-byte reductions, and twice the words to
+//    poll per thread.
 //
 // 2. Both phases run on the tensor cores (mma.sync m16n8k16, bf16 x bf16 -> fp32), not for
 //    their arithmetic rate but because one ldmatrix + one mma replace a hundred unpack and FMA
@@ -40,7 +64,7 @@
 // banks.  An exchange warp does the trip through L2 and leaves the activations.  Inside a
 // layer the consumer warps meet at no block-wide barrier until their sums are reduced.
 //
-// Every wait (mbarrier, exchange words, barrier counters) is bounded; once one has run out
+// Every wait (mbarrier, exchange words, counted sums) is bounded; once one has run out
 // the block records kStatTimeout and skips all later waits, so every thread still passes the
 // same barriers and the kernel drains; the blocks that depend on it follow at their next wait.
 #include <algorithm>
@@ -60,7 +84,10 @@ constexpr int kThreads = kWarps * 32;  // consumer threads
 constexpr int kBlock = kThreads + 64;  // plus one producer warp and one exchange warp
 constexpr int kMaxGroups = 16;         // ring slots
 constexpr int kMaxLayers = 64;         // layers per launch (longer runs are split by the host)
-constexpr int kBarStride = 32;         // one 128-byte line per barrier counter
+constexpr int kBarStride = 32;         // one 128-byte line per counter
+constexpr int kFixShift = 30;          // fixed-point position of the counted sums
+constexpr float kFixLimit = 524288.f;  // |partial sum| a block may add (2^19: 63 of them stay below 2^25 = 2^(55 - kFixShift))
+constexpr int kMaxR = 63;              // row groups whose counts and sums fit a word
 constexpr int kHist = 8;               // pacing history of the producer (> window)
 constexpr int kGroupTarget = 42 * 1024;
 constexpr int kPad = 16;               // bytes between pieces in shared memory
@@ -74,10 +101,13 @@ struct KArgs {
   const uint16_t* x_bf16;      // not NULL: the run starts the stack (layer 0) and reads its input from here (bf16 [D])
   float* xbuf[2];              // x_l of the run's last layer is stored to xbuf[l & 1]
   float* zbuf[3];              // MLP_l(x_l) accumulates into zbuf[l % 3]: kZRep copies of [D]
-  unsigned int* bars;          // [kQ][kBarStride] arrival counters, never reset: the host tracks their value
+  unsigned long long* zfix;    // [2][kZRep][D] counted fixed-point sums of MLP_l(x_l), sets alternate by layer, never cleared
+  unsigned int* bars;          // [kQ][kBarStride] arrival counters, never reset (the host tracks their value).  Counted
+                               // sums: blocks of a slice that have read the sets at the launch's start.  fp32 form:
+                               // blocks that have added their part of a layer (R per layer but the launch's last).
+  unsigned int bar_base;       // value of every counter when the launch starts
   unsigned long long* xch;     // [2][grid][xch_stride] (value, stamp) words
   int32_t* status;
-  unsigned int bar_base;       // value of every counter at launch
   unsigned int seq_base;       // stamp of the launch's first exchange minus one
   unsigned int ng_magic;       // ceil(2^32 / ng): group sequence number -> ring slot without a division
   int l_begin, l_end, D, C, check;
@@ -157,6 +187,9 @@ __device__ __forceinline__ void ld_relaxed_v2u64(const unsigned long long* p, un
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+__device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
 __device__ __forceinline__ unsigned long long stamped(float v, unsigned int stamp) {
   return ((unsigned long long)stamp << 32) | (unsigned long long)__float_as_uint(v);
 }
@@ -218,6 +251,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
   __shared__ int lay_rb[kMaxLayers];       // first active-list index of this block's row group, per layer
   __shared__ int lay_pre[kMaxLayers + 1];  // rows of this row group before each layer (virtual row index)
 
+  constexpr bool kFix = KS == 8;  // counted fixed-point sums between the layers of a launch (one granule per thread)
   const int D = a.D, Ds = D / kQ;
   const int nk = Ds >> 4;     // 16-wide K blocks = 16-column tiles of the slice
   const uint32_t piece_bytes = (uint32_t)Ds * 2u;
@@ -458,6 +492,35 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
   float4 xown[J4];        // x_l of the columns this thread owns, for the whole run
   unsigned int gseq = 0;  // sequence number of the layer's first group
   unsigned int nx = 0;    // exchanges so far
+  // counted sums: what the words of this thread's columns added up to (over the copies) when their set was last complete
+  // (zprev: the set read next, zprev2: the other one; they trade places after every read)
+  unsigned long long zprev[J4][4] = {}, zprev2[J4][4] = {};
+  if (kFix && nl > 1) {
+    unsigned long long seen = 0ull;
+#pragma unroll
+    for (int j = 0; j < J4; ++j) {
+      const int c = tid + j * kThreads;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) zprev[j][e] = zprev2[j][e] = 0ull;
+      if (c < nf4) {
+#pragma unroll
+        for (int rep = 0; rep < kZRep; ++rep) {
+          const ulonglong2* w = reinterpret_cast<const ulonglong2*>(a.zfix + (size_t)rep * D + qoff) + 2 * c;
+          const ulonglong2* w2 = reinterpret_cast<const ulonglong2*>(a.zfix + (size_t)(kZRep + rep) * D + qoff) + 2 * c;
+          const ulonglong2 p0 = __ldcg(w), p1 = __ldcg(w + 1), q0 = __ldcg(w2), q1 = __ldcg(w2 + 1);
+          zprev[j][0] += p0.x, zprev[j][1] += p0.y, zprev[j][2] += p1.x, zprev[j][3] += p1.y;
+          zprev2[j][0] += q0.x, zprev2[j][1] += q0.y, zprev2[j][2] += q1.x, zprev2[j][3] += q1.y;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) seen ^= zprev[j][e] ^ zprev2[j][e];
+      }
+    }
+    // Every value has arrived (it is looked at) before the block counts itself in: only then may any block of
+    // the slice add to these words.  (The words' top bytes hold small counts, so the pattern below cannot occur.)
+    if (seen == 0xffffffffffffffffull) atomicOr(a.status, kStatBadCount);
+    consumer_sync();
+    if (tid == 0) atomicAdd(a.bars + q * kBarStride, 1u);
+  }
   // phase 1, A operand: row = vector rr + 8 (m4 & 1) of the group (clamped into the group), K offset 8 (m4 >> 1)
   const uint32_t a1_off = (uint32_t)((rr + 8 * (m4 & 1)) & (VG - 1)) * pstride + (uint32_t)(m4 >> 1) * 16u;
   // phase 2, A operand (transposed load): stored row = down row rr + 8 (m4 >> 1) of the group, column offset 8 (m4 & 1)
@@ -466,8 +529,12 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
   for (int li = 0; li < nl; ++li) {
     const int l = a.l_begin + li;
     NP_TR(0);
-    // ---- wait until every block of this column slice has added its part of layer l-1 ----
-    if (li > 0) {
+    // ---- the sums of layer l-1 over this thread's columns, once every row group has added its part ----
+    float4 zsum[J4];
+#pragma unroll
+    for (int j = 0; j < J4; ++j) zsum[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!kFix && li > 0) {
+      // fp32 form: wait until every block of this column slice has added its part of layer l-1
       if (tid == 0 && *ok) {
         const unsigned int target = a.bar_base + (unsigned int)li * (unsigned int)R;
         bool arrived = false;
@@ -486,12 +553,73 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       }
       consumer_sync();
     }
+    if (kFix && li > 0) {
+      const int pb = (li - 1) & 1;
+      const unsigned long long* zw = a.zfix + (size_t)pb * kZRep * D + qoff;
+      // One lane per warp watches its own first column until the count is there: 148 x 256 threads polling all
+      // their words would keep the L2 busy with loads that find nothing new.  The blocks add all their columns
+      // in one go, so what the others read afterwards is complete but for stragglers, which they wait out below.
+      if (lane == 0 && tid < nf4) {
+        bool there = !*ok;
+        for (uint32_t spin = 0; spin < npp::kSpinLimit && !there; ++spin) {
+          unsigned long long w[kZRep], sum0 = 0ull;
+#pragma unroll
+          for (int rep = 0; rep < kZRep; ++rep) w[rep] = ld_relaxed_u64(zw + (size_t)rep * D + 4 * tid);
+#pragma unroll
+          for (int rep = 0; rep < kZRep; ++rep) sum0 += w[rep];
+          there = ((((long long)(sum0 - zprev[0][0])) + (1ll << 55)) >> 56) == (long long)R;
+        }
+      }
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < J4; ++j) {  // (one granule per thread in this form)
+        const int c = tid + j * kThreads;
+        if (c >= nf4) continue;
+        unsigned long long sum[4] = {0ull, 0ull, 0ull, 0ull};
+        bool done = !*ok;
+        for (uint32_t spin = 0; spin < npp::kSpinLimit && !done; ++spin) {
+          unsigned long long w[kZRep][4];  // every load of the round is issued before any is looked at
+#pragma unroll
+          for (int rep = 0; rep < kZRep; ++rep) {
+            const unsigned long long* wp = zw + (size_t)rep * D + 4 * c;
+            ld_relaxed_v2u64(wp, w[rep][0], w[rep][1]);
+            ld_relaxed_v2u64(wp + 2, w[rep][2], w[rep][3]);
+          }
+          done = true;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            sum[e] = 0ull;
+#pragma unroll
+            for (int rep = 0; rep < kZRep; ++rep) sum[e] += w[rep][e];
+            const long long delta = (long long)(sum[e] - zprev[j][e]);
+            done = done && ((delta + (1ll << 55)) >> 56) == (long long)R;
+          }
+        }
+        if (!done && *ok) {
+          *ok = 0;
+          atomicOr(a.status, npp::kStatTimeout);
+        }
+        float zv[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const long long value = (long long)(sum[e] - zprev[j][e]) - ((long long)R << 56);
+          zv[e] = done ? __ll2float_rn(value) * (1.f / (float)(1u << kFixShift)) : 0.f;
+          zprev[j][e] = zprev2[j][e];  // the other set is read next; this one, as it stands now, after that
+          zprev2[j][e] = sum[e];
+        }
+        zsum[j] = make_float4(zv[0], zv[1], zv[2], zv[3]);
+      }
+      // the launch's last layer adds into an accumulator that another block cleared one layer earlier (and
+      // fenced before it added the sums read above): the fence that completes that order on this side
+      if (li == nl - 1) __threadfence();
+    }
     NP_TR(1);
     // ---- x_l (this slice): first layer of the run from global, afterwards x_l = x_{l-1} + MLP_{l-1};
     //      each thread updates its own columns and publishes them as three bf16 terms ----
     {
       const float* xa = a.xbuf[(l + 1) & 1] + qoff;
-      const float* zb = l > 0 ? a.zbuf[(l - 1) % 3] + qoff : nullptr;
+      // fp32 sums of the layer before: the previous kernel's; in the fp32 form also those of this launch's layers
+      const float* zb = ((!kFix || li == 0) && l > 0) ? a.zbuf[(l - 1) % 3] + qoff : nullptr;
       float* xst = a.xbuf[l & 1] + qoff;
       float ssq = 0.f;
       float4 w[J4][kZRep];
@@ -520,6 +648,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
         const int c = tid + j * kThreads;
         if (c < nf4) {
           float4 v = xown[j];
+          v.x += zsum[j].x, v.y += zsum[j].y, v.z += zsum[j].z, v.w += zsum[j].w;
           if (zb) {
 #pragma unroll
             for (int rep = 0; rep < kZRep; ++rep) {
@@ -548,16 +677,25 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       }
       ssq = warp_sum(ssq);
       if (lane == 0) ssq_part[wid] = ssq;
-      // clear the next layer's accumulator copies of this slice: every row group takes a share
-      float* znext = a.zbuf[(l + 1) % 3] + qoff;
-      const int zper = (nf4 * kZRep + R - 1) / R;
-      for (int i = r * zper + tid; i < min((r + 1) * zper, nf4 * kZRep); i += kThreads) {
-        int rep = 0, c = i;
-        while (c >= nf4) {
-          c -= nf4;
-          ++rep;
+      // The launch's last layer adds fp32 sums into the stack's rotating accumulators: its own is cleared one
+      // layer ahead (by the layer before it; a launch of one layer finds it cleared by the kernel in front),
+      // and it clears the one the next kernel's first layer adds into.  Every row group takes a share.
+      if (!kFix || li >= nl - 2) {
+        float* znext = a.zbuf[(l + 1) % 3] + qoff;
+        const int zper = (nf4 * kZRep + R - 1) / R;
+        bool cleared = false;
+        for (int i = r * zper + tid; i < min((r + 1) * zper, nf4 * kZRep); i += kThreads) {
+          int rep = 0, c = i;
+          while (c >= nf4) {
+            c -= nf4;
+            ++rep;
+          }
+          reinterpret_cast<float4*>(znext + (size_t)rep * D)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+          cleared = true;
         }
-        reinterpret_cast<float4*>(znext + (size_t)rep * D)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        // the zeros are ahead of this block's counted sums of this layer (added after the barriers below),
+        // which every block reads before it adds to the cleared accumulator
+        if (kFix && cleared && li == nl - 2) __threadfence();
       }
     }
     consumer_sync();  // the terms of x and ssq_part are in place
@@ -702,12 +840,53 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
     gseq += (unsigned int)(n_gu + n_dn);
     NP_TR(5);
 
-    // ---- this block's partial MLP_l(x_l) over its column slice: the three terms are added up and staged
-    //      in shared memory, so that the reductions to the layer's accumulator are 16 bytes wide ----
+    // ---- this block's partial MLP_l(x_l) over its column slice ----
+    if (kFix && li + 1 < nl) {
+      // Between layers of the launch: counted fixed-point sums, straight from the accumulators.  One 64-bit
+      // reduction per column carries the value and this block's arrival (a row group without rows still
+      // counts); a warp's adds leave as soon as its own tiles are done.
+      unsigned long long* zacc = a.zfix + ((size_t)((li & 1) * kZRep + r % kZRep)) * D + qoff;
+      if (li == 0) {  // the launch's first adds: every block of the slice has read what the sets held before
+        if (lane == 0 && *ok) {
+          const unsigned int target = a.bar_base + (unsigned int)R;
+          bool arrived = false;
+          for (uint32_t spin = 0; spin < npp::kSpinLimit && !arrived; ++spin) {
+            unsigned int v;
+            asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a.bars + q * kBarStride) : "memory");
+            arrived = (int)(v - target) >= 0;
+          }
+          if (!arrived) {
+            *ok = 0;
+            atomicOr(a.status, npp::kStatTimeout);
+          }
+        }
+        __syncwarp();
+      }
+#pragma unroll
+      for (int j = 0; j < KS; ++j) {
+        // acc[j]: [0], [1] = (column g8 of tile mt, terms 2 t4, 2 t4 + 1); [2], [3] = (column g8 + 8, same terms)
+        // (columns 3-7 of B are zero: lanes t4 = 0 and 1 hold the three terms between them)
+        float lo = acc[j][0] + acc[j][1];
+        float hi = acc[j][2] + acc[j][3];
+        lo += __shfl_xor_sync(0xffffffffu, lo, 1);
+        hi += __shfl_xor_sync(0xffffffffu, hi, 1);
+        const int mt = wid + kWarps * j;
+        if (t4 < 2 && mt < nk) {  // lane t4 = 0 adds column g8, lane t4 = 1 column g8 + 8
+          const float y = t4 == 0 ? lo : hi;
+          long long fx = 0;
+          if (fabsf(y) < kFixLimit) fx = __float2ll_rn(y * (float)(1u << kFixShift));
+          else atomicOr(a.status, kStatRange);  // also a NaN: the sum would not mean anything
+          red_add_u64(zacc + mt * 16 + g8 + 8 * t4, (unsigned long long)fx + (1ull << 56));
+        }
+      }
+      NP_TR(6);
+      NP_TR(7);
+      continue;
+    }
+    // The launch's last layer: the three terms are added up and staged in shared memory, so that the
+    // reductions to the stack's fp32 accumulator are 16 bytes wide.
 #pragma unroll
     for (int j = 0; j < KS; ++j) {
-      // acc[j]: [0], [1] = (column g8 of tile mt, terms 2 t4, 2 t4 + 1); [2], [3] = (column g8 + 8, same terms)
-      // (columns 3-7 of B are zero: a lane's two columns add up to its share of the three terms)
       float lo = acc[j][0] + acc[j][1];
       float hi = acc[j][2] + acc[j][3];
       lo += __shfl_xor_sync(0xffffffffu, lo, 1);
@@ -727,8 +906,8 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
         if (c < nf4) red_add_v4(yacc + 4 * c, reinterpret_cast<const float4*>(ybuf)[c]);
       }
     }
-    if (li + 1 < nl) {
-      // publish: every warp waits for its own adds (the lanes' adds precede lane 0's fence), then
+    if (!kFix && li + 1 < nl) {
+      // fp32 form, publish: every warp waits for its own adds (the lanes' adds precede lane 0's fence), then
       // one thread counts the block in
       __syncwarp();
       if (lane == 0) __threadfence();
@@ -747,6 +926,7 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   const int ks = (nk + kWarps - 1) / kWarps;
   if (ks > 32) return false;
   const int R = sm_count / kQ;
+  if (R > kMaxR) return false;
   const size_t pstride = (size_t)Ds * 2 + kPad;
   const int max_rows = (d.C + R - 1) / R;  // whatever the active count turns out to be
   // a group: VG vectors (a power of two, at most the 16 rows of an MMA tile), about 32 KB
@@ -774,7 +954,12 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   p->run_layers = (int)std::max<size_t>(1, std::min<size_t>(kMaxLayers, cache_bytes / (4 * (size_t)max_rows)));
   p->slot_cache_rows = p->run_layers * max_rows;
   const size_t fixed = fixed0 + (size_t)p->slot_cache_rows * 4;
-  int window = std::max(1, std::min(ng - 1, (int)(40 * 1024 / group_bytes)));
+  // Groups in flight per block.  Where the hand-over between layers has no fence (counted sums, ks = 8) the
+  // producer runs as far ahead as the ring and its pacing history allow (7B shape: 284 us per 32 layers with one
+  // group in flight, 274 with five).  The fp32 form keeps about 40 KB in flight: a deeper burst queues in front
+  // of its fence and of the short loads behind it (13B shape: 385 us per 40 layers with one 41 KB group in
+  // flight, 411 with two or more; 70B shape: no difference).
+  int window = ks <= 8 ? std::max(1, std::min(ng - 1, kHist - 1)) : std::max(1, std::min(ng - 1, (int)(40 * 1024 / group_bytes)));
 #ifdef NP_TUNE  // development builds only: geometry from the environment
   if (const char* e = getenv("NP_SL_NG")) ng = std::max(2, std::min(ng, atoi(e)));
   if (const char* e = getenv("NP_SL_WIN")) window = std::min(atoi(e), std::min(kHist - 1, ng - 1));
@@ -803,6 +988,7 @@ size_t xch_words(const Dims& d, int sm_count) {
   if (!plan(d, sm_count, &p)) return 16;
   return (size_t)2 * (p.R * kQ) * p.xch_stride;
 }
+size_t zfix_words(const Dims& d) { return (size_t)2 * kZRep * d.D; }
 size_t bar_words() { return (size_t)kQ * kBarStride; }
 
 template <int KS, bool XB>
@@ -829,7 +1015,7 @@ static cudaError_t launch_one(const KArgs& ka, size_t sm, int grid_x, cudaStream
 
 cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s, int sm_count) {
   Plan p;
-  if (!plan(d, sm_count, &p) || !st || !st->bars || !st->xch) return cudaErrorInvalidValue;
+  if (!plan(d, sm_count, &p) || !st || !st->zfix || !st->bars || !st->xch) return cudaErrorInvalidValue;
   cudaError_t e = cudaSuccess;
   for (int l0 = a.l_begin; l0 < a.l_end; l0 += p.run_layers) {
     KArgs ka;
@@ -841,10 +1027,11 @@ cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s,
     ka.x_bf16 = l0 == 0 ? static_cast<const uint16_t*>(a.x_bf16) : nullptr;
     for (int i = 0; i < 2; ++i) ka.xbuf[i] = a.xbuf[i];
     for (int i = 0; i < 3; ++i) ka.zbuf[i] = a.zbuf[i];
+    ka.zfix = st->zfix;
     ka.bars = st->bars;
+    ka.bar_base = st->bar_base;
     ka.xch = st->xch;
     ka.status = a.status;
-    ka.bar_base = st->bar_base;
     ka.seq_base = st->seq_base;
     ka.ng_magic = (unsigned int)((0x100000000ull + p.ng - 1) / p.ng);
     ka.l_begin = l0;
@@ -861,7 +1048,7 @@ cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s,
     ka.group_bytes = (uint32_t)p.group_bytes;
     const int nl = ka.l_end - ka.l_begin;
     // the counters and stamps only ever grow; the next launch starts where this one ends
-    st->bar_base += (unsigned int)(nl - 1) * (unsigned int)p.R;
+    if (nl > 1) st->bar_base += (p.ks == 8 ? 1u : (unsigned int)(nl - 1)) * (unsigned int)p.R;
     st->seq_base += (unsigned int)nl + 1u;
     const bool xb = ((d.D / kQ / 16) >> p.gw_shift) <= 32 && p.ks <= 16;  // phase 1's B operands fit a warp's registers
     if (p.ks == 8) e = xb ? launch_one<8, true>(ka, p.smem, p.R * kQ, s) : launch_one<8, false>(ka, p.smem, p.R * kQ, s);

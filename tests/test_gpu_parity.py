@@ -317,6 +317,26 @@ def test_resident_chain_with_set_sizes_away_from_k(n_set, flags):
         p.close()
 
 
+def test_partial_sums_beyond_the_counted_words_range_are_reported():
+    """Between the layers of a launch the resident kernel hands the MLP's partial sums over as counted
+    fixed-point words (|sum| < 2^19 per block).  Down rows of 3e6 push layer 0 far past that: the launch
+    must say so in the status word (bit 16), not hand on a wrapped sum."""
+    cfg = DENSE
+    p = Pair(cfg, with_oracle=False, chain_layers=cfg.n_layers)
+    try:
+        assert nb.np_mlp_kernel_name(p.eng.ctx, 1) == "k_mlp_slices"
+        p.backing[0, :, 2, :] = 3.0e6                       # record = [gate | up | down] vectors of a neuron
+        words = synth.random_bitmaps(cfg.n_layers, cfg.d_ffn, p.k, 3, 1, 0.6)
+        x = synth.hidden_states(cfg, 1)[0].cuda()
+        out = torch.empty((1, cfg.d_model), dtype=torch.float32, device="cuda")
+        nb.np_step_selected(p.eng.ctx, x, 1, words[0].cuda(), out, p.eng.stream, p.eng.copy_stream)
+        torch.cuda.synchronize()
+        with pytest.raises(nb.NpError, match="0x10"):
+            p.eng.counters()
+    finally:
+        p.close()
+
+
 def test_call_order_and_argument_errors():
     p = Pair(TINY, with_oracle=False)
     try:
