@@ -15,7 +15,7 @@ constexpr int kMaxBatch = 16;
 constexpr int kHostHeaderInts = 16;
 constexpr float kRmsEps = 1e-6f;  // x / sqrt(mean(x^2) + eps) in front of every MLP of the chain
 #ifndef NP_ZREP
-#define NP_ZREP 4
+#define NP_ZREP 2
 #endif
 constexpr int kZRep = NP_ZREP;  // copies of each MLP accumulator vector (spreads same-address adds)  // global header of the host list mirror
 

@@ -88,6 +88,12 @@ constexpr int kBarStride = 32;         // one 128-byte line per counter
 constexpr int kFixShift = 30;          // fixed-point position of the counted sums
 constexpr float kFixLimit = 524288.f;  // |partial sum| a block may add (2^19: 63 of them stay below 2^25 = 2^(55 - kFixShift))
 constexpr int kMaxR = 63;              // row groups whose counts and sums fit a word
+#ifndef NP_SL_FIXREP
+#define NP_SL_FIXREP 1
+#endif
+constexpr int kFixRep = NP_SL_FIXREP;  // copies of the counted words (row group r adds to copy r % kFixRep).  One: the 37
+                                       // adds to a word cost less than reading more copies (7B shape, 32 layers: 250 us
+                                       // with one copy, 252 with two, 262 with four)
 constexpr int kHist = 8;               // pacing history of the producer (> window)
 constexpr int kGroupTarget = 42 * 1024;
 constexpr int kPad = 16;               // bytes between pieces in shared memory
@@ -101,7 +107,7 @@ struct KArgs {
   const uint16_t* x_bf16;      // not NULL: the run starts the stack (layer 0) and reads its input from here (bf16 [D])
   float* xbuf[2];              // x_l of the run's last layer is stored to xbuf[l & 1]
   float* zbuf[3];              // MLP_l(x_l) accumulates into zbuf[l % 3]: kZRep copies of [D]
-  unsigned long long* zfix;    // [2][kZRep][D] counted fixed-point sums of MLP_l(x_l), sets alternate by layer, never cleared
+  unsigned long long* zfix;    // [2][kFixRep][D] counted fixed-point sums of MLP_l(x_l), sets alternate by layer, never cleared
   unsigned int* bars;          // [kQ][kBarStride] arrival counters, never reset (the host tracks their value).  Counted
                                // sums: blocks of a slice that have read the sets at the launch's start.  fp32 form:
                                // blocks that have added their part of a layer (R per layer but the launch's last).
@@ -504,9 +510,9 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       for (int e = 0; e < 4; ++e) zprev[j][e] = zprev2[j][e] = 0ull;
       if (c < nf4) {
 #pragma unroll
-        for (int rep = 0; rep < kZRep; ++rep) {
+        for (int rep = 0; rep < kFixRep; ++rep) {
           const ulonglong2* w = reinterpret_cast<const ulonglong2*>(a.zfix + (size_t)rep * D + qoff) + 2 * c;
-          const ulonglong2* w2 = reinterpret_cast<const ulonglong2*>(a.zfix + (size_t)(kZRep + rep) * D + qoff) + 2 * c;
+          const ulonglong2* w2 = reinterpret_cast<const ulonglong2*>(a.zfix + (size_t)(kFixRep + rep) * D + qoff) + 2 * c;
           const ulonglong2 p0 = __ldcg(w), p1 = __ldcg(w + 1), q0 = __ldcg(w2), q1 = __ldcg(w2 + 1);
           zprev[j][0] += p0.x, zprev[j][1] += p0.y, zprev[j][2] += p1.x, zprev[j][3] += p1.y;
           zprev2[j][0] += q0.x, zprev2[j][1] += q0.y, zprev2[j][2] += q1.x, zprev2[j][3] += q1.y;
@@ -555,22 +561,11 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
     }
     if (kFix && li > 0) {
       const int pb = (li - 1) & 1;
-      const unsigned long long* zw = a.zfix + (size_t)pb * kZRep * D + qoff;
-      // One lane per warp watches its own first column until the count is there: 148 x 256 threads polling all
-      // their words would keep the L2 busy with loads that find nothing new.  The blocks add all their columns
-      // in one go, so what the others read afterwards is complete but for stragglers, which they wait out below.
-      if (lane == 0 && tid < nf4) {
-        bool there = !*ok;
-        for (uint32_t spin = 0; spin < npp::kSpinLimit && !there; ++spin) {
-          unsigned long long w[kZRep], sum0 = 0ull;
-#pragma unroll
-          for (int rep = 0; rep < kZRep; ++rep) w[rep] = ld_relaxed_u64(zw + (size_t)rep * D + 4 * tid);
-#pragma unroll
-          for (int rep = 0; rep < kZRep; ++rep) sum0 += w[rep];
-          there = ((((long long)(sum0 - zprev[0][0])) + (1ll << 55)) >> 56) == (long long)R;
-        }
-      }
-      __syncwarp();
+      const unsigned long long* zw = a.zfix + (size_t)pb * kFixRep * D + qoff;
+      // Every thread polls the words of its own columns (two 16-byte loads per round with one copy of the
+      // words).  With four copies, 148 x 256 threads polling eight loads each kept the L2 busy enough to slow
+      // every other trip through it, and a lane per warp watched one column first; with one copy that watch
+      // only costs a round trip (7B shape, 32 layers: 250 us without it, 253 with it).
 #pragma unroll
       for (int j = 0; j < J4; ++j) {  // (one granule per thread in this form)
         const int c = tid + j * kThreads;
@@ -578,9 +573,9 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
         unsigned long long sum[4] = {0ull, 0ull, 0ull, 0ull};
         bool done = !*ok;
         for (uint32_t spin = 0; spin < npp::kSpinLimit && !done; ++spin) {
-          unsigned long long w[kZRep][4];  // every load of the round is issued before any is looked at
+          unsigned long long w[kFixRep][4];  // every load of the round is issued before any is looked at
 #pragma unroll
-          for (int rep = 0; rep < kZRep; ++rep) {
+          for (int rep = 0; rep < kFixRep; ++rep) {
             const unsigned long long* wp = zw + (size_t)rep * D + 4 * c;
             ld_relaxed_v2u64(wp, w[rep][0], w[rep][1]);
             ld_relaxed_v2u64(wp + 2, w[rep][2], w[rep][3]);
@@ -590,7 +585,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
           for (int e = 0; e < 4; ++e) {
             sum[e] = 0ull;
 #pragma unroll
-            for (int rep = 0; rep < kZRep; ++rep) sum[e] += w[rep][e];
+            for (int rep = 0; rep < kFixRep; ++rep) sum[e] += w[rep][e];
             const long long delta = (long long)(sum[e] - zprev[j][e]);
             done = done && ((delta + (1ll << 55)) >> 56) == (long long)R;
           }
@@ -738,7 +733,8 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
           // free of branches (their A tiles are read from the group's first K block)
 #pragma unroll
           for (int it = 0; it < 32; it += 4) {
-            if (it < trip) {  // warp-uniform; four independent chains, the four loads before the four mma
+            if (it < trip) {  // warp-uniform; four independent chains, the four loads before the four mma (eight
+                              // chains cost registers and measured 271 us per 32 layers against 250)
               uint32_t af[4][4];
 #pragma unroll
               for (int u = 0; u < 4; ++u) ldmatrix_x4(af[u], ap + (it + u < trip ? (uint32_t)(it + u) * kstep : 0u));
@@ -845,7 +841,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       // Between layers of the launch: counted fixed-point sums, straight from the accumulators.  One 64-bit
       // reduction per column carries the value and this block's arrival (a row group without rows still
       // counts); a warp's adds leave as soon as its own tiles are done.
-      unsigned long long* zacc = a.zfix + ((size_t)((li & 1) * kZRep + r % kZRep)) * D + qoff;
+      unsigned long long* zacc = a.zfix + ((size_t)((li & 1) * kFixRep + r % kFixRep)) * D + qoff;
       if (li == 0) {  // the launch's first adds: every block of the slice has read what the sets held before
         if (lane == 0 && *ok) {
           const unsigned int target = a.bar_base + (unsigned int)R;
@@ -988,7 +984,7 @@ size_t xch_words(const Dims& d, int sm_count) {
   if (!plan(d, sm_count, &p)) return 16;
   return (size_t)2 * (p.R * kQ) * p.xch_stride;
 }
-size_t zfix_words(const Dims& d) { return (size_t)2 * kZRep * d.D; }
+size_t zfix_words(const Dims& d) { return (size_t)2 * kFixRep * d.D; }
 size_t bar_words() { return (size_t)kQ * kBarStride; }
 
 template <int KS, bool XB>
