@@ -40,13 +40,11 @@
 //    leaves its sums as fp32 in the stack's rotating accumulators, the form every other kernel of
 //    the chain reads.
 //
-//    This form is used where a thread owns one 4-column granule of the slice (row widths up to
-//    4096).  Wider slices keep the fp32 form between all layers: 16-byte fp32 reductions into the
-//    rotating accumulators (kZRep copies), a fence, one arrival counter per slice that the next
-//    layer's first thread polls, then every thread reads the copies of its columns.  There the
-//    counted words measured slower (13B shape 0.49 against 0.52-0.56 of the HBM peak, 70B shape
-//    0.45 against 0.53): twice the bytes per column, in 8-byte reductions, and twice the words to
-//    poll per thread.
+//    This form is used where a thread owns one or two 4-column granules of the slice (row widths
+//    up to 8192).  Wider slices keep the fp32 form between all layers: 16-byte fp32 reductions into
+//    the rotating accumulators (kZRep copies), a fence, one arrival counter per slice that the next
+//    layer's first thread polls, then every thread reads the copies of its columns (the counted
+//    form would hold the previous sums of four granules in registers there).
 //
 // 2. Both phases run on the tensor cores (mma.sync m16n8k16, bf16 x bf16 -> fp32), not for
 //    their arithmetic rate but because one ldmatrix + one mma replace a hundred unpack and FMA
@@ -88,6 +86,8 @@ constexpr int kBarStride = 32;         // one 128-byte line per counter
 constexpr int kFixShift = 30;          // fixed-point position of the counted sums
 constexpr float kFixLimit = 524288.f;  // |partial sum| a block may add (2^19: 63 of them stay below 2^25 = 2^(55 - kFixShift))
 constexpr int kMaxR = 63;              // row groups whose counts and sums fit a word
+constexpr int kFixMaxKS = 16;          // widest slices (in 16-column tiles per warp) that use the counted words: one or two
+                                       // 4-column granules per thread, row widths up to 8192
 #ifndef NP_SL_FIXREP
 #define NP_SL_FIXREP 1
 #endif
@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
   __shared__ int lay_rb[kMaxLayers];       // first active-list index of this block's row group, per layer
   __shared__ int lay_pre[kMaxLayers + 1];  // rows of this row group before each layer (virtual row index)
 
-  constexpr bool kFix = KS == 8;  // counted fixed-point sums between the layers of a launch (one granule per thread)
+  constexpr bool kFix = KS <= kFixMaxKS;  // counted fixed-point sums between the layers of a launch
   const int D = a.D, Ds = D / kQ;
   const int nk = Ds >> 4;     // 16-wide K blocks = 16-column tiles of the slice
   const uint32_t piece_bytes = (uint32_t)Ds * 2u;
@@ -567,7 +567,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       // every other trip through it, and a lane per warp watched one column first; with one copy that watch
       // only costs a round trip (7B shape, 32 layers: 250 us without it, 253 with it).
 #pragma unroll
-      for (int j = 0; j < J4; ++j) {  // (one granule per thread in this form)
+      for (int j = 0; j < J4; ++j) {  // one or two granules per thread, one after the other
         const int c = tid + j * kThreads;
         if (c >= nf4) continue;
         unsigned long long sum[4] = {0ull, 0ull, 0ull, 0ull};
@@ -950,12 +950,12 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   p->run_layers = (int)std::max<size_t>(1, std::min<size_t>(kMaxLayers, cache_bytes / (4 * (size_t)max_rows)));
   p->slot_cache_rows = p->run_layers * max_rows;
   const size_t fixed = fixed0 + (size_t)p->slot_cache_rows * 4;
-  // Groups in flight per block.  Where the hand-over between layers has no fence (counted sums, ks = 8) the
-  // producer runs as far ahead as the ring and its pacing history allow (7B shape: 284 us per 32 layers with one
-  // group in flight, 274 with five).  The fp32 form keeps about 40 KB in flight: a deeper burst queues in front
-  // of its fence and of the short loads behind it (13B shape: 385 us per 40 layers with one 41 KB group in
-  // flight, 411 with two or more; 70B shape: no difference).
-  int window = ks <= 8 ? std::max(1, std::min(ng - 1, kHist - 1)) : std::max(1, std::min(ng - 1, (int)(40 * 1024 / group_bytes)));
+  // Groups in flight per block.  Where the hand-over between layers has no fence (counted sums) the producer runs
+  // as far ahead as the ring and its pacing history allow (7B shape: 284 us per 32 layers with one group in
+  // flight, 274 with five; 13B shape: 390 us per 40 layers against 357).  The fp32 form keeps about 40 KB in
+  // flight: a deeper burst queues in front of its fence and of the short loads behind it (13B shape, when it
+  // still used this form: 385 us with one 41 KB group in flight, 411 with two or more).
+  int window = ks <= kFixMaxKS ? std::max(1, std::min(ng - 1, kHist - 1)) : std::max(1, std::min(ng - 1, (int)(40 * 1024 / group_bytes)));
 #ifdef NP_TUNE  // development builds only: geometry from the environment
   if (const char* e = getenv("NP_SL_NG")) ng = std::max(2, std::min(ng, atoi(e)));
   if (const char* e = getenv("NP_SL_WIN")) window = std::min(atoi(e), std::min(kHist - 1, ng - 1));
@@ -1044,7 +1044,7 @@ cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s,
     ka.group_bytes = (uint32_t)p.group_bytes;
     const int nl = ka.l_end - ka.l_begin;
     // the counters and stamps only ever grow; the next launch starts where this one ends
-    if (nl > 1) st->bar_base += (p.ks == 8 ? 1u : (unsigned int)(nl - 1)) * (unsigned int)p.R;
+    if (nl > 1) st->bar_base += (p.ks <= kFixMaxKS ? 1u : (unsigned int)(nl - 1)) * (unsigned int)p.R;
     st->seq_base += (unsigned int)nl + 1u;
     const bool xb = ((d.D / kQ / 16) >> p.gw_shift) <= 32 && p.ks <= 16;  // phase 1's B operands fit a warp's registers
     if (p.ks == 8) e = xb ? launch_one<8, true>(ka, p.smem, p.R * kQ, s) : launch_one<8, false>(ka, p.smem, p.R * kQ, s);
