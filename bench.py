@@ -365,7 +365,19 @@ def cuda_arm(args):
     Lp, lp_why = plan_store_layers(cfg, args.store_layers, int(os.environ.get("LOCAL_WORLD_SIZE", world)))
     if Lp < cfg.n_layers and (args.transfer == "file" or args.dense_layers > Lp):
         raise SystemExit("bench.py: an aliased store is not combined with --transfer file or a longer dense prefix here")
-    w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True, store_layers=Lp)
+    # The host may refuse to page-lock a store that MemAvailable said would fit (a limit on locked memory, a
+    # fragmented host): then the store is aliased over three quarters of the layers, and so on.
+    while True:
+        try:
+            w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True, store_layers=Lp)
+            break
+        except RuntimeError as e:
+            if "cudaHostRegister" not in str(e) or Lp <= max(1, cfg.n_layers // 8) or args.transfer == "file" \
+                    or args.store_layers != "auto":
+                raise
+            torch.cuda.synchronize()
+            lp_why = f"the host refused to page-lock {Lp} layers ({Lp * cfg.d_ffn * cfg.record_bytes / 2**30:.0f} GiB)"
+            Lp = max(args.dense_layers, max(1, (3 * Lp) // 4))
     # replicas share one host: the packing threads of the gather transfer are divided among them
     if args.host_threads == 0 and world > 1:
         args.host_threads = nb.replica_host_threads(int(os.environ.get("LOCAL_WORLD_SIZE", world)))
