@@ -1228,10 +1228,14 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
   if (part != kChainTail) ctx->chain_kernel_launches = 0;
   // the sliced kernel widens the stack's bf16 input itself when it runs layer 0
   const bool fold_widen = persistent && (ctx->use_rows || ctx->use_slices) && d.dense == 0;
+  // Where the sliced kernel hands its sums over as counted words, layer 0's fp32 accumulator is used only by a
+  // first launch of one layer that does not end the stack: the clearing waits until the runs are known.
+  const bool lazy_clear = fold_widen && ctx->use_slices && !ctx->use_rows && chain_slices::counted_handover(d, ctx->sm_count);
+  bool out_written = false;  // the last resident launch left x_out itself
   if (part != kChainTail) {
     if (!fold_widen) NP_LAUNCH(ctx, launch_widen_bf16(x_bf16, ctx->ws.xbuf[1], n, s));
     // the accumulator of layer 0 starts at zero (later ones are cleared one layer ahead)
-    NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, (persistent ? (size_t)kZRep * d.D : n) * 4, s));
+    if (!lazy_clear) NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, (persistent ? (size_t)kZRep * d.D : n) * 4, s));
   }
   if (persistent) {
     // runs of layers in one resident kernel each; a run starts once its layers are installed,
@@ -1246,6 +1250,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
     a.check = ctx->cfg.flags & NP_F_CHECK_BOUNDS;
     a.counters = ctx->t.counters;
     a.x_bf16 = fold_widen ? x_bf16 : nullptr;
+    a.x_out = nullptr;
     // the dense prefix first: whole records, every row active, nothing to wait for (it also
     // widens the window in which the sparse layers' rows arrive)
     if (d.dense > 0 && part != kChainTail) {
@@ -1329,7 +1334,11 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
         chain_slices::Plan sp;
         chain_slices::plan(d, ctx->sm_count, &sp);
         ctx->chain_kernel_launches += (l1 - l0 + sp.run_layers - 1) / sp.run_layers;
+        a.x_out = l1 == d.L ? x_out : nullptr;  // the run that ends the stack may leave the result itself
+        if (lazy_clear && l0 == 0 && std::min(l1, sp.run_layers) == 1 && l1 != d.L)
+          NP_CUDA(ctx, cudaMemsetAsync(ctx->ws.zbuf[0], 0, (size_t)kZRep * d.D * 4, s));
         NP_LAUNCH(ctx, chain_slices::launch(d, a, &ctx->slices, s, ctx->sm_count));
+        out_written = a.x_out && ctx->slices.wrote_out;
       } else {
         ctx->chain_kernel_launches += 1;
         NP_LAUNCH(ctx, chain_alu::launch(d, a, s, ctx->sm_count));
@@ -1356,7 +1365,7 @@ static int mlp_chain(np_ctx* ctx, const void* x_bf16, int B, float* x_out, cudaS
       if (rc < 0) return rc;
     }
   }
-  if (part != kChainHead) {
+  if (part != kChainHead && !out_written) {
     if (tc_batch)  // the last accumulator holds the result
       NP_LAUNCH(ctx, launch_add_vec(ctx->ws.zbuf[(d.L - 1) % 3], nullptr, 0, x_out, n, s));
     else

@@ -161,6 +161,7 @@ struct ChainArgs {
   const void* x_bf16;  // sliced kernel only, may be NULL: the stack's input, read by the run that starts at layer 0
   float* xbuf[2];
   float* zbuf[3];
+  float* x_out;  // may be NULL; a kernel that can leave the stack's result itself (the run ends the stack) does so here
   unsigned int* grid_bar;
   int32_t* status;
   int l_begin, l_end, check;
@@ -189,10 +190,12 @@ struct State {
   unsigned int* bars;        // [bar_words()] zero at init / reset
   unsigned long long* xch;   // [xch_words(d, sm_count)] zero at init / reset
   unsigned int bar_base, seq_base;
+  int wrote_out;             // the last launch left the stack's result in ChainArgs::x_out
 };
 bool plan(const Dims& d, int sm_count, Plan* p);
 bool supported(const Dims& d, int sm_count);
 size_t xch_words(const Dims& d, int sm_count);
+bool counted_handover(const Dims& d, int sm_count);  // the sums between layers are counted fixed-point words for this shape
 size_t zfix_words(const Dims& d);
 size_t bar_words();
 cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s, int sm_count);

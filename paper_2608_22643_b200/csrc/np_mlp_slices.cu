@@ -106,6 +106,7 @@ struct KArgs {
   const int32_t* counters;     // [L][NP_N_COUNTERS]
   const uint16_t* x_bf16;      // not NULL: the run starts the stack (layer 0) and reads its input from here (bf16 [D])
   float* xbuf[2];              // x_l of the run's last layer is stored to xbuf[l & 1]
+  float* x_out;                // counted form only, may be NULL: the launch ends the stack and leaves x_L = x_{L-1} + MLP_{L-1} here
   float* zbuf[3];              // MLP_l(x_l) accumulates into zbuf[l % 3]: kZRep copies of [D]
   unsigned long long* zfix;    // [2][kFixRep][D] counted fixed-point sums of MLP_l(x_l), sets alternate by layer, never cleared
   unsigned int* bars;          // [kQ][kBarStride] arrival counters, never reset (the host tracks their value).  Counted
@@ -258,6 +259,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
   __shared__ int lay_pre[kMaxLayers + 1];  // rows of this row group before each layer (virtual row index)
 
   constexpr bool kFix = KS <= kFixMaxKS;  // counted fixed-point sums between the layers of a launch
+  const bool fin = kFix && a.x_out != nullptr;  // ... and behind its last layer: the launch leaves the stack's result itself
   const int D = a.D, Ds = D / kQ;
   const int nk = Ds >> 4;     // 16-wide K blocks = 16-column tiles of the slice
   const uint32_t piece_bytes = (uint32_t)Ds * 2u;
@@ -501,7 +503,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
   // counted sums: what the words of this thread's columns added up to (over the copies) when their set was last complete
   // (zprev: the set read next, zprev2: the other one; they trade places after every read)
   unsigned long long zprev[J4][4] = {}, zprev2[J4][4] = {};
-  if (kFix && nl > 1) {
+  if (kFix && (nl > 1 || fin)) {
     unsigned long long seen = 0ull;
 #pragma unroll
     for (int j = 0; j < J4; ++j) {
@@ -606,7 +608,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       }
       // the launch's last layer adds into an accumulator that another block cleared one layer earlier (and
       // fenced before it added the sums read above): the fence that completes that order on this side
-      if (li == nl - 1) __threadfence();
+      if (li == nl - 1 && !fin) __threadfence();
     }
     NP_TR(1);
     // ---- x_l (this slice): first layer of the run from global, afterwards x_l = x_{l-1} + MLP_{l-1};
@@ -675,7 +677,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       // The launch's last layer adds fp32 sums into the stack's rotating accumulators: its own is cleared one
       // layer ahead (by the layer before it; a launch of one layer finds it cleared by the kernel in front),
       // and it clears the one the next kernel's first layer adds into.  Every row group takes a share.
-      if (!kFix || li >= nl - 2) {
+      if (!kFix || (!fin && li >= nl - 2)) {
         float* znext = a.zbuf[(l + 1) % 3] + qoff;
         const int zper = (nf4 * kZRep + R - 1) / R;
         bool cleared = false;
@@ -837,8 +839,8 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
     NP_TR(5);
 
     // ---- this block's partial MLP_l(x_l) over its column slice ----
-    if (kFix && li + 1 < nl) {
-      // Between layers of the launch: counted fixed-point sums, straight from the accumulators.  One 64-bit
+    if (kFix && (li + 1 < nl || fin)) {
+      // Between layers of the launch (and behind the last one where the launch ends the stack): counted fixed-point sums, straight from the accumulators.  One 64-bit
       // reduction per column carries the value and this block's arrival (a row group without rows still
       // counts); a warp's adds leave as soon as its own tiles are done.
       unsigned long long* zacc = a.zfix + ((size_t)((li & 1) * kFixRep + r % kFixRep)) * D + qoff;
@@ -913,6 +915,45 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
       NP_TR(7);
     }
   }
+  // ---- the launch ends the stack: the blocks of row group 0 wait for the last layer's sums like a next layer
+  //      would and leave x_L (no kernel behind this one has to add the accumulator copies up) ----
+  if (fin && r == 0) {
+    const unsigned long long* zw = a.zfix + (size_t)((nl - 1) & 1) * kFixRep * D + qoff;
+#pragma unroll
+    for (int j = 0; j < J4; ++j) {
+      const int c = tid + j * kThreads;
+      if (c >= nf4) continue;
+      unsigned long long sum[4] = {0ull, 0ull, 0ull, 0ull};
+      bool done = !*ok;
+      for (uint32_t spin = 0; spin < npp::kSpinLimit && !done; ++spin) {
+        unsigned long long w[kFixRep][4];
+#pragma unroll
+        for (int rep = 0; rep < kFixRep; ++rep) {
+          const unsigned long long* wp = zw + (size_t)rep * D + 4 * c;
+          ld_relaxed_v2u64(wp, w[rep][0], w[rep][1]);
+          ld_relaxed_v2u64(wp + 2, w[rep][2], w[rep][3]);
+        }
+        done = true;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          sum[e] = 0ull;
+#pragma unroll
+          for (int rep = 0; rep < kFixRep; ++rep) sum[e] += w[rep][e];
+          done = done && ((((long long)(sum[e] - zprev[j][e])) + (1ll << 55)) >> 56) == (long long)R;
+        }
+      }
+      if (!done && *ok) {
+        *ok = 0;
+        atomicOr(a.status, npp::kStatTimeout);
+      }
+      float zv[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        zv[e] = done ? __ll2float_rn((long long)(sum[e] - zprev[j][e]) - ((long long)R << 56)) * (1.f / (float)(1u << kFixShift)) : 0.f;
+      reinterpret_cast<float4*>(a.x_out + qoff)[c] =
+          make_float4(xown[j].x + zv[0], xown[j].y + zv[1], xown[j].z + zv[2], xown[j].w + zv[3]);
+    }
+  }
 }
 
 bool plan(const Dims& d, int sm_count, Plan* p) {
@@ -979,6 +1020,11 @@ bool supported(const Dims& d, int sm_count) {
   return plan(d, sm_count, &p);
 }
 
+bool counted_handover(const Dims& d, int sm_count) {
+  Plan p;
+  return plan(d, sm_count, &p) && p.ks <= kFixMaxKS;
+}
+
 size_t xch_words(const Dims& d, int sm_count) {
   Plan p;
   if (!plan(d, sm_count, &p)) return 16;
@@ -1022,6 +1068,9 @@ cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s,
     ka.counters = a.counters;
     ka.x_bf16 = l0 == 0 ? static_cast<const uint16_t*>(a.x_bf16) : nullptr;
     for (int i = 0; i < 2; ++i) ka.xbuf[i] = a.xbuf[i];
+    // the launch that ends the stack leaves the result itself where the hand-over is counted
+    ka.x_out = (p.ks <= kFixMaxKS && std::min(a.l_end, l0 + p.run_layers) == a.l_end) ? a.x_out : nullptr;
+    st->wrote_out = ka.x_out != nullptr;
     for (int i = 0; i < 3; ++i) ka.zbuf[i] = a.zbuf[i];
     ka.zfix = st->zfix;
     ka.bars = st->bars;
@@ -1044,7 +1093,8 @@ cudaError_t launch(const Dims& d, const ChainArgs& a, State* st, cudaStream_t s,
     ka.group_bytes = (uint32_t)p.group_bytes;
     const int nl = ka.l_end - ka.l_begin;
     // the counters and stamps only ever grow; the next launch starts where this one ends
-    if (nl > 1) st->bar_base += (p.ks <= kFixMaxKS ? 1u : (unsigned int)(nl - 1)) * (unsigned int)p.R;
+    if (p.ks <= kFixMaxKS) st->bar_base += (nl > 1 || ka.x_out) ? (unsigned int)p.R : 0u;
+    else if (nl > 1) st->bar_base += (unsigned int)(nl - 1) * (unsigned int)p.R;
     st->seq_base += (unsigned int)nl + 1u;
     const bool xb = ((d.D / kQ / 16) >> p.gw_shift) <= 32 && p.ks <= 16;  // phase 1's B operands fit a warp's registers
     if (p.ks == 8) e = xb ? launch_one<8, true>(ka, p.smem, p.R * kQ, s) : launch_one<8, false>(ka, p.smem, p.R * kQ, s);

@@ -317,6 +317,36 @@ def test_resident_chain_with_set_sizes_away_from_k(n_set, flags):
         p.close()
 
 
+def test_chain_in_one_launch_is_reproducible_bit_for_bit():
+    """On resident rows the whole stack is one resident launch, its sums between layers and behind the last one
+    are integer adds (which commute) and the exchange adds its four slices in a fixed order: the result does not
+    depend on the order in which the blocks arrive, so repeated calls give the same bits."""
+    cfg = DENSE
+    p = Pair(cfg, chain_layers=cfg.n_layers)
+    try:
+        assert nb.np_mlp_kernel_name(p.eng.ctx, 1) == "k_mlp_slices"
+        xs = synth.hidden_states(cfg, 2)
+        out = torch.empty((1, cfg.d_model), dtype=torch.float32, device="cuda")
+        logits = torch.empty((1, cfg.n_layers, cfg.d_ffn), dtype=torch.float32, device="cuda")
+        nb.np_predict(p.eng.ctx, xs[0].cuda(), 1, logits, None, p.eng.stream)
+        nb.np_step(p.eng.ctx, xs[0].cuda(), 1, out, p.eng.stream, p.eng.copy_stream)
+        torch.cuda.synchronize()
+        res = p.ora.step(u16(xs[0]), logits_f32=logits.cpu().numpy())
+        runs = []
+        for _ in range(6):
+            o = torch.empty_like(out)
+            nb.np_mlp_chain(p.eng.ctx, xs[0].cuda(), 1, o, p.eng.stream)
+            torch.cuda.synchronize()
+            assert nb.np_chain_launches(p.eng.ctx) == 1
+            runs.append(o.cpu().numpy())
+        assert rel_l2(runs[0], res["x_final"]) < 1e-5
+        for o in runs[1:]:
+            assert (o.view(np.uint32) == runs[0].view(np.uint32)).all()
+        p.eng.counters()
+    finally:
+        p.close()
+
+
 def test_partial_sums_beyond_the_counted_words_range_are_reported():
     """Between the layers of a launch the resident kernel hands the MLP's partial sums over as counted
     fixed-point words (|sum| < 2^19 per block).  Down rows of 3e6 push layer 0 far past that: the launch
