@@ -38,7 +38,8 @@
 //    until every block of its slice has done that reading (one arrival counter per slice, counted
 //    once per launch and long complete by the time the first layer ends).  The launch's last layer
 //    leaves its sums as fp32 in the stack's rotating accumulators, the form every other kernel of
-//    the chain reads.
+//    the chain reads -- unless the launch ends the stack: then the last layer's sums go through the
+//    counted words too, and the blocks of row group 0 wait for them and write the stack's result.
 //
 //    This form is used where a thread owns one or two 4-column granules of the slice (row widths
 //    up to 8192).  Wider slices keep the fp32 form between all layers: 16-byte fp32 reductions into
