@@ -978,8 +978,17 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   // phase 1 deals a layer's gate|up groups to sets of GW warps: as many sets as the expected share has groups
   const long long expect = std::min<long long>(d.C, std::max(1, d.k));
   const int n_gu_typ = (int)((2 * ((expect + R - 1) / R) + VG - 1) / VG);
+  // ... but never a warp alone on a long K range: with more groups than warps (70B shape: ten groups of eight
+  // 4 KB vectors) one warp per group walks through all 128 K blocks twice per layer; pairs walk through 64 three
+  // times (1.51 ms per 80 layers against 1.58).  Four warps per group
+  // measured worse at every shape (70B 1.82 ms, 13B 449 us against 357, 7B 261 us against 248): the layer's groups
+  // are then worked on one or two at a time, and each has to have landed whole.
   int gw_shift = 3;
   while (gw_shift > 0 && (kWarps >> gw_shift) < n_gu_typ) --gw_shift;
+  if (gw_shift == 0 && nk >= 64) gw_shift = 1;
+#ifdef NP_TUNE
+  if (const char* e = getenv("NP_SL_GW")) gw_shift = std::max(0, std::min(3, atoi(e)));
+#endif
   const int GW = 1 << gw_shift;
   // everything but the ring and the slot cache; the cache (the slots of a launch's rows) takes a minimum first
   // and, once the ring's slots are counted, whatever is left, so that a launch can span more layers
