@@ -96,7 +96,8 @@ constexpr int kFixRep = NP_SL_FIXREP;  // copies of the counted words (row group
                                        // adds to a word cost less than reading more copies (7B shape, 32 layers: 250 us
                                        // with one copy, 252 with two, 262 with four)
 constexpr int kHist = 8;               // pacing history of the producer (> window)
-constexpr int kGroupTarget = 42 * 1024;
+constexpr int kGroupTarget = 68 * 1024;  // largest load group: up to 16 vectors, three groups to a ring at least (70B shape:
+                                         // 66 KB groups of 16 vectors, 1.39 ms per 80 layers; 33 KB groups of 8: 1.51 ms)
 constexpr int kPad = 16;               // bytes between pieces in shared memory
 
 struct KArgs {
@@ -967,9 +968,13 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   if (R > kMaxR) return false;
   const size_t pstride = (size_t)Ds * 2 + kPad;
   const int max_rows = (d.C + R - 1) / R;  // whatever the active count turns out to be
-  // a group: VG vectors (a power of two, at most the 16 rows of an MMA tile), about 32 KB
+  // a group: VG vectors (a power of two, at most the 16 rows of an MMA tile), up to kGroupTarget bytes
+  size_t group_target = kGroupTarget;
+#ifdef NP_TUNE
+  if (const char* e = getenv("NP_SL_GT")) group_target = (size_t)atoi(e) * 1024;
+#endif
   int vg_shift = 1;
-  while (vg_shift < 4 && ((size_t)2 << vg_shift) * pstride <= (size_t)kGroupTarget) ++vg_shift;
+  while (vg_shift < 4 && ((size_t)2 << vg_shift) * pstride <= group_target) ++vg_shift;
   const int VG = 1 << vg_shift;
   const size_t group_bytes = (size_t)VG * pstride;
   const size_t budget = 227 * 1024 - 2048;  // static shared memory of the kernel
