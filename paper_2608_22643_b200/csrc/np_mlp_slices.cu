@@ -1012,6 +1012,7 @@ bool plan(const Dims& d, int sm_count, Plan* p) {
   // flight: a deeper burst queues in front of its fence and of the short loads behind it (13B shape, when it
   // still used this form: 385 us with one 41 KB group in flight, 411 with two or more).
   int window = ks <= kFixMaxKS ? std::max(1, std::min(ng - 1, kHist - 1)) : std::max(1, std::min(ng - 1, (int)(40 * 1024 / group_bytes)));
+  if (ng <= 3) window = 1;  // a ring of three large groups (70B shape, 66 KB each): 1.36 ms per 80 layers with one in flight, 1.39 with two
 #ifdef NP_TUNE  // development builds only: geometry from the environment
   if (const char* e = getenv("NP_SL_NG")) ng = std::max(2, std::min(ng, atoi(e)));
   if (const char* e = getenv("NP_SL_WIN")) window = std::min(atoi(e), std::min(kHist - 1, ng - 1));
