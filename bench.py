@@ -228,6 +228,25 @@ def make_workload(cfg, gen_device: str, pin: bool, store_layers=None):
     return w1, w2, store, time.time() - t0
 
 
+def make_pinned_workload(cfg, Lp, lp_why, floor_layers=0, may_shrink=True, make=None):
+    """make_workload with a page-locked store of Lp layers.  The host may refuse to page-lock a store that
+    MemAvailable said would fit (a limit on locked memory, a fragmented host): then the store is aliased over
+    three quarters of the layers, and so on down to an eighth of the stack (or the dense prefix, which must be
+    whole).  Returns (w1, w2, store, seconds, layers held, why)."""
+    make = make or make_workload
+    while True:
+        try:
+            w1, w2, store, gen_s = make(cfg, "cuda", pin=True, store_layers=Lp)
+            return w1, w2, store, gen_s, Lp, lp_why
+        except RuntimeError as e:
+            if "cudaHostRegister" not in str(e) or not may_shrink or Lp <= max(1, floor_layers, cfg.n_layers // 8):
+                raise
+            if torch.cuda.is_available():
+                torch.cuda.synchronize()
+            lp_why = f"the host refused to page-lock {Lp} layers ({Lp * cfg.d_ffn * cfg.record_bytes / 2**30:.0f} GiB)"
+            Lp = max(floor_layers, max(1, cfg.n_layers // 8), (3 * Lp) // 4)
+
+
 def run_oracle_steps(cfg, policy, w1, w2, store, xs, n_steps, layers=None):
     """Times the oracle, as it stands, on steps 1..n_steps of the sequence (step 0 is
     the cold start and is run untimed).  Returns seconds per timed step."""
@@ -365,19 +384,8 @@ def cuda_arm(args):
     Lp, lp_why = plan_store_layers(cfg, args.store_layers, int(os.environ.get("LOCAL_WORLD_SIZE", world)))
     if Lp < cfg.n_layers and (args.transfer == "file" or args.dense_layers > Lp):
         raise SystemExit("bench.py: an aliased store is not combined with --transfer file or a longer dense prefix here")
-    # The host may refuse to page-lock a store that MemAvailable said would fit (a limit on locked memory, a
-    # fragmented host): then the store is aliased over three quarters of the layers, and so on.
-    while True:
-        try:
-            w1, w2, store, gen_s = make_workload(cfg, "cuda", pin=True, store_layers=Lp)
-            break
-        except RuntimeError as e:
-            if "cudaHostRegister" not in str(e) or Lp <= max(1, cfg.n_layers // 8) or args.transfer == "file" \
-                    or args.store_layers != "auto":
-                raise
-            torch.cuda.synchronize()
-            lp_why = f"the host refused to page-lock {Lp} layers ({Lp * cfg.d_ffn * cfg.record_bytes / 2**30:.0f} GiB)"
-            Lp = max(args.dense_layers, max(1, (3 * Lp) // 4))
+    w1, w2, store, gen_s, Lp, lp_why = make_pinned_workload(cfg, Lp, lp_why, floor_layers=args.dense_layers,
+                                                            may_shrink=args.transfer != "file" and args.store_layers == "auto")
     # replicas share one host: the packing threads of the gather transfer are divided among them
     if args.host_threads == 0 and world > 1:
         args.host_threads = nb.replica_host_threads(int(os.environ.get("LOCAL_WORLD_SIZE", world)))

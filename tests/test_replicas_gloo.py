@@ -5,6 +5,8 @@ import os
 import subprocess
 import sys
 
+import pytest
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -56,3 +58,34 @@ def test_reference_arm_runs_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                        env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_store_shrinks_when_the_host_refuses_to_pin_it():
+    """bench.py's store sizing: a refusal to page-lock the store makes it retry with three quarters of the layers
+    (the stack then reads layer l mod Lp), not below an eighth of the stack or the dense prefix; other errors
+    and fixed layer counts are passed on."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2608_22643_b200 import synth
+    cfg = synth.CONFIGS["70b"]
+    asked = []
+
+    def fake(cfg_, dev, pin, store_layers):
+        asked.append(store_layers)
+        if store_layers > 50:
+            raise RuntimeError("cudaHostRegister failed with 2")
+        return "w1", "w2", "store", 0.5
+
+    out = bench.make_pinned_workload(cfg, 74, "host has 195 GiB available", make=fake)
+    assert asked == [74, 55, 41] and out[4] == 41 and "refused to page-lock 55 layers" in out[5]
+    asked.clear()
+    with pytest.raises(RuntimeError):
+        bench.make_pinned_workload(cfg, 74, "", may_shrink=False, make=fake)
+    assert asked == [74]
+    with pytest.raises(RuntimeError):          # never below the dense prefix
+        bench.make_pinned_workload(cfg, 74, "", floor_layers=60, make=fake)
+
+    def other(cfg_, dev, pin, store_layers):
+        raise RuntimeError("out of memory")
+    with pytest.raises(RuntimeError, match="out of memory"):
+        bench.make_pinned_workload(cfg, 74, "", make=other)
