@@ -42,6 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # sparse-MLP kernels, from the ncu captures summarised under profiles/: (kernel, config) -> (bytes, file)
 NCU_TRAFFIC = {
     ("k_mlp_slices", "7b"): (27.236e6, "profiles/k_mlp_slices_7b.md"),
+    ("k_mlp_slices", "13b"): (34.110e6, "profiles/k_mlp_slices_13b.md"),
 }
 
 
