@@ -289,10 +289,11 @@ __global__ void __launch_bounds__(kMlpThreads, 1) k_sparse_mlp_pipe(MlpPipeArgs 
     unsigned char* dst = psm + (size_t)s * rec_bytes;
     const size_t off = (size_t)slot * row_bytes;
     npp::mbar_expect_tx(&full_bar[s], rec_bytes);
-    npp::bulk_g2s(dst, reinterpret_cast<const unsigned char*>(a.gate) + off, row_bytes, &full_bar[s]);
-    npp::bulk_g2s(dst + row_bytes, reinterpret_cast<const unsigned char*>(a.up) + off, row_bytes, &full_bar[s]);
-    npp::bulk_g2s(dst + 2 * row_bytes, reinterpret_cast<const unsigned char*>(a.downT) + off, row_bytes,
-                  &full_bar[s]);
+    const uint64_t pol = npp::policy_evict_first();  // weight rows are read once per token
+    npp::bulk_g2s_stream(dst, reinterpret_cast<const unsigned char*>(a.gate) + off, row_bytes, &full_bar[s], pol);
+    npp::bulk_g2s_stream(dst + row_bytes, reinterpret_cast<const unsigned char*>(a.up) + off, row_bytes, &full_bar[s], pol);
+    npp::bulk_g2s_stream(dst + 2 * row_bytes, reinterpret_cast<const unsigned char*>(a.downT) + off, row_bytes,
+                         &full_bar[s], pol);
   };
 
   if (tid == 0) {

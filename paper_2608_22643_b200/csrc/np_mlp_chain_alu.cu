@@ -170,9 +170,10 @@ __global__ void __launch_bounds__(kChainBlock, 1) k_mlp_chain(ChainKernelArgs a)
         const size_t off = (size_t)(a.l_begin + ll) * layer_bytes + (size_t)slot_cache[v] * row_pitch;
         unsigned char* dst = csm + (size_t)s * rec_bytes;
         npp::mbar_expect_tx(&full_bar[s], rec_bytes);
-        npp::bulk_g2s(dst, a.gate + off, row_bytes, &full_bar[s]);
-        npp::bulk_g2s(dst + row_bytes, a.up + off, row_bytes, &full_bar[s]);
-        npp::bulk_g2s(dst + 2 * row_bytes, a.downT + off, row_bytes, &full_bar[s]);
+        const uint64_t pol = npp::policy_evict_first();  // weight rows are read once per token
+        npp::bulk_g2s_stream(dst, a.gate + off, row_bytes, &full_bar[s], pol);
+        npp::bulk_g2s_stream(dst + row_bytes, a.up + off, row_bytes, &full_bar[s], pol);
+        npp::bulk_g2s_stream(dst + 2 * row_bytes, a.downT + off, row_bytes, &full_bar[s], pol);
         if (++s == n_stages) {
           s = 0;
           ++use;

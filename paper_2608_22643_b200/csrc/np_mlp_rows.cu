@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_rows(KArgs a) {
           good = false;
         } else {
           npp::mbar_expect_tx(&full_bar[s], row_bytes);
-          npp::bulk_g2s(csm + (size_t)s * pstride, src, row_bytes, &full_bar[s]);
+          npp::bulk_g2s_stream(csm + (size_t)s * pstride, src, row_bytes, &full_bar[s], npp::policy_evict_first());
         }
       }
       good = __all_sync(0xffffffffu, good);
@@ -410,9 +410,9 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_rows(KArgs a) {
           return;
         }
         npp::mbar_expect_tx(&ds_full[s], row_bytes);
-        npp::bulk_g2s(dstage + (size_t)s * pstride,
-                      a.downT + (size_t)(a.l_begin + li_n) * layer_bytes + (size_t)slot_cache[lay_pre[li_n] + r_n] * row_bytes, row_bytes,
-                      &ds_full[s]);
+        npp::bulk_g2s_stream(dstage + (size_t)s * pstride,
+                             a.downT + (size_t)(a.l_begin + li_n) * layer_bytes + (size_t)slot_cache[lay_pre[li_n] + r_n] * row_bytes,
+                             row_bytes, &ds_full[s], npp::policy_evict_first());
         ++kn;
         ++r_n;
       };

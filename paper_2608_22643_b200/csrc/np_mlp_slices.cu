@@ -344,6 +344,10 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
     uint32_t hist_par[kHist];
     int issued = 0, slot = 0;
     uint32_t par = 0;
+    // A row is read once per token: the copies mark their lines evict-first, so that the 27 MB a layer streams
+    // through the L2 do not push out the few hundred KB every layer meets in (exchange words, counted sums,
+    // slot lists): 7B shape 236 us per 32 layers against 249, 13B shape 341 us per 40 layers against 358.
+    const uint64_t l2_policy = npp::policy_evict_first();
     const size_t qbytes = (size_t)q * piece_bytes;
     for (int li = 0; li < nl; ++li) {
       const int vbase = lay_pre[li], nrows = lay_pre[li + 1] - vbase;
@@ -381,7 +385,7 @@ __global__ void __launch_bounds__(kBlock, 1) k_mlp_slices(KArgs a) {
             const int i = pass == 0 ? idx >> 1 : idx;
             const size_t off = lbase + (size_t)slot_cache[vbase + r0 + i] * row_bytes;
             const unsigned char* src = (pass == 0 ? ((idx & 1) ? a.up : a.gate) : a.downT) + off;
-            npp::bulk_g2s(dst + (size_t)idx * pstride, src, piece_bytes, &full_bar[slot]);
+            npp::bulk_g2s_stream(dst + (size_t)idx * pstride, src, piece_bytes, &full_bar[slot], l2_policy);
           }
           __syncwarp();
           if (++slot == ng) {

@@ -162,8 +162,9 @@ __device__ __forceinline__ void issue_up_tile(const Blk& k, const unsigned char*
   if (lane < rows) {
     const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r0 + lane) * k.row_pitch + k.slice_off;
     unsigned char* dst = tile + (size_t)lane * k.row_stride;
-    bulk_g2s(dst, gate + src, k.slice_bytes, full);
-    bulk_g2s(dst + (size_t)kUpTile * k.row_stride, up + src, k.slice_bytes, full);
+    const uint64_t pol = policy_evict_first();  // weight rows are read once per token
+    bulk_g2s_stream(dst, gate + src, k.slice_bytes, full, pol);
+    bulk_g2s_stream(dst + (size_t)kUpTile * k.row_stride, up + src, k.slice_bytes, full, pol);
   }
 }
 
@@ -177,7 +178,7 @@ __device__ __forceinline__ void issue_down_tile(const Blk& k, const unsigned cha
   if (lane < kDownTile) {
     const int r = r0 + min(lane, rows - 1);
     const size_t src = (size_t)slot_of(k, slots, s_slots, r_begin, r) * k.row_pitch + k.slice_off;
-    bulk_g2s(tile + (size_t)lane * k.row_stride, downT + src, k.slice_bytes, full);
+    bulk_g2s_stream(tile + (size_t)lane * k.row_stride, downT + src, k.slice_bytes, full, policy_evict_first());
   }
 }
 
