@@ -41,8 +41,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per layer (dram__bytes_read.sum + dram__bytes_write.sum of one launch / its layers) of the
 # sparse-MLP kernels, from the ncu captures summarised under profiles/: (kernel, config) -> (bytes, file)
 NCU_TRAFFIC = {
-    ("k_mlp_slices", "7b"): (27.236e6, "profiles/k_mlp_slices_7b.md"),
-    ("k_mlp_slices", "13b"): (34.110e6, "profiles/k_mlp_slices_13b.md"),
+    ("k_mlp_slices", "7b"): (27.201e6, "profiles/k_mlp_slices_7b.md"),
+    ("k_mlp_slices", "13b"): (34.084e6, "profiles/k_mlp_slices_13b.md"),
 }
 
 
